@@ -1,0 +1,231 @@
+/*
+ * topoep.h -- C boundary of the TopoEP planning step for one GPU (sm_100a).
+ *
+ * One call, topoep_plan(), turns the router's top-k expert ids of a whole
+ * expert-parallel (EP) group into a replica placement x, a token routing q,
+ * a per-token physical-instance assignment and the dispatch layout, for a
+ * batch of independent (layer, microbatch) plans.  Everything is integer
+ * arithmetic; the result is a pure function of (configuration, topk_ids) and
+ * is bitwise reproducible across runs and launch configurations.
+ *
+ * Notation (paper, "System Model"): M NVLink domains (nodes), G GPUs per
+ * node, R = M*G EP ranks, E logical experts, N_slot replica slots per rank,
+ * k experts per token, T tokens per rank, B plans per call.
+ * dom(r) = r / G.  main(e) is the fixed main rank of expert e.
+ *
+ * Physical instances.  E_loc = max_r |{e : main(e) = r}|, S_phys = E_loc +
+ * N_slot, P = R * S_phys.  Instance id p = r * S_phys + l lives on rank r;
+ * l < E_loc is the l-th expert (ascending e) whose main rank is r, and
+ * l = E_loc + j is replica slot j of rank r.  rank(p) = p / S_phys.
+ *
+ * Pointers.  Every pointer named dev_* or documented "device" is a device
+ * pointer owned by the caller; every other pointer is a host pointer.  The
+ * library allocates no device memory: tables and scratch live in a workspace
+ * the caller hands over with topoep_set_workspace().  topoep_plan() and the
+ * other enqueue calls copy nothing to the host, never synchronise, and only
+ * enqueue kernels on the given stream.
+ *
+ * Errors.  Every int-returning function returns TOPOEP_OK (0) or a negative
+ * topoep_status code; nothing aborts or throws.  Conditions only the device
+ * can see (an id outside [0,E) other than -1, the refinement cap binding) set
+ * bits in a device status word read by topoep_read_status(); the plan stays
+ * well defined (invalid ids are ignored and map to -1).
+ */
+#ifndef TOPOEP_H_
+#define TOPOEP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct topoep_ctx* topoep_handle_t;
+/* Same type as cudaStream_t; NULL is the legacy default stream. */
+typedef struct CUstream_st* topoep_stream_t;
+
+typedef enum {
+  TOPOEP_OK = 0,
+  TOPOEP_ERR_NULL = -1,        /* a required pointer is NULL                     */
+  TOPOEP_ERR_CONFIG = -2,      /* topology / expert / slot numbers out of range  */
+  TOPOEP_ERR_MAIN_MAP = -3,    /* main_rank entry outside [0,R), or E % R != 0
+                                  with a NULL map                                */
+  TOPOEP_ERR_COST = -4,        /* negative byte size or cost coefficient         */
+  TOPOEP_ERR_WORKSPACE = -5,   /* workspace missing, too small or misaligned     */
+  TOPOEP_ERR_SIZE = -6,        /* tokens_per_rank or batch outside [0, max]      */
+  TOPOEP_ERR_ALIGN = -7,       /* an int32 buffer is not 4-byte aligned          */
+  TOPOEP_ERR_CUDA = -8,        /* a CUDA runtime call failed (see last error)    */
+  TOPOEP_ERR_SMEM = -9,        /* problem does not fit one SM's shared memory    */
+  TOPOEP_ERR_ARG = -10         /* unknown selector / knob / value                */
+} topoep_status;
+
+/* Device status bits (topoep_read_status). */
+#define TOPOEP_FLAG_BAD_ID      1u  /* some id was outside [0,E) and not -1      */
+#define TOPOEP_FLAG_REFINE_CAP  2u  /* refinement stopped by max_refine_iters    */
+#define TOPOEP_FLAG_INTERNAL    4u  /* a device-side self check failed           */
+
+/*
+ * Cost model (paper, "System Model" and Eq. for b_{d,e}, T_token, T_replica).
+ * The communication-time matrix C has two levels: c_intra between ranks of
+ * one domain, c_inter between domains, 0 on the diagonal.  All experts share
+ * one parameter size.
+ */
+typedef struct {
+  int64_t token_bytes;      /* S_tok: bytes of one routed activation             */
+  int64_t expert_bytes;     /* ||W_e||: bytes of one expert's parameters         */
+  int32_t c_intra;          /* per-byte time inside a domain, integer units      */
+  int32_t c_inter;          /* per-byte time across domains, integer units       */
+  int64_t t_ffn;            /* per-assignment compute time; summaries only       */
+  int32_t max_refine_iters; /* cap per domain; <= 0 selects 256                  */
+  int32_t min_delta;        /* smallest transfer refinement commits; <= 0 -> 1   */
+} topoep_cost_params;
+
+/*
+ * Derived figures of one plan (paper: objective terms T_comp, T_token,
+ * T_replica; max/mean rank-load ratio; inter-node and replica-served
+ * fractions of the "Topology-Aware Token Routing" evaluation).  Integers are
+ * exact; the three doubles are one IEEE division each of the integers beside
+ * them.
+ */
+typedef struct {
+  int64_t assignments;        /* valid (token, expert) pairs = sum_r L_r          */
+  int64_t l_max;              /* max_r L_r                                        */
+  int64_t cross_assignments;  /* executed in another domain than their source     */
+  int64_t replica_served;     /* executed on a rank other than main(e)            */
+  int64_t replicas_inter;     /* replicas in a domain other than their main's     */
+  int64_t replicas_intra;     /* replicas in their main's domain                  */
+  int64_t t_comp;             /* t_ffn * l_max                                    */
+  int64_t t_token;            /* 2 * S_tok * sum c(s,r) q(s,e,r)                  */
+  int64_t t_replica;          /* sum over replicas c(main(e),r) * ||W||           */
+  int64_t cross_token_bytes;  /* 2 * S_tok * cross_assignments (exposed half)     */
+  int64_t refine_iters;       /* refinement commits summed over domains           */
+  int64_t reserved;
+  double  imbalance;          /* l_max * R / assignments  (0 if none)             */
+  double  cross_fraction;     /* cross_assignments / assignments                  */
+  double  replica_fraction;   /* replica_served / assignments                     */
+} topoep_summary_t;
+
+/* Selectors for topoep_debug_tensor (all device int32, laid out as stated). */
+enum {
+  TOPOEP_T_OMEGA = 0,       /* [max_batch][R][E]   routing matrix Omega           */
+  TOPOEP_T_Q = 1,           /* [max_batch][R][P]   q(s, instance)                 */
+  TOPOEP_T_RANK_LOAD = 2,   /* [max_batch][R]      L_r                            */
+  TOPOEP_T_REFINE_ITERS = 3 /* [max_batch][M]      commits per domain             */
+};
+
+/* Knobs for topoep_set_tuning; no knob may change any output bit. */
+enum {
+  TOPOEP_KNOB_TILE_IDS = 0,     /* ids per histogram / reroute tile: 1024..16384,
+                                   power of two                                   */
+  TOPOEP_KNOB_HIST_MODE = 1     /* 0 = warp-aggregated (match) shared atomics,
+                                   1 = plain shared atomics                       */
+};
+
+/*
+ * Create a planner for an M x G topology.  (Paper, "System Model": sets D, R,
+ * E, dom(), main(), N_slot, C, S_tok, ||W||, t_FFN.)
+ *   nodes M in [1,64]; gpus_per_node G in [1,32]; experts E >= 1;
+ *   slots_per_rank N_slot >= 0; top_k k >= 1;
+ *   max_tokens_per_rank, max_batch >= 1 bound later topoep_plan sizes.
+ *   main_rank_host: host array of E ranks, or NULL for the blocked map
+ *   main(e) = e / (E / R), which needs E % R == 0.  Copied; not retained.
+ *   cost: host struct, copied.
+ * Allocates host memory only.  *out is untouched on error.
+ */
+int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int experts,
+                  int slots_per_rank, int top_k, int max_tokens_per_rank,
+                  int max_batch, const int32_t* main_rank_host,
+                  const topoep_cost_params* cost);
+
+/* Frees host state.  The workspace stays the caller's.  NULL is a no-op. */
+void topoep_destroy(topoep_handle_t h);
+
+/* Bytes of device workspace the handle needs (a multiple of 256). 0 if h NULL. */
+size_t topoep_workspace_bytes(topoep_handle_t h);
+
+/*
+ * Hand over the workspace: dev_ptr is device memory, 256-byte aligned, at
+ * least topoep_workspace_bytes(h) long, and stays valid and untouched by the
+ * caller until topoep_destroy or the next topoep_set_workspace.  Uploads the
+ * constant tables and zeroes the counters on the CURRENT device, then
+ * synchronises the device: call it outside stream capture.
+ */
+int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes);
+
+/*
+ * Plan B batches.  (Paper: routing matrix Omega; "Two-Stage GPU-Native
+ * Solver": inter-node placement with b_{d,e}, routing construction, loads
+ * U and L, intra-node refinement with the half-gap delta; constraints
+ * C1-C5; "derives receive counts on the GPU".)
+ *
+ *   dev_topk_ids        in  [B][R][T][k] int32, expert id per assignment; ids
+ *                           outside [0,E) are ignored (-1 is the padding value)
+ *   tokens_per_rank     T in [0, max_tokens_per_rank]
+ *   batch               B in [0, max_batch]
+ *   dev_replica_map     out [B][R][N_slot] expert in replica slot j, -1 if free
+ *                           (may be NULL only when N_slot == 0)
+ *   dev_token_replica   out [B][R][T][k] physical instance id executing the
+ *                           assignment, -1 for an ignored id
+ *   dev_dispatch_counts out [B][R][R]   counts[s][r] = assignments of source s
+ *                           executed on rank r
+ *   dev_dispatch_offsets out [B][2][R][R+1]: [0][s][.] exclusive scan over r of
+ *                           counts[s][.] (send offsets; entry R = row total),
+ *                           [1][r][.] exclusive scan over s of counts[.][r]
+ *                           (receive offsets; entry R = L_r)
+ *   dev_instance_counts out [B][P] U: assignments per physical instance, or NULL
+ *
+ * Within a (plan, source, expert) group, assignments are ranked by flat index
+ * t*k+j and dealt to the expert's instances in ascending rank order, each
+ * taking q(s,e,r) of them.  Enqueues three kernels on `stream`; capturable in
+ * a CUDA graph.  Two plans on one handle must not overlap on the device.
+ */
+int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
+                int batch, int32_t* dev_replica_map, int32_t* dev_token_replica,
+                int32_t* dev_dispatch_counts, int32_t* dev_dispatch_offsets,
+                int32_t* dev_instance_counts, topoep_stream_t stream);
+
+/*
+ * Histogram step alone (paper, Eq. Omega): dev_omega [B][R][E] int32 gets the
+ * number of assignments of source rank s that select expert e.  Uses the
+ * workspace for per-tile counts.  Same argument rules as topoep_plan.
+ */
+int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
+                     int batch, int32_t* dev_omega, topoep_stream_t stream);
+
+/*
+ * Summaries of the last topoep_plan (paper: objective terms and evaluation
+ * ratios, see topoep_summary_t).  dev_out: [batch] topoep_summary_t, 8-byte
+ * aligned.  Enqueues one kernel; off the planning path.
+ */
+int topoep_summary(topoep_handle_t h, int batch, topoep_summary_t* dev_out,
+                   topoep_stream_t stream);
+
+/*
+ * Copy the device status word to *host_flags and clear it.  Synchronises the
+ * stream's device: for tests and health checks, not for the planning path.
+ */
+int topoep_read_status(topoep_handle_t h, uint32_t* host_flags);
+
+/* Device address and byte size of an intermediate tensor inside the workspace. */
+int topoep_debug_tensor(topoep_handle_t h, int which, const void** dev_ptr, size_t* bytes);
+
+/* Change a launch-shape knob; outputs are identical for every legal value. */
+int topoep_set_tuning(topoep_handle_t h, int knob, int value);
+
+/* Derived sizes: E_loc, S_phys, P.  Any output pointer may be NULL. */
+int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances);
+
+/*
+ * Enqueue `count` empty kernels on the stream: the launch floor a plan's
+ * kernel chain is compared against.  Not part of the method.
+ */
+int topoep_launch_floor(int count, topoep_stream_t stream);
+
+/* Static text for a status code. */
+const char* topoep_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOPOEP_H_ */
