@@ -1,0 +1,373 @@
+// C boundary of the TopoEP planning library: argument checks, workspace carving, kernel
+// enqueue.  Nothing here allocates, frees or copies device memory on the planning path; the
+// plan call enqueues three kernels (histogram, solver + layout, reroute) on the caller's stream.
+#include <algorithm>
+#include <new>
+
+#include "topoep_internal.cuh"
+
+using namespace topoep;
+
+struct topoep_ctx {
+  Dims d;
+  int max_tokens, max_batch;
+  topoep_cost_params cost;
+  int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
+  std::vector<int32_t> main_rank, main_local, main_inst_expert;
+  int tile_ids, hist_mode;
+  int max_tiles;
+  // workspace
+  bool have_ws;
+  Workspace ws;
+  size_t off[16];
+  size_t ws_bytes;
+  cudaError_t last_cuda;
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+enum WsSlot {
+  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_STATUS, W_HTICKETS, W_STICKETS, W_OMEGA, W_TILE,
+  W_Q, W_LOAD, W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_SEG, W_INST_SORTED, W_SLOTS
+};
+static_assert(W_SLOTS == 16, "offset table size");
+
+void carve(topoep_ctx* h) {
+  const Dims& d = h->d;
+  const size_t B = (size_t)h->max_batch, R = d.R, E = d.E, P = d.P;
+  size_t sz[W_SLOTS];
+  sz[W_MAIN_RANK] = 4 * E;
+  sz[W_MAIN_LOCAL] = 4 * E;
+  sz[W_MAIN_INST] = 4 * R * (size_t)std::max(d.e_loc, 1);
+  sz[W_STATUS] = 4;
+  sz[W_HTICKETS] = 4 * B * R;
+  sz[W_STICKETS] = 4 * B;
+  sz[W_OMEGA] = 4 * B * R * E;
+  sz[W_TILE] = 4 * B * R * (size_t)h->max_tiles * E;
+  sz[W_Q] = 4 * B * R * P;
+  sz[W_LOAD] = 4 * B * R;
+  sz[W_ITERS] = 4 * B * (size_t)d.M;
+  sz[W_INST_COUNTS] = 4 * B * P;
+  sz[W_REPLICA_MAP] = 4 * B * R * (size_t)std::max(d.N, 1);
+  sz[W_COUNTS] = 4 * B * R * R;
+  sz[W_SEG] = 4 * B * (E + 1);
+  sz[W_INST_SORTED] = 4 * B * P;
+  size_t at = 0;
+  for (int i = 0; i < W_SLOTS; ++i) { h->off[i] = at; at += align_up(sz[i]); }
+  h->ws_bytes = at;
+}
+
+template <typename T>
+T* at(void* base, size_t off) { return reinterpret_cast<T*>(static_cast<char*>(base) + off); }
+
+int check_sizes(topoep_ctx* h, int tokens_per_rank, int batch) {
+  if (!h) return TOPOEP_ERR_NULL;
+  if (!h->have_ws) return TOPOEP_ERR_WORKSPACE;
+  if (tokens_per_rank < 0 || tokens_per_rank > h->max_tokens) return TOPOEP_ERR_SIZE;
+  if (batch < 0 || batch > h->max_batch) return TOPOEP_ERR_SIZE;
+  return TOPOEP_OK;
+}
+
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omega) {
+  HistParams p;
+  p.d = h->d;
+  p.ws = h->ws;
+  p.ids = ids;
+  p.out_omega = out_omega;
+  p.n_ids = T * h->d.k;
+  p.tile_ids = h->tile_ids;
+  p.tiles = std::max(1, (p.n_ids + h->tile_ids - 1) / h->tile_ids);
+  p.max_tiles = h->max_tiles;
+  p.vec_ok = (p.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0);
+  return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int experts,
+                  int slots_per_rank, int top_k, int max_tokens_per_rank, int max_batch,
+                  const int32_t* main_rank_host, const topoep_cost_params* cost) {
+  if (!out || !cost) return TOPOEP_ERR_NULL;
+  if (nodes < 1 || nodes > 64 || gpus_per_node < 1 || gpus_per_node > 32) return TOPOEP_ERR_CONFIG;
+  if (experts < 1 || experts >= (1 << 23) || slots_per_rank < 0 || slots_per_rank > 1024)
+    return TOPOEP_ERR_CONFIG;
+  if (top_k < 1 || max_tokens_per_rank < 1 || max_batch < 1 || max_batch > 65535)
+    return TOPOEP_ERR_CONFIG;
+  const long long R = (long long)nodes * gpus_per_node;
+  const long long n_ids = (long long)max_tokens_per_rank * top_k;
+  if (n_ids * gpus_per_node >= (1ll << 31)) return TOPOEP_ERR_CONFIG;   // D and L stay in int32
+  if (cost->token_bytes < 0 || cost->expert_bytes < 0 || cost->c_intra < 0 || cost->c_inter < 0 ||
+      cost->t_ffn < 0)
+    return TOPOEP_ERR_COST;
+  if (cost->token_bytes > (1ll << 30) || cost->expert_bytes > (1ll << 60)) return TOPOEP_ERR_COST;
+  if (!main_rank_host && experts % R != 0) return TOPOEP_ERR_MAIN_MAP;
+
+  topoep_ctx* h = new (std::nothrow) topoep_ctx();
+  if (!h) return TOPOEP_ERR_CONFIG;
+  Dims& d = h->d;
+  d.M = nodes; d.G = gpus_per_node; d.R = (int)R; d.E = experts; d.N = slots_per_rank; d.k = top_k;
+  h->main_rank.resize(experts);
+  for (int e = 0; e < experts; ++e) {
+    const long long r = main_rank_host ? main_rank_host[e] : e / (experts / R);
+    if (r < 0 || r >= R) { delete h; return TOPOEP_ERR_MAIN_MAP; }
+    h->main_rank[e] = (int32_t)r;
+  }
+  std::vector<int> per_rank((size_t)R, 0);
+  h->main_local.resize(experts);
+  for (int e = 0; e < experts; ++e) h->main_local[e] = per_rank[h->main_rank[e]]++;
+  d.e_loc = *std::max_element(per_rank.begin(), per_rank.end());
+  d.s_phys = d.e_loc + d.N;
+  d.P = d.R * d.s_phys;
+  d.C = d.G * d.s_phys;
+  d.qstride = d.C | 1;
+  if (d.s_phys < 1 || (long long)d.C > 32767) { delete h; return TOPOEP_ERR_CONFIG; }
+  h->main_inst_expert.assign((size_t)R * std::max(d.e_loc, 1), -1);
+  for (int e = 0; e < experts; ++e)
+    h->main_inst_expert[(size_t)h->main_rank[e] * d.e_loc + h->main_local[e]] = e;
+
+  h->cost = *cost;
+  h->max_iters = cost->max_refine_iters > 0 ? cost->max_refine_iters : 256;
+  h->min_delta = cost->min_delta > 0 ? cost->min_delta : 1;
+  // Dense ranks of the replica-creation costs {0, c_intra*W, c_inter*W}: W is common, so the
+  // coefficients are ranked instead (everything ties at 0 when W == 0).
+  {
+    const long long ci = cost->expert_bytes > 0 ? cost->c_intra : 0;
+    const long long cx = cost->expert_bytes > 0 ? cost->c_inter : 0;
+    auto dense_rank = [&](long long c) {
+      int r = 0;
+      if (0 < c) ++r;
+      if (ci < c && ci != 0) ++r;
+      if (cx < c && cx != 0 && cx != ci) ++r;
+      return r;
+    };
+    h->cost_rank_intra = dense_rank(ci);
+    h->cost_rank_inter = dense_rank(cx);
+  }
+  h->max_tokens = max_tokens_per_rank;
+  h->max_batch = max_batch;
+  h->tile_ids = 4096;
+  h->hist_mode = 0;
+  h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
+  h->have_ws = false;
+  h->last_cuda = cudaSuccess;
+  if (solve_smem_bytes(d) > 227 * 1024 || reroute_smem_bytes(d, kMaxTileIds) > 227 * 1024 ||
+      hist_smem_bytes(d) > 48 * 1024) {
+    delete h;
+    return TOPOEP_ERR_SMEM;
+  }
+  carve(h);
+  *out = h;
+  return TOPOEP_OK;
+}
+
+void topoep_destroy(topoep_handle_t h) { delete h; }
+
+size_t topoep_workspace_bytes(topoep_handle_t h) { return h ? h->ws_bytes : 0; }
+
+int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
+  if (!h || !dev_ptr) return TOPOEP_ERR_NULL;
+  if (bytes < h->ws_bytes || (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0)
+    return TOPOEP_ERR_WORKSPACE;
+  h->have_ws = false;
+  Workspace& w = h->ws;
+  w.main_rank = at<int32_t>(dev_ptr, h->off[W_MAIN_RANK]);
+  w.main_local = at<int32_t>(dev_ptr, h->off[W_MAIN_LOCAL]);
+  w.main_inst_expert = at<int32_t>(dev_ptr, h->off[W_MAIN_INST]);
+  w.status = at<uint32_t>(dev_ptr, h->off[W_STATUS]);
+  w.hist_tickets = at<uint32_t>(dev_ptr, h->off[W_HTICKETS]);
+  w.solve_tickets = at<uint32_t>(dev_ptr, h->off[W_STICKETS]);
+  w.omega = at<int32_t>(dev_ptr, h->off[W_OMEGA]);
+  w.tile_pref = at<int32_t>(dev_ptr, h->off[W_TILE]);
+  w.q = at<int32_t>(dev_ptr, h->off[W_Q]);
+  w.rank_load = at<int32_t>(dev_ptr, h->off[W_LOAD]);
+  w.refine_iters = at<int32_t>(dev_ptr, h->off[W_ITERS]);
+  w.inst_counts = at<int32_t>(dev_ptr, h->off[W_INST_COUNTS]);
+  w.replica_map = at<int32_t>(dev_ptr, h->off[W_REPLICA_MAP]);
+  w.counts = at<int32_t>(dev_ptr, h->off[W_COUNTS]);
+  w.seg_start = at<int32_t>(dev_ptr, h->off[W_SEG]);
+  w.inst_sorted = at<int32_t>(dev_ptr, h->off[W_INST_SORTED]);
+
+  cudaError_t e;
+  const size_t E = h->d.E;
+  if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_rank), h->main_rank.data(), 4 * E,
+                      cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+  if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_local), h->main_local.data(), 4 * E,
+                      cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+  if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_inst_expert), h->main_inst_expert.data(),
+                      4 * h->main_inst_expert.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+  // status word and both ticket arrays are contiguous slots: zero them in one go
+  if ((e = cudaMemset(w.status, 0, h->off[W_OMEGA] - h->off[W_STATUS])) != cudaSuccess) goto fail;
+  if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
+  if ((e = configure_reroute(reroute_smem_bytes(h->d, kMaxTileIds))) != cudaSuccess) goto fail;
+  if ((e = cudaDeviceSynchronize()) != cudaSuccess) goto fail;
+  h->have_ws = true;
+  return TOPOEP_OK;
+fail:
+  h->last_cuda = e;
+  return TOPOEP_ERR_CUDA;
+}
+
+int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
+                     int batch, int32_t* dev_omega, topoep_stream_t stream) {
+  int rc = check_sizes(h, tokens_per_rank, batch);
+  if (rc != TOPOEP_OK) return rc;
+  if (batch == 0) return TOPOEP_OK;
+  if (!dev_omega || (!dev_topk_ids && tokens_per_rank > 0)) return TOPOEP_ERR_NULL;
+  if (!aligned4(dev_topk_ids) || !aligned4(dev_omega)) return TOPOEP_ERR_ALIGN;
+  const HistParams hp = make_hist(h, dev_topk_ids, tokens_per_rank, dev_omega);
+  cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank, int batch,
+                int32_t* dev_replica_map, int32_t* dev_token_replica, int32_t* dev_dispatch_counts,
+                int32_t* dev_dispatch_offsets, int32_t* dev_instance_counts,
+                topoep_stream_t stream) {
+  int rc = check_sizes(h, tokens_per_rank, batch);
+  if (rc != TOPOEP_OK) return rc;
+  if (batch == 0) return TOPOEP_OK;
+  if (!dev_dispatch_counts || !dev_dispatch_offsets) return TOPOEP_ERR_NULL;
+  if (h->d.N > 0 && !dev_replica_map) return TOPOEP_ERR_NULL;
+  if (tokens_per_rank > 0 && (!dev_topk_ids || !dev_token_replica)) return TOPOEP_ERR_NULL;
+  if (!aligned4(dev_topk_ids) || !aligned4(dev_replica_map) || !aligned4(dev_token_replica) ||
+      !aligned4(dev_dispatch_counts) || !aligned4(dev_dispatch_offsets) ||
+      !aligned4(dev_instance_counts))
+    return TOPOEP_ERR_ALIGN;
+
+  const HistParams hp = make_hist(h, dev_topk_ids, tokens_per_rank, nullptr);
+  cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+
+  SolveParams sp;
+  sp.d = h->d;
+  sp.ws = h->ws;
+  sp.token_bytes = h->cost.token_bytes;
+  sp.expert_bytes = h->cost.expert_bytes;
+  sp.max_iters = h->max_iters;
+  sp.min_delta = h->min_delta;
+  sp.cost_rank_intra = h->cost_rank_intra;
+  sp.cost_rank_inter = h->cost_rank_inter;
+  sp.out_replica_map = dev_replica_map;
+  sp.out_counts = dev_dispatch_counts;
+  sp.out_offsets = dev_dispatch_offsets;
+  sp.out_inst_counts = dev_instance_counts;
+  e = launch_solve(sp, batch, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+
+  if (tokens_per_rank > 0) {
+    RerouteParams rp;
+    rp.d = h->d;
+    rp.ws = h->ws;
+    rp.ids = dev_topk_ids;
+    rp.out_token_replica = dev_token_replica;
+    rp.n_ids = hp.n_ids;
+    rp.tiles = hp.tiles;
+    rp.max_tiles = hp.max_tiles;
+    rp.tile_ids = hp.tile_ids;
+    e = launch_reroute(rp, batch, stream);
+    if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  }
+  return TOPOEP_OK;
+}
+
+int topoep_summary(topoep_handle_t h, int batch, topoep_summary_t* dev_out, topoep_stream_t stream) {
+  if (!h) return TOPOEP_ERR_NULL;
+  if (!h->have_ws) return TOPOEP_ERR_WORKSPACE;
+  if (batch < 0 || batch > h->max_batch) return TOPOEP_ERR_SIZE;
+  if (batch == 0) return TOPOEP_OK;
+  if (!dev_out) return TOPOEP_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(dev_out) & 7u) return TOPOEP_ERR_ALIGN;
+  SummaryParams p;
+  p.d = h->d;
+  p.ws = h->ws;
+  p.token_bytes = h->cost.token_bytes;
+  p.expert_bytes = h->cost.expert_bytes;
+  p.t_ffn = h->cost.t_ffn;
+  p.c_intra = h->cost.c_intra;
+  p.c_inter = h->cost.c_inter;
+  p.out = dev_out;
+  cudaError_t e = launch_summary(p, batch, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+int topoep_read_status(topoep_handle_t h, uint32_t* host_flags) {
+  if (!h || !host_flags) return TOPOEP_ERR_NULL;
+  if (!h->have_ws) return TOPOEP_ERR_WORKSPACE;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(host_flags, h->ws.status, 4, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemset(h->ws.status, 0, 4);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+int topoep_debug_tensor(topoep_handle_t h, int which, const void** dev_ptr, size_t* bytes) {
+  if (!h || !dev_ptr || !bytes) return TOPOEP_ERR_NULL;
+  if (!h->have_ws) return TOPOEP_ERR_WORKSPACE;
+  const Dims& d = h->d;
+  const size_t B = (size_t)h->max_batch;
+  switch (which) {
+    case TOPOEP_T_OMEGA: *dev_ptr = h->ws.omega; *bytes = 4 * B * d.R * d.E; break;
+    case TOPOEP_T_Q: *dev_ptr = h->ws.q; *bytes = 4 * B * d.R * d.P; break;
+    case TOPOEP_T_RANK_LOAD: *dev_ptr = h->ws.rank_load; *bytes = 4 * B * d.R; break;
+    case TOPOEP_T_REFINE_ITERS: *dev_ptr = h->ws.refine_iters; *bytes = 4 * B * d.M; break;
+    default: return TOPOEP_ERR_ARG;
+  }
+  return TOPOEP_OK;
+}
+
+int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
+  if (!h) return TOPOEP_ERR_NULL;
+  switch (knob) {
+    case TOPOEP_KNOB_TILE_IDS:
+      if (value < kMinTileIds || value > kMaxTileIds || (value & (value - 1))) return TOPOEP_ERR_ARG;
+      h->tile_ids = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_HIST_MODE:
+      if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
+      h->hist_mode = value;
+      return TOPOEP_OK;
+    default:
+      return TOPOEP_ERR_ARG;
+  }
+}
+
+int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances) {
+  if (!h) return TOPOEP_ERR_NULL;
+  if (e_loc) *e_loc = h->d.e_loc;
+  if (s_phys) *s_phys = h->d.s_phys;
+  if (instances) *instances = h->d.P;
+  return TOPOEP_OK;
+}
+
+int topoep_launch_floor(int count, topoep_stream_t stream) {
+  if (count < 0 || count > 1024) return TOPOEP_ERR_ARG;
+  return launch_empty(count, stream) == cudaSuccess ? TOPOEP_OK : TOPOEP_ERR_CUDA;
+}
+
+const char* topoep_strerror(int status) {
+  switch (status) {
+    case TOPOEP_OK: return "ok";
+    case TOPOEP_ERR_NULL: return "a required pointer is NULL";
+    case TOPOEP_ERR_CONFIG: return "topology, expert, slot or size numbers out of range";
+    case TOPOEP_ERR_MAIN_MAP: return "main_rank entry out of range, or E % R != 0 with no map";
+    case TOPOEP_ERR_COST: return "negative or oversized cost parameter";
+    case TOPOEP_ERR_WORKSPACE: return "workspace missing, too small or not 256-byte aligned";
+    case TOPOEP_ERR_SIZE: return "tokens_per_rank or batch outside [0, max]";
+    case TOPOEP_ERR_ALIGN: return "a device buffer is misaligned";
+    case TOPOEP_ERR_CUDA: return "a CUDA runtime call failed";
+    case TOPOEP_ERR_SMEM: return "problem does not fit one SM's shared memory";
+    case TOPOEP_ERR_ARG: return "unknown selector, knob or value";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,134 @@
+"""Convenience holder around the C handle: owns the torch workspace and output tensors.
+
+Marshalling only -- every step of the planning path runs in the CUDA library.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+@dataclass
+class PlanOutputs:
+    replica_map: torch.Tensor       # [B][R][N_slot] int32
+    token_replica: torch.Tensor     # [B][R][T][k]   int32
+    dispatch_counts: torch.Tensor   # [B][R][R]      int32
+    dispatch_offsets: torch.Tensor  # [B][2][R][R+1] int32
+    instance_counts: torch.Tensor   # [B][P]         int32
+
+
+class Planner:
+    """topoep_create + workspace on the current CUDA device."""
+
+    def __init__(self, nodes, gpus_per_node, experts, slots_per_rank, top_k, max_tokens_per_rank,
+                 max_batch=1, token_bytes=0, expert_bytes=0, c_intra=1, c_inter=8, t_ffn=0,
+                 max_refine_iters=0, min_delta=0, main_rank: Optional[np.ndarray] = None,
+                 device: Optional[torch.device] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("TopoEP planning needs a CUDA device; there is no CPU path")
+        self.device = torch.device(device) if device is not None else torch.device(
+            "cuda", torch.cuda.current_device())
+        self.M, self.G, self.E, self.N, self.k = nodes, gpus_per_node, experts, slots_per_rank, top_k
+        self.R = nodes * gpus_per_node
+        self.max_tokens, self.max_batch = max_tokens_per_rank, max_batch
+        cost = B.CostParams(token_bytes, expert_bytes, c_intra, c_inter, t_ffn, max_refine_iters,
+                            min_delta)
+        mr = None if main_rank is None else np.ascontiguousarray(main_rank, dtype=np.int32)
+        rc, self.handle = B.topoep_create(nodes, gpus_per_node, experts, slots_per_rank, top_k,
+                                          max_tokens_per_rank, max_batch, mr, cost)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        rc, self.e_loc, self.s_phys, self.P = B.topoep_get_layout(self.handle)
+        nbytes = B.topoep_workspace_bytes(self.handle)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = self.workspace.data_ptr()
+            self._ws_ptr = (base + 255) // 256 * 256
+            rc = B.topoep_set_workspace(self.handle, self._ws_ptr, nbytes)
+        if rc != B.OK:
+            B.topoep_destroy(self.handle)
+            self.handle = None
+            raise B.TopoEPError(rc)
+
+    def close(self):
+        if getattr(self, "handle", None) is not None:
+            B.topoep_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
+
+    def alloc_outputs(self, batch: int, tokens_per_rank: int) -> PlanOutputs:
+        i32 = dict(dtype=torch.int32, device=self.device)
+        R = self.R
+        return PlanOutputs(torch.empty((batch, R, self.N), **i32),
+                           torch.empty((batch, R, tokens_per_rank, self.k), **i32),
+                           torch.empty((batch, R, R), **i32),
+                           torch.empty((batch, 2, R, R + 1), **i32),
+                           torch.empty((batch, self.P), **i32))
+
+    def plan(self, topk_ids: torch.Tensor, out: Optional[PlanOutputs] = None,
+             stream: Optional[torch.cuda.Stream] = None) -> PlanOutputs:
+        """topoep_plan on ids [B][R][T][k] (int32, contiguous, on this device)."""
+        assert topk_ids.dtype == torch.int32 and topk_ids.is_contiguous() and topk_ids.is_cuda
+        Bn, R, T, k = topk_ids.shape
+        assert R == self.R and k == self.k
+        if out is None:
+            out = self.alloc_outputs(Bn, T)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = B.topoep_plan(self.handle, topk_ids, T, Bn, out.replica_map, out.token_replica,
+                           out.dispatch_counts, out.dispatch_offsets, out.instance_counts,
+                           st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        return out
+
+    def histogram(self, topk_ids: torch.Tensor, stream=None) -> torch.Tensor:
+        Bn, R, T, k = topk_ids.shape
+        omega = torch.empty((Bn, R, self.E), dtype=torch.int32, device=self.device)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = B.topoep_histogram(self.handle, topk_ids, T, Bn, omega, st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        return omega
+
+    def summary(self, batch: int) -> np.ndarray:
+        """Summaries of the last plan as a numpy record array (synchronises)."""
+        n = ctypes.sizeof(B.Summary)
+        buf = torch.empty(batch * n, dtype=torch.uint8, device=self.device)
+        rc = B.topoep_summary(self.handle, batch, buf, torch.cuda.current_stream(self.device).cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        names = [f[0] for f in B.Summary._fields_]
+        dt = np.dtype([(nm, np.int64 if i < 12 else np.float64) for i, nm in enumerate(names)])
+        return np.frombuffer(buf.cpu().numpy().tobytes(), dtype=dt)
+
+    def status(self) -> int:
+        rc, flags = B.topoep_read_status(self.handle)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        return flags
+
+    def debug_tensor(self, which: int, batch: int) -> torch.Tensor:
+        """Copy of an intermediate tensor for the first `batch` plans (int32, on the host)."""
+        rc, ptr, nbytes = B.topoep_debug_tensor(self.handle, which)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        shape = {B.T_OMEGA: (self.R, self.E), B.T_Q: (self.R, self.P), B.T_RANK_LOAD: (self.R,),
+                 B.T_REFINE_ITERS: (self.M,)}[which]
+        off = (ptr - self.workspace.data_ptr())
+        per = int(np.prod(shape)) * 4
+        torch.cuda.synchronize(self.device)
+        raw = self.workspace[off:off + batch * per].cpu().numpy()
+        return torch.from_numpy(raw.view(np.int32).reshape((batch,) + shape).copy())
+
+    def set_tuning(self, knob: int, value: int):
+        rc = B.topoep_set_tuning(self.handle, knob, value)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)

@@ -1,0 +1,248 @@
+"""CUDA library vs CPU oracle, element by element, through the C boundary (needs a B200)."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import workloads as wl
+from plan_checks import check_plan
+from gpu_common import assert_same, make_planner, oracle_config, parity, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+from paper_2609_35481_b200 import binding as B  # noqa: E402
+
+
+# ---- the benchmark configurations at full size -----------------------------------------------
+@pytest.mark.parametrize("name", ["tiny", "mid", "dsv3"])
+@pytest.mark.parametrize("seed", [20260935, 1, 2])
+def test_configs_1_to_3_full_size(name, seed):
+    gpu, ref, _ = parity(wl.CONFIGS[name], seed)
+    assert gpu["flags"] == 0
+
+
+@pytest.mark.parametrize("name", ["scaleout", "scaleout_uniform"])
+def test_config_5_full_size(name):
+    w = wl.CONFIGS[name]
+    gpu, ref, ids = parity(w, wl.BASE_SEED)
+    assert gpu["flags"] == 0
+    check_plan(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k, w.main_rank(),
+               w.token_bytes, w.expert_bytes, ids[0], gpu["replica_map"][0], gpu["token_replica"][0],
+               gpu["dispatch_counts"][0], gpu["dispatch_offsets"][0], gpu["instance_counts"][0],
+               gpu["rank_load"][0])
+
+
+def test_config_4_batched_full_size_sampled_plans():
+    # 232 plans of the dsv3 shape in ONE call, as the bench launches it.  The oracle recomputes a
+    # sample of the plans in full (plans are independent); structural properties are checked on two
+    # more; omega of every plan is checked against bincount.
+    w = wl.CONFIGS["dsv3_batched"]
+    ids = wl.make_topk_ids(w, seed=wl.BASE_SEED)
+    pl = make_planner(w)
+    gpu = run_gpu(pl, ids)
+    assert gpu["flags"] == 0
+    sample = [0, 1, 57, 100, 173, 231]
+    ref = orc.plan(oracle_config(w), ids[sample])
+    assert_same(gpu, ref, plans=sample)
+    for b in (5, 200):
+        check_plan(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k, w.main_rank(),
+                   w.token_bytes, w.expert_bytes, ids[b], gpu["replica_map"][b],
+                   gpu["token_replica"][b], gpu["dispatch_counts"][b], gpu["dispatch_offsets"][b],
+                   gpu["instance_counts"][b], gpu["rank_load"][b])
+    E = w.experts
+    flat = ids.reshape(w.batch * w.ranks, -1).astype(np.int64)
+    flat += (np.arange(flat.shape[0]) * E)[:, None]
+    om = np.bincount(flat.ravel(), minlength=flat.shape[0] * E).reshape(w.batch, w.ranks, E)
+    assert np.array_equal(om, gpu["omega"])
+
+
+# ---- shapes where inter-node placement AND refinement both act ------------------------------
+BOTH_STAGES = [
+    ("dsv3", dict(slots_per_rank=3, tokens_per_rank=2048)),
+    ("dsv3", dict(slots_per_rank=4, tokens_per_rank=2048)),
+    ("dsv3", dict(slots_per_rank=8, tokens_per_rank=4096, zipf_s=0.8)),
+    ("mid", dict(slots_per_rank=3)),
+    ("scaleout", dict(slots_per_rank=4, tokens_per_rank=2048, zipf_s=1.0)),
+    ("tiny", dict(slots_per_rank=3)),
+]
+
+
+@pytest.mark.parametrize("name,over", BOTH_STAGES)
+def test_both_stages_active(name, over):
+    w = wl.CONFIGS[name].replace(**over)
+    gpu, ref, _ = parity(w, 77, batch=3)
+    assert ref.refine_iters.sum() > 0
+    if w.nodes > 1 and name != "tiny":
+        assert ref.summaries["replicas_inter"].sum() > 0
+
+
+# ---- degenerate and ragged shapes --------------------------------------------------------------
+def test_single_domain():
+    w = wl.CONFIGS["mid"].replace(nodes=1, gpus_per_node=8, experts=64, slots_per_rank=2,
+                                  tokens_per_rank=1000)
+    gpu, ref, _ = parity(w, 5, batch=2)
+    assert ref.summaries["replicas_inter"].sum() == 0 and ref.refine_iters.sum() > 0
+
+
+def test_one_gpu_per_node_and_no_slots():
+    parity(wl.CONFIGS["tiny"].replace(nodes=8, gpus_per_node=1, tokens_per_rank=3000), 6)
+    parity(wl.CONFIGS["tiny"].replace(slots_per_rank=0), 6)
+
+
+@pytest.mark.parametrize("T,k", [(1, 1), (3, 1), (7, 3), (1023, 2), (1025, 2), (2049, 3), (4097, 1),
+                                 (5000, 2), (777, 5)])
+def test_ragged_token_counts(T, k):
+    # T*k not a multiple of 4 (scalar loads), of the tile, or smaller than one warp
+    w = wl.CONFIGS["tiny"].replace(tokens_per_rank=T, top_k=k, slots_per_rank=2)
+    parity(w, 100 + T, batch=2)
+
+
+def test_uneven_main_map_and_odd_topology():
+    # 3 nodes x 3 GPUs, 20 experts placed by a seeded random map (some ranks get none)
+    rng = np.random.default_rng(3)
+    w = wl.CONFIGS["tiny"].replace(nodes=3, gpus_per_node=3, experts=20, slots_per_rank=2,
+                                   top_k=3, tokens_per_rank=1500)
+    main = rng.integers(0, 9, size=20).astype(np.int32)
+    ids = wl.make_topk_ids(w, seed=9, batch=2)
+    pl = make_planner(w, max_batch=2, main_rank=main)
+    gpu = run_gpu(pl, ids)
+    ref = orc.plan(oracle_config(w, main_rank=main), ids)
+    assert_same(gpu, ref)
+
+
+def test_random_small_problems():
+    rng = np.random.default_rng(11)
+    for trial in range(40):
+        M, G = int(rng.integers(1, 5)), int(rng.integers(1, 6))
+        R = M * G
+        E = int(rng.integers(1, 40))
+        N = int(rng.integers(0, 4))
+        k = int(rng.integers(1, min(E, 4) + 1))
+        T = int(rng.integers(1, 400))
+        main = rng.integers(0, R, size=E).astype(np.int32)
+        tok, W = int(rng.integers(1, 64)), int(rng.integers(0, 4000))
+        ids = rng.integers(0, E, size=(2, R, T, k)).astype(np.int32)   # duplicates inside a token
+        w = wl.Workload("rnd", M, G, E, N, k, T)
+        over = dict(main_rank=main, token_bytes=tok, expert_bytes=W,
+                    c_intra=int(rng.integers(0, 3)), c_inter=int(rng.integers(0, 9)))
+        pl = make_planner(w, max_batch=2, **over)
+        gpu = run_gpu(pl, ids)
+        ref = orc.plan(oracle_config(w, **over), ids)
+        assert_same(gpu, ref)
+        pl.close()
+
+
+def test_invalid_and_padded_ids():
+    w = wl.CONFIGS["tiny"].replace(slots_per_rank=2)
+    ids = wl.make_topk_ids(w, seed=4, batch=2).copy()
+    ids[0, 1, 100:300, :] = -1                      # padded rows: ignored, no flag
+    gpu, ref, _ = parity(w, 4, ids=ids)
+    assert gpu["flags"] == 0 and (gpu["token_replica"][0, 1, 100:300] == -1).all()
+    ids[1, 2, 7, 0] = w.experts                     # out of range: ignored and flagged
+    ids[1, 3, 9, 1] = -5
+    gpu, ref, _ = parity(w, 4, ids=ids)
+    assert gpu["flags"] == B.FLAG_BAD_ID == ref.flags
+    assert gpu["token_replica"][1, 2, 7, 0] == -1 and gpu["token_replica"][1, 3, 9, 1] == -1
+
+
+def test_refinement_cap_binds_identically():
+    w = wl.CONFIGS["scaleout_uniform"].replace(tokens_per_rank=1024)
+    gpu, ref, _ = parity(w, 8, max_refine_iters=3)
+    assert gpu["flags"] == B.FLAG_REFINE_CAP and (gpu["refine_iters"] <= 3).all()
+    gpu2, ref2, _ = parity(w, 8, min_delta=5)
+    assert gpu2["flags"] == 0
+
+
+def test_empty_batch_and_zero_tokens():
+    w = wl.CONFIGS["tiny"]
+    pl = make_planner(w, max_batch=2)
+    out = pl.alloc_outputs(1, 0)
+    ids = torch.empty((1, w.ranks, 0, w.top_k), dtype=torch.int32, device=pl.device)
+    pl.plan(ids, out)
+    torch.cuda.synchronize()
+    assert (out.dispatch_counts == 0).all() and (out.replica_map == -1).all()
+    assert (out.dispatch_offsets == 0).all() and (out.instance_counts == 0).all()
+    rc = B.topoep_plan(pl.handle, None, 5, 0, None, None, None, None, None, 0)
+    assert rc == B.OK                      # batch 0: nothing to do
+    assert pl.status() == 0
+
+
+# ---- determinism: reruns and launch configurations ----------------------------------------
+def test_bitwise_identical_across_reruns_and_tunings():
+    w = wl.CONFIGS["dsv3"].replace(slots_per_rank=3)
+    ids = wl.make_topk_ids(w, seed=31, batch=2)
+    pl = make_planner(w, max_batch=2)
+    base = run_gpu(pl, ids)
+    for tile in (1024, 2048, 4096, 8192, 16384):
+        for mode in (0, 1):
+            pl.set_tuning(B.KNOB_TILE_IDS, tile)
+            pl.set_tuning(B.KNOB_HIST_MODE, mode)
+            for rep in range(2):
+                again = run_gpu(pl, ids)
+                for key, val in base.items():
+                    if key == "flags":
+                        assert again[key] == val
+                    elif key == "summaries":
+                        assert again[key].tobytes() == val.tobytes()
+                    else:
+                        assert np.array_equal(again[key], val), (key, tile, mode)
+    ref = orc.plan(oracle_config(w), ids)
+    assert_same(base, ref)
+
+
+def test_histogram_entry_point_matches_bincount():
+    w = wl.CONFIGS["mid"]
+    ids = wl.make_topk_ids(w, seed=12, batch=2)
+    pl = make_planner(w, max_batch=2)
+    om = pl.histogram(torch.from_numpy(ids).to(pl.device)).cpu().numpy()
+    for b in range(2):
+        for s in range(w.ranks):
+            assert np.array_equal(om[b, s], np.bincount(ids[b, s].ravel(), minlength=w.experts))
+
+
+# ---- capture: the plan is enqueue-only ---------------------------------------------------------
+def test_plan_is_capturable_in_a_cuda_graph_and_replays_identically():
+    w = wl.CONFIGS["dsv3"]
+    ids = wl.make_topk_ids(w, seed=21)
+    pl = make_planner(w)
+    dev_ids = torch.from_numpy(ids).to(pl.device)
+    out = pl.alloc_outputs(1, w.tokens_per_rank)
+    eager = pl.plan(dev_ids)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        # a host synchronisation, a device-to-host copy or an allocation inside would fail capture
+        with torch.cuda.graph(graph, stream=stream):
+            pl.plan(dev_ids, out, stream=stream)
+    for _ in range(3):
+        out.token_replica.fill_(-7)
+        graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out.token_replica, eager.token_replica)
+    assert torch.equal(out.replica_map, eager.replica_map)
+    assert torch.equal(out.dispatch_offsets, eager.dispatch_offsets)
+    ref = orc.plan(oracle_config(w), ids)
+    assert np.array_equal(out.token_replica.cpu().numpy(), ref.token_replica)
+
+
+# ---- boundary errors that need a live workspace ---------------------------------------------
+def test_size_and_pointer_errors():
+    w = wl.CONFIGS["tiny"]
+    pl = make_planner(w, max_batch=1)
+    out = pl.alloc_outputs(1, w.tokens_per_rank)
+    ids = torch.zeros((1, w.ranks, w.tokens_per_rank, w.top_k), dtype=torch.int32, device=pl.device)
+    args = (out.replica_map, out.token_replica, out.dispatch_counts, out.dispatch_offsets,
+            out.instance_counts, 0)
+    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank + 1, 1, *args) == -6
+    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 2, *args) == -6
+    assert B.topoep_plan(pl.handle, None, w.tokens_per_rank, 1, *args) == -1
+    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 1, None, *args[1:]) == -1
+    assert B.topoep_plan(pl.handle, ids.data_ptr() + 2, w.tokens_per_rank, 1, *args) == -7
+    assert B.topoep_set_workspace(pl.handle, pl._ws_ptr + 4, 1 << 30) == -5
+    assert B.topoep_set_workspace(pl.handle, pl._ws_ptr, 16) == -5
+    assert B.topoep_set_tuning(pl.handle, B.KNOB_TILE_IDS, 3000) == -10
+    # the failed set_workspace calls dropped the workspace: the next plan says so
+    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 1, *args) == -5
