@@ -1,0 +1,472 @@
+#!/usr/bin/env python3
+"""Benchmark of the TopoEP planning step on B200.
+
+One "step" = one topoep_plan call (histogram -> solver + layout -> reroute) over one batch of
+seeded synthetic routing.  Prints ONE JSON line:
+
+  value      top-k assignments planned per second, device-timed with CUDA events over a captured
+             CUDA graph of K plans, inputs resident in HBM, rotating over enough distinct buffer
+             sets to exceed L2 (so every pass reads its ids from DRAM)
+  e2e        the same metric through the public call with HOST buffers: pinned ids copied to the
+             device, the plan, every output copied back, all inside the timed region
+  roofline   for the kernel with the largest share of the plan: algorithmic bytes / its measured
+             launch time against the measured HBM copy bandwidth
+  cpu_baseline  the CPU oracle, as it stands, timed on this machine's host cores on a bounded sample
+
+`--impl reference` times only the oracle (the stand-in for a reference implementation: the paper
+has no released code).  Under torchrun every rank plans its own seeded batches on its own GPU
+(independent replicas, no collective on the data path); times are the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+KERNELS_PER_PLAN = 5
+# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), keyed by
+# (workload, kernel); None until a capture of that pair exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Polls NVML for SM clock, power and clock-event reasons while the GPU is under load."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks",
+               0x10: "sync_boost"}
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self.power = []
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as exc:  # pragma: no cover
+            self.err = repr(exc)
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def finish(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0,
+                    "note": getattr(self, "err", "no samples")}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": round(max(self.power), 1) if self.power else None}
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle leg (CPU baseline / --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_config(w):
+    import oracle as orc
+    return orc.OracleConfig(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
+                            w.token_bytes, w.expert_bytes, w.c_intra, w.c_inter, w.t_ffn,
+                            main_rank=w.main_rank())
+
+
+def time_oracle(w, ids, budget_s):
+    """Run the oracle plan by plan on `ids` [B][R][T][k] until the budget is used up."""
+    import oracle as orc
+    cfg = oracle_config(w)
+    done, t0 = 0, time.perf_counter()
+    while True:
+        b = done % ids.shape[0]
+        orc.plan(cfg, ids[b:b + 1], want_q=False)
+        done += 1
+        if time.perf_counter() - t0 >= budget_s:
+            break
+    dt = time.perf_counter() - t0
+    per_plan = ids.shape[1] * ids.shape[2] * ids.shape[3]
+    return done * per_plan / dt, done, dt
+
+
+def run_reference(args, w):
+    """The oracle as the reference arm: each step plans a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle as orc
+    orc.build()
+    cfg = oracle_config(w)
+    # sample: one plan of the workload's shape, tokens per rank cut so that K+W steps fit ~2 min
+    probe_T = min(w.tokens_per_rank, 1024)
+    ids = wl.make_topk_ids(w.replace(tokens_per_rank=probe_T), seed=wl.BASE_SEED, batch=1)
+    t0 = time.perf_counter()
+    orc.plan(cfg, ids, want_q=False)
+    per_assign = (time.perf_counter() - t0) / ids.size
+    budget = 120.0 / max(args.steps + args.warmup, 1)
+    T = int(min(w.tokens_per_rank, max(64, budget / per_assign / (w.ranks * w.top_k))))
+    ids = wl.make_topk_ids(w.replace(tokens_per_rank=T), seed=wl.BASE_SEED, batch=1)
+    for _ in range(args.warmup):
+        orc.plan(cfg, ids, want_q=False)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.plan(cfg, ids, want_q=False)
+    dt = time.perf_counter() - t0
+    value = args.steps * ids.size / dt
+    sample = "one plan of the %s shape with %d of %d tokens per rank per step" % (w.name, T, w.tokens_per_rank)
+    line = {"impl": "reference", "metric": "topk_assignments_per_s", "value": value,
+            "unit": "assignments/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": workload_config(w, 1, "n/a (CPU)"),
+            "cpu_baseline": {"value": value, "unit": "assignments/s", "cores": 1, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": "assignments/s", "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, nsets, l2_policy):
+    return {"workload": w.name, "nodes": w.nodes, "gpus_per_node": w.gpus_per_node,
+            "ranks": w.ranks, "experts": w.experts, "slots_per_rank": w.slots_per_rank,
+            "top_k": w.top_k, "tokens_per_rank": w.tokens_per_rank, "plans_per_step": w.batch,
+            "assignments_per_step": w.assignments, "main_map": w.main_map, "seed": wl.BASE_SEED,
+            "buffer_sets": nsets, "l2": l2_policy}
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------
+def measure(w, K, W, rank, world, dev, args, stages=True):
+    """Device-timed K plans of workload w inside one captured CUDA graph, plus per-stage graphs."""
+    import torch
+    import torch.distributed as dist
+    from paper_2609_35481_b200 import Planner, binding as B
+
+    # inputs: nsets distinct seeded batches, each with its own planner, workspace and outputs, so
+    # that a rotation over them touches more than twice L2 before any buffer repeats
+    ids_bytes = w.assignments * 4
+    nsets = int(max(1, min(32, -(-2 * L2_BYTES // (2 * ids_bytes)))))
+    l2_policy = ("inputs+outputs of one step exceed L2" if nsets == 1 else
+                 "rotation over %d distinct input/output/workspace sets (%.0f MB) exceeds L2"
+                 % (nsets, nsets * 2 * ids_bytes / 1e6))
+    sets = []
+    for i in range(nsets):
+        ids = wl.make_topk_ids(w, seed=wl.BASE_SEED, plan_base=(rank * 64 + i) * 100000)
+        pl = Planner(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
+                     w.tokens_per_rank, max_batch=w.batch, token_bytes=w.token_bytes,
+                     expert_bytes=w.expert_bytes, c_intra=w.c_intra, c_inter=w.c_inter,
+                     t_ffn=w.t_ffn, main_rank=w.main_rank(), device=dev)
+        if args.tile_ids:
+            pl.set_tuning(B.KNOB_TILE_IDS, args.tile_ids)
+        if args.hist_mode >= 0:
+            pl.set_tuning(B.KNOB_HIST_MODE, args.hist_mode)
+        ids_dev = torch.from_numpy(ids).to(dev)
+        sets.append({"pl": pl, "ids_host": ids, "ids": ids_dev,
+                     "out": pl.alloc_outputs(w.batch, w.tokens_per_rank)})
+
+    stream = torch.cuda.Stream(device=dev)
+    sh = stream.cuda_stream
+
+    def plan(i):
+        s = sets[i % nsets]
+        s["pl"].plan(s["ids"], s["out"], stream=stream)
+
+    def hist(i):
+        s = sets[i % nsets]
+        rc = B.topoep_histogram(s["pl"].handle, s["ids"], w.tokens_per_rank, w.batch, None, sh)
+        assert rc == 0, rc
+
+    def solve(i):
+        s, o = sets[i % nsets], sets[i % nsets]["out"]
+        rc = B.topoep_solve(s["pl"].handle, None, w.batch, o.replica_map, o.dispatch_counts,
+                            o.dispatch_offsets, o.instance_counts, sh)
+        assert rc == 0, rc
+
+    def reroute(i):
+        s = sets[i % nsets]
+        rc = B.topoep_reroute(s["pl"].handle, s["ids"], w.tokens_per_rank, w.batch,
+                              s["out"].token_replica, sh)
+        assert rc == 0, rc
+
+    def floor(i):
+        assert B.topoep_launch_floor(KERNELS_PER_PLAN, sh) == 0
+
+    def capture(fn, n):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(n):
+                    fn(i)
+        return g
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed_replay(g):
+        """ms of one replay of graph g, events on the launching stream, max over ranks."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    # warm-up: W eager plans, and every set at least once so each workspace holds its own plan
+    with torch.cuda.stream(stream):
+        for i in range(max(W, nsets)):
+            plan(i)
+    torch.cuda.synchronize(dev)
+    for s in sets:
+        flags = s["pl"].status()
+        assert flags == 0, "device status flags %d" % flags
+
+    g_plan = capture(plan, K)
+    g_plan.replay()                      # one untimed replay of the captured graph
+    ms_total = timed_replay(g_plan)      # EXACTLY K steps
+    del g_plan
+
+    # per-stage times (same rotation; hist = tile histogram + omega, solve = solver + route
+    # tables, reroute) and the launch floor: the same number of empty kernels
+    stage_us = {}
+    names = (("hist", hist), ("solve", solve), ("reroute", reroute), ("floor", floor))
+    for name, fn in (names if stages else names[3:]):
+        g = capture(fn, K)
+        g.replay()
+        stage_us[name] = timed_replay(g) / K * 1e3
+        del g
+    # leave every workspace consistent again (the stage graphs ran stages out of order)
+    with torch.cuda.stream(stream):
+        for i in range(nsets):
+            plan(i)
+    torch.cuda.synchronize(dev)
+    return {"sets": sets, "nsets": nsets, "l2_policy": l2_policy, "stream": stream,
+            "ms_total": ms_total, "ms_step": ms_total / K, "stage_us": stage_us,
+            "barrier": barrier}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="dsv3_batched", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--no-single-plan", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override plans per step")
+    ap.add_argument("--impl", default="topoep", choices=["topoep", "reference"])
+    ap.add_argument("--tile-ids", type=int, default=0)
+    ap.add_argument("--hist-mode", type=int, default=-1)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    w = wl.CONFIGS[args.workload]
+    if args.batch:
+        w = w.replace(batch=args.batch)
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_35481_b200 import Planner, binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the planning path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    K, W = args.steps, args.warmup
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    m = measure(w, K, W, rank, world, dev, args)
+    sets, nsets, l2_policy, stream = m["sets"], m["nsets"], m["l2_policy"], m["stream"]
+    ms_step, ms_total, stage_us = m["ms_step"], m["ms_total"], m["stage_us"]
+    value = world * w.assignments * K / (ms_total * 1e-3)
+    barrier = m["barrier"]
+
+    # ---- end to end through the public call with host buffers
+    s0 = sets[0]
+    host_ids = torch.from_numpy(s0["ids_host"]).pin_memory()
+    o = s0["out"]
+    dev_outs = [o.replica_map, o.token_replica, o.dispatch_counts, o.dispatch_offsets,
+                o.instance_counts]
+    host_outs = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in dev_outs]
+    h2d = host_ids.numel() * 4
+    d2h = sum(t.numel() * 4 for t in dev_outs)
+
+    def e2e_step():
+        s0["ids"].copy_(host_ids, non_blocking=True)
+        s0["pl"].plan(s0["ids"], o, stream=stream)
+        for hbuf, dbuf in zip(host_outs, dev_outs):
+            hbuf.copy_(dbuf, non_blocking=True)
+
+    k_e2e = max(3, min(K, int(2.0 / max(ms_step * 1e-3 + (h2d + d2h) / 20e9, 1e-6))))
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            e2e_step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(k_e2e):
+            e2e_step()
+        e1.record(stream)
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_value = world * w.assignments * k_e2e / (ms_e2e * 1e-3)
+
+    # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol
+    single = None
+    if w.batch > 1 and not args.no_single_plan:
+        w1 = wl.CONFIGS["dsv3"] if w.name == "dsv3_batched" else w.replace(batch=1)
+        for s_ in sets[1:]:
+            s_["pl"].close()
+        m1 = measure(w1, 200, 20, rank, world, dev, args)
+        single = {"workload": w1.name, "steps": 200, "warmup": 20,
+                  "us_per_layer_plan": round(m1["ms_step"] * 1e3, 3),
+                  "kernel_us": {n: round(m1["stage_us"][n], 3) for n in ("hist", "solve", "reroute")},
+                  "launch_floor_us": round(m1["stage_us"]["floor"], 3),
+                  "vs_launch_floor": round(m1["ms_step"] * 1e3 / m1["stage_us"]["floor"], 2),
+                  "hbm_roofline_us": round(12 * w1.assignments / measured_peak_gbs()[0] / 1e3, 3),
+                  "l2": m1["l2_policy"]}
+        for s_ in m1["sets"]:
+            s_["pl"].close()
+    clocks = sampler.finish()
+
+    # the e2e outputs came back to the host: check them against the device copies of the same plan
+    assert np.array_equal(host_outs[1].numpy(), o.token_replica.cpu().numpy())
+
+    # ---- roofline of the dominant kernel
+    peak, peak_kind = measured_peak_gbs()
+    A = w.assignments
+    algo_bytes = {"hist": 4 * A, "reroute": 8 * A, "solve": None}
+    dominant = max(("hist", "solve", "reroute"), key=lambda n: stage_us[n])
+    hbm_kernels = {n: {"us": round(stage_us[n], 3),
+                       "achieved_gbs": round(algo_bytes[n] / (stage_us[n] * 1e-6) / 1e9, 1),
+                       "frac": round(algo_bytes[n] / (stage_us[n] * 1e-6) / 1e9 / peak, 4)}
+                   for n in ("hist", "reroute")}
+    if dominant == "solve":
+        # latency-bound: a few CTAs of serial integer work; judged against the launch floor, and
+        # reported here with the bytes it has to touch (omega in, q and layout out)
+        dom_bytes = 4 * w.batch * (w.ranks * w.experts + w.ranks * sets[0]["pl"].P
+                                   + 3 * w.ranks * w.ranks)
+    else:
+        dom_bytes = algo_bytes[dominant]
+    achieved = dom_bytes / (stage_us[dominant] * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": {"hist": "hist_kernel", "solve": "solve_kernel",
+                                           "reroute": "reroute_kernel"}[dominant],
+                "achieved": round(achieved, 2), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "peak_source": "of " + peak_kind,
+                "traffic": NCU_TRAFFIC_BYTES.get((w.name, dominant)),
+                "algorithmic_bytes_per_launch": dom_bytes,
+                "plan_bytes": 12 * A,
+                "plan_frac": round(12 * A / (ms_step * 1e-3) / 1e9 / peak, 4),
+                "hbm_kernels": hbm_kernels}
+
+    line = {"metric": "topk_assignments_per_s", "value": value, "unit": "assignments/s",
+            "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms_step,
+            "us_per_layer_plan": ms_step * 1e3 / w.batch,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+            "data": "synthetic", "impl": "topoep_b200",
+            "config": workload_config(w, nsets, l2_policy),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": "assignments/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": k_e2e,
+                    "us_per_layer_plan": ms_e2e * 1e3 / k_e2e / w.batch},
+            "gpu_launches": KERNELS_PER_PLAN * K,
+            "kernel_us": {n: round(stage_us[n], 3) for n in ("hist", "solve", "reroute")},
+            "launch_floor_us": round(stage_us["floor"], 3),
+            "vs_launch_floor": round(ms_step * 1e3 / stage_us["floor"], 2),
+            "roofline": roofline}
+    if single is not None:
+        line["single_plan"] = single
+
+    if rank == 0 and not args.no_cpu_baseline:
+        sample_ids = s0["ids_host"][:min(w.batch, 8)]
+        v, plans, dt = time_oracle(w, sample_ids, args.cpu_seconds)
+        line["cpu_baseline"] = {"value": v, "unit": "assignments/s", "cores": 1, "kind": "oracle",
+                                "sample": "%d whole plans of the %s shape in %.1f s (host has %d cores)"
+                                          % (plans, w.name, dt, os.cpu_count() or 0)}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

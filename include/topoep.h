@@ -116,10 +116,10 @@ enum {
 
 /* Knobs for topoep_set_tuning; no knob may change any output bit. */
 enum {
-  TOPOEP_KNOB_TILE_IDS = 0,     /* ids per histogram / reroute tile: 1024..16384,
+  TOPOEP_KNOB_TILE_IDS = 0,     /* ids per histogram / reroute tile: 1024..8192,
                                    power of two                                   */
-  TOPOEP_KNOB_HIST_MODE = 1     /* 0 = warp-aggregated (match) shared atomics,
-                                   1 = plain shared atomics                       */
+  TOPOEP_KNOB_HIST_MODE = 1     /* 0 = plain shared-memory atomics (default),
+                                   1 = warp-aggregated (__match_any_sync) atomics */
 };
 
 /*
@@ -177,7 +177,8 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes);
  *
  * Within a (plan, source, expert) group, assignments are ranked by flat index
  * t*k+j and dealt to the expert's instances in ascending rank order, each
- * taking q(s,e,r) of them.  Enqueues three kernels on `stream`; capturable in
+ * taking q(s,e,r) of them.  Equivalent to topoep_histogram, topoep_solve and
+ * topoep_reroute in a row: enqueues five kernels on `stream`; capturable in
  * a CUDA graph.  Two plans on one handle must not overlap on the device.
  */
 int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
@@ -187,11 +188,37 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
 
 /*
  * Histogram step alone (paper, Eq. Omega): dev_omega [B][R][E] int32 gets the
- * number of assignments of source rank s that select expert e.  Uses the
- * workspace for per-tile counts.  Same argument rules as topoep_plan.
+ * number of assignments of source rank s that select expert e; it may be NULL,
+ * the routing matrix is always left in the workspace as well (TOPOEP_T_OMEGA).
+ * Uses the workspace for per-tile counts.  Same argument rules as topoep_plan.
  */
 int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
                      int batch, int32_t* dev_omega, topoep_stream_t stream);
+
+/*
+ * Solver step alone (paper, "Two-Stage GPU-Native Solver" and the dispatch
+ * layout): inter-node placement, routing construction, loads, intra-node
+ * refinement, counts and offsets, from a routing matrix.
+ *   dev_omega  in  [B][R][E] int32 routing matrix, or NULL to use the one the
+ *                  last topoep_histogram / topoep_plan on this handle left in
+ *                  the workspace (e.g. rows gathered from other ranks go here)
+ * Outputs as in topoep_plan.  Leaves q, U, L and the per-expert instance lists
+ * in the workspace for topoep_reroute and topoep_summary.
+ */
+int topoep_solve(topoep_handle_t h, const int32_t* dev_omega, int batch,
+                 int32_t* dev_replica_map, int32_t* dev_dispatch_counts,
+                 int32_t* dev_dispatch_offsets, int32_t* dev_instance_counts,
+                 topoep_stream_t stream);
+
+/*
+ * Per-token assignment step alone (paper, "System Design": token-routing
+ * decisions drive dispatch).  Needs, in the workspace, the tile prefixes of a
+ * topoep_histogram over the SAME dev_topk_ids, tokens_per_rank and batch, and
+ * the routing of a topoep_solve after it.  Returns TOPOEP_ERR_SIZE when
+ * tokens_per_rank or batch differ from that histogram call.
+ */
+int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
+                   int batch, int32_t* dev_token_replica, topoep_stream_t stream);
 
 /*
  * Summaries of the last topoep_plan (paper: objective terms and evaluation

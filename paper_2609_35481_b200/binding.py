@@ -20,7 +20,7 @@ T_OMEGA, T_Q, T_RANK_LOAD, T_REFINE_ITERS = 0, 1, 2, 3
 KNOB_TILE_IDS, KNOB_HIST_MODE = 0, 1
 
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
-           "topoep_plan", "topoep_histogram", "topoep_summary", "topoep_read_status",
+           "topoep_plan", "topoep_histogram", "topoep_solve", "topoep_reroute", "topoep_summary", "topoep_read_status",
            "topoep_debug_tensor", "topoep_set_tuning", "topoep_get_layout",
            "topoep_launch_floor", "topoep_strerror")
 
@@ -65,6 +65,10 @@ def lib() -> ctypes.CDLL:
         L.topoep_plan.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, vp, vp]
         L.topoep_histogram.restype = ci
         L.topoep_histogram.argtypes = [vp, vp, ci, ci, vp, vp]
+        L.topoep_solve.restype = ci
+        L.topoep_solve.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp]
+        L.topoep_reroute.restype = ci
+        L.topoep_reroute.argtypes = [vp, vp, ci, ci, vp, vp]
         L.topoep_summary.restype = ci
         L.topoep_summary.argtypes = [vp, ci, vp, vp]
         L.topoep_read_status.restype = ci
@@ -136,6 +140,18 @@ def topoep_plan(h, dev_topk_ids, tokens_per_rank, batch, dev_replica_map, dev_to
 def topoep_histogram(h, dev_topk_ids, tokens_per_rank, batch, dev_omega, stream=0) -> int:
     return lib().topoep_histogram(h, _ptr(dev_topk_ids), tokens_per_rank, batch, _ptr(dev_omega),
                                   stream or None)
+
+
+def topoep_solve(h, dev_omega, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
+                 dev_instance_counts, stream=0) -> int:
+    return lib().topoep_solve(h, _ptr(dev_omega), batch, _ptr(dev_replica_map),
+                              _ptr(dev_dispatch_counts), _ptr(dev_dispatch_offsets),
+                              _ptr(dev_instance_counts), stream or None)
+
+
+def topoep_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream=0) -> int:
+    return lib().topoep_reroute(h, _ptr(dev_topk_ids), tokens_per_rank, batch,
+                                _ptr(dev_token_replica), stream or None)
 
 
 def topoep_summary(h, batch, dev_out, stream=0) -> int:

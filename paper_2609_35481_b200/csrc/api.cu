@@ -1,6 +1,7 @@
 // C boundary of the TopoEP planning library: argument checks, workspace carving, kernel
 // enqueue.  Nothing here allocates, frees or copies device memory on the planning path; the
-// plan call enqueues three kernels (histogram, solver + layout, reroute) on the caller's stream.
+// plan call enqueues five kernels (tile histogram, omega, solver, route tables, reroute) on the
+// caller's stream.
 #include <algorithm>
 #include <new>
 
@@ -16,10 +17,11 @@ struct topoep_ctx {
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode;
   int max_tiles;
+  int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
   // workspace
   bool have_ws;
   Workspace ws;
-  size_t off[16];
+  size_t off[24];
   size_t ws_bytes;
   cudaError_t last_cuda;
 };
@@ -30,10 +32,10 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 enum WsSlot {
-  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_STATUS, W_HTICKETS, W_STICKETS, W_OMEGA, W_TILE,
-  W_Q, W_LOAD, W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_SEG, W_INST_SORTED, W_SLOTS
+  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_STATUS, W_OMEGA, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
+  W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC, W_SLOTS
 };
-static_assert(W_SLOTS == 16, "offset table size");
+static_assert(W_SLOTS <= 24, "offset table size");
 
 void carve(topoep_ctx* h) {
   const Dims& d = h->d;
@@ -43,18 +45,17 @@ void carve(topoep_ctx* h) {
   sz[W_MAIN_LOCAL] = 4 * E;
   sz[W_MAIN_INST] = 4 * R * (size_t)std::max(d.e_loc, 1);
   sz[W_STATUS] = 4;
-  sz[W_HTICKETS] = 4 * B * R;
-  sz[W_STICKETS] = 4 * B;
   sz[W_OMEGA] = 4 * B * R * E;
-  sz[W_TILE] = 4 * B * R * (size_t)h->max_tiles * E;
+  sz[W_TILE_CNT] = 4 * B * R * (size_t)h->max_tiles * E;
+  sz[W_TILE_PREF] = sz[W_TILE_CNT];
   sz[W_Q] = 4 * B * R * P;
   sz[W_LOAD] = 4 * B * R;
   sz[W_ITERS] = 4 * B * (size_t)d.M;
   sz[W_INST_COUNTS] = 4 * B * P;
   sz[W_REPLICA_MAP] = 4 * B * R * (size_t)std::max(d.N, 1);
   sz[W_COUNTS] = 4 * B * R * R;
-  sz[W_SEG] = 4 * B * (E + 1);
-  sz[W_INST_SORTED] = 4 * B * P;
+  sz[W_ROUTE] = 4 * B * R * E;
+  sz[W_SPLIT_REC] = 4 * B * R * (size_t)split_rec_layout(d.E, d.P).ints;
   size_t at = 0;
   for (int i = 0; i < W_SLOTS; ++i) { h->off[i] = at; at += align_up(sz[i]); }
   h->ws_bytes = at;
@@ -156,8 +157,10 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->hist_mode = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
+  h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
   h->last_cuda = cudaSuccess;
   if (solve_smem_bytes(d) > 227 * 1024 || reroute_smem_bytes(d, kMaxTileIds) > 227 * 1024 ||
+      route_smem_bytes(d) > 227 * 1024 ||
       hist_smem_bytes(d) > 48 * 1024) {
     delete h;
     return TOPOEP_ERR_SMEM;
@@ -181,18 +184,17 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.main_local = at<int32_t>(dev_ptr, h->off[W_MAIN_LOCAL]);
   w.main_inst_expert = at<int32_t>(dev_ptr, h->off[W_MAIN_INST]);
   w.status = at<uint32_t>(dev_ptr, h->off[W_STATUS]);
-  w.hist_tickets = at<uint32_t>(dev_ptr, h->off[W_HTICKETS]);
-  w.solve_tickets = at<uint32_t>(dev_ptr, h->off[W_STICKETS]);
   w.omega = at<int32_t>(dev_ptr, h->off[W_OMEGA]);
-  w.tile_pref = at<int32_t>(dev_ptr, h->off[W_TILE]);
+  w.tile_cnt = at<int32_t>(dev_ptr, h->off[W_TILE_CNT]);
+  w.tile_pref = at<int32_t>(dev_ptr, h->off[W_TILE_PREF]);
   w.q = at<int32_t>(dev_ptr, h->off[W_Q]);
   w.rank_load = at<int32_t>(dev_ptr, h->off[W_LOAD]);
   w.refine_iters = at<int32_t>(dev_ptr, h->off[W_ITERS]);
   w.inst_counts = at<int32_t>(dev_ptr, h->off[W_INST_COUNTS]);
   w.replica_map = at<int32_t>(dev_ptr, h->off[W_REPLICA_MAP]);
   w.counts = at<int32_t>(dev_ptr, h->off[W_COUNTS]);
-  w.seg_start = at<int32_t>(dev_ptr, h->off[W_SEG]);
-  w.inst_sorted = at<int32_t>(dev_ptr, h->off[W_INST_SORTED]);
+  w.route = at<int32_t>(dev_ptr, h->off[W_ROUTE]);
+  w.split_rec = at<int32_t>(dev_ptr, h->off[W_SPLIT_REC]);
 
   cudaError_t e;
   const size_t E = h->d.E;
@@ -202,9 +204,9 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
                       cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_inst_expert), h->main_inst_expert.data(),
                       4 * h->main_inst_expert.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
-  // status word and both ticket arrays are contiguous slots: zero them in one go
-  if ((e = cudaMemset(w.status, 0, h->off[W_OMEGA] - h->off[W_STATUS])) != cudaSuccess) goto fail;
+  if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
   if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
+  if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_reroute(reroute_smem_bytes(h->d, kMaxTileIds))) != cudaSuccess) goto fail;
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) goto fail;
   h->have_ws = true;
@@ -214,17 +216,111 @@ fail:
   return TOPOEP_ERR_CUDA;
 }
 
+namespace {
+
+int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* out_omega,
+                 cudaStream_t stream) {
+  const HistParams hp = make_hist(h, ids, T, out_omega);
+  h->hist_tile_ids = hp.tile_ids;
+  h->hist_tokens = T;
+  h->hist_batch = batch;
+  cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
+  if (e == cudaSuccess) e = launch_omega(hp, batch, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+// Solver, then the per-source routing tables.  The tile prefixes are (re)built only when the tile
+// counts in the workspace belong to this batch size.
+int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* replica_map,
+                  int32_t* counts, int32_t* offsets, int32_t* inst_counts, cudaStream_t stream) {
+  SolveParams sp;
+  sp.d = h->d;
+  sp.ws = h->ws;
+  sp.omega = omega ? omega : h->ws.omega;
+  sp.token_bytes = h->cost.token_bytes;
+  sp.expert_bytes = h->cost.expert_bytes;
+  sp.max_iters = h->max_iters;
+  sp.min_delta = h->min_delta;
+  sp.cost_rank_intra = h->cost_rank_intra;
+  sp.cost_rank_inter = h->cost_rank_inter;
+  sp.out_replica_map = replica_map;
+  sp.out_counts = counts;
+  sp.out_offsets = offsets;
+  sp.out_inst_counts = inst_counts;
+  cudaError_t e = launch_solve(sp, batch, stream);
+  if (e == cudaSuccess) {
+    RouteParams rp;
+    rp.d = h->d;
+    rp.ws = h->ws;
+    rp.out_offsets = offsets;
+    rp.max_tiles = h->max_tiles;
+    rp.tiles = 0;
+    if (h->hist_batch == batch && h->hist_tokens >= 0) {
+      const int n_ids = h->hist_tokens * h->d.k;
+      rp.tiles = std::max(1, (n_ids + h->hist_tile_ids - 1) / h->hist_tile_ids);
+    }
+    e = launch_route(rp, batch, stream);
+  }
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* token_replica,
+                    cudaStream_t stream) {
+  if (T == 0) return TOPOEP_OK;
+  RerouteParams rp;
+  rp.d = h->d;
+  rp.ws = h->ws;
+  rp.ids = ids;
+  rp.out_token_replica = token_replica;
+  rp.n_ids = T * h->d.k;
+  rp.tile_ids = h->hist_tile_ids;
+  rp.tiles = std::max(1, (rp.n_ids + rp.tile_ids - 1) / rp.tile_ids);
+  rp.max_tiles = h->max_tiles;
+  rp.vec_ok = (rp.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0) &&
+              ((reinterpret_cast<uintptr_t>(token_replica) & 15u) == 0);
+  const cudaError_t e = launch_reroute(rp, batch, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+}  // namespace
+
 int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
                      int batch, int32_t* dev_omega, topoep_stream_t stream) {
   int rc = check_sizes(h, tokens_per_rank, batch);
   if (rc != TOPOEP_OK) return rc;
   if (batch == 0) return TOPOEP_OK;
-  if (!dev_omega || (!dev_topk_ids && tokens_per_rank > 0)) return TOPOEP_ERR_NULL;
+  if (!dev_topk_ids && tokens_per_rank > 0) return TOPOEP_ERR_NULL;
   if (!aligned4(dev_topk_ids) || !aligned4(dev_omega)) return TOPOEP_ERR_ALIGN;
-  const HistParams hp = make_hist(h, dev_topk_ids, tokens_per_rank, dev_omega);
-  cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
-  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
-  return TOPOEP_OK;
+  return enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, dev_omega, stream);
+}
+
+int topoep_solve(topoep_handle_t h, const int32_t* dev_omega, int batch, int32_t* dev_replica_map,
+                 int32_t* dev_dispatch_counts, int32_t* dev_dispatch_offsets,
+                 int32_t* dev_instance_counts, topoep_stream_t stream) {
+  int rc = check_sizes(h, 0, batch);
+  if (rc != TOPOEP_OK) return rc;
+  if (batch == 0) return TOPOEP_OK;
+  if (!dev_dispatch_counts || !dev_dispatch_offsets) return TOPOEP_ERR_NULL;
+  if (h->d.N > 0 && !dev_replica_map) return TOPOEP_ERR_NULL;
+  if (!aligned4(dev_omega) || !aligned4(dev_replica_map) || !aligned4(dev_dispatch_counts) ||
+      !aligned4(dev_dispatch_offsets) || !aligned4(dev_instance_counts))
+    return TOPOEP_ERR_ALIGN;
+  return enqueue_solve(h, dev_omega, batch, dev_replica_map, dev_dispatch_counts,
+                       dev_dispatch_offsets, dev_instance_counts, stream);
+}
+
+int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank, int batch,
+                   int32_t* dev_token_replica, topoep_stream_t stream) {
+  int rc = check_sizes(h, tokens_per_rank, batch);
+  if (rc != TOPOEP_OK) return rc;
+  if (batch == 0) return TOPOEP_OK;
+  if (tokens_per_rank != h->hist_tokens || batch != h->hist_batch) return TOPOEP_ERR_SIZE;
+  if (tokens_per_rank > 0 && (!dev_topk_ids || !dev_token_replica)) return TOPOEP_ERR_NULL;
+  if (!aligned4(dev_topk_ids) || !aligned4(dev_token_replica)) return TOPOEP_ERR_ALIGN;
+  return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
 }
 
 int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank, int batch,
@@ -241,41 +337,12 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
       !aligned4(dev_dispatch_counts) || !aligned4(dev_dispatch_offsets) ||
       !aligned4(dev_instance_counts))
     return TOPOEP_ERR_ALIGN;
-
-  const HistParams hp = make_hist(h, dev_topk_ids, tokens_per_rank, nullptr);
-  cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
-  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
-
-  SolveParams sp;
-  sp.d = h->d;
-  sp.ws = h->ws;
-  sp.token_bytes = h->cost.token_bytes;
-  sp.expert_bytes = h->cost.expert_bytes;
-  sp.max_iters = h->max_iters;
-  sp.min_delta = h->min_delta;
-  sp.cost_rank_intra = h->cost_rank_intra;
-  sp.cost_rank_inter = h->cost_rank_inter;
-  sp.out_replica_map = dev_replica_map;
-  sp.out_counts = dev_dispatch_counts;
-  sp.out_offsets = dev_dispatch_offsets;
-  sp.out_inst_counts = dev_instance_counts;
-  e = launch_solve(sp, batch, stream);
-  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
-
-  if (tokens_per_rank > 0) {
-    RerouteParams rp;
-    rp.d = h->d;
-    rp.ws = h->ws;
-    rp.ids = dev_topk_ids;
-    rp.out_token_replica = dev_token_replica;
-    rp.n_ids = hp.n_ids;
-    rp.tiles = hp.tiles;
-    rp.max_tiles = hp.max_tiles;
-    rp.tile_ids = hp.tile_ids;
-    e = launch_reroute(rp, batch, stream);
-    if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
-  }
-  return TOPOEP_OK;
+  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream);
+  if (rc != TOPOEP_OK) return rc;
+  rc = enqueue_solve(h, nullptr, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
+                     dev_instance_counts, stream);
+  if (rc != TOPOEP_OK) return rc;
+  return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
 }
 
 int topoep_summary(topoep_handle_t h, int batch, topoep_summary_t* dev_out, topoep_stream_t stream) {

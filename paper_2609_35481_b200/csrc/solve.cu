@@ -9,9 +9,8 @@
 // -- which domains host each expert after inter-node placement -- it recomputes itself, one
 // warp per domain, so no CTA ever waits for another.  Refinement is the serial part: one warp
 // runs the loop, every selection is a warp reduction over a totally ordered key.
-//
-// The last CTA of a plan to finish (ticket counter, no spinning) adds what needs all domains:
-// the send offsets and the (expert, rank)-ordered instance list the reroute kernel walks.
+// What needs every domain's result (send offsets, per-source routing tables) is left to the
+// route kernel that follows.
 #include <limits.h>
 
 #include "topoep_internal.cuh"
@@ -21,7 +20,7 @@ namespace topoep {
 namespace {
 
 struct SolveLayout {
-  size_t hostmask, D, qd, col_expert, col_cr, U, L, used, cnt, tail, hostcol, total;
+  size_t hostmask, D, qd, col_expert, col_cr, U, L, used, cnt, hostcol, total;
 };
 
 __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
@@ -36,7 +35,6 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   o.L = at;          at += sizeof(int) * (size_t)d.G;
   o.used = at;       at += sizeof(int) * (size_t)d.G;
   o.cnt = at;        at += sizeof(int) * (size_t)d.R * d.G;
-  o.tail = at;       at += sizeof(int) * ((size_t)2 * d.E + 2 + (size_t)d.R * d.N);
   o.hostcol = at;    at += sizeof(short) * (size_t)d.G * d.E;
   o.total = (at + 15) & ~(size_t)15;
   return o;
@@ -44,7 +42,6 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
 
 __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
-  __shared__ bool is_last;
   const Dims d = p.d;
   const int M = d.M, G = d.G, R = d.R, E = d.E, N = d.N, C = d.C, QS = d.qstride;
   const int s_phys = d.s_phys, e_loc = d.e_loc;
@@ -62,10 +59,9 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   int* L = reinterpret_cast<int*>(smem + lay.L);
   int* used = reinterpret_cast<int*>(smem + lay.used);
   int* cnt = reinterpret_cast<int*>(smem + lay.cnt);
-  int* tail = reinterpret_cast<int*>(smem + lay.tail);
   short* hostcol = reinterpret_cast<short*>(smem + lay.hostcol);
 
-  const int32_t* om = p.ws.omega + (size_t)b * R * E;
+  const int32_t* om = p.omega + (size_t)b * R * E;
   const int32_t* main_rank = p.ws.main_rank;
 
   // ---- tables of the own domain; candidate demand of every domain -------------------------
@@ -77,15 +73,35 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     U[c] = 0;
   }
   if (tid < G) used[tid] = 0;
-  // D[dd][e], kept only where e is a stage-1 candidate of dd (main outside dd and b > 0), else 0.
-  for (int e = tid; e < E; e += nt) {
-    const int md = main_rank[e] / G;
-    hostmask[e] = 1ull << md;
-    for (int dd = 0; dd < M; ++dd) {
-      int sum = 0;
-      for (int g = 0; g < G; ++g) sum += om[(size_t)(dd * G + g) * E + e];
-      const bool cand = dd != md && 2 * (long long)sum * p.token_bytes - p.expert_bytes > 0;
-      D[dd * E + e] = cand ? sum : 0;
+  for (int e = tid; e < E; e += nt) hostmask[e] = 1ull << (main_rank[e] / G);
+  // D[dd][e] = sum over the G source ranks of domain dd, kept only where e is a stage-1 candidate
+  // of dd (main outside dd and b > 0), else 0.  Loads are issued eight at a time.
+  for (int idx0 = tid; idx0 < M * E; idx0 += 4 * nt) {
+    int sum[4] = {0, 0, 0, 0};
+    for (int g0 = 0; g0 < G; g0 += 8) {
+      int v[4][8];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int idx = idx0 + a * nt;
+        const int dd = idx / E, e = idx - dd * E;
+        const int32_t* col = om + (size_t)dd * G * E + e;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          v[a][u] = (idx < M * E && g0 + u < G) ? __ldg(col + (size_t)(g0 + u) * E) : 0;
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int u = 0; u < 8; ++u) sum[a] += v[a][u];
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const int idx = idx0 + a * nt;
+      if (idx >= M * E) break;
+      const int dd = idx / E, e = idx - dd * E;
+      const bool cand = dd != main_rank[e] / G &&
+                        2 * (long long)sum[a] * p.token_bytes - p.expert_bytes > 0;
+      D[idx] = cand ? sum[a] : 0;
     }
   }
   __syncthreads();
@@ -133,28 +149,42 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   // After stage 1 an expert has at most one instance per domain.  A source keeps everything in
   // its own domain when an instance is there; otherwise it splits over all instances (ascending
   // rank == ascending hosting domain), remainder to `rem` instances starting at (s+e) mod n.
-  for (int idx = tid; idx < R * C; idx += nt) {
-    const int s = idx / C, c = idx - s * C;
-    const int e = col_expert[c];
-    int v = 0;
-    if (e >= 0) {
-      const int w = om[(size_t)s * E + e];
-      const int ds = s / G;
-      if (ds == dm) {
-        v = w;
-      } else {
-        const unsigned long long hm = hostmask[e];
-        if (!((hm >> ds) & 1ull)) {
-          const int n = __popcll(hm);
-          const int i = __popcll(hm & ((1ull << dm) - 1ull));
-          const int base = w / n, rem = w - base * n;
-          int sh = i - (s + e) % n;
-          if (sh < 0) sh += n;
-          v = base + (sh < rem ? 1 : 0);
-        }
+  for (int idx0 = tid; idx0 < R * C; idx0 += 4 * nt) {
+    int w[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {   // the four omega loads go out before any is used
+      const int idx = idx0 + u * nt;
+      w[u] = 0;
+      if (idx < R * C) {
+        const int s = idx / C, e = col_expert[idx - s * C];
+        if (e >= 0) w[u] = __ldg(om + (size_t)s * E + e);
       }
     }
-    qd[s * QS + c] = v;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int idx = idx0 + u * nt;
+      if (idx >= R * C) break;
+      const int s = idx / C, c = idx - s * C;
+      const int e = col_expert[c];
+      int v = 0;
+      if (e >= 0) {
+        const int ds = s / G;
+        if (ds == dm) {
+          v = w[u];
+        } else {
+          const unsigned long long hm = hostmask[e];
+          if (!((hm >> ds) & 1ull)) {
+            const int n = __popcll(hm);
+            const int i = __popcll(hm & ((1ull << dm) - 1ull));
+            const int base = w[u] / n, rem = w[u] - base * n;
+            int sh = i - (s + e) % n;
+            if (sh < 0) sh += n;
+            v = base + (sh < rem ? 1 : 0);
+          }
+        }
+      }
+      qd[s * QS + c] = v;
+    }
   }
   __syncthreads();
   for (int c = tid; c < C; c += nt) {
@@ -294,80 +324,6 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     recv[R] = run;
   }
 
-  // ---- last CTA of the plan: what needs every domain ----------------------------------------
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&p.ws.solve_tickets[b], 1u) == (unsigned)(M - 1));
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-
-  // send offsets of source s: exclusive scan over the destination ranks
-  {
-    const int ch = (R + 31) / 32;
-    for (int s = warp; s < R; s += nwarps) {
-      const int32_t* row = p.ws.counts + ((size_t)b * R + s) * R;
-      int32_t* send = p.out_offsets + (((size_t)b * 2 + 0) * R + s) * (R + 1);
-      const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
-      int sum = 0;
-      for (int r = i0; r < i1; ++r) sum += __ldcg(row + r);
-      int pre = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(full, pre, o);
-        if (lane >= o) pre += t;
-      }
-      if (lane == 31) send[R] = pre;
-      pre -= sum;
-      for (int r = i0; r < i1; ++r) { send[r] = pre; pre += __ldcg(row + r); }
-    }
-  }
-  // instances ordered by (expert, rank): segment of e = [seg[e], seg[e+1])
-  int* cntE = tail;              // [E]
-  int* seg = tail + E;           // [E+1]
-  int* rm = tail + 2 * E + 1;    // [R*N]
-  const int RN = R * N;
-  for (int i = tid; i < RN; i += nt) rm[i] = __ldcg(p.ws.replica_map + (size_t)b * RN + i);
-  for (int e = tid; e < E; e += nt) cntE[e] = 1;   // the main instance
-  __syncthreads();
-  for (int i = tid; i < RN; i += nt)
-    if (rm[i] >= 0) atomicAdd(&cntE[rm[i]], 1);
-  __syncthreads();
-  if (warp == 0) {
-    const int ch = (E + 31) / 32;
-    const int i0 = min(E, lane * ch), i1 = min(E, i0 + ch);
-    int sum = 0;
-    for (int e = i0; e < i1; ++e) sum += cntE[e];
-    int pre = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(full, pre, o);
-      if (lane >= o) pre += t;
-    }
-    if (lane == 31) seg[E] = pre;
-    pre -= sum;
-    for (int e = i0; e < i1; ++e) { seg[e] = pre; pre += cntE[e]; }
-  }
-  __syncthreads();
-  int32_t* inst_sorted = p.ws.inst_sorted + (size_t)b * d.P;
-  for (int e = tid; e < E; e += nt) {
-    const int rmain = main_rank[e];
-    int pos = 0;
-    if (cntE[e] > 1)
-      for (int i = 0; i < RN; ++i) pos += (rm[i] == e && i / N < rmain) ? 1 : 0;
-    inst_sorted[seg[e] + pos] = rmain * s_phys + p.ws.main_local[e];
-  }
-  for (int i = tid; i < RN; i += nt) {
-    const int e = rm[i];
-    if (e < 0) continue;
-    const int r = i / N, j = i - r * N;
-    int pos = main_rank[e] < r ? 1 : 0;
-    for (int i2 = 0; i2 < r * N; ++i2) pos += (rm[i2] == e) ? 1 : 0;
-    inst_sorted[seg[e] + pos] = r * s_phys + e_loc + j;
-  }
-  int32_t* seg_out = p.ws.seg_start + (size_t)b * (E + 1);
-  for (int e = tid; e <= E; e += nt) seg_out[e] = seg[e];
-  if (tid == 0) p.ws.solve_tickets[b] = 0;
 }
 
 }  // namespace

@@ -1,7 +1,7 @@
 // Internal declarations shared by the TopoEP planning kernels (sm_100a).
 //
 // Workspace layout, launch-parameter structs and the host-side launch
-// functions of the three planning kernels plus the summary kernel.
+// functions of the five planning kernels plus the summary kernel.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -15,8 +15,10 @@ namespace topoep {
 
 constexpr int kIdsPerThread = 16;   // every histogram / reroute thread owns 16 ids of its tile
 constexpr int kMinTileIds = 1024;
-constexpr int kMaxTileIds = 16384;
+constexpr int kMaxTileIds = 8192;
 constexpr int kSolveThreads = 512;
+constexpr int kRouteThreads = 256;
+constexpr int kSplitCap = 32;       // split experts the reroute kernel ranks per pass
 
 // Problem constants handed to every kernel by value.
 struct Dims {
@@ -32,19 +34,39 @@ struct Workspace {
   const int32_t* main_local;        // [E] index l of e among the experts of its main rank
   const int32_t* main_inst_expert;  // [R][e_loc] expert of main instance l on rank r, -1 if none
   uint32_t* status;                 // [1]
-  uint32_t* hist_tickets;           // [max_batch][R], zero between launches
-  uint32_t* solve_tickets;          // [max_batch],    zero between launches
   int32_t* omega;                   // [max_batch][R][E]
-  int32_t* tile_pref;               // [max_batch][R][max_tiles][E]: counts, then exclusive prefix
+  int32_t* tile_cnt;                // [max_batch][R][max_tiles][E] per-tile histogram
+  int32_t* tile_pref;               // [max_batch][R][max_tiles][E] exclusive prefix over tiles,
+                                    //   column i = i-th split expert of the source
   int32_t* q;                       // [max_batch][R][P]
   int32_t* rank_load;               // [max_batch][R]
   int32_t* refine_iters;            // [max_batch][M]
   int32_t* inst_counts;             // [max_batch][P]
   int32_t* replica_map;             // [max_batch][R][N]
   int32_t* counts;                  // [max_batch][R][R]
-  int32_t* seg_start;               // [max_batch][E+1] segment of expert e in inst_sorted
-  int32_t* inst_sorted;             // [max_batch][P]   instances ordered by (expert, rank)
+  // per (plan, source) routing tables written by the route kernel
+  int32_t* route;                   // [max_batch][R][E]  >= 0: the one instance; <= -2: -2 - split index
+  int32_t* split_rec;               // [max_batch][R][split_rec_ints(d)]: see SplitRec
 };
+
+// Record of one (plan, source) written by the route kernel, read by the reroute kernel:
+//   [0] n_split  [1] n_list  [2..3] unused
+//   seg  [E+1]  list i of the source's i-th split expert = [seg[i], seg[i+1])
+//   cum  [P]    cumulative quota along each list (instances in ascending rank order)
+//   inst [P]    physical instance ids along each list
+struct SplitRec {
+  int seg, cum, inst, ints;
+};
+__host__ __device__ inline SplitRec split_rec_layout(int E, int P) {
+  SplitRec r;
+  r.seg = 4;
+  r.cum = r.seg + ((E + 1 + 3) & ~3);
+  r.inst = r.cum + ((P + 3) & ~3);
+  r.ints = r.inst + ((P + 3) & ~3);
+  return r;
+}
+constexpr int kFastLists = 128;     // list entries the reroute kernel fetches before it knows n_list
+
 
 struct HistParams {
   Dims d;
@@ -53,7 +75,7 @@ struct HistParams {
   int32_t* out_omega;   // optional caller copy of omega [B][R][E]
   int n_ids;            // T * k
   int tiles;            // tiles per (plan, rank)
-  int max_tiles;        // stride of tile_pref
+  int max_tiles;        // stride of tile_cnt / tile_pref
   int tile_ids;
   int vec_ok;           // rows are 16-byte aligned and n_ids % 4 == 0
 };
@@ -61,6 +83,7 @@ struct HistParams {
 struct SolveParams {
   Dims d;
   Workspace ws;
+  const int32_t* omega;       // [B][R][E] routing matrix to plan from
   int64_t token_bytes, expert_bytes;
   int max_iters, min_delta;
   int cost_rank_intra, cost_rank_inter;   // dense ranks of {0, c_intra*W, c_inter*W}
@@ -70,12 +93,20 @@ struct SolveParams {
   int32_t* out_inst_counts;   // [B][P] or NULL
 };
 
+struct RouteParams {
+  Dims d;
+  Workspace ws;
+  int32_t* out_offsets;       // [B][2][R][R+1]: the send half is written here
+  int tiles, max_tiles;       // shape of the tile counts now in the workspace (tiles 0: none)
+};
+
 struct RerouteParams {
   Dims d;
   Workspace ws;
   const int32_t* ids;
   int32_t* out_token_replica;
   int n_ids, tiles, max_tiles, tile_ids;
+  int vec_ok;
 };
 
 struct SummaryParams {
@@ -88,12 +119,16 @@ struct SummaryParams {
 
 size_t hist_smem_bytes(const Dims& d);
 size_t solve_smem_bytes(const Dims& d);
+size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 
 cudaError_t configure_solve(size_t smem);
+cudaError_t configure_route(size_t smem);
 cudaError_t configure_reroute(size_t smem);
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream);
+cudaError_t launch_omega(const HistParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream);
+cudaError_t launch_route(const RouteParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_summary(const SummaryParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_empty(int count, cudaStream_t stream);
@@ -102,6 +137,34 @@ __device__ __forceinline__ unsigned lanemask_lt() {
   unsigned m;
   asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
   return m;
+}
+
+// Exclusive prefix sum across the lanes of a full warp; *total gets the warp's sum.
+__device__ __forceinline__ int warp_exclusive_scan(int v, int lane, int* total) {
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  *total = __shfl_sync(0xffffffffu, inc, 31);
+  return inc - v;
+}
+
+// The 16 ids a thread owns: four groups of four consecutive ids; group j of thread t is vector
+// j*blockDim.x + t of the tile, so a warp reads 512 contiguous bytes per group.
+__device__ __forceinline__ int4 load_ids4(const int32_t* tile_ids, int vec, int count, bool vec_ok) {
+  if (vec_ok) {
+    return 4 * vec < count ? __ldg(reinterpret_cast<const int4*>(tile_ids) + vec)
+                           : make_int4(-1, -1, -1, -1);
+  }
+  int4 r;
+  const int i = 4 * vec;
+  r.x = i + 0 < count ? __ldg(tile_ids + i + 0) : -1;
+  r.y = i + 1 < count ? __ldg(tile_ids + i + 1) : -1;
+  r.z = i + 2 < count ? __ldg(tile_ids + i + 2) : -1;
+  r.w = i + 3 < count ? __ldg(tile_ids + i + 3) : -1;
+  return r;
 }
 
 }  // namespace topoep

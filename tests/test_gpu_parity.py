@@ -175,7 +175,7 @@ def test_bitwise_identical_across_reruns_and_tunings():
     ids = wl.make_topk_ids(w, seed=31, batch=2)
     pl = make_planner(w, max_batch=2)
     base = run_gpu(pl, ids)
-    for tile in (1024, 2048, 4096, 8192, 16384):
+    for tile in (1024, 2048, 4096, 8192):
         for mode in (0, 1):
             pl.set_tuning(B.KNOB_TILE_IDS, tile)
             pl.set_tuning(B.KNOB_HIST_MODE, mode)
@@ -200,6 +200,31 @@ def test_histogram_entry_point_matches_bincount():
     for b in range(2):
         for s in range(w.ranks):
             assert np.array_equal(om[b, s], np.bincount(ids[b, s].ravel(), minlength=w.experts))
+
+
+def test_stage_entry_points_equal_the_fused_plan():
+    w = wl.CONFIGS["mid"].replace(slots_per_rank=3)
+    ids = wl.make_topk_ids(w, seed=13, batch=2)
+    pl = make_planner(w, max_batch=2)
+    dev = torch.from_numpy(ids).to(pl.device)
+    fused = pl.plan(dev)
+    out = pl.alloc_outputs(2, w.tokens_per_rank)
+    for t in (out.replica_map, out.token_replica, out.dispatch_counts, out.dispatch_offsets,
+              out.instance_counts):
+        t.fill_(-9)
+    omega = torch.empty((2, w.ranks, w.experts), dtype=torch.int32, device=pl.device)
+    T = w.tokens_per_rank
+    assert B.topoep_histogram(pl.handle, dev, T, 2, omega, 0) == 0
+    # the solver accepts the routing matrix from anywhere (e.g. rows gathered from other ranks)
+    assert B.topoep_solve(pl.handle, omega.clone(), 2, out.replica_map, out.dispatch_counts,
+                          out.dispatch_offsets, out.instance_counts, 0) == 0
+    assert B.topoep_reroute(pl.handle, dev, T - 1, 2, out.token_replica, 0) == -6
+    assert B.topoep_reroute(pl.handle, dev, T, 2, out.token_replica, 0) == 0
+    torch.cuda.synchronize()
+    for name in ("replica_map", "token_replica", "dispatch_counts", "dispatch_offsets",
+                 "instance_counts"):
+        assert torch.equal(getattr(out, name), getattr(fused, name)), name
+    assert pl.status() == 0
 
 
 # ---- capture: the plan is enqueue-only ---------------------------------------------------------
@@ -244,5 +269,6 @@ def test_size_and_pointer_errors():
     assert B.topoep_set_workspace(pl.handle, pl._ws_ptr + 4, 1 << 30) == -5
     assert B.topoep_set_workspace(pl.handle, pl._ws_ptr, 16) == -5
     assert B.topoep_set_tuning(pl.handle, B.KNOB_TILE_IDS, 3000) == -10
-    # the failed set_workspace calls dropped the workspace: the next plan says so
-    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 1, *args) == -5
+    # a rejected set_workspace leaves the previous workspace in place
+    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 1, *args) == 0
+    torch.cuda.synchronize()
