@@ -35,7 +35,7 @@ __host__ __device__ inline RerouteLayout reroute_layout(const Dims& d, int tile_
   o.inst = at;  at += sizeof(int) * (size_t)d.P;
   o.tbase = at; at += sizeof(int) * (size_t)kSplitCap;
   o.hdr = at;   at += sizeof(int) * 4;
-  o.work = at;  at += sizeof(unsigned) * (size_t)tile_ids;
+  o.work = at;  at += sizeof(unsigned short) * (size_t)tile_ids;
   o.total = at;
   return o;
 }
@@ -46,14 +46,94 @@ __device__ __forceinline__ int nibble_sum(unsigned x) {
   return (int)((y * 0x01010101u) >> 24);
 }
 
-// Work item: position in the tile (14 bits) | earlier equal ids in the same lane group (2 bits)
-// | split index (16 bits).
-__device__ __forceinline__ void push(unsigned* work, int* n_work, int pos, int prev, int t) {
-  const int slot = atomicAdd(n_work, 1);
-  work[slot] = (unsigned)pos | ((unsigned)prev << 14) | ((unsigned)(-2 - t) << 16);
+// A work item is the position of a split assignment in the tile; its expert and the number of
+// equal ids before it in its group of four are read back from the id array when it is processed.
+
+// Everything the ranking of the split items needs.
+struct SplitCtx {
+  uint4* cnt4; unsigned* cntw; int* base; const int* route; int* seg; int* cum; int* inst;
+  int* tbase; const unsigned short* work; const int32_t* rec; const int32_t* g_tp;
+  const int32_t* ids; int32_t* out; SplitRec rl; int rows, n_split, n_list, n_work;
+  uint32_t* status;
+};
+
+// Rank the split items of the tile and patch their outputs.  Run either by one warp (SOLO:
+// tid = lane, nt = 32, warp-level syncs) or by the whole CTA.
+template <bool SOLO>
+__device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int nt, int warp,
+                                               int nwarps) {
+  const int lane = tid & 31, rows = c.rows;
+  auto sync = [] { if (SOLO) __syncwarp(); else __syncthreads(); };
+  if (c.n_split > kSplitCap || c.n_list > kFastLists) {   // rare: fetch the rest of the record
+    for (int i = tid; i <= c.n_split; i += nt) c.seg[i] = c.rec[c.rl.seg + i];
+    for (int i = tid; i < c.n_list; i += nt) {
+      c.cum[i] = c.rec[c.rl.cum + i];
+      c.inst[i] = c.rec[c.rl.inst + i];
+    }
+  }
+  bool broken = false;
+  for (int p0 = 0; p0 < c.n_split; p0 += kSplitCap) {
+    const int n_here = min(kSplitCap, c.n_split - p0);
+    if (p0 > 0) {   // later passes: fresh counters and tile bases (the first set came up front)
+      for (int i = tid; i < n_here * rows; i += nt) c.cnt4[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (tid < n_here) c.tbase[tid] = c.g_tp[p0 + tid];
+    }
+    if (p0 > 0 || c.n_split > kSplitCap || c.n_list > kFastLists) sync();
+    // every item bumps the 4-bit counter of its (split expert, row, lane)
+    for (int w = tid; w < c.n_work; w += nt) {
+      const int pos = c.work[w];
+      const int i = -2 - c.route[__ldg(c.ids + pos)] - p0;
+      if (i < 0 || i >= n_here) continue;
+      const int vec = pos >> 2;                            // int4 index inside the tile
+      const int rr = vec >> 5, ln = vec & 31;              // row, lane inside the row
+      atomicAdd(&c.cntw[(i * rows + rr) * 4 + (ln >> 3)], 1u << (4 * (ln & 7)));
+    }
+    sync();
+    // base[i][rr] = tile base + ids of split expert i in rows before rr
+    for (int i = warp; i < n_here; i += nwarps) {
+      int carry = c.tbase[i];
+      for (int r0 = 0; r0 < rows; r0 += 32) {
+        const int rr = r0 + lane;
+        int tot = 0;
+        if (rr < rows) {
+          const uint4 q = c.cnt4[i * rows + rr];
+          tot = nibble_sum(q.x) + nibble_sum(q.y) + nibble_sum(q.z) + nibble_sum(q.w);
+        }
+        int all;
+        const int ex = warp_exclusive_scan(tot, lane, &all);
+        if (rr < rows) c.base[i * rows + rr] = carry + ex;
+        carry += all;
+      }
+    }
+    sync();
+    for (int w = tid; w < c.n_work; w += nt) {
+      const int pos = c.work[w], vec = pos >> 2;
+      const int e = __ldg(c.ids + pos);
+      const int i = -2 - c.route[e] - p0;
+      if (i < 0 || i >= n_here) continue;
+      int prev = 0;   // equal ids earlier in the same group of four
+      for (int u = pos & ~3; u < pos; ++u) prev += __ldg(c.ids + u) == e ? 1 : 0;
+      const int rr = vec >> 5, ln = vec & 31, word = ln >> 3, shift = 4 * (ln & 7);
+      const uint4 q = c.cnt4[i * rows + rr];
+      const unsigned cw[4] = {q.x, q.y, q.z, q.w};
+      int rho = c.base[i * rows + rr] + prev;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (u < word) rho += nibble_sum(cw[u]);
+        else if (u == word) rho += nibble_sum(cw[u] & ((1u << shift) - 1u));
+      }
+      int at = c.seg[p0 + i];
+      const int end = c.seg[p0 + i + 1] - 1;
+      while (at < end && rho >= c.cum[at]) ++at;
+      broken |= rho >= c.cum[at];
+      c.out[pos] = c.inst[at];
+    }
+    if (p0 + kSplitCap < c.n_split) sync();
+  }
+  if (broken) atomicOr(c.status, TOPOEP_FLAG_INTERNAL);
 }
 
-__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) reroute_kernel(const RerouteParams p) {
+__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, 4) reroute_kernel(const RerouteParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const Dims d = p.d;
   const int E = d.E, P = d.P;
@@ -70,7 +150,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) reroute_kernel(co
   int* inst = reinterpret_cast<int*>(smem + lay.inst);
   int* tbase = reinterpret_cast<int*>(smem + lay.tbase);
   int* hdr = reinterpret_cast<int*>(smem + lay.hdr);           // n_split, n_list, n_work
-  unsigned* work = reinterpret_cast<unsigned*>(smem + lay.work);
+  unsigned short* work = reinterpret_cast<unsigned short*>(smem + lay.work);
 
   const size_t row = (size_t)b * d.R + s;
   const int begin = tile * p.tile_ids;
@@ -94,26 +174,22 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) reroute_kernel(co
   for (int i = tid; i < fast_list; i += nt) { cum[i] = rec[rl.cum + i]; inst[i] = rec[rl.inst + i]; }
   if (tid < min(E, kSplitCap)) tbase[tid] = g_tp[tid];
   if (tid == 0) { hdr[0] = rec[0]; hdr[1] = rec[1]; hdr[2] = 0; }
+  for (int i = tid; i < kSplitCap * rows; i += nt) cnt4[i] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
 
-  // Stream: look up, store, push the split ones.  An ignored id and a split id both store -1
-  // for now; the split ones are patched below.
+  // Stream: look up and store.  An ignored id and a split id both store -1 for now; the split
+  // ones are remembered in a 16-bit mask, pushed on the work list afterwards and patched below.
   const unsigned uE = (unsigned)E;
+  unsigned split_mask = 0;
 #pragma unroll
   for (int j = 0; j < kIdsPerThread / 4; ++j) {
     const int vec = j * nt + tid;
-    const int e0 = x[j].x, e1 = x[j].y, e2 = x[j].z, e3 = x[j].w;
-    const int t0 = (unsigned)e0 < uE ? route[e0] : -1;
-    const int t1 = (unsigned)e1 < uE ? route[e1] : -1;
-    const int t2 = (unsigned)e2 < uE ? route[e2] : -1;
-    const int t3 = (unsigned)e3 < uE ? route[e3] : -1;
-    if (min(min(t0, t1), min(t2, t3)) <= -2) {
-      int* n_work = hdr + 2;
-      if (t0 <= -2) push(work, n_work, 4 * vec + 0, 0, t0);
-      if (t1 <= -2) push(work, n_work, 4 * vec + 1, (e0 == e1), t1);
-      if (t2 <= -2) push(work, n_work, 4 * vec + 2, (e0 == e2) + (e1 == e2), t2);
-      if (t3 <= -2) push(work, n_work, 4 * vec + 3, (e0 == e3) + (e1 == e3) + (e2 == e3), t3);
-    }
+    const int t0 = (unsigned)x[j].x < uE ? route[x[j].x] : -1;
+    const int t1 = (unsigned)x[j].y < uE ? route[x[j].y] : -1;
+    const int t2 = (unsigned)x[j].z < uE ? route[x[j].z] : -1;
+    const int t3 = (unsigned)x[j].w < uE ? route[x[j].w] : -1;
+    split_mask |= (t0 <= -2 ? 1u : 0u) << (4 * j) | (t1 <= -2 ? 2u : 0u) << (4 * j) |
+                  (t2 <= -2 ? 4u : 0u) << (4 * j) | (t3 <= -2 ? 8u : 0u) << (4 * j);
     const int4 r = make_int4(max(t0, -1), max(t1, -1), max(t2, -1), max(t3, -1));
     if (p.vec_ok) {
       if (4 * vec < count) reinterpret_cast<int4*>(out)[vec] = r;
@@ -124,71 +200,24 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) reroute_kernel(co
       if (4 * vec + 3 < count) out[4 * vec + 3] = r.w;
     }
   }
+  while (split_mask) {   // ~3% of the ids on the benchmark workloads
+    const int k = __ffs(split_mask) - 1;
+    split_mask &= split_mask - 1;
+    work[atomicAdd(hdr + 2, 1)] = (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
+  }
   __syncthreads();   // also orders the stores above before the patches below
   const int n_work = hdr[2];
   if (n_work == 0) return;
 
-  const int n_split = hdr[0], n_list = hdr[1];
-  if (n_split > kSplitCap || n_list > kFastLists) {   // rare: fetch the rest of the record
-    for (int i = tid; i <= n_split; i += nt) seg[i] = rec[rl.seg + i];
-    for (int i = tid; i < n_list; i += nt) { cum[i] = rec[rl.cum + i]; inst[i] = rec[rl.inst + i]; }
+  // Few items (the usual case): one warp ranks and patches them with warp-level syncs only and the
+  // other warps retire; many items: the whole CTA works on them.
+  const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, rec, g_tp, ids, out,
+                      rl, rows, hdr[0], hdr[1], n_work, p.ws.status};
+  if (n_work <= p.solo_items) {
+    if (warp == 0) rank_and_patch<true>(c, lane, 32, 0, 1);
+  } else {
+    rank_and_patch<false>(c, tid, nt, warp, nwarps);
   }
-  bool broken = false;
-  for (int p0 = 0; p0 < n_split; p0 += kSplitCap) {
-    const int n_here = min(kSplitCap, n_split - p0);
-    for (int i = tid; i < n_here * rows; i += nt) cnt4[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (p0 > 0 && tid < n_here) tbase[tid] = g_tp[p0 + tid];
-    __syncthreads();
-    // every item bumps the 4-bit counter of its (split expert, row, lane)
-    for (int w = tid; w < n_work; w += nt) {
-      const unsigned it = work[w];
-      const int i = (int)(it >> 16) - p0;
-      if (i < 0 || i >= n_here) continue;
-      const int vec = (int)(it & 0x3fffu) >> 2;            // int4 index inside the tile
-      const int rr = vec >> 5, ln = vec & 31;              // row, lane inside the row
-      atomicAdd(&cntw[(i * rows + rr) * 4 + (ln >> 3)], 1u << (4 * (ln & 7)));
-    }
-    __syncthreads();
-    // base[i][rr] = tile base + ids of split expert i in rows before rr
-    for (int i = warp; i < n_here; i += nwarps) {
-      int carry = tbase[i];
-      for (int r0 = 0; r0 < rows; r0 += 32) {
-        const int rr = r0 + lane;
-        int tot = 0;
-        if (rr < rows) {
-          const uint4 c = cnt4[i * rows + rr];
-          tot = nibble_sum(c.x) + nibble_sum(c.y) + nibble_sum(c.z) + nibble_sum(c.w);
-        }
-        int all;
-        const int ex = warp_exclusive_scan(tot, lane, &all);
-        if (rr < rows) base[i * rows + rr] = carry + ex;
-        carry += all;
-      }
-    }
-    __syncthreads();
-    for (int w = tid; w < n_work; w += nt) {
-      const unsigned it = work[w];
-      const int i = (int)(it >> 16) - p0;
-      if (i < 0 || i >= n_here) continue;
-      const int pos = (int)(it & 0x3fffu), vec = pos >> 2;
-      const int rr = vec >> 5, ln = vec & 31, word = ln >> 3, shift = 4 * (ln & 7);
-      const uint4 c = cnt4[i * rows + rr];
-      const unsigned cw[4] = {c.x, c.y, c.z, c.w};
-      int rho = base[i * rows + rr] + (int)((it >> 14) & 3u);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (u < word) rho += nibble_sum(cw[u]);
-        else if (u == word) rho += nibble_sum(cw[u] & ((1u << shift) - 1u));
-      }
-      int at = seg[p0 + i];
-      const int end = seg[p0 + i + 1] - 1;
-      while (at < end && rho >= cum[at]) ++at;
-      broken |= rho >= cum[at];
-      out[pos] = inst[at];
-    }
-    __syncthreads();
-  }
-  if (broken) atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
 }
 
 }  // namespace

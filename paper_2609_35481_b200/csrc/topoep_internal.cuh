@@ -18,7 +18,7 @@ constexpr int kMinTileIds = 1024;
 constexpr int kMaxTileIds = 8192;
 constexpr int kSolveThreads = 512;
 constexpr int kRouteThreads = 256;
-constexpr int kSplitCap = 32;       // split experts the reroute kernel ranks per pass
+constexpr int kSplitCap = 16;       // split experts the reroute kernel ranks per pass
 
 // Problem constants handed to every kernel by value.
 struct Dims {
@@ -107,6 +107,7 @@ struct RerouteParams {
   int32_t* out_token_replica;
   int n_ids, tiles, max_tiles, tile_ids;
   int vec_ok;
+  int solo_items;   // up to this many split items, one warp handles a tile's tail alone
 };
 
 struct SummaryParams {
