@@ -41,6 +41,27 @@ KERNELS_PER_PLAN = 5
 NCU_TRAFFIC_BYTES = {}
 
 
+def rank_plan_base(rank: int, set_index: int) -> int:
+    """First plan index of buffer set `set_index` on `rank`: ranks and sets never share a plan."""
+    return (rank * 64 + set_index) * 100000
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time (all-reduce MAX); the job is as fast as its slowest replica."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, assignments_per_step: int, steps: int, ms_total: float) -> float:
+    """Whole-job assignments per second: every rank plans its own batch each step (weak scaling)."""
+    return world * assignments_per_step * steps / (ms_total * 1e-3)
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -206,7 +227,7 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
                  % (nsets, nsets * 2 * ids_bytes / 1e6))
     sets = []
     for i in range(nsets):
-        ids = wl.make_topk_ids(w, seed=wl.BASE_SEED, plan_base=(rank * 64 + i) * 100000)
+        ids = wl.make_topk_ids(w, seed=wl.BASE_SEED, plan_base=rank_plan_base(rank, i))
         pl = Planner(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
                      w.tokens_per_rank, max_batch=w.batch, token_bytes=w.token_bytes,
                      expert_bytes=w.expert_bytes, c_intra=w.c_intra, c_inter=w.c_inter,
@@ -215,8 +236,6 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
             pl.set_tuning(B.KNOB_TILE_IDS, args.tile_ids)
         if args.hist_mode >= 0:
             pl.set_tuning(B.KNOB_HIST_MODE, args.hist_mode)
-        if args.solo_items >= 0:
-            pl.set_tuning(B.KNOB_SOLO_ITEMS, args.solo_items)
         ids_dev = torch.from_numpy(ids).to(dev)
         sets.append({"pl": pl, "ids_host": ids, "ids": ids_dev,
                      "out": pl.alloc_outputs(w.batch, w.tokens_per_rank)})
@@ -271,12 +290,7 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
             g.replay()
             e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     # warm-up: W eager plans, and every set at least once so each workspace holds its own plan
     with torch.cuda.stream(stream):
@@ -322,7 +336,6 @@ def main():
     ap.add_argument("--impl", default="topoep", choices=["topoep", "reference"])
     ap.add_argument("--tile-ids", type=int, default=0)
     ap.add_argument("--hist-mode", type=int, default=-1)
-    ap.add_argument("--solo-items", type=int, default=-1)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -355,7 +368,7 @@ def main():
     m = measure(w, K, W, rank, world, dev, args)
     sets, nsets, l2_policy, stream = m["sets"], m["nsets"], m["l2_policy"], m["stream"]
     ms_step, ms_total, stage_us = m["ms_step"], m["ms_total"], m["stage_us"]
-    value = world * w.assignments * K / (ms_total * 1e-3)
+    value = job_throughput(world, w.assignments, K, ms_total)
     barrier = m["barrier"]
 
     # ---- end to end through the public call with host buffers
@@ -386,12 +399,8 @@ def main():
             e2e_step()
         e1.record(stream)
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * w.assignments * k_e2e / (ms_e2e * 1e-3)
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    e2e_value = job_throughput(world, w.assignments, k_e2e, ms_e2e)
 
     # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol
     single = None

@@ -118,12 +118,8 @@ enum {
 enum {
   TOPOEP_KNOB_TILE_IDS = 0,     /* ids per histogram / reroute tile: 1024..8192,
                                    power of two                                   */
-  TOPOEP_KNOB_HIST_MODE = 1,    /* 0 = plain shared-memory atomics (default),
+  TOPOEP_KNOB_HIST_MODE = 1     /* 0 = plain shared-memory atomics (default),
                                    1 = warp-aggregated (__match_any_sync) atomics */
-  TOPOEP_KNOB_SOLO_ITEMS = 2    /* reroute: a tile with at most this many assignments
-                                   of split experts is finished by one warp instead
-                                   of the whole CTA (default 0 = never: measured
-                                   slower on B200)                                */
 };
 
 /*

@@ -15,7 +15,7 @@ struct topoep_ctx {
   topoep_cost_params cost;
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
-  int tile_ids, hist_mode, solo_items;
+  int tile_ids, hist_mode;
   int max_tiles;
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
   // workspace
@@ -55,7 +55,7 @@ void carve(topoep_ctx* h) {
   sz[W_REPLICA_MAP] = 4 * B * R * (size_t)std::max(d.N, 1);
   sz[W_COUNTS] = 4 * B * R * R;
   sz[W_ROUTE] = 4 * B * R * E;
-  sz[W_SPLIT_REC] = 4 * B * R * (size_t)split_rec_layout(d.E, d.P).ints;
+  sz[W_SPLIT_REC] = 4 * B * R * (size_t)split_rec_layout(d.E, d.P, h->max_tiles).ints;
   size_t at = 0;
   for (int i = 0; i < W_SLOTS; ++i) { h->off[i] = at; at += align_up(sz[i]); }
   h->ws_bytes = at;
@@ -155,7 +155,6 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->max_batch = max_batch;
   h->tile_ids = 4096;
   h->hist_mode = 0;
-  h->solo_items = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
   h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
@@ -279,7 +278,6 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   rp.tile_ids = h->hist_tile_ids;
   rp.tiles = std::max(1, (rp.n_ids + rp.tile_ids - 1) / rp.tile_ids);
   rp.max_tiles = h->max_tiles;
-  rp.solo_items = h->solo_items;
   rp.vec_ok = (rp.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0) &&
               ((reinterpret_cast<uintptr_t>(token_replica) & 15u) == 0);
   const cudaError_t e = launch_reroute(rp, batch, stream);
@@ -403,10 +401,6 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_HIST_MODE:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->hist_mode = value;
-      return TOPOEP_OK;
-    case TOPOEP_KNOB_SOLO_ITEMS:
-      if (value < 0) return TOPOEP_ERR_ARG;
-      h->solo_items = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

@@ -17,27 +17,28 @@ namespace topoep {
 
 namespace {
 
-// Count one id.  `off` accumulates (unsigned)(e + 1) of the ids that were not counted; it stays 0
-// while every skipped id is the padding value -1.
+// Count one id, branch-free in the default mode: an id outside [0,E) is clamped onto the spare
+// bin cnt[E].  `mx` tracks the largest (unsigned)(e + 1) seen: it exceeds E exactly when some id
+// was neither in range nor the padding value -1.
 template <int MODE>
-__device__ __forceinline__ void count_one(int* cnt, int e, unsigned E, unsigned lane, unsigned& off) {
-  const bool valid = (unsigned)e < E;
+__device__ __forceinline__ void count_one(int* cnt, int e, unsigned E, unsigned lane, unsigned& mx) {
+  mx = max(mx, (unsigned)(e + 1));
   if (MODE == 1) {
+    const bool valid = (unsigned)e < E;
     const unsigned mask = __ballot_sync(0xffffffffu, valid);
     if (valid) {
       const unsigned peers = __match_any_sync(mask, e);
       if ((unsigned)(__ffs(peers) - 1) == lane) atomicAdd(&cnt[e], __popc(peers));
     }
   } else {
-    if (valid) atomicAdd(&cnt[e], 1);
+    atomicAdd(&cnt[min((unsigned)e, E)], 1);
   }
-  if (!valid) off |= (unsigned)(e + 1);
 }
 
 // IPT ids per thread (IPT/4 int4 loads in flight per thread); blockDim.x = tile_ids / IPT.
 template <int MODE, int IPT>
 __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const HistParams p) {
-  extern __shared__ int cnt[];   // [E]
+  extern __shared__ int cnt[];   // [E + 1]: the last bin collects ignored ids
   const int E = p.d.E;
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int nt = blockDim.x, tid = threadIdx.x;
@@ -51,17 +52,17 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
 #pragma unroll
   for (int j = 0; j < IPT / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, p.vec_ok);
 
-  for (int e = tid; e < E; e += nt) cnt[e] = 0;
+  for (int e = tid; e <= E; e += nt) cnt[e] = 0;
   __syncthreads();
-  unsigned off = 0;
+  unsigned mx = 0;
 #pragma unroll
   for (int j = 0; j < IPT / 4; ++j) {
-    count_one<MODE>(cnt, x[j].x, E, lane, off);
-    count_one<MODE>(cnt, x[j].y, E, lane, off);
-    count_one<MODE>(cnt, x[j].z, E, lane, off);
-    count_one<MODE>(cnt, x[j].w, E, lane, off);
+    count_one<MODE>(cnt, x[j].x, E, lane, mx);
+    count_one<MODE>(cnt, x[j].y, E, lane, mx);
+    count_one<MODE>(cnt, x[j].z, E, lane, mx);
+    count_one<MODE>(cnt, x[j].w, E, lane, mx);
   }
-  if (off) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);
+  if (mx > (unsigned)E) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);
   __syncthreads();
   int32_t* out = p.ws.tile_cnt + (row * (size_t)p.max_tiles + tile) * E;
   for (int e = tid; e < E; e += nt) out[e] = cnt[e];
@@ -90,7 +91,7 @@ __global__ void empty_kernel() {}
 
 }  // namespace
 
-size_t hist_smem_bytes(const Dims& d) { return sizeof(int) * (size_t)d.E; }
+size_t hist_smem_bytes(const Dims& d) { return sizeof(int) * ((size_t)d.E + 1); }
 
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream) {
   const dim3 grid(p.tiles, p.d.R, batch);

@@ -21,20 +21,23 @@ namespace topoep {
 
 namespace {
 
-struct RerouteLayout { size_t cnt, base, route, seg, cum, inst, tbase, hdr, work, total; };
+struct RerouteLayout { size_t cnt, base, route, hdr, seg, cum, inst, tbase, work, total; };
 
+// Every region starts on a 16-byte boundary (cp.async destinations).  hdr and seg are adjacent,
+// like in the split record, so that one copy brings both.
 __host__ __device__ inline RerouteLayout reroute_layout(const Dims& d, int tile_ids) {
   const int rows = tile_ids / 128;
+  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
   RerouteLayout o;
   size_t at = 0;
   o.cnt = at;   at += sizeof(uint4) * (size_t)kSplitCap * rows;
   o.base = at;  at += sizeof(int) * (size_t)kSplitCap * rows;
-  o.route = at; at += sizeof(int) * (size_t)d.E;
-  o.seg = at;   at += sizeof(int) * (size_t)(d.E + 1);
-  o.cum = at;   at += sizeof(int) * (size_t)d.P;
-  o.inst = at;  at += sizeof(int) * (size_t)d.P;
+  o.route = at; at += sizeof(int) * pad4(d.E + 1);
+  o.hdr = at;   at += sizeof(int) * 4;                       // n_split, n_list, n_work
+  o.seg = at;   at += sizeof(int) * pad4(d.E + 1 > kSplitCap + 4 ? d.E + 1 : kSplitCap + 4);
+  o.cum = at;   at += sizeof(int) * pad4(d.P);
+  o.inst = at;  at += sizeof(int) * pad4(d.P);
   o.tbase = at; at += sizeof(int) * (size_t)kSplitCap;
-  o.hdr = at;   at += sizeof(int) * 4;
   o.work = at;  at += sizeof(unsigned short) * (size_t)tile_ids;
   o.total = at;
   return o;
@@ -57,13 +60,11 @@ struct SplitCtx {
   uint32_t* status;
 };
 
-// Rank the split items of the tile and patch their outputs.  Run either by one warp (SOLO:
-// tid = lane, nt = 32, warp-level syncs) or by the whole CTA.
-template <bool SOLO>
+// Rank the split items of the tile and patch their outputs (whole CTA).
 __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int nt, int warp,
                                                int nwarps) {
   const int lane = tid & 31, rows = c.rows;
-  auto sync = [] { if (SOLO) __syncwarp(); else __syncthreads(); };
+  auto sync = [] { __syncthreads(); };
   if (c.n_split > kSplitCap || c.n_list > kFastLists) {   // rare: fetch the rest of the record
     for (int i = tid; i <= c.n_split; i += nt) c.seg[i] = c.rec[c.rl.seg + i];
     for (int i = tid; i < c.n_list; i += nt) {
@@ -133,7 +134,12 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
   if (broken) atomicOr(c.status, TOPOEP_FLAG_INTERNAL);
 }
 
-__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, 4) reroute_kernel(const RerouteParams p) {
+// 32 registers per thread: eight 256-thread CTAs per SM; measured faster than 40 or 48 registers
+#ifndef TOPOEP_REROUTE_MIN_CTAS
+#define TOPOEP_REROUTE_MIN_CTAS 4
+#endif
+template <bool VEC>
+__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MIN_CTAS) reroute_kernel(const RerouteParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const Dims d = p.d;
   const int E = d.E, P = d.P;
@@ -158,23 +164,53 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, 4) reroute_kernel
   const int32_t* ids = p.ids + row * (size_t)p.n_ids + begin;
   int32_t* out = p.out_token_replica + row * (size_t)p.n_ids + begin;
 
-  // One round of independent loads: the ids, the route table, the head of the split record and
-  // the tile bases of the first kSplitCap split experts (fetched before n_split is known; the
-  // buffers are always large enough, surplus entries are ignored).
+  // The ids go to registers first: sixteen per thread, all four loads in flight.
   int4 x[kIdsPerThread / 4];
 #pragma unroll
-  for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, p.vec_ok);
-  const SplitRec rl = split_rec_layout(E, P);
+  for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+  const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
   const int32_t* rec = p.ws.split_rec + row * (size_t)rl.ints;
   const int32_t* g_route = p.ws.route + row * E;
   const int32_t* g_tp = p.ws.tile_pref + (row * (size_t)p.max_tiles + tile) * E;
-  const int fast_seg = min(E, kSplitCap) + 1, fast_list = min(P, kFastLists);
-  for (int e = tid; e < E; e += nt) route[e] = g_route[e];
-  for (int i = tid; i < fast_seg; i += nt) seg[i] = rec[rl.seg + i];
-  for (int i = tid; i < fast_list; i += nt) { cum[i] = rec[rl.cum + i]; inst[i] = rec[rl.inst + i]; }
-  if (tid < min(E, kSplitCap)) tbase[tid] = g_tp[tid];
-  if (tid == 0) { hdr[0] = rec[0]; hdr[1] = rec[1]; hdr[2] = 0; }
+  // Tables go global -> shared asynchronously, one 16-byte piece per thread, without passing
+  // through registers (the ids above need those): the route table, the head of the split record
+  // (header + first list segments, first kFastLists quotas and instances) and this tile's prefix
+  // bases of the first kSplitCap split experts.  All of it is fetched before n_split is known;
+  // the buffers are always large enough, surplus entries are ignored.
+  {
+    const int n_route = (E % 4 == 0) ? E / 4 : 0;            // 16-byte pieces of the route table
+    const int n_head = (4 + min(E, kSplitCap) + 1 + 3) / 4;  // header + segment starts
+    const int n_list4 = (min(P, kFastLists) + 3) / 4;
+    const int n_tp = kSplitCap / 4;
+    int i = tid;
+    if (i < n_route) cp_async16(route + 4 * i, g_route + 4 * i);
+    i -= n_route;
+    if (i >= 0 && i < n_head) cp_async16(hdr + 4 * i, rec + 4 * i);
+    i -= n_head;
+    if (i >= 0 && i < n_list4) cp_async16(cum + 4 * i, rec + rl.cum + 4 * i);
+    i -= n_list4;
+    if (i >= 0 && i < n_list4) cp_async16(inst + 4 * i, rec + rl.inst + 4 * i);
+    i -= n_list4;
+    if (i >= 0 && i < n_tp) cp_async16(tbase + 4 * i, rec + rl.tp + tile * kSplitCap + 4 * i);
+    // shapes these fixed assignments do not cover: more pieces than threads, or E % 4 != 0
+    for (int j = tid + nt; j < n_route + n_head + 2 * n_list4 + n_tp; j += nt) {
+      int u = j;
+      if (u < n_route) { cp_async16(route + 4 * u, g_route + 4 * u); continue; }
+      u -= n_route;
+      if (u < n_head) { cp_async16(hdr + 4 * u, rec + 4 * u); continue; }
+      u -= n_head;
+      if (u < n_list4) { cp_async16(cum + 4 * u, rec + rl.cum + 4 * u); continue; }
+      u -= n_list4;
+      if (u < n_list4) { cp_async16(inst + 4 * u, rec + rl.inst + 4 * u); continue; }
+      u -= n_list4;
+      cp_async16(tbase + 4 * u, rec + rl.tp + tile * kSplitCap + 4 * u);
+    }
+    if (E % 4 != 0)
+      for (int e = tid; e < E; e += nt) cp_async4(route + e, g_route + e);
+  }
   for (int i = tid; i < kSplitCap * rows; i += nt) cnt4[i] = make_uint4(0u, 0u, 0u, 0u);
+  if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
+  cp_async_wait_all();           // hdr[2], the work-list length, arrives as the record's zero
   __syncthreads();
 
   // Stream: look up and store.  An ignored id and a split id both store -1 for now; the split
@@ -184,14 +220,16 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, 4) reroute_kernel
 #pragma unroll
   for (int j = 0; j < kIdsPerThread / 4; ++j) {
     const int vec = j * nt + tid;
-    const int t0 = (unsigned)x[j].x < uE ? route[x[j].x] : -1;
-    const int t1 = (unsigned)x[j].y < uE ? route[x[j].y] : -1;
-    const int t2 = (unsigned)x[j].z < uE ? route[x[j].z] : -1;
-    const int t3 = (unsigned)x[j].w < uE ? route[x[j].w] : -1;
-    split_mask |= (t0 <= -2 ? 1u : 0u) << (4 * j) | (t1 <= -2 ? 2u : 0u) << (4 * j) |
-                  (t2 <= -2 ? 4u : 0u) << (4 * j) | (t3 <= -2 ? 8u : 0u) << (4 * j);
+    // branch-free lookups: an id outside [0,E) reads the -1 stored at route[E]
+    const int t0 = route[min((unsigned)x[j].x, uE)];
+    const int t1 = route[min((unsigned)x[j].y, uE)];
+    const int t2 = route[min((unsigned)x[j].z, uE)];
+    const int t3 = route[min((unsigned)x[j].w, uE)];
+    // t <= -2  <=>  t + 1 < 0: collect the sign bits
+    split_mask |= (((unsigned)(t0 + 1) >> 31) | ((unsigned)(t1 + 1) >> 31) << 1 |
+                   ((unsigned)(t2 + 1) >> 31) << 2 | ((unsigned)(t3 + 1) >> 31) << 3) << (4 * j);
     const int4 r = make_int4(max(t0, -1), max(t1, -1), max(t2, -1), max(t3, -1));
-    if (p.vec_ok) {
+    if (VEC) {
       if (4 * vec < count) reinterpret_cast<int4*>(out)[vec] = r;
     } else {
       if (4 * vec + 0 < count) out[4 * vec + 0] = r.x;
@@ -209,15 +247,9 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, 4) reroute_kernel
   const int n_work = hdr[2];
   if (n_work == 0) return;
 
-  // Few items (the usual case): one warp ranks and patches them with warp-level syncs only and the
-  // other warps retire; many items: the whole CTA works on them.
   const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, rec, g_tp, ids, out,
                       rl, rows, hdr[0], hdr[1], n_work, p.ws.status};
-  if (n_work <= p.solo_items) {
-    if (warp == 0) rank_and_patch<true>(c, lane, 32, 0, 1);
-  } else {
-    rank_and_patch<false>(c, tid, nt, warp, nwarps);
-  }
+  rank_and_patch(c, tid, nt, warp, nwarps);
 }
 
 }  // namespace
@@ -227,12 +259,15 @@ size_t reroute_smem_bytes(const Dims& d, int tile_ids) { return reroute_layout(d
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.tiles, p.d.R, batch);
   const dim3 block(p.tile_ids / kIdsPerThread);
-  reroute_kernel<<<grid, block, reroute_smem_bytes(p.d, p.tile_ids), stream>>>(p);
+  if (p.vec_ok) reroute_kernel<true><<<grid, block, reroute_smem_bytes(p.d, p.tile_ids), stream>>>(p);
+  else reroute_kernel<false><<<grid, block, reroute_smem_bytes(p.d, p.tile_ids), stream>>>(p);
   return cudaGetLastError();
 }
 
 cudaError_t configure_reroute(size_t smem) {
-  return cudaFuncSetAttribute(reroute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(reroute_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(reroute_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
 }  // namespace topoep

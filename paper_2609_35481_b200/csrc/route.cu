@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   const int n_split = sidx[E], n_list = seg[E];
 
   // second round of loads: tile counts of the split experts (prefix over tiles below)
-  const SplitRec rl = split_rec_layout(E, P);
+  const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
   int32_t* rec = p.ws.split_rec + row * (size_t)rl.ints;
   int32_t* route = p.ws.route + row * E;
   for (int e = tid; e < E; e += nt) {
@@ -132,7 +132,10 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     route[e] = split ? -2 - sidx[e] : single[e];
     if (split) rec[rl.seg + sidx[e]] = seg[e];
   }
-  if (tid == 0) { rec[0] = n_split; rec[1] = n_list; rec[rl.seg + n_split] = n_list; }
+  if (tid == 0) {   // rec[2] doubles as the reroute kernel's initial (empty) work-list length
+    rec[0] = n_split; rec[1] = n_list; rec[2] = 0; rec[3] = 0;
+    rec[rl.seg + n_split] = n_list;
+  }
 
   // Split lists: position of an instance = number of nonzero instances of e on lower ranks.
   for (int e = tid; e < E; e += nt) {
@@ -172,7 +175,10 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
         const int v = lane < p.tiles ? __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e) : 0;
         int total;
         const int ex = warp_exclusive_scan(v, lane, &total);
-        if (lane < p.tiles) p.ws.tile_pref[trow + (size_t)lane * E + sidx[e]] = ex;
+        if (lane < p.tiles) {
+          p.ws.tile_pref[trow + (size_t)lane * E + sidx[e]] = ex;
+          if (sidx[e] < kSplitCap) rec[rl.tp + lane * kSplitCap + sidx[e]] = ex;
+        }
       }
     } else {
       for (int e = tid; e < E; e += nt) {
@@ -186,7 +192,11 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
           for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
 #pragma unroll
           for (int u = 0; u < 8; ++u)
-            if (t0 + u < p.tiles) { o[(size_t)(t0 + u) * E] = run; run += v[u]; }
+            if (t0 + u < p.tiles) {
+              o[(size_t)(t0 + u) * E] = run;
+              if (sidx[e] < kSplitCap) rec[rl.tp + (t0 + u) * kSplitCap + sidx[e]] = run;
+              run += v[u];
+            }
         }
       }
     }

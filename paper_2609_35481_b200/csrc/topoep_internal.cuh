@@ -50,19 +50,23 @@ struct Workspace {
 };
 
 // Record of one (plan, source) written by the route kernel, read by the reroute kernel:
-//   [0] n_split  [1] n_list  [2..3] unused
+//   [0] n_split  [1] n_list  [2..3] zero
 //   seg  [E+1]  list i of the source's i-th split expert = [seg[i], seg[i+1])
 //   cum  [P]    cumulative quota along each list (instances in ascending rank order)
 //   inst [P]    physical instance ids along each list
+//   tp   [max_tiles][kSplitCap]  tile prefixes of the first kSplitCap split experts, so that the
+//               sixteen tiles of a row fetch theirs from one contiguous KB (the full table
+//               tile_pref is only read when a source has more split experts than that)
 struct SplitRec {
-  int seg, cum, inst, ints;
+  int seg, cum, inst, tp, ints;
 };
-__host__ __device__ inline SplitRec split_rec_layout(int E, int P) {
+__host__ __device__ inline SplitRec split_rec_layout(int E, int P, int max_tiles) {
   SplitRec r;
   r.seg = 4;
   r.cum = r.seg + ((E + 1 + 3) & ~3);
   r.inst = r.cum + ((P + 3) & ~3);
-  r.ints = r.inst + ((P + 3) & ~3);
+  r.tp = r.inst + ((P + 3) & ~3);
+  r.ints = r.tp + max_tiles * kSplitCap;
   return r;
 }
 constexpr int kFastLists = 128;     // list entries the reroute kernel fetches before it knows n_list
@@ -107,7 +111,6 @@ struct RerouteParams {
   int32_t* out_token_replica;
   int n_ids, tiles, max_tiles, tile_ids;
   int vec_ok;
-  int solo_items;   // up to this many split items, one warp handles a tile's tail alone
 };
 
 struct SummaryParams {
@@ -150,6 +153,21 @@ __device__ __forceinline__ int warp_exclusive_scan(int v, int lane, int* total) 
   }
   *total = __shfl_sync(0xffffffffu, inc, 31);
   return inc - v;
+}
+
+// Asynchronous global -> shared copies (no register staging); 16-byte form needs both addresses
+// 16-byte aligned.  cp_async_wait_all() makes the calling thread's copies visible to itself; a
+// __syncthreads() after it makes them visible to the CTA.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
 }
 
 // The 16 ids a thread owns: four groups of four consecutive ids; group j of thread t is vector
