@@ -57,7 +57,8 @@ typedef enum {
   TOPOEP_ERR_ALIGN = -7,       /* an int32 buffer is not 4-byte aligned          */
   TOPOEP_ERR_CUDA = -8,        /* a CUDA runtime call failed (see last error)    */
   TOPOEP_ERR_SMEM = -9,        /* problem does not fit one SM's shared memory    */
-  TOPOEP_ERR_ARG = -10         /* unknown selector / knob / value                */
+  TOPOEP_ERR_ARG = -10,        /* unknown selector / knob / value                */
+  TOPOEP_ERR_SCRATCH = -11     /* problem exceeds the library's built-in scratch  */
 } topoep_status;
 
 /* Device status bits (topoep_read_status). */
@@ -194,6 +195,39 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
  */
 int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank,
                      int batch, int32_t* dev_omega, topoep_stream_t stream);
+
+/*
+ * Histogram for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of topoep_histogram, same result.)
+ *
+ * Who needs it: code that may not call cudaMalloc where it runs -- a plugin
+ * living inside another framework's capture region or stream callback, a
+ * process whose device pool is sized once and then frozen, a test harness that
+ * bans allocation after start-up -- and so cannot supply the workspace that
+ * topoep_histogram keeps its per-tile counts in.  Here that scratch is a fixed
+ * 8 MiB array built into the library (held by every GPU context that loads the
+ * library until the context ends).  No handle, no workspace; the call itself
+ * performs no allocation of any kind.
+ *
+ *   dev_topk_ids  in  [batch][ranks][tokens_per_rank][top_k] int32 (device)
+ *   dev_omega     out [batch][ranks][experts] int32 (device)
+ *   dev_flags     out optional device uint32: TOPOEP_FLAG_BAD_ID if some id was
+ *                     outside [0,experts) and not -1; NULL to ignore
+ * Limit: 256 + 4 * batch * ranks * ceil(tokens_per_rank*top_k / 4096) * experts
+ * bytes must fit in the 8 MiB array, else TOPOEP_ERR_SCRATCH (nothing is
+ * enqueued; there is no fallback).  experts <= 12287.
+ *
+ * The first call on a device looks up the array's device address (once per
+ * device, with that device current); make that first call outside any stream
+ * capture.  All calls share the one array, which keeps the previous call's
+ * contents: the call clears the only word that must start at zero itself, and
+ * two calls that overlap on the GPU (different streams, or graphs replayed
+ * concurrently) race on it -- serialise them.
+ */
+int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, int ranks,
+                            int tokens_per_rank, int top_k, int experts,
+                            int32_t* dev_omega, uint32_t* dev_flags,
+                            topoep_stream_t stream);
 
 /*
  * Solver step alone (paper, "Two-Stage GPU-Native Solver" and the dispatch

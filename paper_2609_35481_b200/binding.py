@@ -20,7 +20,7 @@ T_OMEGA, T_Q, T_RANK_LOAD, T_REFINE_ITERS = 0, 1, 2, 3
 KNOB_TILE_IDS, KNOB_HIST_MODE = 0, 1
 
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
-           "topoep_plan", "topoep_histogram", "topoep_solve", "topoep_reroute", "topoep_summary", "topoep_read_status",
+           "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_summary", "topoep_read_status",
            "topoep_debug_tensor", "topoep_set_tuning", "topoep_get_layout",
            "topoep_launch_floor", "topoep_strerror")
 
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.topoep_plan.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, vp, vp]
         L.topoep_histogram.restype = ci
         L.topoep_histogram.argtypes = [vp, vp, ci, ci, vp, vp]
+        L.topoep_histogram_static.restype = ci
+        L.topoep_histogram_static.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp]
         L.topoep_solve.restype = ci
         L.topoep_solve.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp]
         L.topoep_reroute.restype = ci
@@ -140,6 +142,16 @@ def topoep_plan(h, dev_topk_ids, tokens_per_rank, batch, dev_replica_map, dev_to
 def topoep_histogram(h, dev_topk_ids, tokens_per_rank, batch, dev_omega, stream=0) -> int:
     return lib().topoep_histogram(h, _ptr(dev_topk_ids), tokens_per_rank, batch, _ptr(dev_omega),
                                   stream or None)
+
+
+def topoep_histogram_static(dev_topk_ids, batch, ranks, tokens_per_rank, top_k, experts, dev_omega,
+                            dev_flags=None, stream=0) -> int:
+    """Histogram without handle or workspace, for callers that may not allocate device memory:
+    the per-tile scratch is an 8 MiB array inside the library.  Returns -11 when the problem does
+    not fit that array.  Make the first call on a device outside stream capture; calls that
+    overlap on the GPU race on the shared array."""
+    return lib().topoep_histogram_static(_ptr(dev_topk_ids), batch, ranks, tokens_per_rank, top_k,
+                                         experts, _ptr(dev_omega), _ptr(dev_flags), stream or None)
 
 
 def topoep_solve(h, dev_omega, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,

@@ -433,6 +433,7 @@ const char* topoep_strerror(int status) {
     case TOPOEP_ERR_CUDA: return "a CUDA runtime call failed";
     case TOPOEP_ERR_SMEM: return "problem does not fit one SM's shared memory";
     case TOPOEP_ERR_ARG: return "unknown selector, knob or value";
+    case TOPOEP_ERR_SCRATCH: return "problem exceeds the 8 MiB scratch array built into the library";
     default: return "unknown status";
   }
 }
