@@ -36,9 +36,19 @@ import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 KERNELS_PER_PLAN = 5
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/), keyed by
-# (workload, kernel); None until a capture of that pair exists.
-NCU_TRAFFIC_BYTES = {}
+# DRAM read+write bytes per PLAN of the DeepSeek-V3-shaped layer from the committed ncu capture of a
+# 16-plan call (profiles/reroute_kernel_dsv3_batch16.md, profiles/hist_kernel_dsv3_batch16.md);
+# a launch's traffic is this times its plans (every CTA touches only its own tile and tables).
+NCU_TRAFFIC_PER_PLAN = {
+    "reroute": (136071936 + 86523648) / 16,
+    "hist": (134233600 + 6924800) / 16,
+}
+
+
+def ncu_traffic(w, kernel):
+    if w.name in ("dsv3", "dsv3_batched") and kernel in NCU_TRAFFIC_PER_PLAN:
+        return int(NCU_TRAFFIC_PER_PLAN[kernel] * w.batch)
+    return None
 
 
 def rank_plan_base(rank: int, set_index: int) -> int:
@@ -444,7 +454,7 @@ def main():
                                            "reroute": "reroute_kernel"}[dominant],
                 "achieved": round(achieved, 2), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "peak_source": "of " + peak_kind,
-                "traffic": NCU_TRAFFIC_BYTES.get((w.name, dominant)),
+                "traffic": ncu_traffic(w, dominant),
                 "algorithmic_bytes_per_launch": dom_bytes,
                 "plan_bytes": 12 * A,
                 "plan_frac": round(12 * A / (ms_step * 1e-3) / 1e9 / peak, 4),

@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   const Dims d = p.d;
   const int E = d.E, P = d.P;
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
-  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+  const int tid = threadIdx.x, nt = blockDim.x, warp = tid >> 5, nwarps = nt >> 5;
   const int rows = 4 * nwarps;   // 128-id rows of the tile, in flat order
   const RerouteLayout lay = reroute_layout(d, p.tile_ids);
   uint4* cnt4 = reinterpret_cast<uint4*>(smem + lay.cnt);      // [kSplitCap][rows]
