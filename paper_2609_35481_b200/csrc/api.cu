@@ -14,6 +14,7 @@ struct topoep_ctx {
   int max_tokens, max_batch;
   topoep_cost_params cost;
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
+  bool omega_smem;   // solver keeps a plan's routing matrix in shared memory
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode;
   int max_tiles;
@@ -159,7 +160,9 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->have_ws = false;
   h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
   h->last_cuda = cudaSuccess;
-  if (solve_smem_bytes(d) > 227 * 1024 || reroute_smem_bytes(d, kMaxTileIds) > 227 * 1024 ||
+  // the solver stages the routing matrix in shared memory when that leaves room for two CTAs per SM
+  h->omega_smem = solve_smem_bytes(d, true) <= 100 * 1024;
+  if (solve_smem_bytes(d, h->omega_smem) > 227 * 1024 || reroute_smem_bytes(d, kMaxTileIds) > 227 * 1024 ||
       route_smem_bytes(d) > 227 * 1024 ||
       hist_smem_bytes(d) > 48 * 1024) {
     delete h;
@@ -205,7 +208,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_inst_expert), h->main_inst_expert.data(),
                       4 * h->main_inst_expert.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
   if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
-  if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
+  if ((e = configure_solve(solve_smem_bytes(h->d, h->omega_smem))) != cudaSuccess) goto fail;
   if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_reroute(reroute_smem_bytes(h->d, kMaxTileIds))) != cudaSuccess) goto fail;
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) goto fail;
@@ -238,6 +241,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.d = h->d;
   sp.ws = h->ws;
   sp.omega = omega ? omega : h->ws.omega;
+  sp.omega_smem = h->omega_smem ? 1 : 0;
   sp.token_bytes = h->cost.token_bytes;
   sp.expert_bytes = h->cost.expert_bytes;
   sp.max_iters = h->max_iters;

@@ -11,6 +11,11 @@
 // runs the loop, every selection is a warp reduction over a totally ordered key.
 // What needs every domain's result (send offsets, per-source routing tables) is left to the
 // route kernel that follows.
+//
+// The kernel is latency-bound (KBs of state, an L2 round trip costs ~0.7 us on B200), so all
+// global inputs -- the routing matrix when it fits in shared memory, the main-rank tables --
+// arrive in ONE round of cp.async copies before the first barrier, and the phases after it work
+// from shared memory only.
 #include <limits.h>
 
 #include "topoep_internal.cuh"
@@ -19,16 +24,23 @@ namespace topoep {
 
 namespace {
 
+constexpr int kRankCap = 128;   // stage 1 ranks up to this many candidates of a domain all-pairs
+
 struct SolveLayout {
-  size_t hostmask, D, qd, col_expert, col_cr, U, L, used, cnt, hostcol, total;
+  size_t om, cand, D, qd, mrank, host_lo, host_hi, col_expert, col_cr, U, L, used, cnt, hostcol, total;
 };
 
-__host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
+__host__ __device__ inline SolveLayout solve_layout(const Dims& d, bool omega_smem) {
+  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
   SolveLayout o;
   size_t at = 0;
-  o.hostmask = at;   at += sizeof(unsigned long long) * (size_t)d.E;
+  o.om = at;         at += sizeof(int) * (omega_smem ? pad4((size_t)d.R * d.E) : 0);
+  o.cand = at;       at += sizeof(unsigned long long) * (size_t)kRankCap * (kSolveThreads / 32);
+  o.mrank = at;      at += sizeof(int) * pad4(d.E);
   o.D = at;          at += sizeof(int) * (size_t)d.M * d.E;
   o.qd = at;         at += sizeof(int) * (size_t)d.R * d.qstride;
+  o.host_lo = at;    at += sizeof(int) * (size_t)d.E;
+  o.host_hi = at;    at += sizeof(int) * (size_t)d.E;
   o.col_expert = at; at += sizeof(int) * (size_t)d.C;
   o.col_cr = at;     at += sizeof(int) * (size_t)d.C;
   o.U = at;          at += sizeof(int) * (size_t)d.C;
@@ -48,11 +60,15 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   const int dm = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
   const unsigned full = 0xffffffffu;
+  const bool om_smem = p.omega_smem != 0;
 
-  const SolveLayout lay = solve_layout(d);
-  unsigned long long* hostmask = reinterpret_cast<unsigned long long*>(smem + lay.hostmask);
+  const SolveLayout lay = solve_layout(d, om_smem);
+  int* om_s = reinterpret_cast<int*>(smem + lay.om);
+  int* mrank = reinterpret_cast<int*>(smem + lay.mrank);
   int* D = reinterpret_cast<int*>(smem + lay.D);
   int* qd = reinterpret_cast<int*>(smem + lay.qd);
+  unsigned* host_lo = reinterpret_cast<unsigned*>(smem + lay.host_lo);   // hosting domains 0..31
+  unsigned* host_hi = reinterpret_cast<unsigned*>(smem + lay.host_hi);   // hosting domains 32..63
   int* col_expert = reinterpret_cast<int*>(smem + lay.col_expert);
   int* col_cr = reinterpret_cast<int*>(smem + lay.col_cr);
   int* U = reinterpret_cast<int*>(smem + lay.U);
@@ -62,84 +78,152 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   short* hostcol = reinterpret_cast<short*>(smem + lay.hostcol);
 
   const int32_t* om = p.omega + (size_t)b * R * E;
-  const int32_t* main_rank = p.ws.main_rank;
 
-  // ---- tables of the own domain; candidate demand of every domain -------------------------
+  // ---- one round of asynchronous copies: routing matrix, main ranks, the domain's main experts
+  if (om_smem) {
+    const int n = R * E;
+    if ((n & 3) == 0 && (reinterpret_cast<uintptr_t>(om) & 15u) == 0) {
+      for (int i = tid; i < n / 4; i += nt) cp_async16(om_s + 4 * i, om + 4 * i);
+    } else {
+      for (int i = tid; i < n; i += nt) cp_async4(om_s + i, om + i);
+    }
+  }
+  if ((E & 3) == 0) {
+    for (int i = tid; i < E / 4; i += nt) cp_async16(mrank + 4 * i, p.ws.main_rank + 4 * i);
+  } else {
+    for (int i = tid; i < E; i += nt) cp_async4(mrank + i, p.ws.main_rank + i);
+  }
+  for (int i = tid; i < G * e_loc; i += nt) {
+    const int g = i / e_loc, l = i - g * e_loc;
+    cp_async4(col_expert + g * s_phys + l, p.ws.main_inst_expert + (size_t)(dm * G + g) * e_loc + l);
+  }
+  for (int i = tid; i < G * N; i += nt) col_expert[(i / N) * s_phys + e_loc + i % N] = -1;
   for (int i = tid; i < G * E; i += nt) hostcol[i] = -1;
-  for (int c = tid; c < C; c += nt) {
-    const int g = c / s_phys, l = c - g * s_phys;
-    col_expert[c] = l < e_loc ? p.ws.main_inst_expert[(size_t)(dm * G + g) * e_loc + l] : -1;
-    col_cr[c] = p.cost_rank_intra;   // a main instance of this domain: parameters come from inside
-    U[c] = 0;
-  }
+  for (int c = tid; c < C; c += nt) { col_cr[c] = p.cost_rank_intra; U[c] = 0; }
   if (tid < G) used[tid] = 0;
-  for (int e = tid; e < E; e += nt) hostmask[e] = 1ull << (main_rank[e] / G);
-  // D[dd][e] = sum over the G source ranks of domain dd, kept only where e is a stage-1 candidate
-  // of dd (main outside dd and b > 0), else 0.  Loads are issued eight at a time.
-  for (int idx0 = tid; idx0 < M * E; idx0 += 4 * nt) {
-    int sum[4] = {0, 0, 0, 0};
-    for (int g0 = 0; g0 < G; g0 += 8) {
-      int v[4][8];
-#pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        const int idx = idx0 + a * nt;
-        const int dd = idx / E, e = idx - dd * E;
-        const int32_t* col = om + (size_t)dd * G * E + e;
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-          v[a][u] = (idx < M * E && g0 + u < G) ? __ldg(col + (size_t)(g0 + u) * E) : 0;
-      }
-#pragma unroll
-      for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int u = 0; u < 8; ++u) sum[a] += v[a][u];
-    }
-#pragma unroll
-    for (int a = 0; a < 4; ++a) {
-      const int idx = idx0 + a * nt;
-      if (idx >= M * E) break;
-      const int dd = idx / E, e = idx - dd * E;
-      const bool cand = dd != main_rank[e] / G &&
-                        2 * (long long)sum[a] * p.token_bytes - p.expert_bytes > 0;
-      D[idx] = cand ? sum[a] : 0;
-    }
-  }
+  cp_async_wait_all();
   __syncthreads();
+
+  // ---- hosting masks from the main ranks; candidate demand of every domain -------------------
+  for (int e = tid; e < E; e += nt) {
+    const int md = mrank[e] / G;
+    host_lo[e] = md < 32 ? 1u << md : 0u;
+    host_hi[e] = md < 32 ? 0u : 1u << (md - 32);
+  }
   for (int c = tid; c < C; c += nt) {
     const int e = col_expert[c];
     if (e >= 0) hostcol[(c / s_phys) * E + e] = (short)c;
   }
+  // D[dd][e] = sum over the G source ranks of domain dd, kept only where e is a stage-1 candidate
+  // of dd (main outside dd and b > 0), else 0.
+  if (om_smem) {
+    const int chunks = (E + 31) / 32;
+    for (int t = warp; t < M * chunks; t += nwarps) {   // a warp-task = (domain, 32 experts)
+      const int dd = t / chunks, e = (t - dd * chunks) * 32 + lane;
+      if (e >= E) continue;
+      const int* col = om_s + dd * G * E + e;
+      int sum = 0;
+      for (int g = 0; g < G; ++g) sum += col[g * E];
+      const bool cand = dd != mrank[e] / G && 2 * (long long)sum * p.token_bytes - p.expert_bytes > 0;
+      D[dd * E + e] = cand ? sum : 0;
+    }
+  } else {
+    for (int idx0 = tid; idx0 < M * E; idx0 += 4 * nt) {   // 32 loads in flight per thread
+      int sum[4] = {0, 0, 0, 0};
+      for (int g0 = 0; g0 < G; g0 += 8) {
+        int v[4][8];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          const int idx = idx0 + a * nt;
+          const int dd = idx / E, e = idx - dd * E;
+          const int32_t* col = om + (size_t)dd * G * E + e;
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            v[a][u] = (idx < M * E && g0 + u < G) ? __ldg(col + (size_t)(g0 + u) * E) : 0;
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int u = 0; u < 8; ++u) sum[a] += v[a][u];
+      }
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int idx = idx0 + a * nt;
+        if (idx >= M * E) break;
+        const int dd = idx / E, e = idx - dd * E;
+        const bool cand = dd != mrank[e] / G &&
+                          2 * (long long)sum[a] * p.token_bytes - p.expert_bytes > 0;
+        D[idx] = cand ? sum[a] : 0;
+      }
+    }
+  }
+  __syncthreads();
 
   // ---- inter-node placement, every domain, one warp each ------------------------------------
   // Candidates in descending (b, then ascending e) order == descending (D, ascending e) for a
   // uniform ||W|| and S_tok; the i-th goes to rank i mod G, slot i / G (fewest used slots first,
   // ties to the lower rank).
   if (M > 1 && N > 0) {
+    const int slots = G * N;
     for (int dd = warp; dd < M; dd += nwarps) {
       int* Dd = D + dd * E;
-      for (int i = 0; i < G * N; ++i) {
-        int bestD = 0;
-        unsigned bestK = 0;   // ~e: larger means smaller e
-        for (int e = lane; e < E; e += 32) {
-          const int v = Dd[e];
-          if (v > bestD) { bestD = v; bestK = ~(unsigned)e; }   // ascending e: first hit is smallest
-        }
-        const int maxD = __reduce_max_sync(full, bestD);
-        if (maxD <= 0) break;
-        const unsigned k = __reduce_max_sync(full, bestD == maxD ? bestK : 0u);
-        const int e = (int)~k;
-        if (lane == 0) {
-          Dd[e] = 0;   // taken
-          atomicOr(&hostmask[e], 1ull << dd);
-          if (dd == dm) {
-            const int g = i % G, j = i / G, c = g * s_phys + e_loc + j;
-            col_expert[c] = e;
-            col_cr[c] = p.cost_rank_inter;   // its main lies in another domain
-            hostcol[g * E + e] = (short)c;
-            used[g] = j + 1;
+      // compact the candidates (D > 0) of this domain into cand[]: key = (D, -e)
+      unsigned long long* cand = reinterpret_cast<unsigned long long*>(smem + lay.cand) +
+                                 (size_t)warp * kRankCap;
+      int n_c = 0;
+      for (int e0 = 0; e0 < E; e0 += 32) {
+        const int e = e0 + lane;
+        const int v = e < E ? Dd[e] : 0;
+        const unsigned m = __ballot_sync(full, v > 0);
+        const int at = n_c + __popc(m & lanemask_lt());
+        if (v > 0 && at < kRankCap)
+          cand[at] = ((unsigned long long)(unsigned)v << 32) | (unsigned)~(unsigned)e;
+        n_c += __popc(m);
+      }
+      __syncwarp();
+      if (n_c <= kRankCap) {
+        // few candidates: every candidate counts the keys above its own; rank < slots wins
+        for (int c0 = 0; c0 < n_c; c0 += 32) {
+          const int c = c0 + lane;
+          const unsigned long long mine = c < n_c ? cand[c] : 0ull;
+          int rank = 0;
+          for (int o = 0; o < n_c; ++o) rank += cand[o] > mine ? 1 : 0;
+          if (c < n_c && rank < slots) {
+            const int e = (int)~(unsigned)mine;
+            if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
+            if (dd == dm) {
+              const int g = rank % G, j = rank / G, col = g * s_phys + e_loc + j;
+              col_expert[col] = e;
+              col_cr[col] = p.cost_rank_inter;   // its main lies in another domain
+              hostcol[g * E + e] = (short)col;
+              atomicMax(&used[g], j + 1);
+            }
           }
         }
-        __syncwarp();
+      } else {
+        // many candidates: pick the maximum slot by slot
+        for (int i = 0; i < slots; ++i) {
+          int bestD = 0, bestE = INT_MAX;
+          for (int e = lane; e < E; e += 32) {
+            const int x = Dd[e];
+            if (x > bestD) { bestD = x; bestE = e; }   // ascending e: first hit is smallest
+          }
+          const int maxD = __reduce_max_sync(full, bestD);
+          if (maxD <= 0) break;
+          const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
+          if (lane == 0) {
+            Dd[e] = 0;   // taken
+            if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
+            if (dd == dm) {
+              const int g = i % G, j = i / G, col = g * s_phys + e_loc + j;
+              col_expert[col] = e;
+              col_cr[col] = p.cost_rank_inter;
+              hostcol[g * E + e] = (short)col;
+              used[g] = j + 1;
+            }
+          }
+          __syncwarp();
+        }
       }
     }
   }
@@ -149,48 +233,31 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   // After stage 1 an expert has at most one instance per domain.  A source keeps everything in
   // its own domain when an instance is there; otherwise it splits over all instances (ascending
   // rank == ascending hosting domain), remainder to `rem` instances starting at (s+e) mod n.
-  for (int idx0 = tid; idx0 < R * C; idx0 += 4 * nt) {
-    int w[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {   // the four omega loads go out before any is used
-      const int idx = idx0 + u * nt;
-      w[u] = 0;
-      if (idx < R * C) {
-        const int s = idx / C, e = col_expert[idx - s * C];
-        if (e >= 0) w[u] = __ldg(om + (size_t)s * E + e);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int idx = idx0 + u * nt;
-      if (idx >= R * C) break;
-      const int s = idx / C, c = idx - s * C;
+  // Warps walk the sources, lanes the columns; U accumulates by shared atomics (sums commute).
+  for (int s = warp; s < R; s += nwarps) {
+    const int ds = s / G;
+    for (int c = lane; c < C; c += 32) {
       const int e = col_expert[c];
       int v = 0;
       if (e >= 0) {
-        const int ds = s / G;
+        const int w = om_smem ? om_s[s * E + e] : __ldg(om + (size_t)s * E + e);
         if (ds == dm) {
-          v = w[u];
+          v = w;
         } else {
-          const unsigned long long hm = hostmask[e];
+          const unsigned long long hm = ((unsigned long long)host_hi[e] << 32) | host_lo[e];
           if (!((hm >> ds) & 1ull)) {
             const int n = __popcll(hm);
             const int i = __popcll(hm & ((1ull << dm) - 1ull));
-            const int base = w[u] / n, rem = w[u] - base * n;
+            const int base = w / n, rem = w - base * n;
             int sh = i - (s + e) % n;
             if (sh < 0) sh += n;
             v = base + (sh < rem ? 1 : 0);
           }
         }
+        if (v) atomicAdd(&U[c], v);
       }
       qd[s * QS + c] = v;
     }
-  }
-  __syncthreads();
-  for (int c = tid; c < C; c += nt) {
-    int sum = 0;
-    for (int s = 0; s < R; ++s) sum += qd[s * QS + c];
-    U[c] = sum;
   }
   __syncthreads();
   if (tid < G) {
@@ -204,28 +271,35 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   if (warp == 0) {
     int it = 0;
     const int chunk = (R + 31) / 32;
+    // lane -> (target rank gt, start slot k0): lanes gt, gt+G, ... share a target and stride the
+    // instance slots of the busiest rank
+    const int gt = lane % G, k0 = lane / G, kstep = max(32 / G, 1);
+    const bool lane_on = lane < G * kstep;
     for (;;) {
       const int Lg = lane < G ? L[lane] : -1;
       const int Lb = __reduce_max_sync(full, Lg);
       const int gb = __ffs(__ballot_sync(full, Lg == Lb)) - 1;   // busiest, lowest id on ties
       int bd = 0, bl = INT_MAX;
       unsigned bk = 0xffffffffu;
-      for (int idx = lane; idx < s_phys * G; idx += 32) {
-        const int l = idx / G, gt = idx - l * G;
-        const int cb = gb * s_phys + l;
-        const int e = col_expert[cb];
-        if (gt == gb || e < 0) continue;
-        const int u = U[cb];
-        if (u <= 0) continue;
-        const int hc = hostcol[gt * E + e];
-        if (hc < 0 && used[gt] >= N) continue;              // neither hosts e nor has a free slot
+      if (lane_on && gt != gb) {
         const int Lt = L[gt];
-        const int delta = min(u, (Lb - Lt) >> 1);           // half-gap bound
-        if (delta < p.min_delta) continue;
-        const unsigned cr = hc >= 0 ? 0u : (unsigned)col_cr[cb];
-        const unsigned key = (cr << 28) | ((unsigned)e << 5) | (unsigned)gt;
-        if (delta > bd || (delta == bd && (Lt < bl || (Lt == bl && key < bk)))) {
-          bd = delta; bl = Lt; bk = key;
+        const int half = (Lb - Lt) >> 1;                         // half-gap bound
+        const bool has_slot = used[gt] < N;
+        if (half >= p.min_delta) {
+          for (int l = k0; l < s_phys; l += kstep) {
+            const int cb = gb * s_phys + l;
+            const int e = col_expert[cb];
+            const int u = U[cb];
+            if (e < 0 || u <= 0) continue;
+            const int hc = hostcol[gt * E + e];
+            if (hc < 0 && !has_slot) continue;                   // neither hosts e nor has a slot
+            const int delta = min(u, half);
+            if (delta < p.min_delta) continue;
+            const unsigned cr = hc >= 0 ? 0u : (unsigned)col_cr[cb];
+            const unsigned key = (cr << 28) | ((unsigned)e << 5) | (unsigned)gt;
+            if (delta > bd || (delta == bd && key < bk)) { bd = delta; bk = key; }
+          }
+          bl = Lt;
         }
       }
       const int md = __reduce_max_sync(full, bd);
@@ -236,22 +310,22 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         if (lane == 0) atomicOr(p.ws.status, TOPOEP_FLAG_REFINE_CAP);
         break;
       }
-      const int e = (int)((mk >> 5) & 0x7fffffu), gt = (int)(mk & 31u);
+      const int e = (int)((mk >> 5) & 0x7fffffu), wt = (int)(mk & 31u);
       const int cb = hostcol[gb * E + e];
-      int ct = hostcol[gt * E + e];
+      int ct = hostcol[wt * E + e];
       if (ct < 0) {   // create the replica in the target's next free slot
-        ct = gt * s_phys + e_loc + used[gt];
+        ct = wt * s_phys + e_loc + used[wt];
         __syncwarp();
         if (lane == 0) {
           col_expert[ct] = e;
           col_cr[ct] = col_cr[cb];
-          hostcol[gt * E + e] = (short)ct;
-          used[gt] += 1;
+          hostcol[wt * E + e] = (short)ct;
+          used[wt] += 1;
         }
       }
       // Move md units of q from column cb to ct; sources in the order: the target rank itself,
       // then the others ascending, the busiest rank last.
-      const int rb = dm * G + gb, rt = dm * G + gt;
+      const int rb = dm * G + gb, rt = dm * G + wt;
       const int lo = min(rb, rt), hi = max(rb, rt);
       const int i0 = min(R, lane * chunk), i1 = min(R, i0 + chunk);
       int sum = 0;
@@ -260,13 +334,8 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         if (i != 0 && i != R - 1) { if (s >= lo) ++s; if (s >= hi) ++s; }
         sum += qd[s * QS + cb];
       }
-      int pre = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(full, pre, o);
-        if (lane >= o) pre += t;
-      }
-      pre -= sum;
+      int total;
+      int pre = warp_exclusive_scan(sum, lane, &total);
       for (int i = i0; i < i1; ++i) {
         int s = i == 0 ? rt : (i == R - 1 ? rb : i - 1);
         if (i != 0 && i != R - 1) { if (s >= lo) ++s; if (s >= hi) ++s; }
@@ -280,7 +349,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       }
       if (lane == 0) {
         U[cb] -= md; U[ct] += md;
-        L[gb] -= md; L[gt] += md;
+        L[gb] -= md; L[wt] += md;
       }
       __syncwarp();
       ++it;
@@ -297,42 +366,46 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     p.ws.replica_map[at] = e;
     if (p.out_replica_map) p.out_replica_map[at] = e;
   }
-  for (int idx = tid; idx < R * C; idx += nt) {
-    const int s = idx / C, c = idx - s * C;
-    p.ws.q[((size_t)b * R + s) * d.P + (size_t)dm * C + c] = qd[s * QS + c];
-  }
   for (int c = tid; c < C; c += nt) {
     const size_t at = (size_t)b * d.P + (size_t)dm * C + c;
     p.ws.inst_counts[at] = U[c];
     if (p.out_inst_counts) p.out_inst_counts[at] = U[c];
   }
   if (tid < G) p.ws.rank_load[(size_t)b * R + dm * G + tid] = L[tid];
-  for (int idx = tid; idx < R * G; idx += nt) {
-    const int s = idx / G, g = idx - s * G;
-    int sum = 0;
-    for (int l = 0; l < s_phys; ++l) sum += qd[s * QS + g * s_phys + l];
-    cnt[idx] = sum;
-    const size_t at = ((size_t)b * R + s) * R + dm * G + g;
-    p.ws.counts[at] = sum;
-    p.out_counts[at] = sum;
+  for (int s = warp; s < R; s += nwarps) {
+    int32_t* qrow = p.ws.q + ((size_t)b * R + s) * d.P + (size_t)dm * C;
+    for (int c = lane; c < C; c += 32) qrow[c] = qd[s * QS + c];
+    if (lane < G) {   // counts[s][r] for the ranks r of this domain
+      int sum = 0;
+      for (int l = 0; l < s_phys; ++l) sum += qd[s * QS + lane * s_phys + l];
+      cnt[s * G + lane] = sum;
+      const size_t at = ((size_t)b * R + s) * R + dm * G + lane;
+      p.ws.counts[at] = sum;
+      p.out_counts[at] = sum;
+    }
   }
   __syncthreads();
-  if (tid < G) {   // receive offsets of rank r: exclusive scan over the sources
-    int32_t* recv = p.out_offsets + (((size_t)b * 2 + 1) * R + dm * G + tid) * (R + 1);
-    int run = 0;
-    for (int s = 0; s < R; ++s) { recv[s] = run; run += cnt[s * G + tid]; }
-    recv[R] = run;
+  // receive offsets of rank r: exclusive scan over the sources, one warp per rank
+  for (int g = warp; g < G; g += nwarps) {
+    int32_t* recv = p.out_offsets + (((size_t)b * 2 + 1) * R + dm * G + g) * (R + 1);
+    const int ch = (R + 31) / 32;
+    const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
+    int sum = 0;
+    for (int s = i0; s < i1; ++s) sum += cnt[s * G + g];
+    int total;
+    int pre = warp_exclusive_scan(sum, lane, &total);
+    for (int s = i0; s < i1; ++s) { recv[s] = pre; pre += cnt[s * G + g]; }
+    if (lane == 0) recv[R] = total;
   }
-
 }
 
 }  // namespace
 
-size_t solve_smem_bytes(const Dims& d) { return solve_layout(d).total; }
+size_t solve_smem_bytes(const Dims& d, bool omega_smem) { return solve_layout(d, omega_smem).total; }
 
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.d.M, batch);
-  solve_kernel<<<grid, kSolveThreads, solve_smem_bytes(p.d), stream>>>(p);
+  solve_kernel<<<grid, kSolveThreads, solve_smem_bytes(p.d, p.omega_smem != 0), stream>>>(p);
   return cudaGetLastError();
 }
 

@@ -88,6 +88,7 @@ struct SolveParams {
   Dims d;
   Workspace ws;
   const int32_t* omega;       // [B][R][E] routing matrix to plan from
+  int omega_smem;             // the routing matrix of one plan fits in shared memory
   int64_t token_bytes, expert_bytes;
   int max_iters, min_delta;
   int cost_rank_intra, cost_rank_inter;   // dense ranks of {0, c_intra*W, c_inter*W}
@@ -122,7 +123,7 @@ struct SummaryParams {
 };
 
 size_t hist_smem_bytes(const Dims& d);
-size_t solve_smem_bytes(const Dims& d);
+size_t solve_smem_bytes(const Dims& d, bool omega_smem);
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 

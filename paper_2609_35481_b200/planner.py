@@ -62,7 +62,10 @@ class Planner:
             self.handle = None
 
     def __del__(self):
-        self.close()
+        try:
+            self.close()
+        except Exception:   # interpreter shutdown: the binding module may already be gone
+            pass
 
     def alloc_outputs(self, batch: int, tokens_per_rank: int) -> PlanOutputs:
         i32 = dict(dtype=torch.int32, device=self.device)
