@@ -14,7 +14,6 @@ struct topoep_ctx {
   int max_tokens, max_batch;
   topoep_cost_params cost;
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
-  bool omega_smem;   // solver keeps a plan's routing matrix in shared memory
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode;
   int max_tiles;
@@ -33,7 +32,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 enum WsSlot {
-  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_STATUS, W_OMEGA, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
+  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
   W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC, W_SLOTS
 };
 static_assert(W_SLOTS <= 24, "offset table size");
@@ -47,6 +46,8 @@ void carve(topoep_ctx* h) {
   sz[W_MAIN_INST] = 4 * R * (size_t)std::max(d.e_loc, 1);
   sz[W_STATUS] = 4;
   sz[W_OMEGA] = 4 * B * R * E;
+  sz[W_OMEGA_M] = 4 * B * R * (size_t)std::max(d.e_loc, 1) * R;
+  sz[W_DEMAND] = 4 * B * (size_t)d.M * E;
   sz[W_TILE_CNT] = 4 * B * R * (size_t)h->max_tiles * E;
   sz[W_TILE_PREF] = sz[W_TILE_CNT];
   sz[W_Q] = 4 * B * R * P;
@@ -87,6 +88,20 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   p.max_tiles = h->max_tiles;
   p.vec_ok = (p.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0);
   return p;
+}
+
+OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, int tiles) {
+  OmegaParams op;
+  op.d = h->d;
+  op.ws = h->ws;
+  op.src_omega = src;
+  op.out_omega = out_omega;
+  op.tiles = tiles;
+  op.max_tiles = h->max_tiles;
+  int gpad = 1;
+  while (gpad < h->d.G) gpad <<= 1;
+  op.epw = 32 / gpad;
+  return op;
 }
 
 }  // namespace
@@ -160,9 +175,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->have_ws = false;
   h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
   h->last_cuda = cudaSuccess;
-  // the solver stages the routing matrix in shared memory when that leaves room for two CTAs per SM
-  h->omega_smem = solve_smem_bytes(d, true) <= 100 * 1024;
-  if (solve_smem_bytes(d, h->omega_smem) > 227 * 1024 || reroute_smem_bytes(d, kMaxTileIds) > 227 * 1024 ||
+  if (solve_smem_bytes(d) > 227 * 1024 || reroute_smem_bytes(d, kMaxTileIds) > 227 * 1024 ||
       route_smem_bytes(d) > 227 * 1024 ||
       hist_smem_bytes(d) > 48 * 1024) {
     delete h;
@@ -188,6 +201,8 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.main_inst_expert = at<int32_t>(dev_ptr, h->off[W_MAIN_INST]);
   w.status = at<uint32_t>(dev_ptr, h->off[W_STATUS]);
   w.omega = at<int32_t>(dev_ptr, h->off[W_OMEGA]);
+  w.omega_m = at<int32_t>(dev_ptr, h->off[W_OMEGA_M]);
+  w.demand = at<int32_t>(dev_ptr, h->off[W_DEMAND]);
   w.tile_cnt = at<int32_t>(dev_ptr, h->off[W_TILE_CNT]);
   w.tile_pref = at<int32_t>(dev_ptr, h->off[W_TILE_PREF]);
   w.q = at<int32_t>(dev_ptr, h->off[W_Q]);
@@ -208,7 +223,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_inst_expert), h->main_inst_expert.data(),
                       4 * h->main_inst_expert.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
   if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
-  if ((e = configure_solve(solve_smem_bytes(h->d, h->omega_smem))) != cudaSuccess) goto fail;
+  if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_reroute(reroute_smem_bytes(h->d, kMaxTileIds))) != cudaSuccess) goto fail;
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) goto fail;
@@ -228,7 +243,7 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
   h->hist_tokens = T;
   h->hist_batch = batch;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
-  if (e == cudaSuccess) e = launch_omega(hp, batch, stream);
+  if (e == cudaSuccess) e = launch_omega(make_omega(h, nullptr, out_omega, hp.tiles), batch, stream);
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
 }
@@ -240,8 +255,6 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   SolveParams sp;
   sp.d = h->d;
   sp.ws = h->ws;
-  sp.omega = omega ? omega : h->ws.omega;
-  sp.omega_smem = h->omega_smem ? 1 : 0;
   sp.token_bytes = h->cost.token_bytes;
   sp.expert_bytes = h->cost.expert_bytes;
   sp.max_iters = h->max_iters;
@@ -252,7 +265,10 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.out_counts = counts;
   sp.out_offsets = offsets;
   sp.out_inst_counts = inst_counts;
-  cudaError_t e = launch_solve(sp, batch, stream);
+  cudaError_t e = cudaSuccess;
+  // a routing matrix handed in from outside: derive the demand and the transposed copy from it
+  if (omega) e = launch_omega(make_omega(h, omega, nullptr, 0), batch, stream);
+  if (e == cudaSuccess) e = launch_solve(sp, batch, stream);
   if (e == cudaSuccess) {
     RouteParams rp;
     rp.d = h->d;

@@ -2,7 +2,8 @@
 //   omega[s][e] = number of (token, expert) assignments of source rank s that select expert e.
 //
 // hist_kernel: one CTA counts one tile of one source rank's flat id array in shared memory and
-// writes the tile's counts.  omega_kernel: omega[s][e] = sum of the tile counts.  No global
+// writes the tile's counts.  omega_kernel: omega[s][e] = sum of the tile counts (plus the two
+// derived layouts the solver reads).  No global
 // atomics, no zero-fill pass, no inter-CTA hand-off: the result cannot depend on arrival order,
 // and the per-tile counts are what the later kernels turn into the cross-tile base of an
 // assignment's stable rank.
@@ -68,23 +69,42 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   for (int e = tid; e < E; e += nt) out[e] = cnt[e];
 }
 
-// omega[b][s][e] = sum over tiles; one thread per (b, s, e), tile counts read coalesced over e.
-__global__ void omega_kernel(const HistParams p) {
-  const int E = p.d.E;
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= E) return;
-  const size_t row = (size_t)blockIdx.z * p.d.R + blockIdx.y;
-  const int32_t* c = p.ws.tile_cnt + row * (size_t)p.max_tiles * E + e;
-  int sum = 0;
-  for (int t0 = 0; t0 < p.tiles; t0 += 8) {
-    int v[8];
+// omega[b][s][e] = sum over the row's tiles (or a routing matrix handed in), written three ways
+// for the solver: omega[s][e]; omega_m[main instance of e][s] (transposed, so that the columns a
+// solver CTA needs are contiguous rows); and the domain demand D[d][e] = sum over the G ranks of d
+// (paper, "System Model", Eq. D).  A warp covers one domain and epw = 32 / Gpad experts: lane =
+// g * epw + i holds omega[d*G + g][e0 + i], and a butterfly over the g bits yields D.
+__global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
+  const int E = p.d.E, G = p.d.G, R = p.d.R, epw = p.epw;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int dm = blockIdx.y, b = blockIdx.z;
+  const int g = lane / epw, e = (blockIdx.x * 4 + warp) * epw + (lane - g * epw);
+  const bool on = g < G && e < E;
+  const int s = dm * G + g;
+  const size_t row = (size_t)b * R + s;
+  int sum = 0, mi = 0;
+  if (on) {
+    if (p.ws.omega_m)   // row of the transposed copy; fetched alongside the counts
+      mi = __ldg(p.ws.main_rank + e) * p.d.e_loc + __ldg(p.ws.main_local + e);
+    if (p.src_omega) {
+      sum = __ldg(p.src_omega + row * E + e);
+    } else {
+      const int32_t* c = p.ws.tile_cnt + row * (size_t)p.max_tiles * E + e;
+      for (int t0 = 0; t0 < p.tiles; t0 += 16) {
+        int v[16];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
+        for (int u = 0; u < 16; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) sum += v[u];
+        for (int u = 0; u < 16; ++u) sum += v[u];
+      }
+    }
+    if (p.ws.omega) p.ws.omega[row * E + e] = sum;
+    if (p.out_omega) p.out_omega[row * E + e] = sum;
+    if (p.ws.omega_m) p.ws.omega_m[((size_t)b * R * p.d.e_loc + mi) * R + s] = sum;
   }
-  p.ws.omega[row * E + e] = sum;
-  if (p.out_omega) p.out_omega[row * E + e] = sum;
+  int dsum = sum;
+  for (int o = epw; o < 32; o <<= 1) dsum += __shfl_xor_sync(0xffffffffu, dsum, o);
+  if (g == 0 && e < E && p.ws.demand) p.ws.demand[((size_t)b * p.d.M + dm) * E + e] = dsum;
 }
 
 __global__ void empty_kernel() {}
@@ -108,8 +128,8 @@ cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t s
   return cudaGetLastError();
 }
 
-cudaError_t launch_omega(const HistParams& p, int batch, cudaStream_t stream) {
-  const dim3 grid((p.d.E + 127) / 128, p.d.R, batch);
+cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream) {
+  const dim3 grid((p.d.E + 4 * p.epw - 1) / (4 * p.epw), p.d.M, batch);
   omega_kernel<<<grid, 128, 0, stream>>>(p);
   return cudaGetLastError();
 }

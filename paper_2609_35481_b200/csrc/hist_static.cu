@@ -82,7 +82,6 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   hp.d.k = top_k;
   hp.ws.status = flags;
   hp.ws.tile_cnt = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(base) + kFlagsBytes);
-  hp.ws.omega = dev_omega;
   hp.ids = dev_topk_ids;
   hp.out_omega = nullptr;
   hp.n_ids = (int)n_ids;
@@ -91,6 +90,18 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   hp.max_tiles = (int)tiles;
   hp.vec_ok = (n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(dev_topk_ids) & 15u) == 0);
   e = launch_hist(hp, batch, 0, stream);
-  if (e == cudaSuccess) e = launch_omega(hp, batch, stream);
+  if (e == cudaSuccess) {
+    OmegaParams op = {};   // every rank its own "domain": plain tile sums into dev_omega
+    op.d.R = ranks;
+    op.d.M = ranks;
+    op.d.G = 1;
+    op.d.E = experts;
+    op.ws.tile_cnt = hp.ws.tile_cnt;
+    op.out_omega = dev_omega;
+    op.tiles = hp.tiles;
+    op.max_tiles = hp.max_tiles;
+    op.epw = 32;
+    e = launch_omega(op, batch, stream);
+  }
   return e == cudaSuccess ? TOPOEP_OK : TOPOEP_ERR_CUDA;
 }

@@ -20,7 +20,7 @@ namespace topoep {
 
 namespace {
 
-struct RouteLayout { size_t rm, qrow, mr, ml, nz, single, sidx, seg, cum, crow, warp_tot, total; };
+struct RouteLayout { size_t rm, qrow, mr, ml, nz, single, sidx, seg, cum, crow, split_e, warp_tot, total; };
 
 __host__ __device__ inline RouteLayout route_layout(const Dims& d) {
   RouteLayout o;
@@ -35,6 +35,7 @@ __host__ __device__ inline RouteLayout route_layout(const Dims& d) {
   o.seg = at;      at += sizeof(int) * (size_t)(d.E + 1);
   o.cum = at;      at += sizeof(int) * (size_t)d.P;
   o.crow = at;     at += sizeof(int) * (size_t)d.R;
+  o.split_e = at;  at += sizeof(int) * (size_t)d.E;
   o.warp_tot = at; at += sizeof(int) * 2 * (kRouteThreads / 32);
   o.total = at;
   return o;
@@ -90,6 +91,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   int* seg = reinterpret_cast<int*>(smem + lay.seg);       // [E+1] list start of e (split only)
   int* cum = reinterpret_cast<int*>(smem + lay.cum);       // [P]   quotas in list order
   int* crow = reinterpret_cast<int*>(smem + lay.crow);     // [R]   counts[s][.]
+  int* split_e = reinterpret_cast<int*>(smem + lay.split_e); // [E]   expert of split index i
   int* warp_tot = reinterpret_cast<int*>(smem + lay.warp_tot);
 
   const size_t row = (size_t)b * R + s;
@@ -130,7 +132,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   for (int e = tid; e < E; e += nt) {
     const bool split = nz[e] >= 2;
     route[e] = split ? -2 - sidx[e] : single[e];
-    if (split) rec[rl.seg + sidx[e]] = seg[e];
+    if (split) { rec[rl.seg + sidx[e]] = seg[e]; split_e[sidx[e]] = e; }
   }
   if (tid == 0) {   // rec[2] doubles as the reroute kernel's initial (empty) work-list length
     rec[0] = n_split; rec[1] = n_list; rec[2] = 0; rec[3] = 0;
@@ -170,14 +172,14 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     const size_t trow = row * (size_t)p.max_tiles * E;
     if (p.tiles <= 32) {
       // a warp owns a split expert, a lane owns a tile
-      for (int e = warp; e < E; e += nt >> 5) {
-        if (nz[e] < 2) continue;
+      for (int i = warp; i < n_split; i += nt >> 5) {
+        const int e = split_e[i];
         const int v = lane < p.tiles ? __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e) : 0;
         int total;
         const int ex = warp_exclusive_scan(v, lane, &total);
         if (lane < p.tiles) {
-          p.ws.tile_pref[trow + (size_t)lane * E + sidx[e]] = ex;
-          if (sidx[e] < kSplitCap) rec[rl.tp + lane * kSplitCap + sidx[e]] = ex;
+          p.ws.tile_pref[trow + (size_t)lane * E + i] = ex;
+          if (i < kSplitCap) rec[rl.tp + lane * kSplitCap + i] = ex;
         }
       }
     } else {

@@ -12,10 +12,13 @@
 // What needs every domain's result (send offsets, per-source routing tables) is left to the
 // route kernel that follows.
 //
-// The kernel is latency-bound (KBs of state, an L2 round trip costs ~0.7 us on B200), so all
-// global inputs -- the routing matrix when it fits in shared memory, the main-rank tables --
-// arrive in ONE round of cp.async copies before the first barrier, and the phases after it work
-// from shared memory only.
+// The kernel is latency-bound (KBs of state; an L2 round trip costs ~0.7 us on B200 and a lone
+// warp retires a dependent instruction every ~5 cycles), so:
+//  * its inputs arrive by cp.async in one round before the first barrier: the demand D of every
+//    domain (summed by omega_kernel), the main-rank tables, and the routing-matrix columns of the
+//    domain's main instances, which omega_kernel stored as contiguous rows;
+//  * the columns of the replicas chosen in stage 1 are fetched while the main columns are routed;
+//  * stage 1 ranks the candidates of a domain all-pairs instead of selecting one maximum at a time.
 #include <limits.h>
 
 #include "topoep_internal.cuh"
@@ -27,17 +30,20 @@ namespace {
 constexpr int kRankCap = 128;   // stage 1 ranks up to this many candidates of a domain all-pairs
 
 struct SolveLayout {
-  size_t om, cand, D, qd, mrank, host_lo, host_hi, col_expert, col_cr, U, L, used, cnt, hostcol, total;
+  size_t cand, col_main, col_rep, mrank, mlocal, D, qd, host_lo, host_hi, col_expert, col_cr, U, L,
+      used, cnt, hostcol, sdom, total;
 };
 
-__host__ __device__ inline SolveLayout solve_layout(const Dims& d, bool omega_smem) {
+__host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
   SolveLayout o;
   size_t at = 0;
-  o.om = at;         at += sizeof(int) * (omega_smem ? pad4((size_t)d.R * d.E) : 0);
   o.cand = at;       at += sizeof(unsigned long long) * (size_t)kRankCap * (kSolveThreads / 32);
+  o.col_main = at;   at += sizeof(int) * pad4((size_t)d.G * d.e_loc * d.R);   // [G*e_loc][R]
+  o.col_rep = at;    at += sizeof(int) * pad4((size_t)d.G * d.N * d.R);       // [G*N][R]
   o.mrank = at;      at += sizeof(int) * pad4(d.E);
-  o.D = at;          at += sizeof(int) * (size_t)d.M * d.E;
+  o.mlocal = at;     at += sizeof(int) * pad4(d.E);
+  o.D = at;          at += sizeof(int) * pad4((size_t)d.M * d.E);
   o.qd = at;         at += sizeof(int) * (size_t)d.R * d.qstride;
   o.host_lo = at;    at += sizeof(int) * (size_t)d.E;
   o.host_hi = at;    at += sizeof(int) * (size_t)d.E;
@@ -48,8 +54,18 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d, bool omega_sm
   o.used = at;       at += sizeof(int) * (size_t)d.G;
   o.cnt = at;        at += sizeof(int) * (size_t)d.R * d.G;
   o.hostcol = at;    at += sizeof(short) * (size_t)d.G * d.E;
+  o.sdom = at;       at += sizeof(short) * (size_t)d.R;
   o.total = (at + 15) & ~(size_t)15;
   return o;
+}
+
+// n ints global -> shared, 16 bytes at a time when both sides allow it.
+__device__ __forceinline__ void copy_async(int* dst, const int32_t* src, int n, int tid, int nt) {
+  if ((n & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    for (int i = tid; i < n / 4; i += nt) cp_async16(dst + 4 * i, src + 4 * i);
+  } else {
+    for (int i = tid; i < n; i += nt) cp_async4(dst + i, src + i);
+  }
 }
 
 __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams p) {
@@ -60,11 +76,13 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   const int dm = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
   const unsigned full = 0xffffffffu;
-  const bool om_smem = p.omega_smem != 0;
 
-  const SolveLayout lay = solve_layout(d, om_smem);
-  int* om_s = reinterpret_cast<int*>(smem + lay.om);
+  const SolveLayout lay = solve_layout(d);
+  unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);
+  int* col_main = reinterpret_cast<int*>(smem + lay.col_main);
+  int* col_rep = reinterpret_cast<int*>(smem + lay.col_rep);
   int* mrank = reinterpret_cast<int*>(smem + lay.mrank);
+  int* mlocal = reinterpret_cast<int*>(smem + lay.mlocal);
   int* D = reinterpret_cast<int*>(smem + lay.D);
   int* qd = reinterpret_cast<int*>(smem + lay.qd);
   unsigned* host_lo = reinterpret_cast<unsigned*>(smem + lay.host_lo);   // hosting domains 0..31
@@ -76,86 +94,41 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   int* used = reinterpret_cast<int*>(smem + lay.used);
   int* cnt = reinterpret_cast<int*>(smem + lay.cnt);
   short* hostcol = reinterpret_cast<short*>(smem + lay.hostcol);
+  short* sdom = reinterpret_cast<short*>(smem + lay.sdom);
 
-  const int32_t* om = p.omega + (size_t)b * R * E;
+  const int32_t* om_m = p.ws.omega_m + (size_t)b * R * e_loc * R;   // rows = main instances
 
-  // ---- one round of asynchronous copies: routing matrix, main ranks, the domain's main experts
-  if (om_smem) {
-    const int n = R * E;
-    if ((n & 3) == 0 && (reinterpret_cast<uintptr_t>(om) & 15u) == 0) {
-      for (int i = tid; i < n / 4; i += nt) cp_async16(om_s + 4 * i, om + 4 * i);
-    } else {
-      for (int i = tid; i < n; i += nt) cp_async4(om_s + i, om + i);
-    }
-  }
-  if ((E & 3) == 0) {
-    for (int i = tid; i < E / 4; i += nt) cp_async16(mrank + 4 * i, p.ws.main_rank + 4 * i);
-  } else {
-    for (int i = tid; i < E; i += nt) cp_async4(mrank + i, p.ws.main_rank + i);
-  }
+  // ---- round 1 of asynchronous copies ---------------------------------------------------------
+  copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
+  copy_async(mrank, p.ws.main_rank, E, tid, nt);
+  copy_async(mlocal, p.ws.main_local, E, tid, nt);
+  copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
   for (int i = tid; i < G * e_loc; i += nt) {
     const int g = i / e_loc, l = i - g * e_loc;
     cp_async4(col_expert + g * s_phys + l, p.ws.main_inst_expert + (size_t)(dm * G + g) * e_loc + l);
   }
   for (int i = tid; i < G * N; i += nt) col_expert[(i / N) * s_phys + e_loc + i % N] = -1;
   for (int i = tid; i < G * E; i += nt) hostcol[i] = -1;
-  for (int c = tid; c < C; c += nt) { col_cr[c] = p.cost_rank_intra; U[c] = 0; }
+  for (int c = tid; c < C; c += nt) col_cr[c] = p.cost_rank_intra;
+  for (int s = tid; s < R; s += nt) sdom[s] = (short)(s / G);
   if (tid < G) used[tid] = 0;
   cp_async_wait_all();
   __syncthreads();
 
-  // ---- hosting masks from the main ranks; candidate demand of every domain -------------------
+  // ---- hosting masks from the main ranks; keep D only where e is a stage-1 candidate ----------
   for (int e = tid; e < E; e += nt) {
     const int md = mrank[e] / G;
     host_lo[e] = md < 32 ? 1u << md : 0u;
     host_hi[e] = md < 32 ? 0u : 1u << (md - 32);
+    for (int dd = 0; dd < M; ++dd) {
+      const int v = D[dd * E + e];
+      const bool cand = dd != md && 2 * (long long)v * p.token_bytes - p.expert_bytes > 0;
+      if (!cand) D[dd * E + e] = 0;
+    }
   }
   for (int c = tid; c < C; c += nt) {
     const int e = col_expert[c];
     if (e >= 0) hostcol[(c / s_phys) * E + e] = (short)c;
-  }
-  // D[dd][e] = sum over the G source ranks of domain dd, kept only where e is a stage-1 candidate
-  // of dd (main outside dd and b > 0), else 0.
-  if (om_smem) {
-    const int chunks = (E + 31) / 32;
-    for (int t = warp; t < M * chunks; t += nwarps) {   // a warp-task = (domain, 32 experts)
-      const int dd = t / chunks, e = (t - dd * chunks) * 32 + lane;
-      if (e >= E) continue;
-      const int* col = om_s + dd * G * E + e;
-      int sum = 0;
-      for (int g = 0; g < G; ++g) sum += col[g * E];
-      const bool cand = dd != mrank[e] / G && 2 * (long long)sum * p.token_bytes - p.expert_bytes > 0;
-      D[dd * E + e] = cand ? sum : 0;
-    }
-  } else {
-    for (int idx0 = tid; idx0 < M * E; idx0 += 4 * nt) {   // 32 loads in flight per thread
-      int sum[4] = {0, 0, 0, 0};
-      for (int g0 = 0; g0 < G; g0 += 8) {
-        int v[4][8];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-          const int idx = idx0 + a * nt;
-          const int dd = idx / E, e = idx - dd * E;
-          const int32_t* col = om + (size_t)dd * G * E + e;
-#pragma unroll
-          for (int u = 0; u < 8; ++u)
-            v[a][u] = (idx < M * E && g0 + u < G) ? __ldg(col + (size_t)(g0 + u) * E) : 0;
-        }
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int u = 0; u < 8; ++u) sum[a] += v[a][u];
-      }
-#pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        const int idx = idx0 + a * nt;
-        if (idx >= M * E) break;
-        const int dd = idx / E, e = idx - dd * E;
-        const bool cand = dd != mrank[e] / G &&
-                          2 * (long long)sum[a] * p.token_bytes - p.expert_bytes > 0;
-        D[idx] = cand ? sum[a] : 0;
-      }
-    }
   }
   __syncthreads();
 
@@ -168,8 +141,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     for (int dd = warp; dd < M; dd += nwarps) {
       int* Dd = D + dd * E;
       // compact the candidates (D > 0) of this domain into cand[]: key = (D, -e)
-      unsigned long long* cand = reinterpret_cast<unsigned long long*>(smem + lay.cand) +
-                                 (size_t)warp * kRankCap;
+      unsigned long long* cand = cand_all + (size_t)warp * kRankCap;
       int n_c = 0;
       for (int e0 = 0; e0 < E; e0 += 32) {
         const int e = e0 + lane;
@@ -229,34 +201,60 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   }
   __syncthreads();
 
+  // ---- round 2 of asynchronous copies: the routing-matrix columns of this domain's replicas ----
+  for (int i = warp; i < G * N; i += nwarps) {
+    const int e = col_expert[(i / N) * s_phys + e_loc + i % N];
+    if (e < 0) continue;
+    const int32_t* src = om_m + (size_t)(mrank[e] * e_loc + mlocal[e]) * R;
+    copy_async(col_rep + i * R, src, R, lane, 32);
+  }
+
   // ---- routing construction for the columns of this domain ----------------------------------
   // After stage 1 an expert has at most one instance per domain.  A source keeps everything in
   // its own domain when an instance is there; otherwise it splits over all instances (ascending
   // rank == ascending hosting domain), remainder to `rem` instances starting at (s+e) mod n.
-  // Warps walk the sources, lanes the columns; U accumulates by shared atomics (sums commute).
-  for (int s = warp; s < R; s += nwarps) {
-    const int ds = s / G;
-    for (int c = lane; c < C; c += 32) {
+  // A warp takes a column, its lanes the sources; main columns first, replica columns once their
+  // copies have landed.
+  for (int pass = 0; pass < 2; ++pass) {
+    if (pass == 1) {
+      cp_async_wait_all();
+      __syncthreads();
+    }
+    const int ncols = pass == 0 ? G * e_loc : G * N;
+    for (int i = warp; i < ncols; i += nwarps) {
+      const int per = pass == 0 ? e_loc : N;
+      const int g = i / per, l = i - g * per;
+      const int c = g * s_phys + (pass == 0 ? l : e_loc + l);
       const int e = col_expert[c];
-      int v = 0;
+      const int* w_col = (pass == 0 ? col_main : col_rep) + i * R;
+      unsigned long long hm = 0;
+      int n = 1, idx = 0;
       if (e >= 0) {
-        const int w = om_smem ? om_s[s * E + e] : __ldg(om + (size_t)s * E + e);
-        if (ds == dm) {
-          v = w;
-        } else {
-          const unsigned long long hm = ((unsigned long long)host_hi[e] << 32) | host_lo[e];
-          if (!((hm >> ds) & 1ull)) {
-            const int n = __popcll(hm);
-            const int i = __popcll(hm & ((1ull << dm) - 1ull));
+        hm = ((unsigned long long)host_hi[e] << 32) | host_lo[e];
+        n = __popcll(hm);
+        idx = __popcll(hm & ((1ull << dm) - 1ull));
+      }
+      int usum = 0;
+      for (int s0 = 0; s0 < R; s0 += 32) {
+        const int s = s0 + lane;
+        int v = 0;
+        if (s < R && e >= 0) {
+          const int w = w_col[s];
+          const int ds = sdom[s];
+          if (ds == dm || n == 1) {   // own domain, or the only instance anywhere
+            v = w;
+          } else if (!((hm >> ds) & 1ull)) {
             const int base = w / n, rem = w - base * n;
-            int sh = i - (s + e) % n;
+            int sh = idx - (s + e) % n;
             if (sh < 0) sh += n;
             v = base + (sh < rem ? 1 : 0);
           }
         }
-        if (v) atomicAdd(&U[c], v);
+        if (s < R) qd[s * QS + c] = v;
+        usum += v;
       }
-      qd[s * QS + c] = v;
+      usum = __reduce_add_sync(full, usum);
+      if (lane == 0) U[c] = usum;
     }
   }
   __syncthreads();
@@ -367,9 +365,10 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     if (p.out_replica_map) p.out_replica_map[at] = e;
   }
   for (int c = tid; c < C; c += nt) {
+    const int u = col_expert[c] >= 0 ? U[c] : 0;
     const size_t at = (size_t)b * d.P + (size_t)dm * C + c;
-    p.ws.inst_counts[at] = U[c];
-    if (p.out_inst_counts) p.out_inst_counts[at] = U[c];
+    p.ws.inst_counts[at] = u;
+    if (p.out_inst_counts) p.out_inst_counts[at] = u;
   }
   if (tid < G) p.ws.rank_load[(size_t)b * R + dm * G + tid] = L[tid];
   for (int s = warp; s < R; s += nwarps) {
@@ -401,11 +400,11 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
 
 }  // namespace
 
-size_t solve_smem_bytes(const Dims& d, bool omega_smem) { return solve_layout(d, omega_smem).total; }
+size_t solve_smem_bytes(const Dims& d) { return solve_layout(d).total; }
 
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.d.M, batch);
-  solve_kernel<<<grid, kSolveThreads, solve_smem_bytes(p.d, p.omega_smem != 0), stream>>>(p);
+  solve_kernel<<<grid, kSolveThreads, solve_smem_bytes(p.d), stream>>>(p);
   return cudaGetLastError();
 }
 

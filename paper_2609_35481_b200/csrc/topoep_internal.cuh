@@ -35,6 +35,9 @@ struct Workspace {
   const int32_t* main_inst_expert;  // [R][e_loc] expert of main instance l on rank r, -1 if none
   uint32_t* status;                 // [1]
   int32_t* omega;                   // [max_batch][R][E]
+  int32_t* omega_m;                 // [max_batch][R*e_loc][R] omega transposed, one row per main
+                                    //   instance (row = main_rank(e)*e_loc + main_local(e))
+  int32_t* demand;                  // [max_batch][M][E] domain demand D
   int32_t* tile_cnt;                // [max_batch][R][max_tiles][E] per-tile histogram
   int32_t* tile_pref;               // [max_batch][R][max_tiles][E] exclusive prefix over tiles,
                                     //   column i = i-th split expert of the source
@@ -84,11 +87,18 @@ struct HistParams {
   int vec_ok;           // rows are 16-byte aligned and n_ids % 4 == 0
 };
 
+struct OmegaParams {
+  Dims d;
+  Workspace ws;
+  const int32_t* src_omega;   // given routing matrix [B][R][E], or NULL: sum the tile counts
+  int32_t* out_omega;         // optional caller copy of omega [B][R][E]
+  int tiles, max_tiles;
+  int epw;                    // experts per warp = 32 / (G rounded up to a power of two)
+};
+
 struct SolveParams {
   Dims d;
   Workspace ws;
-  const int32_t* omega;       // [B][R][E] routing matrix to plan from
-  int omega_smem;             // the routing matrix of one plan fits in shared memory
   int64_t token_bytes, expert_bytes;
   int max_iters, min_delta;
   int cost_rank_intra, cost_rank_inter;   // dense ranks of {0, c_intra*W, c_inter*W}
@@ -123,7 +133,7 @@ struct SummaryParams {
 };
 
 size_t hist_smem_bytes(const Dims& d);
-size_t solve_smem_bytes(const Dims& d, bool omega_smem);
+size_t solve_smem_bytes(const Dims& d);
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 
@@ -131,7 +141,7 @@ cudaError_t configure_solve(size_t smem);
 cudaError_t configure_route(size_t smem);
 cudaError_t configure_reroute(size_t smem);
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream);
-cudaError_t launch_omega(const HistParams& p, int batch, cudaStream_t stream);
+cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_route(const RouteParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream);
