@@ -47,9 +47,12 @@ def lib() -> ctypes.CDLL:
     """Load the CUDA library (built in-tree by paper_2609_35481_b200.build)."""
     global _lib
     if _lib is None:
+        # Stale or missing library: compile it in-tree (nvcc, sm_100a).  There is no other
+        # implementation to fall back to; a failed build raises.
+        from . import build as _build
+        _build.build()
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError("libtopoep.so is not built: run `python -m paper_2609_35481_b200.build` "
-                               "(there is no CPU fallback)")
+            raise RuntimeError("libtopoep.so could not be built (there is no CPU fallback)")
         L = ctypes.CDLL(LIB_PATH)
         vp, ci, i32p = ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p
         L.topoep_create.restype = ci

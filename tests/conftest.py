@@ -12,6 +12,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def _built_once():
+    """Compile the CUDA library, the oracle and the input generator if they are missing or stale."""
+    import __graft_entry__
+    __graft_entry__.build()
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch
