@@ -112,6 +112,24 @@ def test_uneven_main_map_and_odd_topology():
     assert_same(gpu, ref)
 
 
+def test_many_domains_wide_nodes_and_many_candidates():
+    # 40 single-GPU nodes (hosting masks beyond bit 31), a 32-GPU node (one refinement lane per
+    # target), and a cheap expert (tiny ||W||) so that a domain has far more than 128 stage-1
+    # candidates (slot-by-slot selection path) and many split experts per source (several passes
+    # of the reroute ranking)
+    w = wl.CONFIGS["tiny"].replace(nodes=40, gpus_per_node=1, experts=80, slots_per_rank=2, top_k=4,
+                                   tokens_per_rank=700, zipf_s=0.9)
+    parity(w, 21, batch=2, expert_bytes=4096)
+    w = wl.CONFIGS["tiny"].replace(nodes=2, gpus_per_node=32, experts=128, slots_per_rank=2, top_k=4,
+                                   tokens_per_rank=900, zipf_s=1.3)
+    gpu, ref, _ = parity(w, 22, batch=2)
+    assert ref.refine_iters.sum() > 0
+    w = wl.CONFIGS["tiny"].replace(nodes=3, gpus_per_node=4, experts=600, slots_per_rank=24,
+                                   top_k=8, tokens_per_rank=4096, zipf_s=0.3)
+    gpu, ref, _ = parity(w, 23, batch=1, expert_bytes=64, token_bytes=64)
+    assert ref.summaries["replicas_inter"][0] > 128
+
+
 def test_random_small_problems():
     rng = np.random.default_rng(11)
     for trial in range(40):
