@@ -69,6 +69,8 @@ def _load():
         lib.oracle_layout.argtypes = [vp] * 8
         lib.oracle_summary_of.restype = None
         lib.oracle_summary_of.argtypes = [vp] * 7
+        lib.oracle_dispatch_positions.restype = None
+        lib.oracle_dispatch_positions.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, vp]
         lib.oracle_plan.restype = ctypes.c_int
         lib.oracle_plan.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int] + [vp] * 11
         _lib = lib
@@ -215,6 +217,19 @@ def summary(cfg: OracleConfig, res: SolveResult) -> np.ndarray:
     _load().oracle_summary_of(ctypes.addressof(c), _p(cfg.main_rank), _p(res.x), _p(res.q),
                               _p(res.L), _p(res.iters), _p(out))
     return out[0]
+
+
+def dispatch_positions(cfg: OracleConfig, token_replica: np.ndarray):
+    """O10 for one plan: token_replica [R][T][k] -> (send_pos, recv_pos, instance_offsets)."""
+    R = cfg.ranks
+    tr = np.ascontiguousarray(token_replica, dtype=np.int32).reshape(R, -1, cfg.top_k)
+    send = np.empty_like(tr)
+    recv = np.empty_like(tr)
+    inst_off = np.zeros((R, cfg.s_phys + 1), np.int32)
+    c = cfg.c_struct()
+    _load().oracle_dispatch_positions(ctypes.addressof(c), _p(cfg.main_rank), tr.shape[1], _p(tr),
+                                      _p(send), _p(recv), _p(inst_off))
+    return send, recv, inst_off
 
 
 @dataclass

@@ -23,6 +23,8 @@
  *   O9 summaries                                 (objective terms T_comp, T_token, T_replica;
  *                                                 max/mean load ratio; inter-node and
  *                                                 replica-served fractions)
+ *   O10 dispatch permutation                     (the step after the path; layout defined at
+ *                                                 the function, pinned to numpy.lexsort)
  *
  * Where the paper is silent the readings are (all listed in the design notes
  * of the repository, none of them pinned by the paper itself):
@@ -501,4 +503,49 @@ int oracle_plan(const oracle_config* c, const int32_t* main_rank, const int32_t*
   free(omega); free(x); free(slotmap); free(q); free(U); free(L); free(D); free(iters);
   free(cnt_tmp); free(off_tmp);
   return 0;
+}
+
+/*
+ * O10 -- dispatch permutation (the step right after the planning path; the paper leaves the
+ * buffer layout to its dispatch library, so this is a definition of ours, stated here):
+ *   send_pos: index of an assignment in its source rank's send buffer, which is ordered by
+ *             (destination rank, physical instance, flat index t*k+j);
+ *   recv_pos: index in its destination rank's receive buffer, which is ordered by
+ *             (physical instance, source rank, flat index) -- every instance's tokens contiguous,
+ *             ready for a grouped GEMM;
+ *   instance_offsets[r][l]: start of instance l's segment in rank r's receive buffer
+ *             (entry S_phys = L_r).
+ * Written as counting walks, one buffer slot at a time; ignored ids get -1.
+ */
+void oracle_dispatch_positions(const oracle_config* c, const int32_t* main_rank, int T,
+                               const int32_t* token_replica /*[R][T][k]*/, int32_t* send_pos,
+                               int32_t* recv_pos, int32_t* instance_offsets /*[R][S_phys+1]*/) {
+  const int R = c->nodes * c->gpus_per_node, k = c->top_k;
+  const int s_phys = oracle_e_loc(c, main_rank) + c->slots_per_rank;
+  const int64_t n = (int64_t)T * k;
+  /* send side: for each source, walk the instances in ascending id (= ascending rank, then
+     instance) and hand out consecutive slots in flat order */
+  for (int s = 0; s < R; ++s) {
+    int64_t next = 0;
+    for (int p = 0; p < R * s_phys; ++p)
+      for (int64_t f = 0; f < n; ++f)
+        if (token_replica[(size_t)s * n + f] == p) send_pos[(size_t)s * n + f] = (int32_t)next++;
+    for (int64_t f = 0; f < n; ++f)
+      if (token_replica[(size_t)s * n + f] < 0) send_pos[(size_t)s * n + f] = -1;
+  }
+  /* receive side: for each rank, instance by instance, source by source, in flat order */
+  for (int r = 0; r < R; ++r) {
+    int64_t next = 0;
+    for (int l = 0; l < s_phys; ++l) {
+      instance_offsets[(size_t)r * (s_phys + 1) + l] = (int32_t)next;
+      const int p = r * s_phys + l;
+      for (int s = 0; s < R; ++s)
+        for (int64_t f = 0; f < n; ++f)
+          if (token_replica[(size_t)s * n + f] == p) recv_pos[(size_t)s * n + f] = (int32_t)next++;
+    }
+    instance_offsets[(size_t)r * (s_phys + 1) + s_phys] = (int32_t)next;
+  }
+  for (int s = 0; s < R; ++s)
+    for (int64_t f = 0; f < n; ++f)
+      if (token_replica[(size_t)s * n + f] < 0) recv_pos[(size_t)s * n + f] = -1;
 }

@@ -127,3 +127,36 @@ def objective(nodes, gpus_per_node, main_rank, token_bytes, expert_bytes, c_intr
             if x[e, r] and r != main_rank[e]:
                 t_replica += int(C[main_rank[e], r]) * expert_bytes
     return t_comp, t_token, t_replica
+
+
+def dispatch_positions_by_sorting(ranks, s_phys, token_replica):
+    """Independent definition of the dispatch permutation with numpy.lexsort.
+
+    send buffer of a source: ordered by (instance id, flat index) -- instance ids ascend with
+    (rank, instance); receive buffer of a rank: ordered by (instance, source, flat index).
+    Returns (send_pos, recv_pos, instance_offsets) for one plan; ignored ids (-1) get -1.
+    """
+    tr = np.asarray(token_replica, np.int64).reshape(ranks, -1)
+    n = tr.shape[1]
+    send = np.full(tr.shape, -1, np.int64)
+    flat = np.arange(n)
+    for s in range(ranks):
+        ok = tr[s] >= 0
+        order = np.lexsort((flat[ok], tr[s][ok]))
+        pos = np.empty(order.size, np.int64)
+        pos[order] = np.arange(order.size)
+        send[s][ok] = pos
+    recv = np.full(tr.shape, -1, np.int64)
+    src = np.broadcast_to(np.arange(ranks)[:, None], tr.shape)
+    fl = np.broadcast_to(flat[None, :], tr.shape)
+    inst_off = np.zeros((ranks, s_phys + 1), np.int64)
+    for r in range(ranks):
+        sel = (tr >= 0) & (tr // s_phys == r)
+        p, s_, f_ = tr[sel], src[sel], fl[sel]
+        order = np.lexsort((f_, s_, p))
+        pos = np.empty(order.size, np.int64)
+        pos[order] = np.arange(order.size)
+        recv[sel] = pos
+        counts = np.bincount(p - r * s_phys, minlength=s_phys)
+        inst_off[r, 1:] = np.cumsum(counts)
+    return send, recv, inst_off

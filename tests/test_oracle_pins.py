@@ -14,7 +14,7 @@ import pytest
 
 import oracle as orc
 import workloads as wl
-from plan_checks import check_plan, objective
+from plan_checks import check_plan, dispatch_positions_by_sorting, objective
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 MiB = 1 << 20
@@ -389,6 +389,32 @@ def test_token_assignment_brute_force():
                     cursor += n
                 assert cursor == len(pos)
             assert (out[s].ravel()[flat < 0] == -1).all()
+
+
+def test_dispatch_positions_are_the_sorted_order():
+    # O10 against numpy.lexsort: the send buffer is the assignments of a source sorted by
+    # (instance, flat index), the receive buffer those of a rank sorted by (instance, source, flat)
+    for name, over in (("tiny", dict(slots_per_rank=2)), ("mid", dict(tokens_per_rank=300, slots_per_rank=3))):
+        w = wl.CONFIGS[name].replace(**over)
+        ids = wl.make_topk_ids(w, seed=17).copy()
+        ids[0, 1, 5:9, :] = -1
+        cfg = _wl_cfg(w)
+        p = orc.plan(cfg, ids)
+        send, recv, off = orc.dispatch_positions(cfg, p.token_replica[0])
+        s2, r2, o2 = dispatch_positions_by_sorting(w.ranks, cfg.s_phys, p.token_replica[0])
+        assert (send.reshape(w.ranks, -1) == s2).all()
+        assert (recv.reshape(w.ranks, -1) == r2).all()
+        assert (off == o2).all()
+        # the offsets are the exclusive scan of the instance counts, the last one is L_r
+        U = p.instance_counts[0].reshape(w.ranks, cfg.s_phys)
+        assert (off[:, 1:] == np.cumsum(U, axis=1)).all() and (off[:, -1] == p.rank_load[0]).all()
+        # a source's block for destination rank r starts at its send offset
+        tr = p.token_replica[0].reshape(w.ranks, -1)
+        for s in range(w.ranks):
+            for r in range(w.ranks):
+                sel = (tr[s] >= 0) & (tr[s] // cfg.s_phys == r)
+                if sel.any():
+                    assert send.reshape(w.ranks, -1)[s][sel].min() == p.dispatch_offsets[0, 0, s, r]
 
 
 # ----------------------------------------------------------------------------------------------
