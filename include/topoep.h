@@ -255,6 +255,39 @@ int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_pe
                    int batch, int32_t* dev_token_replica, topoep_stream_t stream);
 
 /*
+ * Dispatch permutation of the last topoep_plan (the step after the planning
+ * path; the paper's "DeepEP dispatch and combine" leaves the buffer layout to
+ * its dispatch library, so the layout is defined here):
+ *   send buffer of source rank s: its assignments ordered by (physical instance
+ *     executing them, flat index t*k+j).  Instance ids ascend with (rank,
+ *     instance), so destination r's block is contiguous and starts at
+ *     dev_dispatch_offsets[0][s][r].
+ *   receive buffer of rank r: the assignments it executes ordered by (instance,
+ *     source rank, flat index): every instance's tokens are contiguous, ready for
+ *     a grouped GEMM, sources in rank order inside.
+ *
+ *   dev_token_replica    in  [B][R][T][k] as written by topoep_plan
+ *   dev_send_pos         out [B][R][T][k] index in the source's send buffer, -1
+ *                            for an ignored id
+ *   dev_recv_pos         out [B][R][T][k] index in the destination rank's receive
+ *                            buffer, -1 for an ignored id
+ *   dev_instance_offsets out [B][R][S_phys+1] start of each instance's segment in
+ *                            its rank's receive buffer (entry S_phys = L_r); or NULL
+ *   dev_scratch          device memory, 256-byte aligned, at least
+ *                            topoep_dispatch_scratch_bytes(h, T, B) long; contents
+ *                            need not be kept between calls
+ * Uses q and U of the plan still in the workspace: call it after topoep_plan
+ * (or topoep_solve + topoep_reroute) of the same batch.  Enqueues three kernels;
+ * capturable after its first call.  Off the planning path: the ranking kernel is
+ * bound by warp-match issue cost, not by HBM.
+ */
+size_t topoep_dispatch_scratch_bytes(topoep_handle_t h, int tokens_per_rank, int batch);
+int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replica,
+                              int tokens_per_rank, int batch, int32_t* dev_send_pos,
+                              int32_t* dev_recv_pos, int32_t* dev_instance_offsets,
+                              void* dev_scratch, size_t scratch_bytes, topoep_stream_t stream);
+
+/*
  * Summaries of the last topoep_plan (paper: objective terms and evaluation
  * ratios, see topoep_summary_t).  dev_out: [batch] topoep_summary_t, 8-byte
  * aligned.  Enqueues one kernel; off the planning path.

@@ -20,7 +20,8 @@ T_OMEGA, T_Q, T_RANK_LOAD, T_REFINE_ITERS = 0, 1, 2, 3
 KNOB_TILE_IDS, KNOB_HIST_MODE = 0, 1
 
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
-           "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_summary", "topoep_read_status",
+           "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions",
+           "topoep_summary", "topoep_read_status",
            "topoep_debug_tensor", "topoep_set_tuning", "topoep_get_layout",
            "topoep_launch_floor", "topoep_strerror")
 
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.topoep_solve.argtypes = [vp, vp, ci, vp, vp, vp, vp, vp]
         L.topoep_reroute.restype = ci
         L.topoep_reroute.argtypes = [vp, vp, ci, ci, vp, vp]
+        L.topoep_dispatch_scratch_bytes.restype = ctypes.c_size_t
+        L.topoep_dispatch_scratch_bytes.argtypes = [vp, ci, ci]
+        L.topoep_dispatch_positions.restype = ci
+        L.topoep_dispatch_positions.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.topoep_summary.restype = ci
         L.topoep_summary.argtypes = [vp, ci, vp, vp]
         L.topoep_read_status.restype = ci
@@ -167,6 +172,19 @@ def topoep_solve(h, dev_omega, batch, dev_replica_map, dev_dispatch_counts, dev_
 def topoep_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream=0) -> int:
     return lib().topoep_reroute(h, _ptr(dev_topk_ids), tokens_per_rank, batch,
                                 _ptr(dev_token_replica), stream or None)
+
+
+def topoep_dispatch_scratch_bytes(h, tokens_per_rank, batch) -> int:
+    return int(lib().topoep_dispatch_scratch_bytes(h, tokens_per_rank, batch))
+
+
+def topoep_dispatch_positions(h, dev_token_replica, tokens_per_rank, batch, dev_send_pos,
+                              dev_recv_pos, dev_instance_offsets, dev_scratch, scratch_bytes,
+                              stream=0) -> int:
+    return lib().topoep_dispatch_positions(h, _ptr(dev_token_replica), tokens_per_rank, batch,
+                                           _ptr(dev_send_pos), _ptr(dev_recv_pos),
+                                           _ptr(dev_instance_offsets), _ptr(dev_scratch),
+                                           scratch_bytes, stream or None)
 
 
 def topoep_summary(h, batch, dev_out, stream=0) -> int:

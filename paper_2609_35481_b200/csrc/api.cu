@@ -16,6 +16,7 @@ struct topoep_ctx {
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode;
+  size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
   int max_tiles;
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
   // workspace
@@ -171,6 +172,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->max_batch = max_batch;
   h->tile_ids = 4096;
   h->hist_mode = 0;
+  h->dispatch_smem = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
   h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
@@ -363,6 +365,60 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
                      dev_instance_counts, stream);
   if (rc != TOPOEP_OK) return rc;
   return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
+}
+
+size_t topoep_dispatch_scratch_bytes(topoep_handle_t h, int tokens_per_rank, int batch) {
+  if (!h || tokens_per_rank < 0 || batch < 0) return 0;
+  const size_t n_ids = (size_t)tokens_per_rank * h->d.k;
+  const size_t tiles = std::max<size_t>(1, (n_ids + h->tile_ids - 1) / h->tile_ids);
+  const size_t rows = (size_t)batch * h->d.R;
+  return kAlign + align_up(4 * rows * h->d.P) * 2 + align_up(4 * rows * tiles * h->d.P);
+}
+
+int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replica,
+                              int tokens_per_rank, int batch, int32_t* dev_send_pos,
+                              int32_t* dev_recv_pos, int32_t* dev_instance_offsets,
+                              void* dev_scratch, size_t scratch_bytes, topoep_stream_t stream) {
+  int rc = check_sizes(h, tokens_per_rank, batch);
+  if (rc != TOPOEP_OK) return rc;
+  if (batch == 0) return TOPOEP_OK;
+  if (!dev_scratch) return TOPOEP_ERR_NULL;
+  if (tokens_per_rank > 0 && (!dev_token_replica || !dev_send_pos || !dev_recv_pos))
+    return TOPOEP_ERR_NULL;
+  if (!aligned4(dev_token_replica) || !aligned4(dev_send_pos) || !aligned4(dev_recv_pos) ||
+      !aligned4(dev_instance_offsets))
+    return TOPOEP_ERR_ALIGN;
+  if (scratch_bytes < topoep_dispatch_scratch_bytes(h, tokens_per_rank, batch) ||
+      (reinterpret_cast<uintptr_t>(dev_scratch) % kAlign) != 0)
+    return TOPOEP_ERR_WORKSPACE;
+  if (((size_t)h->d.P + 1) * sizeof(int) > 48 * 1024 ||
+      pos_rank_smem_bytes(h->d, h->tile_ids) > 227 * 1024)
+    return TOPOEP_ERR_SMEM;
+  PosParams p;
+  p.d = h->d;
+  p.ws = h->ws;
+  p.token_replica = dev_token_replica;
+  p.out_send_pos = dev_send_pos;
+  p.out_recv_pos = dev_recv_pos;
+  p.out_instance_offsets = dev_instance_offsets;
+  p.n_ids = tokens_per_rank * h->d.k;
+  p.tile_ids = h->tile_ids;
+  p.tiles = std::max(1, (p.n_ids + p.tile_ids - 1) / p.tile_ids);
+  const size_t rows = (size_t)batch * h->d.R;
+  char* base = static_cast<char*>(dev_scratch);
+  p.scratch_status = reinterpret_cast<uint32_t*>(base);
+  p.pos_a = reinterpret_cast<int32_t*>(base + kAlign);
+  p.pos_b = reinterpret_cast<int32_t*>(base + kAlign + align_up(4 * rows * h->d.P));
+  p.pos_cnt = reinterpret_cast<int32_t*>(base + kAlign + 2 * align_up(4 * rows * h->d.P));
+  cudaError_t e = cudaSuccess;
+  if (pos_rank_smem_bytes(h->d, kMaxTileIds) != h->dispatch_smem) {
+    // first use: opt in to the shared memory the ranking kernel needs (host-side attribute only)
+    e = configure_dispatch(pos_rank_smem_bytes(h->d, kMaxTileIds));
+    if (e == cudaSuccess) h->dispatch_smem = pos_rank_smem_bytes(h->d, kMaxTileIds);
+  }
+  if (e == cudaSuccess) e = launch_dispatch(p, batch, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
 }
 
 int topoep_summary(topoep_handle_t h, int batch, topoep_summary_t* dev_out, topoep_stream_t stream) {

@@ -1,0 +1,209 @@
+// Dispatch permutation: where every assignment sits in its source rank's send buffer and in its
+// destination rank's receive buffer (the step right after the planning path; the paper's
+// "DeepEP dispatch and combine" paragraph leaves the buffer layout to its dispatch library, so
+// the layout is defined here, in include/topoep.h).
+//
+//   send buffer of source s : ordered by (physical instance p, flat index) -- p ascends with
+//                             (destination rank, instance), so each destination's block is
+//                             contiguous and starts at the plan's send offset;
+//   recv buffer of rank r   : ordered by (instance, source rank, flat index) -- every instance's
+//                             tokens contiguous (grouped GEMM), sources in rank order inside.
+//
+// Both are stable sorts of token_replica, done as counting sorts with P bins in three kernels:
+//   1. per-tile histogram of p            (the histogram kernel, P bins instead of E)
+//   2. pos_prefix_kernel, CTA = (plan, source): prefix over tiles of the tile counts, and the
+//      per-(source, instance) bases A0[p] (send) and B0[p] (receive) from the plan's q and U
+//   3. pos_rank_kernel, CTA = tile: stable rank of each assignment among the tile's equal p
+//      (__match_any_sync inside a warp, per-warp counters scanned across warps), added to the
+//      bases.
+// Ranks come from counts and prefix sums only, never from atomic arrival order.  Kernel 3 is
+// bound by the issue cost of match.any on B200 (~160-250 cycles per warp instruction), not by
+// HBM; it is off the planning path.
+#include "topoep_internal.cuh"
+
+namespace topoep {
+
+namespace {
+
+constexpr int kPosThreads = 256;
+
+__global__ void __launch_bounds__(kPosThreads) pos_prefix_kernel(const PosParams p) {
+  extern __shared__ int sm[];   // [P] q row, then [P+1] scratch
+  const Dims d = p.d;
+  const int R = d.R, P = d.P, s_phys = d.s_phys;
+  const int s = blockIdx.x, b = blockIdx.y;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+  int* qrow = sm;
+  int* warp_tot = sm + P;
+  const size_t row = (size_t)b * R + s;
+  for (int i = tid; i < P; i += nt) qrow[i] = p.ws.q[row * P + i];
+  __syncthreads();
+
+  // A0[p] = number of assignments of source s executed on instances below p (exclusive scan)
+  int32_t* A0 = p.pos_a + row * P;
+  {
+    const int chunk = (P + nt - 1) / nt;
+    const int i0 = min(P, tid * chunk), i1 = min(P, i0 + chunk);
+    int sum = 0;
+    for (int i = i0; i < i1; ++i) sum += qrow[i];
+    int total;
+    int ex = warp_exclusive_scan(sum, lane, &total);
+    if (lane == 0) warp_tot[warp] = total;
+    __syncthreads();
+    for (int w = 0; w < warp; ++w) ex += warp_tot[w];
+    for (int i = i0; i < i1; ++i) { A0[i] = ex; ex += qrow[i]; }
+  }
+  // B0[p] = start of instance p's segment in its rank's receive buffer + assignments of lower
+  // source ranks on p
+  int32_t* B0 = p.pos_b + row * P;
+  const int32_t* U = p.ws.inst_counts + (size_t)b * P;
+  for (int i = tid; i < P; i += nt) {
+    const int r = i / s_phys;
+    int acc = 0;
+    for (int j = r * s_phys; j < i; ++j) acc += U[j];                        // instance offset
+    const int32_t* col = p.ws.q + (size_t)b * R * P + i;
+    for (int s2 = 0; s2 < s; ++s2) acc += col[(size_t)s2 * P];               // lower sources
+    B0[i] = acc;
+  }
+  if (s == 0 && p.out_instance_offsets) {
+    int32_t* off = p.out_instance_offsets + (size_t)b * R * (s_phys + 1);
+    for (int i = tid; i < R * (s_phys + 1); i += nt) {
+      const int r = i / (s_phys + 1), l = i - r * (s_phys + 1);
+      int acc = 0;
+      for (int j = 0; j < l; ++j) acc += U[r * s_phys + j];
+      off[i] = acc;
+    }
+  }
+  // exclusive prefix over tiles of the per-tile counts, in place
+  int32_t* cnt = p.pos_cnt + row * (size_t)p.tiles * P;
+  for (int i = tid; i < P; i += nt) {
+    int run = 0;
+    for (int t0 = 0; t0 < p.tiles; t0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? cnt[(size_t)(t0 + u) * P + i] : 0;
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (t0 + u < p.tiles) { cnt[(size_t)(t0 + u) * P + i] = run; run += v[u]; }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(const PosParams p) {
+  extern __shared__ int sm[];   // base_a[P], base_b[P], wh[nwarps][P]
+  const Dims d = p.d;
+  const int P = d.P;
+  const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+  int* base_a = sm;
+  int* base_b = sm + P;
+  int* wh = sm + 2 * P;
+  const size_t row = (size_t)b * d.R + s;
+  const int begin = tile * p.tile_ids;
+  const int count = min(p.tile_ids, p.n_ids - begin);
+  const int32_t* tr = p.token_replica + row * (size_t)p.n_ids + begin;
+
+  // this warp's 512 assignments: step j covers 32 consecutive ones, so (step, lane) is flat order
+  const int wbase = warp * (32 * kIdsPerThread);
+  int x[kIdsPerThread];
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread; ++j) {
+    const int i = wbase + j * 32 + lane;
+    x[j] = i < count ? __ldg(tr + i) : -1;
+  }
+  const int32_t* tp = p.pos_cnt + (row * (size_t)p.tiles + tile) * P;
+  for (int i = tid; i < P; i += nt) {
+    const int t = tp[i];
+    base_a[i] = p.pos_a[row * P + i] + t;
+    base_b[i] = p.pos_b[row * P + i] + t;
+  }
+  for (int i = tid; i < nwarps * P; i += nt) wh[i] = 0;
+  __syncthreads();
+
+  int* my = wh + warp * P;
+  int rho[kIdsPerThread];
+  const unsigned lt = lanemask_lt();
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread; ++j) {
+    const int v = x[j];
+    const bool valid = v >= 0 && v < P;
+    const unsigned mask = __ballot_sync(0xffffffffu, valid);
+    int r = 0;
+    if (valid) {
+      const unsigned peers = __match_any_sync(mask, v);
+      const int leader = __ffs(peers) - 1;
+      int old = 0;
+      if (lane == leader) { old = my[v]; my[v] = old + __popc(peers); }
+      old = __shfl_sync(peers, old, leader);
+      r = old + __popc(peers & lt);
+    }
+    rho[j] = r;
+    __syncwarp();
+  }
+  __syncthreads();
+  // per-warp totals -> exclusive prefix over the warps of the tile
+  for (int i = tid; i < P; i += nt) {
+    int run = 0;
+    for (int w = 0; w < nwarps; ++w) {
+      const int t = wh[w * P + i];
+      wh[w * P + i] = run;
+      run += t;
+    }
+  }
+  __syncthreads();
+  int32_t* send = p.out_send_pos + row * (size_t)p.n_ids + begin;
+  int32_t* recv = p.out_recv_pos + row * (size_t)p.n_ids + begin;
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread; ++j) {
+    const int i = wbase + j * 32 + lane;
+    const int v = x[j];
+    int a = -1, c = -1;
+    if (v >= 0 && v < P) {
+      const int k = rho[j] + my[v];
+      a = base_a[v] + k;
+      c = base_b[v] + k;
+    }
+    if (i < count) { send[i] = a; recv[i] = c; }
+  }
+}
+
+}  // namespace
+
+size_t pos_rank_smem_bytes(const Dims& d, int tile_ids) {
+  return sizeof(int) * ((size_t)2 * d.P + (size_t)(tile_ids / 512) * d.P);
+}
+
+cudaError_t configure_dispatch(size_t smem) {
+  return cudaFuncSetAttribute(pos_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)smem);
+}
+
+cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) {
+  // 1. per-tile histogram of the instance ids: the histogram kernel with P bins
+  HistParams hp = {};
+  hp.d = p.d;
+  hp.d.E = p.d.P;
+  hp.ws = p.ws;
+  hp.ws.tile_cnt = p.pos_cnt;
+  hp.ids = p.token_replica;
+  hp.n_ids = p.n_ids;
+  hp.tiles = p.tiles;
+  hp.max_tiles = p.tiles;
+  hp.tile_ids = p.tile_ids;
+  hp.vec_ok = (p.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.token_replica) & 15u) == 0);
+  hp.ws.status = p.scratch_status;   // a stray instance id must not raise the plan's BAD_ID flag
+  cudaError_t e = launch_hist(hp, batch, 0, stream);
+  if (e != cudaSuccess) return e;
+  // 2. bases and tile prefixes
+  pos_prefix_kernel<<<dim3(p.d.R, batch), kPosThreads,
+                      sizeof(int) * ((size_t)p.d.P + kPosThreads / 32 + 1), stream>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  // 3. stable ranks inside the tile
+  const dim3 grid(p.tiles, p.d.R, batch);
+  const dim3 block(p.tile_ids / kIdsPerThread);
+  pos_rank_kernel<<<grid, block, pos_rank_smem_bytes(p.d, p.tile_ids), stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace topoep

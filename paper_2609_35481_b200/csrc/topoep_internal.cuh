@@ -124,6 +124,20 @@ struct RerouteParams {
   int vec_ok;
 };
 
+struct PosParams {
+  Dims d;
+  Workspace ws;
+  const int32_t* token_replica;   // [B][R][n_ids]
+  int32_t* out_send_pos;          // [B][R][n_ids]
+  int32_t* out_recv_pos;          // [B][R][n_ids]
+  int32_t* out_instance_offsets;  // [B][R][S_phys+1] or NULL
+  int32_t* pos_cnt;               // scratch [B][R][tiles][P]: tile counts, then prefixes over tiles
+  int32_t* pos_a;                 // scratch [B][R][P] send base of (source, instance)
+  int32_t* pos_b;                 // scratch [B][R][P] receive base of (source, instance)
+  uint32_t* scratch_status;       // scratch word for the histogram kernel's flag
+  int n_ids, tiles, tile_ids;
+};
+
 struct SummaryParams {
   Dims d;
   Workspace ws;
@@ -136,15 +150,18 @@ size_t hist_smem_bytes(const Dims& d);
 size_t solve_smem_bytes(const Dims& d);
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
+size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
 
 cudaError_t configure_solve(size_t smem);
 cudaError_t configure_route(size_t smem);
 cudaError_t configure_reroute(size_t smem);
+cudaError_t configure_dispatch(size_t smem);
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream);
 cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_route(const RouteParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream);
+cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_summary(const SummaryParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_empty(int count, cudaStream_t stream);
 

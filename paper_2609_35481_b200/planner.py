@@ -92,6 +92,24 @@ class Planner:
             raise B.TopoEPError(rc)
         return out
 
+    def dispatch_positions(self, token_replica: torch.Tensor, stream=None):
+        """(send_pos, recv_pos, instance_offsets) of the plan that produced token_replica."""
+        Bn, R, T, k = token_replica.shape
+        i32 = dict(dtype=torch.int32, device=self.device)
+        send = torch.empty((Bn, R, T, k), **i32)
+        recv = torch.empty((Bn, R, T, k), **i32)
+        inst_off = torch.empty((Bn, R, self.s_phys + 1), **i32)
+        nbytes = B.topoep_dispatch_scratch_bytes(self.handle, T, Bn)
+        scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        ptr = (scratch.data_ptr() + 255) // 256 * 256
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = B.topoep_dispatch_positions(self.handle, token_replica, T, Bn, send, recv, inst_off,
+                                         ptr, nbytes, st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        st.synchronize()   # the scratch tensor is released when this returns
+        return send, recv, inst_off
+
     def histogram(self, topk_ids: torch.Tensor, stream=None) -> torch.Tensor:
         Bn, R, T, k = topk_ids.shape
         omega = torch.empty((Bn, R, self.E), dtype=torch.int32, device=self.device)

@@ -7,7 +7,7 @@ import torch
 
 import oracle as orc
 import workloads as wl
-from plan_checks import check_plan
+from plan_checks import check_plan, dispatch_positions_by_sorting
 from gpu_common import assert_same, make_planner, oracle_config, parity, run_gpu
 
 pytestmark = pytest.mark.gpu
@@ -243,6 +243,53 @@ def test_stage_entry_points_equal_the_fused_plan():
                  "instance_counts"):
         assert torch.equal(getattr(out, name), getattr(fused, name)), name
     assert pl.status() == 0
+
+
+# ---- dispatch permutation (the step after the path) --------------------------------------------
+@pytest.mark.parametrize("name,over,batch", [
+    ("tiny", dict(slots_per_rank=2), 2),
+    ("mid", dict(tokens_per_rank=777, slots_per_rank=3, top_k=5), 2),
+    ("dsv3", dict(tokens_per_rank=1024), 1),
+])
+def test_dispatch_positions_match_the_oracle(name, over, batch):
+    w = wl.CONFIGS[name].replace(**over)
+    ids = wl.make_topk_ids(w, seed=41, batch=batch).copy()
+    ids[0, 1, 3:20, :] = -1
+    pl = make_planner(w, max_batch=batch)
+    out = pl.plan(torch.from_numpy(ids).to(pl.device))
+    send, recv, off = pl.dispatch_positions(out.token_replica)
+    cfg = oracle_config(w)
+    ref = orc.plan(cfg, ids)
+    assert np.array_equal(out.token_replica.cpu().numpy(), ref.token_replica)
+    for b in range(batch):
+        s_ref, r_ref, o_ref = orc.dispatch_positions(cfg, ref.token_replica[b])
+        assert np.array_equal(send[b].cpu().numpy(), s_ref)
+        assert np.array_equal(recv[b].cpu().numpy(), r_ref)
+        assert np.array_equal(off[b].cpu().numpy(), o_ref)
+    assert pl.status() == 0
+
+
+@pytest.mark.parametrize("name", ["dsv3", "scaleout"])
+def test_dispatch_positions_full_size_are_the_sorted_order(name):
+    # at full size the permutation is checked against its definition: a stable sort
+    w = wl.CONFIGS[name]
+    ids = wl.make_topk_ids(w, seed=43)
+    pl = make_planner(w)
+    out = pl.plan(torch.from_numpy(ids).to(pl.device))
+    send, recv, off = pl.dispatch_positions(out.token_replica)
+    tr = out.token_replica[0].cpu().numpy()
+    s2, r2, o2 = dispatch_positions_by_sorting(w.ranks, pl.s_phys, tr)
+    assert np.array_equal(send[0].cpu().numpy().reshape(w.ranks, -1), s2)
+    assert np.array_equal(recv[0].cpu().numpy().reshape(w.ranks, -1), r2)
+    assert np.array_equal(off[0].cpu().numpy(), o2)
+    # a destination's block in a source's send buffer starts at the plan's send offset
+    send_off = out.dispatch_offsets[0, 0].cpu().numpy()
+    trf = tr.reshape(w.ranks, -1)
+    for s in (0, w.ranks - 1):
+        for r in (0, w.ranks // 2, w.ranks - 1):
+            sel = (trf[s] // pl.s_phys == r) & (trf[s] >= 0)
+            if sel.any():
+                assert s2[s][sel].min() == send_off[s, r]
 
 
 # ---- capture: the plan is enqueue-only ---------------------------------------------------------
