@@ -342,6 +342,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="dsv3_batched", choices=sorted(wl.CONFIGS))
     ap.add_argument("--no-single-plan", action="store_true")
+    ap.add_argument("--no-dispatch", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override plans per step")
     ap.add_argument("--impl", default="topoep", choices=["topoep", "reference"])
     ap.add_argument("--tile-ids", type=int, default=0)
@@ -412,6 +413,43 @@ def main():
     ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
     e2e_value = job_throughput(world, w.assignments, k_e2e, ms_e2e)
 
+    # ---- the step after the path: dispatch permutation of the same batch (reported, not timed
+    # into `value`)
+    dispatch = None
+    if not args.no_dispatch:
+        pl0 = s0["pl"]
+        nb = B.topoep_dispatch_scratch_bytes(pl0.handle, w.tokens_per_rank, w.batch)
+        scratch = torch.empty(nb + 256, dtype=torch.uint8, device=dev)
+        sptr = (scratch.data_ptr() + 255) // 256 * 256
+        send = torch.empty_like(o.token_replica)
+        recv = torch.empty_like(o.token_replica)
+        ioff = torch.empty((w.batch, w.ranks, pl0.s_phys + 1), dtype=torch.int32, device=dev)
+
+        def dispatch_once():
+            rc = B.topoep_dispatch_positions(pl0.handle, o.token_replica, w.tokens_per_rank, w.batch,
+                                             send, recv, ioff, sptr, nb, stream.cuda_stream)
+            assert rc == 0, rc
+
+        with torch.cuda.stream(stream):
+            s0["pl"].plan(s0["ids"], o, stream=stream)
+            for _ in range(3):
+                dispatch_once()
+        n_d = 10
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        with torch.cuda.stream(stream):
+            d0.record(stream)
+            for _ in range(n_d):
+                dispatch_once()
+            d1.record(stream)
+        barrier()
+        us = max_over_ranks(d0.elapsed_time(d1), world, dev) / n_d * 1e3
+        dispatch = {"us_per_call": round(us, 2), "us_per_layer_plan": round(us / w.batch, 3),
+                    "bytes_per_assignment": 16,
+                    "hbm_frac": round(16 * w.assignments / (us * 1e-6) / 1e9 / measured_peak_gbs()[0], 4),
+                    "note": "send/recv positions; ranking kernel is bound by warp-match issue cost"}
+        del scratch, send, recv, ioff
+
     # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol
     single = None
     if w.batch > 1 and not args.no_single_plan:
@@ -477,6 +515,8 @@ def main():
             "roofline": roofline}
     if single is not None:
         line["single_plan"] = single
+    if dispatch is not None:
+        line["dispatch_positions"] = dispatch
 
     if rank == 0 and not args.no_cpu_baseline:
         sample_ids = s0["ids_host"][:min(w.batch, 8)]

@@ -411,10 +411,10 @@ int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replic
   p.pos_b = reinterpret_cast<int32_t*>(base + kAlign + align_up(4 * rows * h->d.P));
   p.pos_cnt = reinterpret_cast<int32_t*>(base + kAlign + 2 * align_up(4 * rows * h->d.P));
   cudaError_t e = cudaSuccess;
-  if (pos_rank_smem_bytes(h->d, kMaxTileIds) != h->dispatch_smem) {
-    // first use: opt in to the shared memory the ranking kernel needs (host-side attribute only)
-    e = configure_dispatch(pos_rank_smem_bytes(h->d, kMaxTileIds));
-    if (e == cudaSuccess) h->dispatch_smem = pos_rank_smem_bytes(h->d, kMaxTileIds);
+  if (!h->dispatch_smem) {
+    // first use: opt in to the shared memory the kernels need (host-side attribute only)
+    e = configure_dispatch(h->d);
+    if (e == cudaSuccess) h->dispatch_smem = 1;
   }
   if (e == cudaSuccess) e = launch_dispatch(p, batch, stream);
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }

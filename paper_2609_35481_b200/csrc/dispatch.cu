@@ -28,7 +28,7 @@ namespace {
 constexpr int kPosThreads = 256;
 
 __global__ void __launch_bounds__(kPosThreads) pos_prefix_kernel(const PosParams p) {
-  extern __shared__ int sm[];   // [P] q row, then [P+1] scratch
+  extern __shared__ int sm[];   // [P] q row, per-warp totals, [P] instance counts
   const Dims d = p.d;
   const int R = d.R, P = d.P, s_phys = d.s_phys;
   const int s = blockIdx.x, b = blockIdx.y;
@@ -54,15 +54,24 @@ __global__ void __launch_bounds__(kPosThreads) pos_prefix_kernel(const PosParams
     for (int i = i0; i < i1; ++i) { A0[i] = ex; ex += qrow[i]; }
   }
   // B0[p] = start of instance p's segment in its rank's receive buffer + assignments of lower
-  // source ranks on p
+  // source ranks on p (loads issued eight at a time)
   int32_t* B0 = p.pos_b + row * P;
+  int* Us = warp_tot + nw + 1;   // [P] instance counts U
   const int32_t* U = p.ws.inst_counts + (size_t)b * P;
+  for (int i = tid; i < P; i += nt) Us[i] = U[i];
+  __syncthreads();
   for (int i = tid; i < P; i += nt) {
     const int r = i / s_phys;
     int acc = 0;
-    for (int j = r * s_phys; j < i; ++j) acc += U[j];                        // instance offset
+    for (int j = r * s_phys; j < i; ++j) acc += Us[j];                       // instance offset
     const int32_t* col = p.ws.q + (size_t)b * R * P + i;
-    for (int s2 = 0; s2 < s; ++s2) acc += col[(size_t)s2 * P];               // lower sources
+    for (int s0 = 0; s0 < s; s0 += 8) {                                      // lower sources
+      int v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = s0 + u < s ? __ldg(col + (size_t)(s0 + u) * P) : 0;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc += v[u];
+    }
     B0[i] = acc;
   }
   if (s == 0 && p.out_instance_offsets) {
@@ -70,7 +79,7 @@ __global__ void __launch_bounds__(kPosThreads) pos_prefix_kernel(const PosParams
     for (int i = tid; i < R * (s_phys + 1); i += nt) {
       const int r = i / (s_phys + 1), l = i - r * (s_phys + 1);
       int acc = 0;
-      for (int j = 0; j < l; ++j) acc += U[r * s_phys + j];
+      for (int j = 0; j < l; ++j) acc += Us[r * s_phys + j];
       off[i] = acc;
     }
   }
@@ -173,9 +182,16 @@ size_t pos_rank_smem_bytes(const Dims& d, int tile_ids) {
   return sizeof(int) * ((size_t)2 * d.P + (size_t)(tile_ids / 512) * d.P);
 }
 
-cudaError_t configure_dispatch(size_t smem) {
-  return cudaFuncSetAttribute(pos_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)smem);
+size_t pos_prefix_smem_bytes(const Dims& d) {
+  return sizeof(int) * ((size_t)2 * d.P + kPosThreads / 32 + 1);
+}
+
+cudaError_t configure_dispatch(const Dims& d) {
+  cudaError_t e = cudaFuncSetAttribute(pos_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)pos_rank_smem_bytes(d, kMaxTileIds));
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(pos_prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)pos_prefix_smem_bytes(d));
 }
 
 cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) {
@@ -195,8 +211,7 @@ cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) 
   cudaError_t e = launch_hist(hp, batch, 0, stream);
   if (e != cudaSuccess) return e;
   // 2. bases and tile prefixes
-  pos_prefix_kernel<<<dim3(p.d.R, batch), kPosThreads,
-                      sizeof(int) * ((size_t)p.d.P + kPosThreads / 32 + 1), stream>>>(p);
+  pos_prefix_kernel<<<dim3(p.d.R, batch), kPosThreads, pos_prefix_smem_bytes(p.d), stream>>>(p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // 3. stable ranks inside the tile

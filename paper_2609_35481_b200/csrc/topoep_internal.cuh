@@ -155,7 +155,7 @@ size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
 cudaError_t configure_solve(size_t smem);
 cudaError_t configure_route(size_t smem);
 cudaError_t configure_reroute(size_t smem);
-cudaError_t configure_dispatch(size_t smem);
+cudaError_t configure_dispatch(const Dims& d);
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream);
 cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream);
