@@ -16,7 +16,7 @@ namespace topoep {
 constexpr int kIdsPerThread = 16;   // every histogram / reroute thread owns 16 ids of its tile
 constexpr int kMinTileIds = 1024;
 constexpr int kMaxTileIds = 8192;
-constexpr int kSolveThreads = 512;
+constexpr int kSolveThreads = 512;   // at most; large batches launch 256 (more CTAs per SM)
 constexpr int kRouteThreads = 256;
 constexpr int kSplitCap = 16;       // split experts the reroute kernel ranks per pass
 
