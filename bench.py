@@ -246,6 +246,8 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
             pl.set_tuning(B.KNOB_TILE_IDS, args.tile_ids)
         if args.hist_mode >= 0:
             pl.set_tuning(B.KNOB_HIST_MODE, args.hist_mode)
+        if args.pdl >= 0:
+            pl.set_tuning(B.KNOB_PDL, args.pdl)
         ids_dev = torch.from_numpy(ids).to(dev)
         sets.append({"pl": pl, "ids_host": ids, "ids": ids_dev,
                      "out": pl.alloc_outputs(w.batch, w.tokens_per_rank)})
@@ -347,6 +349,7 @@ def main():
     ap.add_argument("--impl", default="topoep", choices=["topoep", "reference"])
     ap.add_argument("--tile-ids", type=int, default=0)
     ap.add_argument("--hist-mode", type=int, default=-1)
+    ap.add_argument("--pdl", type=int, default=-1)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

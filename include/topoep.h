@@ -119,8 +119,12 @@ enum {
 enum {
   TOPOEP_KNOB_TILE_IDS = 0,     /* ids per histogram / reroute tile: 1024..8192,
                                    power of two                                   */
-  TOPOEP_KNOB_HIST_MODE = 1     /* 0 = plain shared-memory atomics (default),
+  TOPOEP_KNOB_HIST_MODE = 1,    /* 0 = plain shared-memory atomics (default),
                                    1 = warp-aggregated (__match_any_sync) atomics */
+  TOPOEP_KNOB_PDL = 2           /* 1 (default): the kernels after the histogram are
+                                   launched with programmatic dependent launch and
+                                   overlap their predecessor's tail; 0: plain
+                                   stream order                                   */
 };
 
 /*

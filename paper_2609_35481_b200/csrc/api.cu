@@ -15,7 +15,7 @@ struct topoep_ctx {
   topoep_cost_params cost;
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
-  int tile_ids, hist_mode;
+  int tile_ids, hist_mode, pdl;
   size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
   int max_tiles;
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
@@ -88,6 +88,9 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   p.tiles = std::max(1, (p.n_ids + h->tile_ids - 1) / h->tile_ids);
   p.max_tiles = h->max_tiles;
   p.vec_ok = (p.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0);
+  // The first kernel of the chain is never launched early: whatever produced the ids (a router
+  // kernel, a copy) must be complete before it reads them.
+  p.pdl = 0;
   return p;
 }
 
@@ -95,6 +98,7 @@ OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, in
   OmegaParams op;
   op.d = h->d;
   op.ws = h->ws;
+  op.pdl = h->pdl;
   op.src_omega = src;
   op.out_omega = out_omega;
   op.tiles = tiles;
@@ -172,6 +176,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->max_batch = max_batch;
   h->tile_ids = 4096;
   h->hist_mode = 0;
+  h->pdl = 1;
   h->dispatch_smem = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
@@ -257,6 +262,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   SolveParams sp;
   sp.d = h->d;
   sp.ws = h->ws;
+  sp.pdl = h->pdl;
   sp.token_bytes = h->cost.token_bytes;
   sp.expert_bytes = h->cost.expert_bytes;
   sp.max_iters = h->max_iters;
@@ -275,6 +281,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
     RouteParams rp;
     rp.d = h->d;
     rp.ws = h->ws;
+    rp.pdl = h->pdl;
     rp.out_offsets = offsets;
     rp.max_tiles = h->max_tiles;
     rp.tiles = 0;
@@ -294,6 +301,7 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   RerouteParams rp;
   rp.d = h->d;
   rp.ws = h->ws;
+  rp.pdl = h->pdl;
   rp.ids = ids;
   rp.out_token_replica = token_replica;
   rp.n_ids = T * h->d.k;
@@ -477,6 +485,10 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_HIST_MODE:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->hist_mode = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_PDL:
+      if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
+      h->pdl = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

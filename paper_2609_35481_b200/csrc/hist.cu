@@ -63,6 +63,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
     count_one<MODE>(cnt, x[j].z, E, lane, mx);
     count_one<MODE>(cnt, x[j].w, E, lane, mx);
   }
+  pdl_wait();   // the ids are nobody's output; everything written below may still be in use
   if (mx > (unsigned)E) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);
   __syncthreads();
   int32_t* out = p.ws.tile_cnt + (row * (size_t)p.max_tiles + tile) * E;
@@ -83,9 +84,10 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
   const int s = dm * G + g;
   const size_t row = (size_t)b * R + s;
   int sum = 0, mi = 0;
+  if (on && p.ws.omega_m)   // row of the transposed copy: static tables, fetched before the wait
+    mi = __ldg(p.ws.main_rank + e) * p.d.e_loc + __ldg(p.ws.main_local + e);
+  pdl_wait();
   if (on) {
-    if (p.ws.omega_m)   // row of the transposed copy; fetched alongside the counts
-      mi = __ldg(p.ws.main_rank + e) * p.d.e_loc + __ldg(p.ws.main_local + e);
     if (p.src_omega) {
       sum = __ldg(p.src_omega + row * E + e);
     } else {
@@ -118,20 +120,18 @@ cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t s
   const size_t smem = hist_smem_bytes(p.d);
   const bool wide = p.tile_ids >= 2048;   // 32 ids per thread once the CTA still has 2+ warps
   const dim3 block(p.tile_ids / (wide ? 32 : 16));
+  const bool pdl = p.pdl != 0;
   if (mode == 1) {
-    if (wide) hist_kernel<1, 32><<<grid, block, smem, stream>>>(p);
-    else hist_kernel<1, 16><<<grid, block, smem, stream>>>(p);
-  } else {
-    if (wide) hist_kernel<0, 32><<<grid, block, smem, stream>>>(p);
-    else hist_kernel<0, 16><<<grid, block, smem, stream>>>(p);
+    return wide ? launch_kernel(hist_kernel<1, 32>, grid, block, smem, stream, pdl, p)
+                : launch_kernel(hist_kernel<1, 16>, grid, block, smem, stream, pdl, p);
   }
-  return cudaGetLastError();
+  return wide ? launch_kernel(hist_kernel<0, 32>, grid, block, smem, stream, pdl, p)
+              : launch_kernel(hist_kernel<0, 16>, grid, block, smem, stream, pdl, p);
 }
 
 cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream) {
   const dim3 grid((p.d.E + 4 * p.epw - 1) / (4 * p.epw), p.d.M, batch);
-  omega_kernel<<<grid, 128, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(omega_kernel, grid, dim3(128), 0, stream, p.pdl != 0, p);
 }
 
 cudaError_t launch_empty(int count, cudaStream_t stream) {

@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   int4 x[kIdsPerThread / 4];
 #pragma unroll
   for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+  pdl_wait();   // the ids above are nobody's output; the tables below are the route kernel's
   const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
   const int32_t* rec = p.ws.split_rec + row * (size_t)rl.ints;
   const int32_t* g_route = p.ws.route + row * E;
@@ -259,9 +260,9 @@ size_t reroute_smem_bytes(const Dims& d, int tile_ids) { return reroute_layout(d
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.tiles, p.d.R, batch);
   const dim3 block(p.tile_ids / kIdsPerThread);
-  if (p.vec_ok) reroute_kernel<true><<<grid, block, reroute_smem_bytes(p.d, p.tile_ids), stream>>>(p);
-  else reroute_kernel<false><<<grid, block, reroute_smem_bytes(p.d, p.tile_ids), stream>>>(p);
-  return cudaGetLastError();
+  const size_t smem = reroute_smem_bytes(p.d, p.tile_ids);
+  return p.vec_ok ? launch_kernel(reroute_kernel<true>, grid, block, smem, stream, p.pdl != 0, p)
+                  : launch_kernel(reroute_kernel<false>, grid, block, smem, stream, p.pdl != 0, p);
 }
 
 cudaError_t configure_reroute(size_t smem) {

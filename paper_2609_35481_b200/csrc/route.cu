@@ -96,14 +96,15 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
 
   const size_t row = (size_t)b * R + s;
   const int RN = R * N;
-  // one round of independent loads
-  for (int i = tid; i < RN; i += nt) rm[i] = p.ws.replica_map[(size_t)b * RN + i];
-  for (int i = tid; i < P; i += nt) qrow[i] = p.ws.q[row * P + i];
+  // static tables before the solver is known to be done, its results after
   for (int e = tid; e < E; e += nt) {
     const int r = p.ws.main_rank[e];
     mr[e] = r;
     ml[e] = r * s_phys + p.ws.main_local[e];
   }
+  pdl_wait();
+  for (int i = tid; i < RN; i += nt) rm[i] = p.ws.replica_map[(size_t)b * RN + i];
+  for (int i = tid; i < P; i += nt) qrow[i] = p.ws.q[row * P + i];
   for (int r = tid; r < R; r += nt) crow[r] = p.ws.counts[row * R + r];
   __syncthreads();
 
@@ -224,8 +225,8 @@ size_t route_smem_bytes(const Dims& d) { return route_layout(d).total; }
 
 cudaError_t launch_route(const RouteParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.d.R, batch);
-  route_kernel<<<grid, kRouteThreads, route_smem_bytes(p.d), stream>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(route_kernel, grid, dim3(kRouteThreads), route_smem_bytes(p.d), stream,
+                       p.pdl != 0, p);
 }
 
 cudaError_t configure_route(size_t smem) {

@@ -98,11 +98,10 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
 
   const int32_t* om_m = p.ws.omega_m + (size_t)b * R * e_loc * R;   // rows = main instances
 
-  // ---- round 1 of asynchronous copies ---------------------------------------------------------
-  copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
+  // ---- round 1 of asynchronous copies: static tables first, then (once the omega kernel is
+  // done) the demand and this domain's main columns
   copy_async(mrank, p.ws.main_rank, E, tid, nt);
   copy_async(mlocal, p.ws.main_local, E, tid, nt);
-  copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
   for (int i = tid; i < G * e_loc; i += nt) {
     const int g = i / e_loc, l = i - g * e_loc;
     cp_async4(col_expert + g * s_phys + l, p.ws.main_inst_expert + (size_t)(dm * G + g) * e_loc + l);
@@ -112,6 +111,9 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   for (int c = tid; c < C; c += nt) col_cr[c] = p.cost_rank_intra;
   for (int s = tid; s < R; s += nt) sdom[s] = (short)(s / G);
   if (tid < G) used[tid] = 0;
+  pdl_wait();
+  copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
+  copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
   cp_async_wait_all();
   __syncthreads();
 
@@ -407,8 +409,8 @@ cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream) {
   // few CTAs: 512 threads shorten each CTA's phases (33.6 vs 35.1 us per single plan); enough
   // CTAs to fill the GPU twice over: 256 threads fit more CTAs per SM (91 vs 106 us per 232 plans)
   const int threads = (long long)p.d.M * batch >= 2 * 148 ? 256 : kSolveThreads;
-  solve_kernel<<<grid, threads, solve_smem_bytes(p.d), stream>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(solve_kernel, grid, dim3(threads), solve_smem_bytes(p.d), stream,
+                       p.pdl != 0, p);
 }
 
 cudaError_t configure_solve(size_t smem) {
