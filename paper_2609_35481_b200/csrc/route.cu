@@ -20,7 +20,7 @@ namespace topoep {
 
 namespace {
 
-struct RouteLayout { size_t rm, qrow, mr, ml, nz, single, sidx, seg, cum, crow, split_e, warp_tot, total; };
+struct RouteLayout { size_t rm, qrow, mr, ml, nz, single, sidx, seg, crow, split_e, warp_tot, total; };
 
 __host__ __device__ inline RouteLayout route_layout(const Dims& d) {
   RouteLayout o;
@@ -33,7 +33,6 @@ __host__ __device__ inline RouteLayout route_layout(const Dims& d) {
   o.single = at;   at += sizeof(int) * (size_t)d.E;
   o.sidx = at;     at += sizeof(int) * (size_t)(d.E + 1);
   o.seg = at;      at += sizeof(int) * (size_t)(d.E + 1);
-  o.cum = at;      at += sizeof(int) * (size_t)d.P;
   o.crow = at;     at += sizeof(int) * (size_t)d.R;
   o.split_e = at;  at += sizeof(int) * (size_t)d.E;
   o.warp_tot = at; at += sizeof(int) * 2 * (kRouteThreads / 32);
@@ -89,7 +88,6 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   int* single = reinterpret_cast<int*>(smem + lay.single); // [E]
   int* sidx = reinterpret_cast<int*>(smem + lay.sidx);     // [E+1] split index of e
   int* seg = reinterpret_cast<int*>(smem + lay.seg);       // [E+1] list start of e (split only)
-  int* cum = reinterpret_cast<int*>(smem + lay.cum);       // [P]   quotas in list order
   int* crow = reinterpret_cast<int*>(smem + lay.crow);     // [R]   counts[s][.]
   int* split_e = reinterpret_cast<int*>(smem + lay.split_e); // [E]   expert of split index i
   int* warp_tot = reinterpret_cast<int*>(smem + lay.warp_tot);
@@ -140,33 +138,39 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     rec[rl.seg + n_split] = n_list;
   }
 
-  // Split lists: position of an instance = number of nonzero instances of e on lower ranks.
+  // Split lists: position of an instance = number of nonzero instances of e on lower ranks; its
+  // cumulative quota = its own share plus the shares of those.
   for (int e = tid; e < E; e += nt) {
     if (nz[e] < 2 || qrow[ml[e]] <= 0) continue;
-    int pos = 0;
-    for (int i = 0; i < mr[e] * N; ++i)
-      pos += (rm[i] == e && qrow[(i / N) * s_phys + e_loc + i % N] > 0) ? 1 : 0;
-    cum[seg[e] + pos] = qrow[ml[e]];
+    int pos = 0, below = 0;
+    const int lim = mr[e] * N;
+    for (int i = 0, r = 0, j = 0; i < lim; ++i) {
+      const int v = qrow[r * s_phys + e_loc + j];
+      if (rm[i] == e && v > 0) { ++pos; below += v; }
+      if (++j == N) { j = 0; ++r; }
+    }
+    rec[rl.cum + seg[e] + pos] = below + qrow[ml[e]];
     rec[rl.inst + seg[e] + pos] = ml[e];
   }
   for (int i = tid; i < RN; i += nt) {
     const int e = rm[i];
     if (e < 0 || nz[e] < 2) continue;
-    const int r = i / N, pi = r * s_phys + e_loc + i % N;
+    const int r = i / N, pi = r * s_phys + e_loc + (i - r * N);
     if (qrow[pi] <= 0) continue;
-    int pos = (mr[e] < r && qrow[ml[e]] > 0) ? 1 : 0;
-    for (int i2 = 0; i2 < r * N; ++i2)
-      pos += (rm[i2] == e && qrow[(i2 / N) * s_phys + e_loc + i2 % N] > 0) ? 1 : 0;
-    cum[seg[e] + pos] = qrow[pi];
+    const int qm = qrow[ml[e]];
+    int pos = 0, below = 0;
+    if (mr[e] < r && qm > 0) { pos = 1; below = qm; }
+    const int lim = r * N;
+    for (int i2 = 0, r2 = 0, j2 = 0; i2 < lim; ++i2) {
+      const int v = qrow[r2 * s_phys + e_loc + j2];
+      if (rm[i2] == e && v > 0) { ++pos; below += v; }
+      if (++j2 == N) { j2 = 0; ++r2; }
+    }
+    rec[rl.cum + seg[e] + pos] = below + qrow[pi];
     rec[rl.inst + seg[e] + pos] = pi;
   }
-  __syncthreads();
-  for (int e = tid; e < E; e += nt) {
-    if (nz[e] < 2) continue;
-    int run = 0;
-    for (int i = seg[e]; i < seg[e] + nz[e]; ++i) { run += cum[i]; rec[rl.cum + i] = run; }
-  }
 
+  __syncthreads();   // split_e is complete
   // Cross-tile base of the stable rank, split experts only: exclusive prefix over the row's tiles.
   // One (split expert, tile) pair per thread-iteration so that all loads of a sweep are in flight.
   if (p.tiles > 0 && n_split > 0) {
