@@ -450,7 +450,7 @@ def main():
         dispatch = {"us_per_call": round(us, 2), "us_per_layer_plan": round(us / w.batch, 3),
                     "bytes_per_assignment": 16,
                     "hbm_frac": round(16 * w.assignments / (us * 1e-6) / 1e9 / measured_peak_gbs()[0], 4),
-                    "note": "send/recv positions; ranking kernel is bound by warp-match issue cost"}
+                    "note": "send/recv positions of every assignment; off the planning path, issue-bound"}
         del scratch, send, recv, ioff
 
     # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol

@@ -283,7 +283,7 @@ int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_pe
  * Uses q and U of the plan still in the workspace: call it after topoep_plan
  * (or topoep_solve + topoep_reroute) of the same batch.  Enqueues three kernels;
  * capturable after its first call.  Off the planning path: the ranking kernel is
- * bound by warp-match issue cost, not by HBM.
+ * bound by instruction issue, not by HBM.
  */
 size_t topoep_dispatch_scratch_bytes(topoep_handle_t h, int tokens_per_rank, int batch);
 int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replica,

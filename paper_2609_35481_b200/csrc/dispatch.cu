@@ -14,11 +14,10 @@
 //   2. pos_prefix_kernel, CTA = (plan, source): prefix over tiles of the tile counts, and the
 //      per-(source, instance) bases A0[p] (send) and B0[p] (receive) from the plan's q and U
 //   3. pos_rank_kernel, CTA = tile: stable rank of each assignment among the tile's equal p
-//      (__match_any_sync inside a warp, per-warp counters scanned across warps), added to the
-//      bases.
+//      (per-warp counters; lanes of a warp step that share an instance are ordered by ballots),
+//      added to the bases.
 // Ranks come from counts and prefix sums only, never from atomic arrival order.  Kernel 3 is
-// bound by the issue cost of match.any on B200 (~160-250 cycles per warp instruction), not by
-// HBM; it is off the planning path.
+// bound by instruction issue, not by HBM; it is off the planning path.
 #include "topoep_internal.cuh"
 
 namespace topoep {
@@ -129,6 +128,11 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
   for (int i = tid; i < nwarps * P; i += nt) wh[i] = 0;
   __syncthreads();
 
+  // In-warp stable rank, 32 assignments per step.  All lanes add 1 to their instance's per-warp
+  // counter; the counter value before the step is the rank of the step's FIRST lane with that
+  // instance.  Only instances met twice or more in the step (the counter grew by more than one)
+  // need their lanes ordered, which takes one ballot per such instance -- instead of a
+  // __match_any_sync per step, whose cost on B200 grows with every distinct value in the warp.
   int* my = wh + warp * P;
   int rho[kIdsPerThread];
   const unsigned lt = lanemask_lt();
@@ -136,18 +140,20 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
   for (int j = 0; j < kIdsPerThread; ++j) {
     const int v = x[j];
     const bool valid = v >= 0 && v < P;
-    const unsigned mask = __ballot_sync(0xffffffffu, valid);
-    int r = 0;
-    if (valid) {
-      const unsigned peers = __match_any_sync(mask, v);
-      const int leader = __ffs(peers) - 1;
-      int old = 0;
-      if (lane == leader) { old = my[v]; my[v] = old + __popc(peers); }
-      old = __shfl_sync(peers, old, leader);
-      r = old + __popc(peers & lt);
+    const int before = valid ? my[v] : 0;
+    __syncwarp();
+    if (valid) atomicAdd(&my[v], 1);
+    __syncwarp();
+    const int grown = valid ? my[v] - before : 0;
+    int r = before;
+    unsigned todo = __ballot_sync(0xffffffffu, grown > 1);
+    while (todo) {   // uniform across the warp
+      const int key = __shfl_sync(0xffffffffu, v, __ffs(todo) - 1);
+      const unsigned peers = __ballot_sync(0xffffffffu, valid && v == key);
+      if (valid && v == key) r = before + __popc(peers & lt);
+      todo &= ~peers;
     }
     rho[j] = r;
-    __syncwarp();
   }
   __syncthreads();
   // per-warp totals -> exclusive prefix over the warps of the tile
