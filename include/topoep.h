@@ -311,6 +311,21 @@ int topoep_debug_tensor(topoep_handle_t h, int which, const void** dev_ptr, size
 /* Change a launch-shape knob; outputs are identical for every legal value. */
 int topoep_set_tuning(topoep_handle_t h, int knob, int value);
 
+/*
+ * Sharded deployment (paper, "GPU-Native Load Balancer": an EP-group all-gather gives every rank
+ * the same routing matrix, and every rank derives the same plan without a coordinator).  A GPU
+ * that IS EP rank r holds only its own tokens.  After topoep_set_rank_window(h, first, count):
+ *   topoep_histogram  takes dev_topk_ids [B][count][T][k] of source ranks first..first+count-1
+ *                     and writes dev_omega [B][count][E] (the rows to all-gather);
+ *   topoep_solve      must be given the gathered dev_omega [B][R][E]; it plans the whole group
+ *                     (outputs for all R ranks, identical on every rank) and builds the
+ *                     routing tables of the window;
+ *   topoep_reroute    takes dev_topk_ids / writes dev_token_replica [B][count][T][k].
+ * topoep_plan and topoep_dispatch_positions need the full window (0, R) and return
+ * TOPOEP_ERR_ARG otherwise.  The default window is (0, R).
+ */
+int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count);
+
 /* Derived sizes: E_loc, S_phys, P.  Any output pointer may be NULL. */
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances);
 

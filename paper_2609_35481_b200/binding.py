@@ -22,7 +22,7 @@ KNOB_TILE_IDS, KNOB_HIST_MODE, KNOB_PDL = 0, 1, 2
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
            "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions",
            "topoep_summary", "topoep_read_status",
-           "topoep_debug_tensor", "topoep_set_tuning", "topoep_get_layout",
+           "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_get_layout",
            "topoep_launch_floor", "topoep_strerror")
 
 
@@ -87,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.topoep_debug_tensor.argtypes = [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
         L.topoep_set_tuning.restype = ci
         L.topoep_set_tuning.argtypes = [vp, ci, ci]
+        L.topoep_set_rank_window.restype = ci
+        L.topoep_set_rank_window.argtypes = [vp, ci, ci]
         L.topoep_get_layout.restype = ci
         L.topoep_get_layout.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.topoep_launch_floor.restype = ci
@@ -207,6 +209,10 @@ def topoep_debug_tensor(h, which: int):
 
 def topoep_set_tuning(h, knob: int, value: int) -> int:
     return lib().topoep_set_tuning(h, knob, value)
+
+
+def topoep_set_rank_window(h, first_rank: int, rank_count: int) -> int:
+    return lib().topoep_set_rank_window(h, first_rank, rank_count)
 
 
 def topoep_get_layout(h):

@@ -16,6 +16,7 @@ struct topoep_ctx {
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode, pdl;
+  int rank_first, rank_count;   // window of source ranks of the histogram / reroute buffers
   size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
   int max_tiles;
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
@@ -91,6 +92,8 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   // The first kernel of the chain is never launched early: whatever produced the ids (a router
   // kernel, a copy) must be complete before it reads them.
   p.pdl = 0;
+  p.rank_first = h->rank_first;
+  p.rank_count = h->rank_count;
   return p;
 }
 
@@ -106,6 +109,8 @@ OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, in
   int gpad = 1;
   while (gpad < h->d.G) gpad <<= 1;
   op.epw = 32 / gpad;
+  op.rank_first = 0;
+  op.rank_count = h->d.R;
   return op;
 }
 
@@ -177,6 +182,8 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->tile_ids = 4096;
   h->hist_mode = 0;
   h->pdl = 1;
+  h->rank_first = 0;
+  h->rank_count = (int)R;
   h->dispatch_smem = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
@@ -250,7 +257,21 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
   h->hist_tokens = T;
   h->hist_batch = batch;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
-  if (e == cudaSuccess) e = launch_omega(make_omega(h, nullptr, out_omega, hp.tiles), batch, stream);
+  if (e == cudaSuccess) {
+    OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles);
+    if (h->rank_count != h->d.R) {
+      // a window of ranks: plain tile sums, rank by rank; the demand and the transposed copy need
+      // every rank's row and are derived later, from the gathered matrix handed to topoep_solve
+      op.d.M = h->rank_count;
+      op.d.G = 1;
+      op.epw = 32;
+      op.ws.omega_m = nullptr;
+      op.ws.demand = nullptr;
+      op.rank_first = h->rank_first;
+      op.rank_count = h->rank_count;
+    }
+    e = launch_omega(op, batch, stream);
+  }
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
 }
@@ -282,6 +303,8 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
     rp.d = h->d;
     rp.ws = h->ws;
     rp.pdl = h->pdl;
+    rp.rank_first = h->rank_first;
+    rp.rank_count = h->rank_count;
     rp.out_offsets = offsets;
     rp.max_tiles = h->max_tiles;
     rp.tiles = 0;
@@ -302,6 +325,8 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   rp.d = h->d;
   rp.ws = h->ws;
   rp.pdl = h->pdl;
+  rp.rank_first = h->rank_first;
+  rp.rank_count = h->rank_count;
   rp.ids = ids;
   rp.out_token_replica = token_replica;
   rp.n_ids = T * h->d.k;
@@ -338,6 +363,8 @@ int topoep_solve(topoep_handle_t h, const int32_t* dev_omega, int batch, int32_t
   if (!aligned4(dev_omega) || !aligned4(dev_replica_map) || !aligned4(dev_dispatch_counts) ||
       !aligned4(dev_dispatch_offsets) || !aligned4(dev_instance_counts))
     return TOPOEP_ERR_ALIGN;
+  // with a window of ranks the workspace holds only the window's rows: the gathered matrix is required
+  if (h->rank_count != h->d.R && !dev_omega) return TOPOEP_ERR_NULL;
   return enqueue_solve(h, dev_omega, batch, dev_replica_map, dev_dispatch_counts,
                        dev_dispatch_offsets, dev_instance_counts, stream);
 }
@@ -367,6 +394,7 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
       !aligned4(dev_dispatch_counts) || !aligned4(dev_dispatch_offsets) ||
       !aligned4(dev_instance_counts))
     return TOPOEP_ERR_ALIGN;
+  if (h->rank_count != h->d.R) return TOPOEP_ERR_ARG;   // a whole plan needs every rank's ids
   rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream);
   if (rc != TOPOEP_OK) return rc;
   rc = enqueue_solve(h, nullptr, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
@@ -391,6 +419,7 @@ int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replic
   if (rc != TOPOEP_OK) return rc;
   if (batch == 0) return TOPOEP_OK;
   if (!dev_scratch) return TOPOEP_ERR_NULL;
+  if (h->rank_count != h->d.R) return TOPOEP_ERR_ARG;   // needs every rank's assignments
   if (tokens_per_rank > 0 && (!dev_token_replica || !dev_send_pos || !dev_recv_pos))
     return TOPOEP_ERR_NULL;
   if (!aligned4(dev_token_replica) || !aligned4(dev_send_pos) || !aligned4(dev_recv_pos) ||
@@ -493,6 +522,15 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     default:
       return TOPOEP_ERR_ARG;
   }
+}
+
+int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count) {
+  if (!h) return TOPOEP_ERR_NULL;
+  if (first_rank < 0 || rank_count < 1 || first_rank + rank_count > h->d.R) return TOPOEP_ERR_ARG;
+  h->rank_first = first_rank;
+  h->rank_count = rank_count;
+  h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;   // earlier tile counts no longer apply
+  return TOPOEP_OK;
 }
 
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances) {

@@ -208,6 +208,8 @@ cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) 
   hp.ws = p.ws;
   hp.ws.tile_cnt = p.pos_cnt;
   hp.ids = p.token_replica;
+  hp.rank_first = 0;
+  hp.rank_count = p.d.R;
   hp.n_ids = p.n_ids;
   hp.tiles = p.tiles;
   hp.max_tiles = p.tiles;

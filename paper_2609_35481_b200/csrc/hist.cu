@@ -45,10 +45,11 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   const int nt = blockDim.x, tid = threadIdx.x;
   const unsigned lane = tid & 31;
 
-  const size_t row = (size_t)b * p.d.R + s;
+  // workspace rows are indexed by the global source rank, the caller's buffer by its window
+  const size_t row = (size_t)b * p.d.R + p.rank_first + s;
   const int begin = tile * p.tile_ids;
   const int count = min(p.tile_ids, p.n_ids - begin);   // <= 0 only when n_ids == 0
-  const int32_t* ids = p.ids + row * (size_t)p.n_ids + begin;
+  const int32_t* ids = p.ids + ((size_t)b * p.rank_count + s) * (size_t)p.n_ids + begin;
   int4 x[IPT / 4];
 #pragma unroll
   for (int j = 0; j < IPT / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, p.vec_ok);
@@ -81,8 +82,9 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
   const int dm = blockIdx.y, b = blockIdx.z;
   const int g = lane / epw, e = (blockIdx.x * 4 + warp) * epw + (lane - g * epw);
   const bool on = g < G && e < E;
-  const int s = dm * G + g;
+  const int s = p.rank_first + dm * G + g;   // global source rank
   const size_t row = (size_t)b * R + s;
+  const size_t user_row = (size_t)b * p.rank_count + dm * G + g;   // row in the caller's window
   int sum = 0, mi = 0;
   if (on && p.ws.omega_m)   // row of the transposed copy: static tables, fetched before the wait
     mi = __ldg(p.ws.main_rank + e) * p.d.e_loc + __ldg(p.ws.main_local + e);
@@ -101,7 +103,7 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
       }
     }
     if (p.ws.omega) p.ws.omega[row * E + e] = sum;
-    if (p.out_omega) p.out_omega[row * E + e] = sum;
+    if (p.out_omega) p.out_omega[user_row * E + e] = sum;
     if (p.ws.omega_m) p.ws.omega_m[((size_t)b * R * p.d.e_loc + mi) * R + s] = sum;
   }
   int dsum = sum;
@@ -116,7 +118,7 @@ __global__ void empty_kernel() {}
 size_t hist_smem_bytes(const Dims& d) { return sizeof(int) * ((size_t)d.E + 1); }
 
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream) {
-  const dim3 grid(p.tiles, p.d.R, batch);
+  const dim3 grid(p.tiles, p.rank_count, batch);
   const size_t smem = hist_smem_bytes(p.d);
   const bool wide = p.tile_ids >= 2048;   // 32 ids per thread once the CTA still has 2+ warps
   const dim3 block(p.tile_ids / (wide ? 32 : 16));

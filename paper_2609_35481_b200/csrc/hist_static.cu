@@ -80,6 +80,8 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   hp.d.R = ranks;
   hp.d.E = experts;
   hp.d.k = top_k;
+  hp.rank_first = 0;
+  hp.rank_count = ranks;
   hp.ws.status = flags;
   hp.ws.tile_cnt = reinterpret_cast<int32_t*>(static_cast<unsigned char*>(base) + kFlagsBytes);
   hp.ids = dev_topk_ids;
@@ -101,6 +103,8 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
     op.tiles = hp.tiles;
     op.max_tiles = hp.max_tiles;
     op.epw = 32;
+    op.rank_first = 0;
+    op.rank_count = ranks;
     e = launch_omega(op, batch, stream);
   }
   return e == cudaSuccess ? TOPOEP_OK : TOPOEP_ERR_CUDA;

@@ -158,11 +158,13 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   int* hdr = reinterpret_cast<int*>(smem + lay.hdr);           // n_split, n_list, n_work
   unsigned short* work = reinterpret_cast<unsigned short*>(smem + lay.work);
 
-  const size_t row = (size_t)b * d.R + s;
+  // workspace rows are indexed by the global source rank, the caller's buffers by their window
+  const size_t row = (size_t)b * d.R + p.rank_first + s;
+  const size_t user_row = (size_t)b * p.rank_count + s;
   const int begin = tile * p.tile_ids;
   const int count = min(p.tile_ids, p.n_ids - begin);
-  const int32_t* ids = p.ids + row * (size_t)p.n_ids + begin;
-  int32_t* out = p.out_token_replica + row * (size_t)p.n_ids + begin;
+  const int32_t* ids = p.ids + user_row * (size_t)p.n_ids + begin;
+  int32_t* out = p.out_token_replica + user_row * (size_t)p.n_ids + begin;
 
   // The ids go to registers first: sixteen per thread, all four loads in flight.
   int4 x[kIdsPerThread / 4];
@@ -258,7 +260,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
 size_t reroute_smem_bytes(const Dims& d, int tile_ids) { return reroute_layout(d, tile_ids).total; }
 
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream) {
-  const dim3 grid(p.tiles, p.d.R, batch);
+  const dim3 grid(p.tiles, p.rank_count, batch);
   const dim3 block(p.tile_ids / kIdsPerThread);
   const size_t smem = reroute_smem_bytes(p.d, p.tile_ids);
   return p.vec_ok ? launch_kernel(reroute_kernel<true>, grid, block, smem, stream, p.pdl != 0, p)

@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   __syncthreads();   // split_e is complete
   // Cross-tile base of the stable rank, split experts only: exclusive prefix over the row's tiles.
   // One (split expert, tile) pair per thread-iteration so that all loads of a sweep are in flight.
-  if (p.tiles > 0 && n_split > 0) {
+  if (p.tiles > 0 && n_split > 0 && s >= p.rank_first && s < p.rank_first + p.rank_count) {
     const size_t trow = row * (size_t)p.max_tiles * E;
     if (p.tiles <= 32) {
       // a warp owns a split expert, a lane owns a tile

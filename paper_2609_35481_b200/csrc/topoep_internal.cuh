@@ -79,6 +79,7 @@ struct HistParams {
   Dims d;
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
+  int rank_first, rank_count;   // window of source ranks the caller's id buffers cover
   const int32_t* ids;   // [B][R][n_ids]
   int32_t* out_omega;   // optional caller copy of omega [B][R][E]
   int n_ids;            // T * k
@@ -92,6 +93,7 @@ struct OmegaParams {
   Dims d;
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
+  int rank_first, rank_count;   // window of source ranks the caller's id buffers cover
   const int32_t* src_omega;   // given routing matrix [B][R][E], or NULL: sum the tile counts
   int32_t* out_omega;         // optional caller copy of omega [B][R][E]
   int tiles, max_tiles;
@@ -115,6 +117,7 @@ struct RouteParams {
   Dims d;
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
+  int rank_first, rank_count;   // window of source ranks the caller's id buffers cover
   int32_t* out_offsets;       // [B][2][R][R+1]: the send half is written here
   int tiles, max_tiles;       // shape of the tile counts now in the workspace (tiles 0: none)
 };
@@ -123,6 +126,7 @@ struct RerouteParams {
   Dims d;
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
+  int rank_first, rank_count;   // window of source ranks the caller's id buffers cover
   const int32_t* ids;
   int32_t* out_token_replica;
   int n_ids, tiles, max_tiles, tile_ids;

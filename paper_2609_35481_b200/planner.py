@@ -45,6 +45,7 @@ class Planner:
         if rc != B.OK:
             raise B.TopoEPError(rc)
         rc, self.e_loc, self.s_phys, self.P = B.topoep_get_layout(self.handle)
+        self.window = (0, self.R)
         nbytes = B.topoep_workspace_bytes(self.handle)
         with torch.cuda.device(self.device):
             self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
@@ -71,7 +72,7 @@ class Planner:
         i32 = dict(dtype=torch.int32, device=self.device)
         R = self.R
         return PlanOutputs(torch.empty((batch, R, self.N), **i32),
-                           torch.empty((batch, R, tokens_per_rank, self.k), **i32),
+                           torch.empty((batch, self.window[1], tokens_per_rank, self.k), **i32),
                            torch.empty((batch, R, R), **i32),
                            torch.empty((batch, 2, R, R + 1), **i32),
                            torch.empty((batch, self.P), **i32))
@@ -111,13 +112,76 @@ class Planner:
         return send, recv, inst_off
 
     def histogram(self, topk_ids: torch.Tensor, stream=None) -> torch.Tensor:
+        """topoep_histogram on ids [B][rank window][T][k]; returns Omega rows [B][window][E]."""
         Bn, R, T, k = topk_ids.shape
+        assert R == self.window[1]
         omega = torch.empty((Bn, R, self.E), dtype=torch.int32, device=self.device)
         st = stream if stream is not None else torch.cuda.current_stream(self.device)
         rc = B.topoep_histogram(self.handle, topk_ids, T, Bn, omega, st.cuda_stream)
         if rc != B.OK:
             raise B.TopoEPError(rc)
         return omega
+
+    def set_rank_window(self, first_rank: int, rank_count: int):
+        """Sharded deployment: this process holds the ids of ranks first..first+count-1 only."""
+        rc = B.topoep_set_rank_window(self.handle, first_rank, rank_count)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        self.window = (first_rank, rank_count)
+
+    def solve(self, omega: Optional[torch.Tensor], batch: int, out: Optional[PlanOutputs] = None,
+              tokens_per_rank: int = 0, stream=None) -> PlanOutputs:
+        """topoep_solve on the gathered Omega [B][R][E] (None: the one topoep_histogram left)."""
+        if out is None:
+            out = self.alloc_outputs(batch, tokens_per_rank)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = B.topoep_solve(self.handle, omega, batch, out.replica_map, out.dispatch_counts,
+                            out.dispatch_offsets, out.instance_counts, st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        return out
+
+    def reroute(self, topk_ids: torch.Tensor, stream=None) -> torch.Tensor:
+        """topoep_reroute on the ids given to histogram(); returns token_replica of the window."""
+        Bn, R, T, k = topk_ids.shape
+        assert R == self.window[1]
+        tr = torch.empty((Bn, R, T, k), dtype=torch.int32, device=self.device)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = B.topoep_reroute(self.handle, topk_ids, T, Bn, tr, st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        return tr
+
+    def plan_sharded(self, my_topk_ids: torch.Tensor, group=None,
+                     out: Optional[PlanOutputs] = None) -> PlanOutputs:
+        """One planning step of a process that owns a window of source ranks.
+
+        Every process of `group` (torch.distributed, NCCL) calls this with the ids of its own
+        window [B][count][T][k]; windows are equal-sized and ordered by group rank.  The rows of
+        the routing matrix are all-gathered (the only exchange: B*R*E int32, never the ids), every
+        process solves the whole group's plan from the same matrix, and reroutes its own ids.
+        token_replica of the result covers this process's window; the other outputs cover all
+        ranks and are identical on every process.
+        """
+        import torch.distributed as dist
+        Bn, cnt, T, _ = my_topk_ids.shape
+        world = dist.get_world_size(group)
+        me = dist.get_rank(group)
+        if cnt * world != self.R:
+            raise ValueError("windows of %d ranks x %d processes do not cover %d ranks"
+                             % (cnt, world, self.R))
+        if self.window != (me * cnt, cnt):
+            self.set_rank_window(me * cnt, cnt)
+        rows = self.histogram(my_topk_ids)                       # [B][cnt][E]
+        allrows = torch.empty((world,) + tuple(rows.shape), dtype=rows.dtype, device=self.device)
+        dist.all_gather_into_tensor(allrows, rows, group=group)
+        omega = allrows.permute(1, 0, 2, 3).reshape(Bn, self.R, self.E).contiguous()
+        out = self.solve(omega, Bn, out=out, tokens_per_rank=T)
+        rc = B.topoep_reroute(self.handle, my_topk_ids, T, Bn, out.token_replica,
+                              torch.cuda.current_stream(self.device).cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        return out
 
     def summary(self, batch: int) -> np.ndarray:
         """Summaries of the last plan as a numpy record array (synchronises)."""

@@ -246,6 +246,87 @@ def test_stage_entry_points_equal_the_fused_plan():
     assert pl.status() == 0
 
 
+# ---- sharded deployment: every rank plans from the gathered routing matrix -----------------------
+@pytest.mark.parametrize("name,over,batch,window", [
+    ("mid", dict(slots_per_rank=3), 2, 1),
+    ("mid", dict(slots_per_rank=2, tokens_per_rank=777), 1, 3),   # ragged last window and tile
+    ("dsv3", dict(tokens_per_rank=4099), 1, 8),                    # one process per node
+    ("scaleout", dict(tokens_per_rank=1500), 1, 16),
+])
+def test_sharded_ranks_reach_the_same_plan_as_the_oracle(name, over, batch, window):
+    """Each emulated process owns a window of source ranks: it histograms its own ids, the rows
+    are gathered, every process solves the whole group from the gathered matrix and reroutes its
+    own ids.  The processes run one after the other on this GPU, each with its own handle and
+    workspace.  Every process must hold the same plan, bit for bit, and the union of their
+    per-token outputs must equal the oracle's single-process result."""
+    w = wl.CONFIGS[name].replace(**over)
+    ids = wl.make_topk_ids(w, seed=21, batch=batch)
+    ref = orc.plan(oracle_config(w), ids)
+    R, T = w.ranks, w.tokens_per_rank
+    windows = [(f, min(window, R - f)) for f in range(0, R, window)]
+    procs = []
+    for first, count in windows:
+        pl = make_planner(w, max_batch=batch)
+        pl.set_rank_window(first, count)
+        procs.append((pl, torch.from_numpy(np.ascontiguousarray(ids[:, first:first + count])).to(pl.device)))
+    rows = [pl.histogram(mine) for pl, mine in procs]
+    for (first, count), r in zip(windows, rows):
+        assert np.array_equal(r.cpu().numpy(), ref.omega[:, first:first + count])
+    gathered = torch.cat(rows, dim=1).contiguous()          # the EP-group all-gather
+    outs = [pl.solve(gathered, batch, tokens_per_rank=T) for pl, _ in procs]
+    parts = [pl.reroute(mine) for pl, mine in procs]
+    torch.cuda.synchronize()
+    for (pl, _), out in zip(procs, outs):
+        for field in ("replica_map", "dispatch_counts", "dispatch_offsets", "instance_counts"):
+            assert np.array_equal(getattr(out, field).cpu().numpy(), getattr(ref, field)), field
+        assert pl.status() == 0
+        assert np.array_equal(pl.debug_tensor(B.T_Q, batch).numpy(), ref.q_instances)
+    assert np.array_equal(torch.cat(parts, dim=1).cpu().numpy(), ref.token_replica)
+
+
+def test_plan_sharded_over_a_one_process_nccl_group():
+    """The NCCL form of the same step, in a group of one process (one GPU here): the all-gather,
+    the row permutation and the window bookkeeping run as they would in a larger group."""
+    import socket
+    import torch.distributed as dist
+    w = wl.CONFIGS["mid"].replace(slots_per_rank=2)
+    ids = wl.make_topk_ids(w, seed=22, batch=2)
+    ref = orc.plan(oracle_config(w), ids)
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % port, rank=0, world_size=1,
+                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        pl = make_planner(w, max_batch=2)
+        out = pl.plan_sharded(torch.from_numpy(ids).to(pl.device))
+        torch.cuda.synchronize()
+        for field in ("replica_map", "token_replica", "dispatch_counts", "dispatch_offsets",
+                      "instance_counts"):
+            assert np.array_equal(getattr(out, field).cpu().numpy(), getattr(ref, field)), field
+        assert pl.status() == 0
+    finally:
+        dist.destroy_process_group()
+
+
+def test_rank_window_argument_errors():
+    w = wl.CONFIGS["tiny"]
+    pl = make_planner(w)
+    ids = torch.from_numpy(wl.make_topk_ids(w, seed=3)).to(pl.device)
+    for first, count in ((-1, 1), (0, 0), (w.ranks, 1), (1, w.ranks)):
+        assert B.topoep_set_rank_window(pl.handle, first, count) == -10
+    pl.set_rank_window(1, 2)
+    out = pl.alloc_outputs(1, w.tokens_per_rank)
+    # a whole plan, the solver without a gathered matrix, and the dispatch permutation need all ranks
+    assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 1, out.replica_map, out.token_replica,
+                         out.dispatch_counts, out.dispatch_offsets, out.instance_counts, 0) == -10
+    assert B.topoep_solve(pl.handle, None, 1, out.replica_map, out.dispatch_counts,
+                          out.dispatch_offsets, out.instance_counts, 0) == -1
+    pl.set_rank_window(0, w.ranks)
+    run = pl.plan(ids)
+    assert pl.status() == 0 and run.token_replica.shape[1] == w.ranks
+
+
 # ---- dispatch permutation (the step after the path) --------------------------------------------
 @pytest.mark.parametrize("name,over,batch", [
     ("tiny", dict(slots_per_rank=2), 2),
