@@ -71,6 +71,10 @@ def _load():
         lib.oracle_summary_of.argtypes = [vp] * 7
         lib.oracle_dispatch_positions.restype = None
         lib.oracle_dispatch_positions.argtypes = [vp, vp, ctypes.c_int, vp, vp, vp, vp]
+        lib.oracle_replica_pull.restype = None
+        lib.oracle_replica_pull.argtypes = [vp, vp, vp, ctypes.c_int64, vp, vp]
+        lib.oracle_replica_grad_return.restype = None
+        lib.oracle_replica_grad_return.argtypes = [vp, vp, vp, ctypes.c_int64, vp, vp]
         lib.oracle_plan.restype = ctypes.c_int
         lib.oracle_plan.argtypes = [vp, vp, vp, ctypes.c_int, ctypes.c_int] + [vp] * 11
         _lib = lib
@@ -230,6 +234,36 @@ def dispatch_positions(cfg: OracleConfig, token_replica: np.ndarray):
     _load().oracle_dispatch_positions(ctypes.addressof(c), _p(cfg.main_rank), tr.shape[1], _p(tr),
                                       _p(send), _p(recv), _p(inst_off))
     return send, recv, inst_off
+
+
+def replica_pull(cfg: OracleConfig, slotmap: np.ndarray, main_params: np.ndarray,
+                 replica_buf: np.ndarray) -> np.ndarray:
+    """O11: main_params [R][E_loc][W] uint8, replica_buf [R][N_slot][W] uint8 -> updated copy."""
+    R, N = cfg.ranks, cfg.slots_per_rank
+    mp = np.ascontiguousarray(main_params, dtype=np.uint8)
+    out = np.array(replica_buf, dtype=np.uint8, order="C", copy=True)
+    W = mp.shape[-1]
+    assert mp.shape == (R, cfg.e_loc, W) and out.shape == (R, N, W)
+    sm = np.concatenate([np.asarray(slotmap, np.int32).ravel(), [-1]]).astype(np.int32)
+    c = cfg.c_struct()
+    _load().oracle_replica_pull(ctypes.addressof(c), _p(cfg.main_rank), _p(sm), ctypes.c_int64(W),
+                                _p(mp), _p(out))
+    return out
+
+
+def replica_grad_return(cfg: OracleConfig, slotmap: np.ndarray, replica_buf: np.ndarray,
+                        grad_acc: np.ndarray) -> np.ndarray:
+    """O12: replica_buf [R][N_slot][W], grad_acc [R][R][E_loc][W] uint8 -> updated copy."""
+    R, N = cfg.ranks, cfg.slots_per_rank
+    rb = np.ascontiguousarray(replica_buf, dtype=np.uint8)
+    out = np.array(grad_acc, dtype=np.uint8, order="C", copy=True)
+    W = rb.shape[-1]
+    assert rb.shape == (R, N, W) and out.shape == (R, R, cfg.e_loc, W)
+    sm = np.concatenate([np.asarray(slotmap, np.int32).ravel(), [-1]]).astype(np.int32)
+    c = cfg.c_struct()
+    _load().oracle_replica_grad_return(ctypes.addressof(c), _p(cfg.main_rank), _p(sm),
+                                       ctypes.c_int64(W), _p(rb), _p(out))
+    return out
 
 
 @dataclass

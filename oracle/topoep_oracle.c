@@ -25,6 +25,9 @@
  *                                                 replica-served fractions)
  *   O10 dispatch permutation                     (the step after the path; layout defined at
  *                                                 the function, pinned to numpy.lexsort)
+ *   O11 replica parameter pull, O12 replica      ("Device-initiated replica transfers" with the
+ *       gradient return                           three buffers of the same subsection; pinned by
+ *                                                 hand-written byte fixtures and an identity code)
  *
  * Where the paper is silent the readings are (all listed in the design notes
  * of the repository, none of them pinned by the paper itself):
@@ -548,4 +551,57 @@ void oracle_dispatch_positions(const oracle_config* c, const int32_t* main_rank,
   for (int s = 0; s < R; ++s)
     for (int64_t f = 0; f < n; ++f)
       if (token_replica[(size_t)s * n + f] < 0) recv_pos[(size_t)s * n + f] = -1;
+}
+
+
+/* l(e): position of e among the experts whose main rank is main_rank[e], ascending e. */
+static int main_local_index(const int32_t* main_rank, int e) {
+  int l = 0;
+  for (int e2 = 0; e2 < e; ++e2) l += (main_rank[e2] == main_rank[e]);
+  return l;
+}
+
+/*
+ * O11 -- replica parameter pull ("Device-initiated replica transfers", forward direction).
+ * Buffers as the subsection lists them, for all ranks of the simulated group side by side:
+ *   main_params [R][E_loc][W]  rank m's main instances, by local index l(e);
+ *   replica_buf [R][N_slot][W] rank r's replica slots.
+ * For every occupied slot j of rank r (slotmap[r][j] = e >= 0) the slot receives the W bytes of
+ * e's main instance; an empty slot keeps its bytes.
+ */
+void oracle_replica_pull(const oracle_config* c, const int32_t* main_rank, const int32_t* slotmap,
+                         int64_t W, const uint8_t* main_params, uint8_t* replica_buf) {
+  const int R = c->nodes * c->gpus_per_node, N = c->slots_per_rank;
+  const int e_loc = oracle_e_loc(c, main_rank);
+  for (int r = 0; r < R; ++r)
+    for (int j = 0; j < N; ++j) {
+      const int e = slotmap[(size_t)r * N + j];
+      if (e < 0) continue;
+      const uint8_t* src = main_params + ((size_t)main_rank[e] * e_loc + main_local_index(main_rank, e)) * W;
+      uint8_t* dst = replica_buf + ((size_t)r * N + j) * W;
+      for (int64_t i = 0; i < W; ++i) dst[i] = src[i];
+    }
+}
+
+/*
+ * O12 -- replica gradient return (same subsection, backward direction).  The slot that held the
+ * parameters now holds the replica's gradient; it goes to the gradient-accumulation buffer of
+ * the expert's main rank, which is partitioned by SOURCE rank into R regions of E_loc blocks:
+ *   grad_acc [R main][R source][E_loc][W];  grad_acc[main(e)][r][l(e)] = replica_buf[r][j].
+ * Everything else in grad_acc keeps its bytes (the copy does not accumulate: each region has
+ * exactly one writer, and the main rank sums its regions later).
+ */
+void oracle_replica_grad_return(const oracle_config* c, const int32_t* main_rank,
+                                const int32_t* slotmap, int64_t W, const uint8_t* replica_buf,
+                                uint8_t* grad_acc) {
+  const int R = c->nodes * c->gpus_per_node, N = c->slots_per_rank;
+  const int e_loc = oracle_e_loc(c, main_rank);
+  for (int r = 0; r < R; ++r)
+    for (int j = 0; j < N; ++j) {
+      const int e = slotmap[(size_t)r * N + j];
+      if (e < 0) continue;
+      const uint8_t* src = replica_buf + ((size_t)r * N + j) * W;
+      uint8_t* dst = grad_acc + (((size_t)main_rank[e] * R + r) * e_loc + main_local_index(main_rank, e)) * W;
+      for (int64_t i = 0; i < W; ++i) dst[i] = src[i];
+    }
 }

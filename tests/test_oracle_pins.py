@@ -550,3 +550,73 @@ def test_summary_floats_are_the_integer_ratios():
     assert s["cross_fraction"] == s["cross_assignments"] / s["assignments"]
     assert s["replica_fraction"] == s["replica_served"] / s["assignments"]
     assert s["t_comp"] == w.t_ffn * s["l_max"]
+
+
+# ---- O11 / O12: replica parameter pull and gradient return ---------------------------------------
+def _transfer_cfg(fx):
+    return orc.OracleConfig(fx["nodes"], fx["gpus_per_node"], fx["experts"], fx["slots_per_rank"], 1, 0, 0,
+                            main_rank=np.array(fx["main_rank"], np.int32))
+
+
+def test_replica_pull_and_grad_return_hand_written_bytes():
+    fx = _load("replica_transfer.json")
+    cfg = _transfer_cfg(fx)
+    rmap = np.array(fx["replica_map"], np.int32)
+    after = orc.replica_pull(cfg, rmap, np.array(fx["main_params"], np.uint8),
+                             np.array(fx["replica_before"], np.uint8))
+    assert np.array_equal(after, np.array(fx["replica_after_pull"], np.uint8))
+    R, W = cfg.ranks, fx["param_bytes"]
+    expect = np.zeros((R, R, cfg.e_loc, W), np.uint8)
+    for m, s, l, b in fx["grad_acc_entries"]:
+        expect[m, s, l] = b
+    got = orc.replica_grad_return(cfg, rmap, np.array(fx["replica_grads"], np.uint8),
+                                  np.zeros_like(expect))
+    assert np.array_equal(got, expect)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_replica_transfers_identity_code(seed):
+    """Every byte of expert e's main block is e: a pulled slot must read back its own map entry,
+    an empty slot its old bytes; returned gradients coded (source, slot) must land once each in
+    the region [main(e)][source], and pull followed by return reproduces the main block there."""
+    rng = np.random.default_rng(seed)
+    M, G, E, N, W = 2, 3, 24, 3, 48
+    R = M * G
+    main_rank = rng.integers(0, R, E).astype(np.int32)
+    cfg = orc.OracleConfig(M, G, E, N, 1, 0, 0, main_rank=main_rank)
+    e_loc = cfg.e_loc
+    mp = np.full((R, e_loc, W), 255, np.uint8)
+    nxt = np.zeros(R, int)
+    where = {}
+    for e in range(E):
+        mp[main_rank[e], nxt[main_rank[e]]] = e
+        where[e] = (int(main_rank[e]), int(nxt[main_rank[e]]))
+        nxt[main_rank[e]] += 1
+    rmap = np.full((R, N), -1, np.int32)
+    for r in range(R):
+        others = [e for e in range(E) if main_rank[e] != r]
+        n = int(rng.integers(0, N + 1))
+        rmap[r, :n] = rng.choice(others, n, replace=False)
+    before = np.full((R, N, W), 254, np.uint8)
+    after = orc.replica_pull(cfg, rmap, mp, before)
+    assert np.array_equal(after[:, :, 0], np.where(rmap >= 0, rmap, 254).astype(np.uint8))
+    assert (after == after[:, :, :1]).all()
+    # backward, bytes coded by (source rank, slot)
+    grads = (np.arange(R)[:, None, None] * 16 + np.arange(N)[None, :, None]
+             + np.zeros((1, 1, W), int)).astype(np.uint8)
+    acc = orc.replica_grad_return(cfg, rmap, grads, np.full((R, R, e_loc, W), 253, np.uint8))
+    written = 0
+    for r in range(R):
+        for j in range(N):
+            if rmap[r, j] >= 0:
+                m, l = where[int(rmap[r, j])]
+                assert (acc[m, r, l] == r * 16 + j).all()
+                written += 1
+    assert (acc != 253).sum() == written * W          # nothing else was touched
+    # pull then return: the main rank gets its own parameters back in the source's region
+    acc2 = orc.replica_grad_return(cfg, rmap, after, np.full((R, R, e_loc, W), 253, np.uint8))
+    for r in range(R):
+        for j in range(N):
+            if rmap[r, j] >= 0:
+                m, l = where[int(rmap[r, j])]
+                assert np.array_equal(acc2[m, r, l], mp[m, l])
