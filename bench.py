@@ -345,6 +345,7 @@ def main():
     ap.add_argument("--workload", default="dsv3_batched", choices=sorted(wl.CONFIGS))
     ap.add_argument("--no-single-plan", action="store_true")
     ap.add_argument("--no-dispatch", action="store_true")
+    ap.add_argument("--no-transfer", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override plans per step")
     ap.add_argument("--impl", default="topoep", choices=["topoep", "reference"])
     ap.add_argument("--tile-ids", type=int, default=0)
@@ -453,6 +454,56 @@ def main():
                     "note": "send/recv positions of every assignment; off the planning path, issue-bound"}
         del scratch, send, recv, ioff
 
+    # ---- replica parameter executor driven by plan 0 of the batch (reported, not timed into
+    # `value`): forward pull at the layer's full expert size, gradient return at 1/16 of it (the
+    # accumulation buffers of all simulated ranks, R*R*E_loc blocks, must fit one GPU)
+    transfer = None
+    if not args.no_transfer and w.slots_per_rank > 0 and w.expert_bytes >= 256:
+        pl0 = s0["pl"]
+        R, N, e_loc = w.ranks, w.slots_per_rank, pl0.e_loc
+        w_pull = w.expert_bytes // 16 * 16
+        while R * e_loc * w_pull > 48 * 2**30:
+            w_pull = w_pull // 32 * 16
+        w_ret = w_pull
+        while R * R * e_loc * w_ret > 48 * 2**30:
+            w_ret = w_ret // 32 * 16
+        rmap = o.replica_map[0]
+        n_occ = int((rmap >= 0).sum().item())
+        u8 = dict(dtype=torch.uint8, device=dev)
+        main = torch.empty((R, e_loc, w_pull), **u8)
+        slots = torch.empty((R, N, w_pull), **u8)
+        gslots = torch.empty((R, N, w_ret), **u8)
+        acc = torch.empty((R, R, e_loc, w_ret), **u8)
+        peak = measured_peak_gbs()[0]
+
+        def time_transfer(fn, a, b_, wb, n_it=10):
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    assert fn(pl0.handle, rmap, a, b_, wb, stream.cuda_stream) == 0
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            with torch.cuda.stream(stream):
+                t0.record(stream)
+                for _ in range(n_it):
+                    fn(pl0.handle, rmap, a, b_, wb, stream.cuda_stream)
+                t1.record(stream)
+            barrier()
+            us = max_over_ranks(t0.elapsed_time(t1), world, dev) / n_it * 1e3
+            gbs = 2.0 * wb * n_occ / (us * 1e-6) / 1e9 if n_occ else 0.0
+            return {"us": round(us, 2), "gbs": round(gbs, 1), "hbm_frac": round(gbs / peak, 4),
+                    "param_bytes": wb}
+
+        transfer = {"occupied_slots": n_occ, "slots": R * N,
+                    "bytes_per_slot": "read |W| + write |W|"}
+        for mode, name in ((0, "bulk"), (1, "plain")):
+            pl0.set_tuning(B.KNOB_TRANSFER_MODE, mode)
+            transfer[name] = {"pull": time_transfer(B.topoep_replica_pull, main, slots, w_pull),
+                              "grad_return": time_transfer(B.topoep_replica_grad_return, gslots,
+                                                           acc, w_ret)}
+        pl0.set_tuning(B.KNOB_TRANSFER_MODE, 0)
+        assert pl0.status() == 0
+        del main, slots, gslots, acc
+
     # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol
     single = None
     if w.batch > 1 and not args.no_single_plan:
@@ -520,6 +571,8 @@ def main():
         line["single_plan"] = single
     if dispatch is not None:
         line["dispatch_positions"] = dispatch
+    if transfer is not None:
+        line["replica_transfer"] = transfer
 
     if rank == 0 and not args.no_cpu_baseline:
         sample_ids = s0["ids_host"][:min(w.batch, 8)]

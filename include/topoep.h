@@ -121,10 +121,13 @@ enum {
                                    power of two                                   */
   TOPOEP_KNOB_HIST_MODE = 1,    /* 0 = plain shared-memory atomics (default),
                                    1 = warp-aggregated (__match_any_sync) atomics */
-  TOPOEP_KNOB_PDL = 2           /* 1 (default): the kernels after the histogram are
+  TOPOEP_KNOB_PDL = 2,          /* 1 (default): the kernels after the histogram are
                                    launched with programmatic dependent launch and
                                    overlap their predecessor's tail; 0: plain
                                    stream order                                   */
+  TOPOEP_KNOB_TRANSFER_MODE = 3 /* replica transfers: 0 (default) the bulk
+                                   asynchronous copy unit through shared memory,
+                                   1 plain 16-byte loads and stores               */
 };
 
 /*
@@ -310,6 +313,32 @@ int topoep_debug_tensor(topoep_handle_t h, int which, const void** dev_ptr, size
 
 /* Change a launch-shape knob; outputs are identical for every legal value. */
 int topoep_set_tuning(topoep_handle_t h, int knob, int value);
+
+/*
+ * Replica parameter executor (paper, "Device-initiated replica transfers", with the three
+ * buffers that subsection lists).  Copies driven by the device-resident replica map of ONE plan
+ * (dev_replica_map [R][N_slot], e.g. one plan's slice of topoep_plan's output): no host read of
+ * the plan, nothing allocated, asynchronous on `stream`, capturable.  Buffers hold all ranks of
+ * the simulated group side by side, blocks of param_bytes bytes each (|W|):
+ *   dev_main_params [R][E_loc][W]     rank m's main instances by local index l (ascending e);
+ *   dev_replica_buf [R][N_slot][W]    rank r's replica slots;
+ *   dev_grad_acc    [R][R][E_loc][W]  [main rank][source rank][local index]: the accumulation
+ *                                     buffer of each main rank, partitioned by source rank.
+ * topoep_replica_pull (forward): for every occupied slot (r, j) with expert e,
+ *   replica_buf[r][j] <- main_params[main(e)][l(e)]; empty slots keep their bytes.
+ * topoep_replica_grad_return (backward): the slot now holds the replica's gradient;
+ *   grad_acc[main(e)][r][l(e)] <- replica_buf[r][j]; every other block keeps its bytes (plain
+ *   copy, one writer per block; summing the regions is the main rank's later step).
+ * param_bytes must be a multiple of 16 and the two data pointers 16-byte aligned
+ * (TOPOEP_ERR_ALIGN); the buffers must not overlap.  A map entry >= E sets TOPOEP_FLAG_BAD_ID
+ * and is skipped.  param_bytes == 0 or N_slot == 0: nothing is done, TOPOEP_OK.
+ */
+int topoep_replica_pull(topoep_handle_t h, const int32_t* dev_replica_map,
+                        const void* dev_main_params, void* dev_replica_buf, size_t param_bytes,
+                        topoep_stream_t stream);
+int topoep_replica_grad_return(topoep_handle_t h, const int32_t* dev_replica_map,
+                               const void* dev_replica_buf, void* dev_grad_acc, size_t param_bytes,
+                               topoep_stream_t stream);
 
 /*
  * Sharded deployment (paper, "GPU-Native Load Balancer": an EP-group all-gather gives every rank

@@ -17,12 +17,13 @@ LIB_PATH = os.path.join(_HERE, "libtopoep.so")
 OK = 0
 FLAG_BAD_ID, FLAG_REFINE_CAP, FLAG_INTERNAL = 1, 2, 4
 T_OMEGA, T_Q, T_RANK_LOAD, T_REFINE_ITERS = 0, 1, 2, 3
-KNOB_TILE_IDS, KNOB_HIST_MODE, KNOB_PDL = 0, 1, 2
+KNOB_TILE_IDS, KNOB_HIST_MODE, KNOB_PDL, KNOB_TRANSFER_MODE = 0, 1, 2, 3
 
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
            "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions",
            "topoep_summary", "topoep_read_status",
-           "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_get_layout",
+           "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_replica_pull", "topoep_replica_grad_return",
+           "topoep_get_layout",
            "topoep_launch_floor", "topoep_strerror")
 
 
@@ -89,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.topoep_set_tuning.argtypes = [vp, ci, ci]
         L.topoep_set_rank_window.restype = ci
         L.topoep_set_rank_window.argtypes = [vp, ci, ci]
+        for fn in (L.topoep_replica_pull, L.topoep_replica_grad_return):
+            fn.restype = ci
+            fn.argtypes = [vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.topoep_get_layout.restype = ci
         L.topoep_get_layout.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.topoep_launch_floor.restype = ci
@@ -213,6 +217,18 @@ def topoep_set_tuning(h, knob: int, value: int) -> int:
 
 def topoep_set_rank_window(h, first_rank: int, rank_count: int) -> int:
     return lib().topoep_set_rank_window(h, first_rank, rank_count)
+
+
+def topoep_replica_pull(h, dev_replica_map, dev_main_params, dev_replica_buf, param_bytes,
+                        stream=0) -> int:
+    return lib().topoep_replica_pull(h, _ptr(dev_replica_map), _ptr(dev_main_params),
+                                     _ptr(dev_replica_buf), param_bytes, stream or None)
+
+
+def topoep_replica_grad_return(h, dev_replica_map, dev_replica_buf, dev_grad_acc, param_bytes,
+                               stream=0) -> int:
+    return lib().topoep_replica_grad_return(h, _ptr(dev_replica_map), _ptr(dev_replica_buf),
+                                            _ptr(dev_grad_acc), param_bytes, stream or None)
 
 
 def topoep_get_layout(h):

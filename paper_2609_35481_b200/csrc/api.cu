@@ -18,6 +18,7 @@ struct topoep_ctx {
   int tile_ids, hist_mode, pdl;
   int rank_first, rank_count;   // window of source ranks of the histogram / reroute buffers
   size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
+  int transfer_ready, transfer_mode, sms;   // replica executor: configured?, copy engine, SM count
   int max_tiles;
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
   // workspace
@@ -185,6 +186,9 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->rank_first = 0;
   h->rank_count = (int)R;
   h->dispatch_smem = 0;
+  h->transfer_ready = 0;
+  h->transfer_mode = 0;
+  h->sms = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
   h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
@@ -458,6 +462,60 @@ int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replic
   return TOPOEP_OK;
 }
 
+namespace {
+
+// Shared body of the two replica transfers.
+int enqueue_transfer(topoep_handle_t h, int direction, const int32_t* dev_replica_map,
+                     const void* src, void* dst, size_t param_bytes, cudaStream_t stream) {
+  if (!h) return TOPOEP_ERR_NULL;
+  if (!h->have_ws) return TOPOEP_ERR_WORKSPACE;
+  if (h->d.N == 0 || param_bytes == 0) return TOPOEP_OK;   // no slots or nothing to move
+  if (!dev_replica_map || !src || !dst) return TOPOEP_ERR_NULL;
+  if (!aligned4(dev_replica_map) || (reinterpret_cast<uintptr_t>(src) & 15u) ||
+      (reinterpret_cast<uintptr_t>(dst) & 15u) || (param_bytes & 15u))
+    return TOPOEP_ERR_ALIGN;
+  // block indices are 32-bit: [R][R][e_loc] blocks in the largest buffer
+  if ((unsigned long long)h->d.R * h->d.R * h->d.e_loc >= (1ull << 32)) return TOPOEP_ERR_SIZE;
+  if (transfer_smem_bytes(h->d, h->transfer_mode) > 113 * 1024) return TOPOEP_ERR_SMEM;
+  cudaError_t e = cudaSuccess;
+  if (!h->transfer_ready) {
+    // first use: host-side attributes only (shared-memory opt-in, SM count)
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = configure_transfer(h->d);
+    if (e == cudaSuccess) h->transfer_ready = 1;
+  }
+  if (e == cudaSuccess) {
+    TransferParams p;
+    p.d = h->d;
+    p.ws = h->ws;
+    p.replica_map = dev_replica_map;
+    p.src = src;
+    p.dst = dst;
+    p.param_bytes = param_bytes;
+    e = launch_transfer(p, direction, h->transfer_mode, h->sms, stream);
+  }
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+}  // namespace
+
+int topoep_replica_pull(topoep_handle_t h, const int32_t* dev_replica_map,
+                        const void* dev_main_params, void* dev_replica_buf, size_t param_bytes,
+                        topoep_stream_t stream) {
+  return enqueue_transfer(h, 0, dev_replica_map, dev_main_params, dev_replica_buf, param_bytes,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int topoep_replica_grad_return(topoep_handle_t h, const int32_t* dev_replica_map,
+                               const void* dev_replica_buf, void* dev_grad_acc, size_t param_bytes,
+                               topoep_stream_t stream) {
+  return enqueue_transfer(h, 1, dev_replica_map, dev_replica_buf, dev_grad_acc, param_bytes,
+                          static_cast<cudaStream_t>(stream));
+}
+
 int topoep_summary(topoep_handle_t h, int batch, topoep_summary_t* dev_out, topoep_stream_t stream) {
   if (!h) return TOPOEP_ERR_NULL;
   if (!h->have_ws) return TOPOEP_ERR_WORKSPACE;
@@ -518,6 +576,10 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_PDL:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->pdl = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_TRANSFER_MODE:
+      if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
+      h->transfer_mode = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

@@ -147,6 +147,15 @@ struct PosParams {
   int n_ids, tiles, tile_ids;
 };
 
+struct TransferParams {
+  Dims d;
+  Workspace ws;
+  const int32_t* replica_map;   // [R][N] of ONE plan
+  const void* src;              // pull: main_params [R][e_loc][W]; return: replica_buf [R][N][W]
+  void* dst;                    // pull: replica_buf;  return: grad_acc [R][R][e_loc][W]
+  unsigned long long param_bytes;   // W, a multiple of 16
+};
+
 struct SummaryParams {
   Dims d;
   Workspace ws;
@@ -172,6 +181,11 @@ cudaError_t launch_route(const RouteParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_reroute(const RerouteParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream);
 cudaError_t launch_summary(const SummaryParams& p, int batch, cudaStream_t stream);
+size_t transfer_smem_bytes(const Dims& d, int mode);
+cudaError_t configure_transfer(const Dims& d);
+// direction 0 = parameter pull, 1 = gradient return; mode 0 = bulk copy unit, 1 = plain loads
+cudaError_t launch_transfer(const TransferParams& p, int direction, int mode, int sms,
+                            cudaStream_t stream);
 cudaError_t launch_empty(int count, cudaStream_t stream);
 
 // Programmatic dependent launch (PDL).  The kernels after the histogram are launched with the

@@ -183,6 +183,31 @@ class Planner:
             raise B.TopoEPError(rc)
         return out
 
+    def replica_pull(self, replica_map: torch.Tensor, main_params: torch.Tensor,
+                     replica_buf: torch.Tensor, stream=None):
+        """topoep_replica_pull for ONE plan: replica_map [R][N_slot] int32, main_params
+        [R][E_loc][W] and replica_buf [R][N_slot][W] as uint8 (contiguous, on this device)."""
+        self._transfer(B.topoep_replica_pull, replica_map, main_params, replica_buf,
+                       (self.R, self.e_loc), (self.R, self.N), stream)
+
+    def replica_grad_return(self, replica_map: torch.Tensor, replica_buf: torch.Tensor,
+                            grad_acc: torch.Tensor, stream=None):
+        """topoep_replica_grad_return for ONE plan: grad_acc [R][R][E_loc][W] uint8."""
+        self._transfer(B.topoep_replica_grad_return, replica_map, replica_buf, grad_acc,
+                       (self.R, self.N), (self.R, self.R, self.e_loc), stream)
+
+    def _transfer(self, fn, replica_map, src, dst, src_lead, dst_lead, stream):
+        assert replica_map.dtype == torch.int32 and replica_map.is_contiguous()
+        assert tuple(replica_map.shape) == (self.R, self.N)
+        W = src.shape[-1]
+        for t, lead in ((src, src_lead), (dst, dst_lead)):
+            assert t.dtype == torch.uint8 and t.is_contiguous() and t.is_cuda
+            assert tuple(t.shape) == tuple(lead) + (W,)
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = fn(self.handle, replica_map, src, dst, W, st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+
     def summary(self, batch: int) -> np.ndarray:
         """Summaries of the last plan as a numpy record array (synchronises)."""
         n = ctypes.sizeof(B.Summary)

@@ -185,3 +185,8 @@ def make_topk_ids(w: Workload, seed: int = BASE_SEED, batch: Optional[int] = Non
         if rc != 0:
             raise ValueError("wl_gen_topk rejected the shape (k > E or k > 64)")
     return out.reshape(B, R, T, k)
+
+
+def make_param_bytes(shape, seed: int) -> np.ndarray:
+    """Seeded stand-in for expert parameters or gradients: uniform random bytes of `shape`."""
+    return np.random.default_rng(seed).integers(0, 256, size=shape, dtype=np.uint8)
