@@ -346,6 +346,8 @@ def main():
     ap.add_argument("--no-single-plan", action="store_true")
     ap.add_argument("--no-dispatch", action="store_true")
     ap.add_argument("--no-transfer", action="store_true")
+    ap.add_argument("--transfer-bytes", type=int, default=0,
+                    help="bytes per expert block of the replica transfers (default: the layer's)")
     ap.add_argument("--batch", type=int, default=0, help="override plans per step")
     ap.add_argument("--impl", default="topoep", choices=["topoep", "reference"])
     ap.add_argument("--tile-ids", type=int, default=0)
@@ -461,7 +463,7 @@ def main():
     if not args.no_transfer and w.slots_per_rank > 0 and w.expert_bytes >= 256:
         pl0 = s0["pl"]
         R, N, e_loc = w.ranks, w.slots_per_rank, pl0.e_loc
-        w_pull = w.expert_bytes // 16 * 16
+        w_pull = (args.transfer_bytes or w.expert_bytes) // 16 * 16
         while R * e_loc * w_pull > 48 * 2**30:
             w_pull = w_pull // 32 * 16
         w_ret = w_pull

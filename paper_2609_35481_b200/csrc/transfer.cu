@@ -25,8 +25,11 @@ namespace topoep {
 
 namespace {
 
-constexpr int kStageBytes = 16 * 1024;   // one chunk = one ring stage
-constexpr int kStages = 6;               // 96 KiB of ring per CTA, two CTAs per SM
+// Measured on B200 for 32 blocks of 88 MB: 32 KiB x 3 stages 0.955 of the copy peak,
+// 16 KiB x 6 0.942, 8 KiB x 12 0.937 (two CTAs per SM each); four CTAs of 16 KiB x 3 0.942.
+constexpr int kStageBytes = 32 * 1024;   // one chunk = one ring stage
+constexpr int kStages = 3;               // 96 KiB of ring per CTA
+constexpr int kBulkCtasPerSm = 2;
 constexpr int kBulkThreads = 32;
 constexpr int kPlainThreads = 256;
 constexpr unsigned kWaitLimit = 1u << 22;   // polls (about 0.1 s) before a wait is given up
@@ -232,7 +235,7 @@ cudaError_t launch_transfer(const TransferParams& p, int direction, int mode, in
                             cudaStream_t stream) {
   const size_t smem = transfer_smem_bytes(p.d, mode);
   if (mode == 0) {
-    const dim3 grid(2 * sms), block(kBulkThreads);
+    const dim3 grid(kBulkCtasPerSm * sms), block(kBulkThreads);
     if (direction == 0) transfer_bulk_kernel<0><<<grid, block, smem, stream>>>(p);
     else transfer_bulk_kernel<1><<<grid, block, smem, stream>>>(p);
   } else {
