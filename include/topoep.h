@@ -121,10 +121,12 @@ enum {
                                    power of two                                   */
   TOPOEP_KNOB_HIST_MODE = 1,    /* 0 = plain shared-memory atomics (default),
                                    1 = warp-aggregated (__match_any_sync) atomics */
-  TOPOEP_KNOB_PDL = 2,          /* 1 (default): the kernels after the histogram are
-                                   launched with programmatic dependent launch and
-                                   overlap their predecessor's tail; 0: plain
-                                   stream order                                   */
+  TOPOEP_KNOB_PDL = 2,          /* programmatic dependent launch of the kernels after
+                                   the histogram.  0: plain stream order; 1 (default):
+                                   on, and a call small enough to be resident on the
+                                   GPU all at once also lets each kernel start its
+                                   dependents early; 2: on, never early; 3: on,
+                                   always early                                   */
   TOPOEP_KNOB_TRANSFER_MODE = 3 /* replica transfers: 0 (default) the bulk
                                    asynchronous copy unit through shared memory,
                                    1 plain 16-byte loads and stores               */

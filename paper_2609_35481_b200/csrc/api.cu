@@ -98,11 +98,25 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   return p;
 }
 
-OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, int tiles) {
+// How the kernels after the histogram are launched for a call of `batch` plans: 0 plain stream
+// order, 1 programmatic launch with the implicit trigger, 2 also triggering dependents at kernel
+// start.  The early trigger pays only while the whole chain fits the GPU at once: at most one
+// wave of reroute blocks (eight per SM).
+int chain_pdl(const topoep_ctx* h, int batch) {
+  if (h->pdl == 0) return 0;
+  if (h->pdl == 2) return 1;
+  if (h->pdl == 3) return 2;
+  long long tiles = 1;
+  if (h->hist_tokens >= 0 && h->hist_tile_ids > 0)
+    tiles = std::max(1ll, ((long long)h->hist_tokens * h->d.k + h->hist_tile_ids - 1) / h->hist_tile_ids);
+  return tiles * h->rank_count * batch <= 8ll * 148 ? 2 : 1;
+}
+
+OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, int tiles, int batch) {
   OmegaParams op;
   op.d = h->d;
   op.ws = h->ws;
-  op.pdl = h->pdl;
+  op.pdl = chain_pdl(h, batch);
   op.src_omega = src;
   op.out_omega = out_omega;
   op.tiles = tiles;
@@ -262,7 +276,7 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
   h->hist_batch = batch;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
   if (e == cudaSuccess) {
-    OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles);
+    OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles, batch);
     if (h->rank_count != h->d.R) {
       // a window of ranks: plain tile sums, rank by rank; the demand and the transposed copy need
       // every rank's row and are derived later, from the gathered matrix handed to topoep_solve
@@ -287,7 +301,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   SolveParams sp;
   sp.d = h->d;
   sp.ws = h->ws;
-  sp.pdl = h->pdl;
+  sp.pdl = chain_pdl(h, batch);
   sp.token_bytes = h->cost.token_bytes;
   sp.expert_bytes = h->cost.expert_bytes;
   sp.max_iters = h->max_iters;
@@ -300,13 +314,13 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.out_inst_counts = inst_counts;
   cudaError_t e = cudaSuccess;
   // a routing matrix handed in from outside: derive the demand and the transposed copy from it
-  if (omega) e = launch_omega(make_omega(h, omega, nullptr, 0), batch, stream);
+  if (omega) e = launch_omega(make_omega(h, omega, nullptr, 0, batch), batch, stream);
   if (e == cudaSuccess) e = launch_solve(sp, batch, stream);
   if (e == cudaSuccess) {
     RouteParams rp;
     rp.d = h->d;
     rp.ws = h->ws;
-    rp.pdl = h->pdl;
+    rp.pdl = chain_pdl(h, batch);
     rp.rank_first = h->rank_first;
     rp.rank_count = h->rank_count;
     rp.out_offsets = offsets;
@@ -328,7 +342,7 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   RerouteParams rp;
   rp.d = h->d;
   rp.ws = h->ws;
-  rp.pdl = h->pdl;
+  rp.pdl = chain_pdl(h, batch) != 0;
   rp.rank_first = h->rank_first;
   rp.rank_count = h->rank_count;
   rp.ids = ids;
@@ -574,7 +588,7 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
       h->hist_mode = value;
       return TOPOEP_OK;
     case TOPOEP_KNOB_PDL:
-      if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
+      if (value < 0 || value > 3) return TOPOEP_ERR_ARG;
       h->pdl = value;
       return TOPOEP_OK;
     case TOPOEP_KNOB_TRANSFER_MODE:

@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
   const int E = p.d.E, G = p.d.G, R = p.d.R, epw = p.epw;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int dm = blockIdx.y, b = blockIdx.z;
+  if (p.pdl == 2) pdl_trigger();
   const int g = lane / epw, e = (blockIdx.x * 4 + warp) * epw + (lane - g * epw);
   const bool on = g < G && e < E;
   const int s = p.rank_first + dm * G + g;   // global source rank

@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   const int R = d.R, E = d.E, N = d.N, P = d.P, s_phys = d.s_phys, e_loc = d.e_loc;
   const int s = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  if (p.pdl == 2) pdl_trigger();
   const RouteLayout lay = route_layout(d);
   int* rm = reinterpret_cast<int*>(smem + lay.rm);         // [R*N] expert in replica slot
   int* qrow = reinterpret_cast<int*>(smem + lay.qrow);     // [P]   q(s, instance)

@@ -76,6 +76,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   const int dm = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
   const unsigned full = 0xffffffffu;
+  if (p.pdl == 2) pdl_trigger();
 
   const SolveLayout lay = solve_layout(d);
   unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);

@@ -194,11 +194,19 @@ cudaError_t launch_empty(int count, cudaStream_t stream);
 // depend on the predecessor -- loading the ids, static tables, clearing shared memory -- before
 // pdl_wait(), which returns once the predecessor grid has completed and its writes are visible.
 // Every block calls pdl_wait() before its first global write and before it exits, so completion
-// stays transitive along the chain.  No kernel triggers its dependents early: measured on B200,
-// early-resident successor blocks take SM resources from the running kernel (a 232-plan call
-// went from 1.15 ms to 1.32 ms), while the implicit trigger at block exit costs nothing there
-// and saves ~1.5 us on a single plan.
+// stays transitive along the chain.  Whether a kernel also triggers its dependents at its own
+// start (pdl == 2) depends on the size of the call: measured on B200, early-resident successor
+// blocks take SM resources from the running kernel when the call fills the GPU (a 232-plan call
+// went from 1.15 ms to 1.32 ms), so large calls rely on the implicit trigger at block exit
+// (pdl == 1, ~1.5 us saved per plan over plain stream order); when the whole chain fits the GPU
+// at once (a single plan), the early trigger lets every later kernel finish its prologue --
+// static tables, the ids of the reroute tiles -- before its predecessor is done (1-2 us more).
+// The histogram never triggers early: the reroute blocks would read the ids at the same time.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the dependent kernel's blocks become resident now (they still stop at their pdl_wait()).
+__device__ __forceinline__ void pdl_trigger() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // Launch `kernel`, allowing it to overlap the tail of the previous kernel in the stream when
 // `pdl` is set (the kernel must then follow the protocol above).

@@ -197,7 +197,8 @@ def test_bitwise_identical_across_reruns_and_tunings():
         for mode in (0, 1):
             pl.set_tuning(B.KNOB_TILE_IDS, tile)
             pl.set_tuning(B.KNOB_HIST_MODE, mode)
-            pl.set_tuning(B.KNOB_PDL, mode)
+            # launch protocol: plain order, automatic, never early, always early
+            pl.set_tuning(B.KNOB_PDL, (tile // 1024 + mode) % 4)
             for rep in range(2):
                 again = run_gpu(pl, ids)
                 for key, val in base.items():
