@@ -3,6 +3,7 @@
 // plan call enqueues five kernels (tile histogram, omega, solver, route tables, reroute) on the
 // caller's stream.
 #include <algorithm>
+#include <climits>
 #include <new>
 
 #include "topoep_internal.cuh"
@@ -35,7 +36,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 enum WsSlot {
-  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
+  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
   W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC, W_SLOTS
 };
 static_assert(W_SLOTS <= 24, "offset table size");
@@ -47,6 +48,7 @@ void carve(topoep_ctx* h) {
   sz[W_MAIN_RANK] = 4 * E;
   sz[W_MAIN_LOCAL] = 4 * E;
   sz[W_MAIN_INST] = 4 * R * (size_t)std::max(d.e_loc, 1);
+  sz[W_SOLVE_STATIC] = (size_t)d.M * solve_static_bytes(d);
   sz[W_STATUS] = 4;
   sz[W_OMEGA] = 4 * B * R * E;
   sz[W_OMEGA_M] = 4 * B * R * (size_t)std::max(d.e_loc, 1) * R;
@@ -231,6 +233,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.main_rank = at<int32_t>(dev_ptr, h->off[W_MAIN_RANK]);
   w.main_local = at<int32_t>(dev_ptr, h->off[W_MAIN_LOCAL]);
   w.main_inst_expert = at<int32_t>(dev_ptr, h->off[W_MAIN_INST]);
+  w.solve_static = at<int32_t>(dev_ptr, h->off[W_SOLVE_STATIC]);
   w.status = at<uint32_t>(dev_ptr, h->off[W_STATUS]);
   w.omega = at<int32_t>(dev_ptr, h->off[W_OMEGA]);
   w.omega_m = at<int32_t>(dev_ptr, h->off[W_OMEGA_M]);
@@ -254,6 +257,16 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
                       cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_inst_expert), h->main_inst_expert.data(),
                       4 * h->main_inst_expert.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+  {
+    const size_t per = solve_static_bytes(h->d) / sizeof(int32_t);
+    std::vector<int32_t> blocks((size_t)h->d.M * per);
+    for (int dm = 0; dm < h->d.M; ++dm)
+      solve_static_fill(h->d, dm, h->main_rank.data(), h->main_local.data(),
+                        h->main_inst_expert.data(), h->cost_rank_intra, blocks.data() + dm * per);
+    e = cudaMemcpy(const_cast<int32_t*>(w.solve_static), blocks.data(), 4 * blocks.size(),
+                   cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) goto fail;
+  }
   if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
   if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
@@ -306,6 +319,12 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.expert_bytes = h->cost.expert_bytes;
   sp.max_iters = h->max_iters;
   sp.min_delta = h->min_delta;
+  // 2 D S_tok - ||W|| > 0  <=>  D > floor(||W|| / (2 S_tok)); S_tok = 0 admits no candidate
+  {
+    const long long st = h->cost.token_bytes, wb = h->cost.expert_bytes;
+    const long long thr = st > 0 ? wb / (2 * st) : (long long)INT_MAX;
+    sp.cand_thr = (int)std::min<long long>(thr, INT_MAX);
+  }
   sp.cost_rank_intra = h->cost_rank_intra;
   sp.cost_rank_inter = h->cost_rank_inter;
   sp.out_replica_map = replica_map;

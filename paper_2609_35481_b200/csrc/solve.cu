@@ -30,9 +30,19 @@ namespace {
 constexpr int kRankCap = 128;   // stage 1 ranks up to this many candidates of a domain all-pairs
 
 struct SolveLayout {
-  size_t cand, col_main, col_rep, mrank, mlocal, D, qd, host_lo, host_hi, col_expert, col_cr, U, L,
-      used, cnt, hostcol, sdom, total;
+  size_t cand, col_main, col_rep, stat, mrank, mlocal, host_lo, host_hi, col_expert, col_cr, hostcol,
+      sdom, col_rank, D, qd, U, L, used, cnt, total;
 };
+
+// The static block: everything that depends only on the handle and the domain, laid out in the
+// workspace exactly as in shared memory so that one contiguous copy brings it in.
+//   ints:   mrank[E] mlocal[E] host_lo[E] host_hi[E] col_expert[C] col_cr[C]
+//   shorts: hostcol[G*E] sdom[R] col_rank[C]
+__host__ __device__ inline size_t solve_static_ints(const Dims& d) {
+  const size_t ints = 4 * (size_t)d.E + 2 * (size_t)d.C;
+  const size_t shorts = (size_t)d.G * d.E + d.R + d.C;
+  return (ints + (shorts + 1) / 2 + 3) & ~(size_t)3;
+}
 
 __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
@@ -41,20 +51,23 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   o.cand = at;       at += sizeof(unsigned long long) * (size_t)kRankCap * (kSolveThreads / 32);
   o.col_main = at;   at += sizeof(int) * pad4((size_t)d.G * d.e_loc * d.R);   // [G*e_loc][R]
   o.col_rep = at;    at += sizeof(int) * pad4((size_t)d.G * d.N * d.R);       // [G*N][R]
-  o.mrank = at;      at += sizeof(int) * pad4(d.E);
-  o.mlocal = at;     at += sizeof(int) * pad4(d.E);
-  o.D = at;          at += sizeof(int) * pad4((size_t)d.M * d.E);
-  o.qd = at;         at += sizeof(int) * (size_t)d.R * d.qstride;
+  o.stat = at;
+  o.mrank = at;      at += sizeof(int) * (size_t)d.E;
+  o.mlocal = at;     at += sizeof(int) * (size_t)d.E;
   o.host_lo = at;    at += sizeof(int) * (size_t)d.E;
   o.host_hi = at;    at += sizeof(int) * (size_t)d.E;
   o.col_expert = at; at += sizeof(int) * (size_t)d.C;
   o.col_cr = at;     at += sizeof(int) * (size_t)d.C;
+  o.hostcol = at;    at += sizeof(short) * (size_t)d.G * d.E;
+  o.sdom = at;       at += sizeof(short) * (size_t)d.R;
+  o.col_rank = at;   at += sizeof(short) * (size_t)d.C;
+  at = o.stat + sizeof(int) * solve_static_ints(d);
+  o.D = at;          at += sizeof(int) * pad4((size_t)d.M * d.E);
+  o.qd = at;         at += sizeof(int) * (size_t)d.R * d.qstride;
   o.U = at;          at += sizeof(int) * (size_t)d.C;
   o.L = at;          at += sizeof(int) * (size_t)d.G;
   o.used = at;       at += sizeof(int) * (size_t)d.G;
   o.cnt = at;        at += sizeof(int) * (size_t)d.R * d.G;
-  o.hostcol = at;    at += sizeof(short) * (size_t)d.G * d.E;
-  o.sdom = at;       at += sizeof(short) * (size_t)d.R;
   o.total = (at + 15) & ~(size_t)15;
   return o;
 }
@@ -95,44 +108,22 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   int* used = reinterpret_cast<int*>(smem + lay.used);
   int* cnt = reinterpret_cast<int*>(smem + lay.cnt);
   short* hostcol = reinterpret_cast<short*>(smem + lay.hostcol);
-  short* sdom = reinterpret_cast<short*>(smem + lay.sdom);
+  const short* sdom = reinterpret_cast<const short*>(smem + lay.sdom);
+  const short* col_rank = reinterpret_cast<const short*>(smem + lay.col_rank);   // rank of a column
 
   const int32_t* om_m = p.ws.omega_m + (size_t)b * R * e_loc * R;   // rows = main instances
 
-  // ---- round 1 of asynchronous copies: static tables first, then (once the omega kernel is
-  // done) the demand and this domain's main columns
-  copy_async(mrank, p.ws.main_rank, E, tid, nt);
-  copy_async(mlocal, p.ws.main_local, E, tid, nt);
-  for (int i = tid; i < G * e_loc; i += nt) {
-    const int g = i / e_loc, l = i - g * e_loc;
-    cp_async4(col_expert + g * s_phys + l, p.ws.main_inst_expert + (size_t)(dm * G + g) * e_loc + l);
-  }
-  for (int i = tid; i < G * N; i += nt) col_expert[(i / N) * s_phys + e_loc + i % N] = -1;
-  for (int i = tid; i < G * E; i += nt) hostcol[i] = -1;
-  for (int c = tid; c < C; c += nt) col_cr[c] = p.cost_rank_intra;
-  for (int s = tid; s < R; s += nt) sdom[s] = (short)(s / G);
+  // ---- round 1 of asynchronous copies: the static block of this domain first (main-rank tables,
+  // hosting masks and column tables as they are before any replica exists), then -- once the
+  // omega kernel is done -- the demand and this domain's main columns
+  copy_async(reinterpret_cast<int*>(smem + lay.stat),
+             p.ws.solve_static + (size_t)dm * solve_static_ints(d), (int)solve_static_ints(d), tid, nt);
   if (tid < G) used[tid] = 0;
+  for (int i = tid; i < R * G; i += nt) cnt[i] = 0;
   pdl_wait();
   copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
   copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
   cp_async_wait_all();
-  __syncthreads();
-
-  // ---- hosting masks from the main ranks; keep D only where e is a stage-1 candidate ----------
-  for (int e = tid; e < E; e += nt) {
-    const int md = mrank[e] / G;
-    host_lo[e] = md < 32 ? 1u << md : 0u;
-    host_hi[e] = md < 32 ? 0u : 1u << (md - 32);
-    for (int dd = 0; dd < M; ++dd) {
-      const int v = D[dd * E + e];
-      const bool cand = dd != md && 2 * (long long)v * p.token_bytes - p.expert_bytes > 0;
-      if (!cand) D[dd * E + e] = 0;
-    }
-  }
-  for (int c = tid; c < C; c += nt) {
-    const int e = col_expert[c];
-    if (e >= 0) hostcol[(c / s_phys) * E + e] = (short)c;
-  }
   __syncthreads();
 
   // ---- inter-node placement, every domain, one warp each ------------------------------------
@@ -148,7 +139,14 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       int n_c = 0;
       for (int e0 = 0; e0 < E; e0 += 32) {
         const int e = e0 + lane;
-        const int v = e < E ? Dd[e] : 0;
+        int v = 0;
+        if (e < E) {
+          // a candidate has positive benefit (D above the threshold) and its main elsewhere; bit dd
+          // of the mask is still the main-domain bit here: only this warp ever sets it, below
+          const unsigned hosted = dd < 32 ? host_lo[e] >> dd : host_hi[e] >> (dd - 32);
+          v = (hosted & 1u) ? 0 : Dd[e];
+          v = v > p.cand_thr ? v : 0;
+        }
         const unsigned m = __ballot_sync(full, v > 0);
         const int at = n_c + __popc(m & lanemask_lt());
         if (v > 0 && at < kRankCap)
@@ -176,7 +174,12 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           }
         }
       } else {
-        // many candidates: pick the maximum slot by slot
+        // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
+        for (int e = lane; e < E; e += 32) {
+          const unsigned hosted = dd < 32 ? host_lo[e] >> dd : host_hi[e] >> (dd - 32);
+          if ((hosted & 1u) || Dd[e] <= p.cand_thr) Dd[e] = 0;
+        }
+        __syncwarp();
         for (int i = 0; i < slots; ++i) {
           int bestD = 0, bestE = INT_MAX;
           for (int e = lane; e < E; e += 32) {
@@ -224,40 +227,58 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       __syncthreads();
     }
     const int ncols = pass == 0 ? G * e_loc : G * N;
-    for (int i = warp; i < ncols; i += nwarps) {
-      const int per = pass == 0 ? e_loc : N;
-      const int g = i / per, l = i - g * per;
-      const int c = g * s_phys + (pass == 0 ? l : e_loc + l);
-      const int e = col_expert[c];
-      const int* w_col = (pass == 0 ? col_main : col_rep) + i * R;
-      unsigned long long hm = 0;
-      int n = 1, idx = 0;
-      if (e >= 0) {
-        hm = ((unsigned long long)host_hi[e] << 32) | host_lo[e];
-        n = __popcll(hm);
-        idx = __popcll(hm & ((1ull << dm) - 1ull));
+    const int per = pass == 0 ? e_loc : N;
+    const int* w_base = pass == 0 ? col_main : col_rep;
+    // four columns of a warp at a time, so that their dependent shared-memory reads overlap
+    constexpr int kCols = 4;
+    for (int i0 = warp; i0 < ncols; i0 += kCols * nwarps) {
+      int c[kCols], e[kCols], n[kCols], idx[kCols], usum[kCols];
+      unsigned long long hm[kCols];
+#pragma unroll
+      for (int u = 0; u < kCols; ++u) {
+        const int i = i0 + u * nwarps;
+        const int g = i / per, l = i - g * per;
+        c[u] = g * s_phys + (pass == 0 ? l : e_loc + l);
+        e[u] = i < ncols ? col_expert[c[u]] : -2;   // -1: empty slot, -2: no such column
+        usum[u] = 0;
       }
-      int usum = 0;
+#pragma unroll
+      for (int u = 0; u < kCols; ++u) {
+        hm[u] = 0;
+        n[u] = 1;
+        idx[u] = 0;
+        if (e[u] >= 0) {
+          hm[u] = ((unsigned long long)host_hi[e[u]] << 32) | host_lo[e[u]];
+          n[u] = __popcll(hm[u]);
+          idx[u] = __popcll(hm[u] & ((1ull << dm) - 1ull));
+        }
+      }
       for (int s0 = 0; s0 < R; s0 += 32) {
         const int s = s0 + lane;
-        int v = 0;
-        if (s < R && e >= 0) {
-          const int w = w_col[s];
-          const int ds = sdom[s];
-          if (ds == dm || n == 1) {   // own domain, or the only instance anywhere
-            v = w;
-          } else if (!((hm >> ds) & 1ull)) {
-            const int base = w / n, rem = w - base * n;
-            int sh = idx - (s + e) % n;
-            if (sh < 0) sh += n;
-            v = base + (sh < rem ? 1 : 0);
+        const int ds = s < R ? sdom[s] : 0;
+#pragma unroll
+        for (int u = 0; u < kCols; ++u) {
+          int v = 0;
+          if (s < R && e[u] >= 0) {
+            const int w = w_base[(i0 + u * nwarps) * R + s];
+            if (ds == dm || n[u] == 1) {   // own domain, or the only instance anywhere
+              v = w;
+            } else if (!((hm[u] >> ds) & 1ull)) {
+              const int base = w / n[u], rem = w - base * n[u];
+              int sh = idx[u] - (s + e[u]) % n[u];
+              if (sh < 0) sh += n[u];
+              v = base + (sh < rem ? 1 : 0);
+            }
           }
+          if (s < R && e[u] >= -1) qd[s * QS + c[u]] = v;
+          usum[u] += v;
         }
-        if (s < R) qd[s * QS + c] = v;
-        usum += v;
       }
-      usum = __reduce_add_sync(full, usum);
-      if (lane == 0) U[c] = usum;
+#pragma unroll
+      for (int u = 0; u < kCols; ++u) {
+        const int tot = __reduce_add_sync(full, usum[u]);
+        if (lane == 0 && e[u] >= -1) U[c[u]] = tot;
+      }
     }
   }
   __syncthreads();
@@ -276,7 +297,10 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     // instance slots of the busiest rank
     const int gt = lane % G, k0 = lane / G, kstep = max(32 / G, 1);
     const bool lane_on = lane < G * kstep;
-    for (;;) {
+    // Inter-node placement leaves an expert at most one instance per domain, so a move needs a
+    // target with a free slot; when every slot of the domain is taken there is nothing to do.
+    const bool any_free = __any_sync(full, lane < G && used[lane] < N);
+    for (; any_free;) {
       const int Lg = lane < G ? L[lane] : -1;
       const int Lb = __reduce_max_sync(full, Lg);
       const int gb = __ffs(__ballot_sync(full, Lg == Lb)) - 1;   // busiest, lowest id on ties
@@ -374,19 +398,22 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     if (p.out_inst_counts) p.out_inst_counts[at] = u;
   }
   if (tid < G) p.ws.rank_load[(size_t)b * R + dm * G + tid] = L[tid];
+  // q rows of this domain's columns; counts[s][r] accumulated per (source, rank) on the way
   for (int s = warp; s < R; s += nwarps) {
     int32_t* qrow = p.ws.q + ((size_t)b * R + s) * d.P + (size_t)dm * C;
-    for (int c = lane; c < C; c += 32) qrow[c] = qd[s * QS + c];
-    if (lane < G) {   // counts[s][r] for the ranks r of this domain
-      int sum = 0;
-      for (int l = 0; l < s_phys; ++l) sum += qd[s * QS + lane * s_phys + l];
-      cnt[s * G + lane] = sum;
-      const size_t at = ((size_t)b * R + s) * R + dm * G + lane;
-      p.ws.counts[at] = sum;
-      p.out_counts[at] = sum;
+    for (int c = lane; c < C; c += 32) {
+      const int v = qd[s * QS + c];
+      qrow[c] = v;
+      if (v != 0) atomicAdd(&cnt[s * G + col_rank[c]], v);
     }
   }
   __syncthreads();
+  for (int i = tid; i < R * G; i += nt) {
+    const int s = i / G, g = i - s * G;
+    const size_t at = ((size_t)b * R + s) * R + dm * G + g;
+    p.ws.counts[at] = cnt[i];
+    p.out_counts[at] = cnt[i];
+  }
   // receive offsets of rank r: exclusive scan over the sources, one warp per rank
   for (int g = warp; g < G; g += nwarps) {
     int32_t* recv = p.out_offsets + (((size_t)b * 2 + 1) * R + dm * G + g) * (R + 1);
@@ -404,6 +431,40 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
 }  // namespace
 
 size_t solve_smem_bytes(const Dims& d) { return solve_layout(d).total; }
+
+size_t solve_static_bytes(const Dims& d) { return sizeof(int32_t) * solve_static_ints(d); }
+
+void solve_static_fill(const Dims& d, int dm, const int32_t* main_rank, const int32_t* main_local,
+                       const int32_t* main_inst_expert, int cost_rank_intra, int32_t* out) {
+  const int E = d.E, G = d.G, C = d.C, R = d.R;
+  int32_t* mrank = out;
+  int32_t* mlocal = mrank + E;
+  int32_t* host_lo = mlocal + E;
+  int32_t* host_hi = host_lo + E;
+  int32_t* col_expert = host_hi + E;
+  int32_t* col_cr = col_expert + C;
+  short* hostcol = reinterpret_cast<short*>(col_cr + C);
+  short* sdom = hostcol + (size_t)G * E;
+  short* col_rank = sdom + R;
+  for (size_t i = 0; i < solve_static_ints(d); ++i) out[i] = 0;
+  for (int e = 0; e < E; ++e) {
+    mrank[e] = main_rank[e];
+    mlocal[e] = main_local[e];
+    const int md = main_rank[e] / G;   // the expert's main domain hosts it from the start
+    host_lo[e] = md < 32 ? (int32_t)(1u << md) : 0;
+    host_hi[e] = md < 32 ? 0 : (int32_t)(1u << (md - 32));
+  }
+  for (int i = 0; i < G * E; ++i) hostcol[i] = -1;
+  for (int c = 0; c < C; ++c) {
+    const int g = c / d.s_phys, l = c - g * d.s_phys;
+    const int e = l < d.e_loc ? main_inst_expert[(size_t)(dm * G + g) * d.e_loc + l] : -1;
+    col_expert[c] = e;
+    col_cr[c] = cost_rank_intra;
+    col_rank[c] = (short)g;
+    if (e >= 0) hostcol[(size_t)g * E + e] = (short)c;
+  }
+  for (int s = 0; s < R; ++s) sdom[s] = (short)(s / G);
+}
 
 cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.d.M, batch);

@@ -33,6 +33,7 @@ struct Workspace {
   const int32_t* main_rank;         // [E]
   const int32_t* main_local;        // [E] index l of e among the experts of its main rank
   const int32_t* main_inst_expert;  // [R][e_loc] expert of main instance l on rank r, -1 if none
+  const int32_t* solve_static;      // [M][solve_static_ints]: per-domain static block of the solver
   uint32_t* status;                 // [1]
   int32_t* omega;                   // [max_batch][R][E]
   int32_t* omega_m;                 // [max_batch][R*e_loc][R] omega transposed, one row per main
@@ -106,6 +107,7 @@ struct SolveParams {
   int pdl;   // launched with programmatic dependent launch
   int64_t token_bytes, expert_bytes;
   int max_iters, min_delta;
+  int cand_thr;   // demand D of a stage-1 candidate exceeds this: floor(||W|| / (2 S_tok))
   int cost_rank_intra, cost_rank_inter;   // dense ranks of {0, c_intra*W, c_inter*W}
   int32_t* out_replica_map;   // [B][R][N]
   int32_t* out_counts;        // [B][R][R]
@@ -166,6 +168,10 @@ struct SummaryParams {
 
 size_t hist_smem_bytes(const Dims& d);
 size_t solve_smem_bytes(const Dims& d);
+size_t solve_static_bytes(const Dims& d);   // bytes of one domain's static block
+// fills one domain's static block (host memory) from the main-rank tables
+void solve_static_fill(const Dims& d, int dm, const int32_t* main_rank, const int32_t* main_local,
+                       const int32_t* main_inst_expert, int cost_rank_intra, int32_t* out);
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
