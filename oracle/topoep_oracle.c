@@ -51,6 +51,10 @@
  *     flat index t*k+j and dealt to the instances in ascending rank order,
  *     instance r taking q[s][e][r] of them.
  *   - ids outside [0,E) are ignored everywhere and map to -1.
+ *   - the paper does not say whether inter-node placement leaves slots for the refinement; by
+ *     default it does not (its slot-count experiment reports no gain from refinement with one
+ *     slot per rank).  reserve_slots > 0 is a policy variant of ours: stage 1 fills at most
+ *     N_slot - reserve_slots slots of a rank.
  *
  * Parity status: O1, O8 are pinned to library routines (bincount, cumsum);
  * O3-O6 are pinned by the paper's worked two-domain example, hand-derived
@@ -74,6 +78,9 @@ typedef struct {
   int32_t max_refine_iters; /* <= 0 -> 256 */
   int32_t min_delta;        /* <= 0 -> 1   */
   int32_t stages;           /* bit 0: run inter-node placement; bit 1: run refinement */
+  int32_t reserve_slots;    /* non-default policy: slots per rank that inter-node placement
+                               must leave free for the refinement (0 = the paper's behaviour) */
+  int32_t pad_;
   int64_t token_bytes;      /* S_tok */
   int64_t expert_bytes;     /* ||W|| */
   int64_t t_ffn;            /* t_FFN */
@@ -159,6 +166,9 @@ static void domain_demand(const oracle_config* c, const int64_t* omega, int64_t*
 static void inter_node_placement(const oracle_config* c, const int32_t* main_rank,
                                  const int64_t* D, int8_t* x, int32_t* slotmap, int32_t* used) {
   const int M = c->nodes, G = c->gpus_per_node, E = c->experts, R = M * G, N = c->slots_per_rank;
+  /* slots this stage may fill on a rank: all of them unless the reservation policy is on */
+  int cap = N - (c->reserve_slots > 0 ? c->reserve_slots : 0);
+  if (cap < 0) cap = 0;
   if (M == 1) return;
   int8_t* taken = (int8_t*)malloc((size_t)E);
   for (int d = 0; d < M; ++d) {
@@ -177,7 +187,7 @@ static void inter_node_placement(const oracle_config* c, const int32_t* main_ran
       /* least occupied rank of d that still has a free slot */
       int best_r = -1;
       for (int r = d * G; r < (d + 1) * G; ++r)
-        if (used[r] < N && (best_r < 0 || used[r] < used[best_r])) best_r = r;
+        if (used[r] < cap && (best_r < 0 || used[r] < used[best_r])) best_r = r;
       if (best_r < 0) break;
       slotmap[(size_t)best_r * N + used[best_r]] = best_e;
       x[(size_t)best_e * R + best_r] = 1;

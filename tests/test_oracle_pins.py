@@ -620,3 +620,65 @@ def test_replica_transfers_identity_code(seed):
             if rmap[r, j] >= 0:
                 m, l = where[int(rmap[r, j])]
                 assert np.array_equal(acc2[m, r, l], mp[m, l])
+
+
+# ---- policy variant: slots reserved for the refinement -------------------------------------------
+def _skewed_case(seed, nodes=2, gpus=4, experts=32, slots=3, tokens=600, k=2):
+    w = wl.CONFIGS["tiny"].replace(nodes=nodes, gpus_per_node=gpus, experts=experts,
+                                   slots_per_rank=slots, tokens_per_rank=tokens, top_k=k,
+                                   zipf_s=1.4, ffn=16)   # small experts: many candidates
+    ids = wl.make_topk_ids(w, seed=seed)
+    return w, ids
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_reserved_slots_stage1_takes_the_top_candidates_only(seed):
+    """With r slots reserved, inter-node placement alone (stages = 1) must fill exactly the
+    (N - r) * G best candidates of each domain, in the order (benefit down, expert id up), dealt
+    round-robin over the ranks -- recomputed here with a plain sort."""
+    w, ids = _skewed_case(seed)
+    M, G, E, N = w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank
+    mr = w.main_rank()
+    for reserve in (0, 1, 2, 3):
+        cfg = orc.OracleConfig(M, G, E, N, w.top_k, w.token_bytes, w.expert_bytes, main_rank=mr,
+                               stages=1, reserve_slots=reserve)
+        res = orc.plan(cfg, ids)
+        omega = res.omega[0]
+        D = omega.reshape(M, G, E).sum(axis=1)
+        for d in range(M):
+            b = 2 * D[d] * w.token_bytes - w.expert_bytes
+            cands = [e for e in range(E) if mr[e] // G != d and b[e] > 0]
+            cands.sort(key=lambda e: (-b[e], e))
+            assert len(cands) > (N - 1) * G          # the capacity binds whenever reserve >= 1
+            take = cands[:(N - reserve) * G]
+            want = np.full((G, N), -1, np.int32)
+            for i, e in enumerate(take):
+                want[i % G, i // G] = e
+            assert np.array_equal(res.replica_map[0, d * G:(d + 1) * G], want), (reserve, d)
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_reserving_every_slot_equals_refinement_only(seed):
+    w, ids = _skewed_case(seed)
+    kw = dict(main_rank=w.main_rank())
+    a = orc.plan(orc.OracleConfig(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
+                                  w.token_bytes, w.expert_bytes, reserve_slots=w.slots_per_rank,
+                                  **kw), ids)
+    b = orc.plan(orc.OracleConfig(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
+                                  w.token_bytes, w.expert_bytes, stages=2, **kw), ids)
+    for name in ("replica_map", "token_replica", "dispatch_counts", "instance_counts", "rank_load"):
+        assert np.array_equal(getattr(a, name), getattr(b, name)), name
+    assert a.refine_iters.sum() > 0
+
+
+@pytest.mark.parametrize("reserve", [1, 2])
+def test_reserved_slots_keep_every_constraint(reserve):
+    w, ids = _skewed_case(7)
+    cfg = orc.OracleConfig(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
+                           w.token_bytes, w.expert_bytes, main_rank=w.main_rank(),
+                           reserve_slots=reserve)
+    res = orc.plan(cfg, ids)
+    check_plan(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k, w.main_rank(),
+               w.token_bytes, w.expert_bytes, ids[0], res.replica_map[0], res.token_replica[0],
+               res.dispatch_counts[0], res.dispatch_offsets[0], res.instance_counts[0],
+               res.rank_load[0])
