@@ -317,6 +317,18 @@ int topoep_debug_tensor(topoep_handle_t h, int which, const void** dev_ptr, size
 int topoep_set_tuning(topoep_handle_t h, int knob, int value);
 
 /*
+ * Policy variants (NOT tuning: they change the plan).  The defaults reproduce the paper's
+ * procedure as read here.
+ *   TOPOEP_POLICY_RESERVE_SLOTS = r (0 <= r <= N_slot, default 0): inter-node placement fills at
+ *     most N_slot - r replica slots of a rank, leaving r to the intra-node refinement.  The paper
+ *     does not say whether slots are held back; by default none are, and with one slot per rank
+ *     the refinement then has nothing to work with (paper, slot-count experiment).
+ * Takes effect from the next topoep_plan / topoep_solve.
+ */
+enum { TOPOEP_POLICY_RESERVE_SLOTS = 0 };
+int topoep_set_policy(topoep_handle_t h, int policy, int value);
+
+/*
  * Replica parameter executor (paper, "Device-initiated replica transfers", with the three
  * buffers that subsection lists).  Copies driven by the device-resident replica map of ONE plan
  * (dev_replica_map [R][N_slot], e.g. one plan's slice of topoep_plan's output): no host read of

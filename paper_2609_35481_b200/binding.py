@@ -22,7 +22,7 @@ KNOB_TILE_IDS, KNOB_HIST_MODE, KNOB_PDL, KNOB_TRANSFER_MODE = 0, 1, 2, 3
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
            "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions",
            "topoep_summary", "topoep_read_status",
-           "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_replica_pull", "topoep_replica_grad_return",
+           "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_set_policy", "topoep_replica_pull", "topoep_replica_grad_return",
            "topoep_get_layout",
            "topoep_launch_floor", "topoep_strerror")
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.topoep_debug_tensor.argtypes = [vp, ci, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
         L.topoep_set_tuning.restype = ci
         L.topoep_set_tuning.argtypes = [vp, ci, ci]
+        L.topoep_set_policy.restype = ci
+        L.topoep_set_policy.argtypes = [vp, ci, ci]
         L.topoep_set_rank_window.restype = ci
         L.topoep_set_rank_window.argtypes = [vp, ci, ci]
         for fn in (L.topoep_replica_pull, L.topoep_replica_grad_return):
@@ -213,6 +215,13 @@ def topoep_debug_tensor(h, which: int):
 
 def topoep_set_tuning(h, knob: int, value: int) -> int:
     return lib().topoep_set_tuning(h, knob, value)
+
+
+POLICY_RESERVE_SLOTS = 0
+
+
+def topoep_set_policy(h, policy: int, value: int) -> int:
+    return lib().topoep_set_policy(h, policy, value)
 
 
 def topoep_set_rank_window(h, first_rank: int, rank_count: int) -> int:

@@ -17,6 +17,7 @@ struct topoep_ctx {
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode, pdl;
+  int reserve_slots;   // policy: slots per rank left to the refinement by inter-node placement
   int rank_first, rank_count;   // window of source ranks of the histogram / reroute buffers
   size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
   int transfer_ready, transfer_mode, sms;   // replica executor: configured?, copy engine, SM count
@@ -199,6 +200,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->tile_ids = 4096;
   h->hist_mode = 0;
   h->pdl = 1;
+  h->reserve_slots = 0;
   h->rank_first = 0;
   h->rank_count = (int)R;
   h->dispatch_smem = 0;
@@ -325,6 +327,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
     const long long thr = st > 0 ? wb / (2 * st) : (long long)INT_MAX;
     sp.cand_thr = (int)std::min<long long>(thr, INT_MAX);
   }
+  sp.stage1_slots = std::max(0, h->d.N - h->reserve_slots);
   sp.cost_rank_intra = h->cost_rank_intra;
   sp.cost_rank_inter = h->cost_rank_inter;
   sp.out_replica_map = replica_map;
@@ -613,6 +616,18 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_TRANSFER_MODE:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->transfer_mode = value;
+      return TOPOEP_OK;
+    default:
+      return TOPOEP_ERR_ARG;
+  }
+}
+
+int topoep_set_policy(topoep_handle_t h, int policy, int value) {
+  if (!h) return TOPOEP_ERR_NULL;
+  switch (policy) {
+    case TOPOEP_POLICY_RESERVE_SLOTS:
+      if (value < 0 || value > h->d.N) return TOPOEP_ERR_ARG;
+      h->reserve_slots = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

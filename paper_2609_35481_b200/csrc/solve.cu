@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   // Candidates in descending (b, then ascending e) order == descending (D, ascending e) for a
   // uniform ||W|| and S_tok; the i-th goes to rank i mod G, slot i / G (fewest used slots first,
   // ties to the lower rank).
-  if (M > 1 && N > 0) {
-    const int slots = G * N;
+  if (M > 1 && p.stage1_slots > 0) {
+    const int slots = G * p.stage1_slots;   // all N per rank unless some are reserved
     for (int dd = warp; dd < M; dd += nwarps) {
       int* Dd = D + dd * E;
       // compact the candidates (D > 0) of this domain into cand[]: key = (D, -e)

@@ -238,6 +238,12 @@ class Planner:
         raw = self.workspace[off:off + batch * per].cpu().numpy()
         return torch.from_numpy(raw.view(np.int32).reshape((batch,) + shape).copy())
 
+    def set_policy(self, policy: int, value: int):
+        """Policy variants change the plan (unlike tuning knobs); see topoep_set_policy."""
+        rc = B.topoep_set_policy(self.handle, policy, value)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+
     def set_tuning(self, knob: int, value: int):
         rc = B.topoep_set_tuning(self.handle, knob, value)
         if rc != B.OK:

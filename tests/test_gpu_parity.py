@@ -247,6 +247,29 @@ def test_stage_entry_points_equal_the_fused_plan():
     assert pl.status() == 0
 
 
+# ---- policy variant: slots reserved for the refinement ------------------------------------------
+@pytest.mark.parametrize("name,over,reserve", [
+    ("dsv3", dict(slots_per_rank=2, tokens_per_rank=2048), 1),
+    ("dsv3", dict(slots_per_rank=4, tokens_per_rank=2048), 3),
+    ("mid", dict(slots_per_rank=1), 1),                    # everything reserved: refinement only
+    ("scaleout", dict(slots_per_rank=3, tokens_per_rank=2048, zipf_s=1.0), 2),
+    ("tiny", dict(slots_per_rank=3, ffn=16), 1),           # many candidates, capacity binds
+])
+def test_reserved_slots_policy_matches_the_oracle(name, over, reserve):
+    w = wl.CONFIGS[name].replace(**over)
+    ids = wl.make_topk_ids(w, seed=41, batch=2)
+    pl = make_planner(w, max_batch=2)
+    pl.set_policy(B.POLICY_RESERVE_SLOTS, reserve)
+    gpu = run_gpu(pl, ids)
+    ref = orc.plan(oracle_config(w, reserve_slots=reserve), ids)
+    assert_same(gpu, ref)
+    assert ref.refine_iters.sum() > 0
+    assert B.topoep_set_policy(pl.handle, B.POLICY_RESERVE_SLOTS, w.slots_per_rank + 1) == -10
+    # back to the default: the paper's procedure again
+    pl.set_policy(B.POLICY_RESERVE_SLOTS, 0)
+    assert_same(run_gpu(pl, ids), orc.plan(oracle_config(w), ids))
+
+
 # ---- sharded deployment: every rank plans from the gathered routing matrix -----------------------
 @pytest.mark.parametrize("name,over,batch,window", [
     ("mid", dict(slots_per_rank=3), 2, 1),
@@ -420,3 +443,28 @@ def test_size_and_pointer_errors():
     # a rejected set_workspace leaves the previous workspace in place
     assert B.topoep_plan(pl.handle, ids, w.tokens_per_rank, 1, *args) == 0
     torch.cuda.synchronize()
+
+
+def test_imbalance_against_slot_count_on_the_slot_experiment_shape():
+    """The shape of the paper's slot-count experiment (32 ranks, 640 experts, top-8; its routing
+    trace is not public, so Zipf-skewed synthetic routing stands in): the max/mean rank load of the
+    CUDA plan equals the oracle's for every slot count and policy, replicas never make it worse
+    than no replicas, and holding one slot back for the refinement helps when slots are scarce."""
+    base = wl.CONFIGS["dsv3"].replace(experts=640, tokens_per_rank=2048, zipf_s=1.2, bursts=0)
+    ids = wl.make_topk_ids(base, seed=51)
+    table = {}
+    for slots in (0, 1, 2, 4):
+        for reserve in (0, 1):
+            if reserve > slots:
+                continue
+            w = base.replace(slots_per_rank=slots)
+            pl = make_planner(w)
+            pl.set_policy(B.POLICY_RESERVE_SLOTS, reserve)
+            gpu = run_gpu(pl, ids)
+            ref = orc.plan(oracle_config(w, reserve_slots=reserve), ids)
+            assert_same(gpu, ref)
+            table[(slots, reserve)] = float(gpu["summaries"]["imbalance"][0])
+    print("imbalance (slots, reserve):", {k: round(v, 3) for k, v in table.items()})
+    none = table[(0, 0)]
+    assert all(v <= none + 1e-9 for v in table.values())
+    assert table[(1, 1)] < table[(1, 0)]
