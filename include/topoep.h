@@ -285,12 +285,36 @@ int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_pe
  *   dev_scratch          device memory, 256-byte aligned, at least
  *                            topoep_dispatch_scratch_bytes(h, T, B) long; contents
  *                            need not be kept between calls
- * Uses q and U of the plan still in the workspace: call it after topoep_plan
- * (or topoep_solve + topoep_reroute) of the same batch.  Enqueues three kernels;
- * capturable after its first call.  Off the planning path: the ranking kernel is
- * bound by instruction issue, not by HBM.
+ * Works from dev_token_replica alone (nothing of the plan in the workspace is
+ * read).  Enqueues four kernels; capturable after its first call.  Off the
+ * planning path: the ranking kernel is bound by instruction issue, not by HBM.
+ *
+ * topoep_dispatch_window is the same for a window of tokens, first_token ..
+ * first_token + token_count - 1 of every source rank -- one chunk of the paper's
+ * two-chunk pipeline ("Fine-Grained Pipelined Execution": the routed tokens are
+ * partitioned into two disjoint chunks that are dispatched one after the other;
+ * the paper does not say how they are cut, here a chunk is a range of token
+ * indices).  dev_token_replica stays the whole [B][R][T][k] tensor; the chunk has
+ * its own send and receive buffers:
+ *   dev_send_pos, dev_recv_pos out [B][R][token_count][k] positions inside the
+ *                                  chunk's buffers
+ *   dev_instance_offsets       out [B][R][S_phys+1] of the chunk, or NULL
+ *   dev_counts                 out [B][R][R] assignments of the chunk from source
+ *                                  s executed on rank r, or NULL
+ *   dev_offsets                out [B][2][R][R+1] the chunk's send / receive
+ *                                  offsets (layout of dev_dispatch_offsets), or NULL
+ *   dev_scratch                at least topoep_dispatch_scratch_bytes(h,
+ *                                  token_count, B) long
+ * The counts of disjoint windows that cover all tokens add up to the plan's
+ * dev_dispatch_counts.  TOPOEP_ERR_SIZE if the window leaves [0, T].
  */
 size_t topoep_dispatch_scratch_bytes(topoep_handle_t h, int tokens_per_rank, int batch);
+int topoep_dispatch_window(topoep_handle_t h, const int32_t* dev_token_replica,
+                           int tokens_per_rank, int batch, int first_token, int token_count,
+                           int32_t* dev_send_pos, int32_t* dev_recv_pos,
+                           int32_t* dev_instance_offsets, int32_t* dev_counts,
+                           int32_t* dev_offsets, void* dev_scratch, size_t scratch_bytes,
+                           topoep_stream_t stream);
 int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replica,
                               int tokens_per_rank, int batch, int32_t* dev_send_pos,
                               int32_t* dev_recv_pos, int32_t* dev_instance_offsets,

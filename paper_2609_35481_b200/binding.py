@@ -20,7 +20,7 @@ T_OMEGA, T_Q, T_RANK_LOAD, T_REFINE_ITERS = 0, 1, 2, 3
 KNOB_TILE_IDS, KNOB_HIST_MODE, KNOB_PDL, KNOB_TRANSFER_MODE = 0, 1, 2, 3
 
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
-           "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions",
+           "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions", "topoep_dispatch_window",
            "topoep_summary", "topoep_read_status",
            "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_set_policy", "topoep_replica_pull", "topoep_replica_grad_return",
            "topoep_get_layout",
@@ -80,6 +80,9 @@ def lib() -> ctypes.CDLL:
         L.topoep_dispatch_scratch_bytes.argtypes = [vp, ci, ci]
         L.topoep_dispatch_positions.restype = ci
         L.topoep_dispatch_positions.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.topoep_dispatch_window.restype = ci
+        L.topoep_dispatch_window.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp,
+                                             ctypes.c_size_t, vp]
         L.topoep_summary.restype = ci
         L.topoep_summary.argtypes = [vp, ci, vp, vp]
         L.topoep_read_status.restype = ci
@@ -193,6 +196,16 @@ def topoep_dispatch_positions(h, dev_token_replica, tokens_per_rank, batch, dev_
                                            _ptr(dev_send_pos), _ptr(dev_recv_pos),
                                            _ptr(dev_instance_offsets), _ptr(dev_scratch),
                                            scratch_bytes, stream or None)
+
+
+def topoep_dispatch_window(h, dev_token_replica, tokens_per_rank, batch, first_token, token_count,
+                           dev_send_pos, dev_recv_pos, dev_instance_offsets, dev_counts,
+                           dev_offsets, dev_scratch, scratch_bytes, stream=0) -> int:
+    return lib().topoep_dispatch_window(h, _ptr(dev_token_replica), tokens_per_rank, batch,
+                                        first_token, token_count, _ptr(dev_send_pos),
+                                        _ptr(dev_recv_pos), _ptr(dev_instance_offsets),
+                                        _ptr(dev_counts), _ptr(dev_offsets), _ptr(dev_scratch),
+                                        scratch_bytes, stream or None)
 
 
 def topoep_summary(h, batch, dev_out, stream=0) -> int:

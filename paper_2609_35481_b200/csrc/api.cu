@@ -89,6 +89,8 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   p.ids = ids;
   p.out_omega = out_omega;
   p.n_ids = T * h->d.k;
+  p.row_stride = p.n_ids;
+  p.first_id = 0;
   p.tile_ids = h->tile_ids;
   p.tiles = std::max(1, (p.n_ids + h->tile_ids - 1) / h->tile_ids);
   p.max_tiles = h->max_tiles;
@@ -448,28 +450,33 @@ size_t topoep_dispatch_scratch_bytes(topoep_handle_t h, int tokens_per_rank, int
   const size_t n_ids = (size_t)tokens_per_rank * h->d.k;
   const size_t tiles = std::max<size_t>(1, (n_ids + h->tile_ids - 1) / h->tile_ids);
   const size_t rows = (size_t)batch * h->d.R;
-  return kAlign + align_up(4 * rows * h->d.P) * 2 + align_up(4 * rows * tiles * h->d.P);
+  return kAlign + align_up(4 * rows * h->d.P) * 3 + align_up(4 * rows * tiles * h->d.P);
 }
 
-int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replica,
-                              int tokens_per_rank, int batch, int32_t* dev_send_pos,
-                              int32_t* dev_recv_pos, int32_t* dev_instance_offsets,
-                              void* dev_scratch, size_t scratch_bytes, topoep_stream_t stream) {
+int topoep_dispatch_window(topoep_handle_t h, const int32_t* dev_token_replica,
+                           int tokens_per_rank, int batch, int first_token, int token_count,
+                           int32_t* dev_send_pos, int32_t* dev_recv_pos,
+                           int32_t* dev_instance_offsets, int32_t* dev_counts,
+                           int32_t* dev_offsets, void* dev_scratch, size_t scratch_bytes,
+                           topoep_stream_t stream) {
   int rc = check_sizes(h, tokens_per_rank, batch);
   if (rc != TOPOEP_OK) return rc;
+  if (first_token < 0 || token_count < 0 || first_token > tokens_per_rank - token_count)
+    return TOPOEP_ERR_SIZE;
   if (batch == 0) return TOPOEP_OK;
   if (!dev_scratch) return TOPOEP_ERR_NULL;
   if (h->rank_count != h->d.R) return TOPOEP_ERR_ARG;   // needs every rank's assignments
-  if (tokens_per_rank > 0 && (!dev_token_replica || !dev_send_pos || !dev_recv_pos))
+  if (token_count > 0 && (!dev_token_replica || !dev_send_pos || !dev_recv_pos))
     return TOPOEP_ERR_NULL;
   if (!aligned4(dev_token_replica) || !aligned4(dev_send_pos) || !aligned4(dev_recv_pos) ||
-      !aligned4(dev_instance_offsets))
+      !aligned4(dev_instance_offsets) || !aligned4(dev_counts) || !aligned4(dev_offsets))
     return TOPOEP_ERR_ALIGN;
-  if (scratch_bytes < topoep_dispatch_scratch_bytes(h, tokens_per_rank, batch) ||
+  if (scratch_bytes < topoep_dispatch_scratch_bytes(h, token_count, batch) ||
       (reinterpret_cast<uintptr_t>(dev_scratch) % kAlign) != 0)
     return TOPOEP_ERR_WORKSPACE;
   if (((size_t)h->d.P + 1) * sizeof(int) > 48 * 1024 ||
-      pos_rank_smem_bytes(h->d, h->tile_ids) > 227 * 1024)
+      pos_rank_smem_bytes(h->d, h->tile_ids) > 227 * 1024 ||
+      pos_prefix_smem_bytes(h->d) > 227 * 1024)
     return TOPOEP_ERR_SMEM;
   PosParams p;
   p.d = h->d;
@@ -478,24 +485,39 @@ int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replic
   p.out_send_pos = dev_send_pos;
   p.out_recv_pos = dev_recv_pos;
   p.out_instance_offsets = dev_instance_offsets;
-  p.n_ids = tokens_per_rank * h->d.k;
+  p.out_counts = dev_counts;
+  p.out_offsets = dev_offsets;
+  p.n_ids = token_count * h->d.k;
+  p.row_stride = (long long)tokens_per_rank * h->d.k;
+  p.first_id = (long long)first_token * h->d.k;
   p.tile_ids = h->tile_ids;
   p.tiles = std::max(1, (p.n_ids + p.tile_ids - 1) / p.tile_ids);
   const size_t rows = (size_t)batch * h->d.R;
+  const size_t per = align_up(4 * rows * h->d.P);
   char* base = static_cast<char*>(dev_scratch);
   p.scratch_status = reinterpret_cast<uint32_t*>(base);
   p.pos_a = reinterpret_cast<int32_t*>(base + kAlign);
-  p.pos_b = reinterpret_cast<int32_t*>(base + kAlign + align_up(4 * rows * h->d.P));
-  p.pos_cnt = reinterpret_cast<int32_t*>(base + kAlign + 2 * align_up(4 * rows * h->d.P));
+  p.pos_b = reinterpret_cast<int32_t*>(base + kAlign + per);
+  p.pos_tot = reinterpret_cast<int32_t*>(base + kAlign + 2 * per);
+  p.pos_cnt = reinterpret_cast<int32_t*>(base + kAlign + 3 * per);
   cudaError_t e = cudaSuccess;
   if (!h->dispatch_smem) {
     // first use: opt in to the shared memory the kernels need (host-side attribute only)
     e = configure_dispatch(h->d);
     if (e == cudaSuccess) h->dispatch_smem = 1;
   }
-  if (e == cudaSuccess) e = launch_dispatch(p, batch, stream);
+  if (e == cudaSuccess) e = launch_dispatch(p, batch, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
+}
+
+int topoep_dispatch_positions(topoep_handle_t h, const int32_t* dev_token_replica,
+                              int tokens_per_rank, int batch, int32_t* dev_send_pos,
+                              int32_t* dev_recv_pos, int32_t* dev_instance_offsets,
+                              void* dev_scratch, size_t scratch_bytes, topoep_stream_t stream) {
+  return topoep_dispatch_window(h, dev_token_replica, tokens_per_rank, batch, 0, tokens_per_rank,
+                                dev_send_pos, dev_recv_pos, dev_instance_offsets, nullptr, nullptr,
+                                dev_scratch, scratch_bytes, stream);
 }
 
 namespace {

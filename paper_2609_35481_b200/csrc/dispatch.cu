@@ -9,10 +9,12 @@
 //   recv buffer of rank r   : ordered by (instance, source rank, flat index) -- every instance's
 //                             tokens contiguous (grouped GEMM), sources in rank order inside.
 //
-// Both are stable sorts of token_replica, done as counting sorts with P bins in three kernels:
+// Both are stable sorts of token_replica, done as counting sorts with P bins in four kernels:
 //   1. per-tile histogram of p            (the histogram kernel, P bins instead of E)
-//   2. pos_prefix_kernel, CTA = (plan, source): prefix over tiles of the tile counts, and the
-//      per-(source, instance) bases A0[p] (send) and B0[p] (receive) from the plan's q and U
+//   2. pos_tile_prefix_kernel, CTA = (plan, source): prefix over tiles of the tile counts and the
+//      totals per (source, instance); pos_base_kernel, CTA = (plan, source): from the totals of
+//      all sources the bases A0[p] (send) and B0[p] (receive), the instance offsets and, for a
+//      window of tokens, its own dispatch counts and offsets
 //   3. pos_rank_kernel, CTA = tile: stable rank of each assignment among the tile's equal p
 //      (per-warp counters; lanes of a warp step that share an instance are ordered by ballots),
 //      added to the bases.
@@ -26,51 +28,83 @@ namespace {
 
 constexpr int kPosThreads = 256;
 
-__global__ void __launch_bounds__(kPosThreads) pos_prefix_kernel(const PosParams p) {
-  extern __shared__ int sm[];   // [P] q row, per-warp totals, [P] instance counts
+// 2a. CTA = (plan, source): exclusive prefix over tiles of the tile counts, in place, and the
+// totals tot[s][p] = assignments of source s on instance p inside the window.
+__global__ void __launch_bounds__(kPosThreads) pos_tile_prefix_kernel(const PosParams p) {
+  const int P = p.d.P;
+  const int s = blockIdx.x, b = blockIdx.y;
+  const size_t row = (size_t)b * p.d.R + s;
+  int32_t* cnt = p.pos_cnt + row * (size_t)p.tiles * P;
+  for (int i = threadIdx.x; i < P; i += blockDim.x) {
+    int run = 0;
+    for (int t0 = 0; t0 < p.tiles; t0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? cnt[(size_t)(t0 + u) * P + i] : 0;
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (t0 + u < p.tiles) { cnt[(size_t)(t0 + u) * P + i] = run; run += v[u]; }
+    }
+    p.pos_tot[row * P + i] = run;
+  }
+}
+
+// 2b. CTA = (plan, source): bases of (source, instance) in the send and receive buffers, from the
+// totals of every source -- nothing here depends on the plan in the workspace, so the positions
+// of any window of tokens (a chunk of a two-chunk pipeline) come out the same way as a whole
+// plan's.  Also the window's dispatch counts and offsets (row s) and the instance offsets.
+__global__ void __launch_bounds__(kPosThreads) pos_base_kernel(const PosParams p) {
+  extern __shared__ int sm[];   // mine[P], lower[P], U[P], per-warp totals, crow[R], lrow[R]
   const Dims d = p.d;
   const int R = d.R, P = d.P, s_phys = d.s_phys;
   const int s = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
-  int* qrow = sm;
-  int* warp_tot = sm + P;
+  int* mine = sm;
+  int* lower = sm + P;
+  int* Us = sm + 2 * P;
+  int* warp_tot = sm + 3 * P;
+  int* crow = warp_tot + nw + 1;
+  int* lrow = crow + R;
   const size_t row = (size_t)b * R + s;
-  for (int i = tid; i < P; i += nt) qrow[i] = p.ws.q[row * P + i];
+  const int32_t* tot = p.pos_tot + (size_t)b * R * P;
+  // column sums over the sources: everything (U) and the sources below s (loads eight at a time)
+  for (int i = tid; i < P; i += nt) {
+    int lo = 0, all = 0;
+    for (int s0 = 0; s0 < R; s0 += 8) {
+      int v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = s0 + u < R ? __ldg(tot + (size_t)(s0 + u) * P + i) : 0;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        all += v[u];
+        lo += s0 + u < s ? v[u] : 0;
+      }
+    }
+    Us[i] = all;
+    lower[i] = lo;
+    mine[i] = __ldg(tot + (size_t)s * P + i);
+  }
   __syncthreads();
-
-  // A0[p] = number of assignments of source s executed on instances below p (exclusive scan)
+  // A0[p] = assignments of source s on instances below p (exclusive scan over p)
   int32_t* A0 = p.pos_a + row * P;
   {
     const int chunk = (P + nt - 1) / nt;
     const int i0 = min(P, tid * chunk), i1 = min(P, i0 + chunk);
     int sum = 0;
-    for (int i = i0; i < i1; ++i) sum += qrow[i];
+    for (int i = i0; i < i1; ++i) sum += mine[i];
     int total;
     int ex = warp_exclusive_scan(sum, lane, &total);
     if (lane == 0) warp_tot[warp] = total;
     __syncthreads();
     for (int w = 0; w < warp; ++w) ex += warp_tot[w];
-    for (int i = i0; i < i1; ++i) { A0[i] = ex; ex += qrow[i]; }
+    for (int i = i0; i < i1; ++i) { A0[i] = ex; ex += mine[i]; }
   }
-  // B0[p] = start of instance p's segment in its rank's receive buffer + assignments of lower
-  // source ranks on p (loads issued eight at a time)
+  // B0[p] = start of instance p's segment in its rank's receive buffer + lower sources on p
   int32_t* B0 = p.pos_b + row * P;
-  int* Us = warp_tot + nw + 1;   // [P] instance counts U
-  const int32_t* U = p.ws.inst_counts + (size_t)b * P;
-  for (int i = tid; i < P; i += nt) Us[i] = U[i];
-  __syncthreads();
   for (int i = tid; i < P; i += nt) {
     const int r = i / s_phys;
-    int acc = 0;
-    for (int j = r * s_phys; j < i; ++j) acc += Us[j];                       // instance offset
-    const int32_t* col = p.ws.q + (size_t)b * R * P + i;
-    for (int s0 = 0; s0 < s; s0 += 8) {                                      // lower sources
-      int v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = s0 + u < s ? __ldg(col + (size_t)(s0 + u) * P) : 0;
-#pragma unroll
-      for (int u = 0; u < 8; ++u) acc += v[u];
-    }
+    int acc = lower[i];
+    for (int j = r * s_phys; j < i; ++j) acc += Us[j];
     B0[i] = acc;
   }
   if (s == 0 && p.out_instance_offsets) {
@@ -82,17 +116,34 @@ __global__ void __launch_bounds__(kPosThreads) pos_prefix_kernel(const PosParams
       off[i] = acc;
     }
   }
-  // exclusive prefix over tiles of the per-tile counts, in place
-  int32_t* cnt = p.pos_cnt + row * (size_t)p.tiles * P;
-  for (int i = tid; i < P; i += nt) {
-    int run = 0;
-    for (int t0 = 0; t0 < p.tiles; t0 += 8) {
-      int v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? cnt[(size_t)(t0 + u) * P + i] : 0;
-#pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (t0 + u < p.tiles) { cnt[(size_t)(t0 + u) * P + i] = run; run += v[u]; }
+  if (p.out_counts || p.out_offsets) {
+    // row s of the counts, and for each destination what the lower sources send to it
+    for (int r = tid; r < R; r += nt) {
+      int c = 0, lo = 0;
+      for (int l = 0; l < s_phys; ++l) { c += mine[r * s_phys + l]; lo += lower[r * s_phys + l]; }
+      crow[r] = c;
+      lrow[r] = lo;
+      if (p.out_counts) p.out_counts[row * R + r] = c;
+    }
+    __syncthreads();
+    if (p.out_offsets) {
+      int32_t* send = p.out_offsets + (((size_t)b * 2 + 0) * R + s) * (R + 1);
+      int32_t* recv = p.out_offsets + ((size_t)b * 2 + 1) * R * (R + 1);
+      if (warp == 0) {   // send offsets of source s: exclusive scan over the destinations
+        const int ch = (R + 31) / 32;
+        const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
+        int sum = 0;
+        for (int r = i0; r < i1; ++r) sum += crow[r];
+        int total;
+        int pre = warp_exclusive_scan(sum, lane, &total);
+        for (int r = i0; r < i1; ++r) { send[r] = pre; pre += crow[r]; }
+        if (lane == 0) send[R] = total;
+      }
+      // receive offsets: entry s of every destination's row; the last source appends the total
+      for (int r = tid; r < R; r += nt) {
+        recv[(size_t)r * (R + 1) + s] = lrow[r];
+        if (s == R - 1) recv[(size_t)r * (R + 1) + R] = lrow[r] + crow[r];
+      }
     }
   }
 }
@@ -109,7 +160,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
   const size_t row = (size_t)b * d.R + s;
   const int begin = tile * p.tile_ids;
   const int count = min(p.tile_ids, p.n_ids - begin);
-  const int32_t* tr = p.token_replica + row * (size_t)p.n_ids + begin;
+  const int32_t* tr = p.token_replica + row * (size_t)p.row_stride + p.first_id + begin;
 
   // this warp's 512 assignments: step j covers 32 consecutive ones, so (step, lane) is flat order
   const int wbase = warp * (32 * kIdsPerThread);
@@ -189,14 +240,14 @@ size_t pos_rank_smem_bytes(const Dims& d, int tile_ids) {
 }
 
 size_t pos_prefix_smem_bytes(const Dims& d) {
-  return sizeof(int) * ((size_t)2 * d.P + kPosThreads / 32 + 1);
+  return sizeof(int) * ((size_t)3 * d.P + kPosThreads / 32 + 1 + 2 * (size_t)d.R);
 }
 
 cudaError_t configure_dispatch(const Dims& d) {
   cudaError_t e = cudaFuncSetAttribute(pos_rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)pos_rank_smem_bytes(d, kMaxTileIds));
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(pos_prefix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  return cudaFuncSetAttribute(pos_base_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)pos_prefix_smem_bytes(d));
 }
 
@@ -211,15 +262,21 @@ cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) 
   hp.rank_first = 0;
   hp.rank_count = p.d.R;
   hp.n_ids = p.n_ids;
+  hp.row_stride = p.row_stride;
+  hp.first_id = p.first_id;
   hp.tiles = p.tiles;
   hp.max_tiles = p.tiles;
   hp.tile_ids = p.tile_ids;
-  hp.vec_ok = (p.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.token_replica) & 15u) == 0);
+  hp.vec_ok = (p.n_ids % 4 == 0) && (p.row_stride % 4 == 0) && (p.first_id % 4 == 0) &&
+              ((reinterpret_cast<uintptr_t>(p.token_replica) & 15u) == 0);
   hp.ws.status = p.scratch_status;   // a stray instance id must not raise the plan's BAD_ID flag
   cudaError_t e = launch_hist(hp, batch, 0, stream);
   if (e != cudaSuccess) return e;
   // 2. bases and tile prefixes
-  pos_prefix_kernel<<<dim3(p.d.R, batch), kPosThreads, pos_prefix_smem_bytes(p.d), stream>>>(p);
+  pos_tile_prefix_kernel<<<dim3(p.d.R, batch), kPosThreads, 0, stream>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  pos_base_kernel<<<dim3(p.d.R, batch), kPosThreads, pos_prefix_smem_bytes(p.d), stream>>>(p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   // 3. stable ranks inside the tile

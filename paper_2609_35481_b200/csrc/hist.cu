@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   const size_t row = (size_t)b * p.d.R + p.rank_first + s;
   const int begin = tile * p.tile_ids;
   const int count = min(p.tile_ids, p.n_ids - begin);   // <= 0 only when n_ids == 0
-  const int32_t* ids = p.ids + ((size_t)b * p.rank_count + s) * (size_t)p.n_ids + begin;
+  const int32_t* ids = p.ids + ((size_t)b * p.rank_count + s) * (size_t)p.row_stride + p.first_id + begin;
   int4 x[IPT / 4];
 #pragma unroll
   for (int j = 0; j < IPT / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, p.vec_ok);

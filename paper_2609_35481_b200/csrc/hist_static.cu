@@ -87,6 +87,8 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   hp.ids = dev_topk_ids;
   hp.out_omega = nullptr;
   hp.n_ids = (int)n_ids;
+  hp.row_stride = n_ids;
+  hp.first_id = 0;
   hp.tile_ids = kStaticTileIds;
   hp.tiles = (int)tiles;
   hp.max_tiles = (int)tiles;

@@ -83,7 +83,9 @@ struct HistParams {
   int rank_first, rank_count;   // window of source ranks the caller's id buffers cover
   const int32_t* ids;   // [B][R][n_ids]
   int32_t* out_omega;   // optional caller copy of omega [B][R][E]
-  int n_ids;            // T * k
+  int n_ids;            // ids of a row that are counted (T * k, or the ids of a token window)
+  long long row_stride; // ids between the starts of consecutive rows of the buffer
+  long long first_id;   // offset of the first counted id inside its row
   int tiles;            // tiles per (plan, rank)
   int max_tiles;        // stride of tile_cnt / tile_pref
   int tile_ids;
@@ -146,6 +148,10 @@ struct PosParams {
   int32_t* pos_cnt;               // scratch [B][R][tiles][P]: tile counts, then prefixes over tiles
   int32_t* pos_a;                 // scratch [B][R][P] send base of (source, instance)
   int32_t* pos_b;                 // scratch [B][R][P] receive base of (source, instance)
+  int32_t* pos_tot;               // scratch [B][R][P] assignments of (source, instance) in the window
+  int32_t* out_counts;            // [B][R][R] dispatch counts of the window, or NULL
+  int32_t* out_offsets;           // [B][2][R][R+1] send / receive offsets of the window, or NULL
+  long long row_stride, first_id; // the window inside token_replica's rows (ids)
   uint32_t* scratch_status;       // scratch word for the histogram kernel's flag
   int n_ids, tiles, tile_ids;
 };
@@ -176,6 +182,7 @@ void solve_static_fill(const Dims& d, int dm, const int32_t* main_rank, const in
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
+size_t pos_prefix_smem_bytes(const Dims& d);
 
 cudaError_t configure_solve(size_t smem);
 cudaError_t configure_route(size_t smem);

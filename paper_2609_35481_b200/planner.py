@@ -111,6 +111,29 @@ class Planner:
         st.synchronize()   # the scratch tensor is released when this returns
         return send, recv, inst_off
 
+    def dispatch_window(self, token_replica: torch.Tensor, first_token: int, token_count: int,
+                        stream=None):
+        """(send_pos, recv_pos, instance_offsets, counts, offsets) of one chunk of tokens,
+        first_token .. first_token + token_count - 1 of every source rank."""
+        Bn, R, T, k = token_replica.shape
+        i32 = dict(dtype=torch.int32, device=self.device)
+        send = torch.empty((Bn, R, token_count, k), **i32)
+        recv = torch.empty((Bn, R, token_count, k), **i32)
+        inst_off = torch.empty((Bn, R, self.s_phys + 1), **i32)
+        counts = torch.empty((Bn, R, R), **i32)
+        offsets = torch.empty((Bn, 2, R, R + 1), **i32)
+        nbytes = B.topoep_dispatch_scratch_bytes(self.handle, token_count, Bn)
+        scratch = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        ptr = (scratch.data_ptr() + 255) // 256 * 256
+        st = stream if stream is not None else torch.cuda.current_stream(self.device)
+        rc = B.topoep_dispatch_window(self.handle, token_replica, T, Bn, first_token, token_count,
+                                      send, recv, inst_off, counts, offsets, ptr, nbytes,
+                                      st.cuda_stream)
+        if rc != B.OK:
+            raise B.TopoEPError(rc)
+        st.synchronize()   # the scratch tensor is released when this returns
+        return send, recv, inst_off, counts, offsets
+
     def histogram(self, topk_ids: torch.Tensor, stream=None) -> torch.Tensor:
         """topoep_histogram on ids [B][rank window][T][k]; returns Omega rows [B][window][E]."""
         Bn, R, T, k = topk_ids.shape

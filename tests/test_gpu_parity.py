@@ -468,3 +468,44 @@ def test_imbalance_against_slot_count_on_the_slot_experiment_shape():
     none = table[(0, 0)]
     assert all(v <= none + 1e-9 for v in table.values())
     assert table[(1, 1)] < table[(1, 0)]
+
+
+# ---- two-chunk pipeline: dispatch layout of a window of tokens ----------------------------------
+@pytest.mark.parametrize("name,over,batch,cut", [
+    ("mid", dict(slots_per_rank=3), 2, 2048),                      # the even split of the paper
+    ("tiny", dict(slots_per_rank=2), 1, 511),                      # odd cut: ragged, unaligned rows
+    ("dsv3", dict(slots_per_rank=2, tokens_per_rank=1024), 1, 384),
+])
+def test_two_chunk_dispatch_windows_match_the_oracle(name, over, batch, cut):
+    """The routed tokens are cut into chunks c1 = tokens [0, cut) and c2 = [cut, T) of every source.
+    Each chunk's send/receive positions and instance offsets must equal the oracle's dispatch
+    permutation of that slice of token_replica; its counts are a bincount of the slice, its offsets
+    their cumulative sums; the two chunks' counts add up to the plan's dispatch counts."""
+    w = wl.CONFIGS[name].replace(**over)
+    cfg = oracle_config(w)
+    ids = wl.make_topk_ids(w, seed=61, batch=batch)
+    pl = make_planner(w, max_batch=batch)
+    out = pl.plan(torch.from_numpy(ids).to(pl.device))
+    tr = out.token_replica.cpu().numpy()
+    R, T, S = w.ranks, w.tokens_per_rank, pl.s_phys
+    total = np.zeros((batch, R, R), np.int64)
+    for first, count in ((0, cut), (cut, T - cut)):
+        send, recv, ioff, counts, offsets = (t.cpu().numpy() for t in
+                                             pl.dispatch_window(out.token_replica, first, count))
+        for b in range(batch):
+            part = np.ascontiguousarray(tr[b][:, first:first + count])
+            want_send, want_recv, want_ioff = orc.dispatch_positions(cfg, part)
+            assert np.array_equal(send[b], want_send) and np.array_equal(recv[b], want_recv)
+            assert np.array_equal(ioff[b], want_ioff)
+            flat = part.reshape(R, -1)
+            want_counts = np.stack([np.bincount(flat[s][flat[s] >= 0] // S, minlength=R)
+                                    for s in range(R)])
+            assert np.array_equal(counts[b], want_counts)
+            zero = np.zeros((R, 1), np.int64)
+            assert np.array_equal(offsets[b, 0], np.concatenate([zero, np.cumsum(want_counts, 1)], 1))
+            assert np.array_equal(offsets[b, 1], np.concatenate([zero, np.cumsum(want_counts.T, 1)], 1))
+        total += counts
+    assert np.array_equal(total, out.dispatch_counts.cpu().numpy())
+    # window errors
+    assert B.topoep_dispatch_window(pl.handle, out.token_replica, T, batch, T - 1, 2, None, None,
+                                    None, None, None, 256, 0, 0) == -6
