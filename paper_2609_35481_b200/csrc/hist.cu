@@ -112,6 +112,61 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
   if (g == 0 && e < E && p.ws.demand) p.ws.demand[((size_t)b * p.d.M + dm) * E + e] = dsum;
 }
 
+// The same with 16-byte accesses: a lane holds FOUR consecutive experts of its rank (E % 4 == 0
+// and 16-byte aligned rows), so a tile row is read in full sectors and a warp covers
+// 4 * epw experts.  Used for calls that fill the GPU.
+__global__ void __launch_bounds__(128) omega4_kernel(const OmegaParams p) {
+  const int E = p.d.E, G = p.d.G, R = p.d.R, epw = p.epw;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int dm = blockIdx.y, b = blockIdx.z;
+  if (p.pdl == 2) pdl_trigger();
+  const int g = lane / epw, e = 4 * ((blockIdx.x * 4 + warp) * epw + (lane - g * epw));
+  const bool on = g < G && e < E;
+  const int s = p.rank_first + dm * G + g;   // global source rank
+  const size_t row = (size_t)b * R + s;
+  const size_t user_row = (size_t)b * p.rank_count + dm * G + g;
+  int4 sum = make_int4(0, 0, 0, 0), mr = sum, ml = sum;
+  if (on && p.ws.omega_m) {   // static tables, fetched before the wait
+    mr = __ldg(reinterpret_cast<const int4*>(p.ws.main_rank + e));
+    ml = __ldg(reinterpret_cast<const int4*>(p.ws.main_local + e));
+  }
+  pdl_wait();
+  if (on) {
+    if (p.src_omega) {
+      sum = __ldg(reinterpret_cast<const int4*>(p.src_omega + row * E + e));
+    } else {
+      const int4* c = reinterpret_cast<const int4*>(p.ws.tile_cnt + row * (size_t)p.max_tiles * E + e);
+      const size_t stride = (size_t)E / 4;
+      for (int t0 = 0; t0 < p.tiles; t0 += 8) {
+        int4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * stride) : make_int4(0, 0, 0, 0);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { sum.x += v[u].x; sum.y += v[u].y; sum.z += v[u].z; sum.w += v[u].w; }
+      }
+    }
+    if (p.ws.omega) *reinterpret_cast<int4*>(p.ws.omega + row * E + e) = sum;
+    if (p.out_omega) *reinterpret_cast<int4*>(p.out_omega + user_row * E + e) = sum;
+    if (p.ws.omega_m) {
+      int32_t* om = p.ws.omega_m + (size_t)b * R * p.d.e_loc * R + s;
+      om[(size_t)(mr.x * p.d.e_loc + ml.x) * R] = sum.x;
+      om[(size_t)(mr.y * p.d.e_loc + ml.y) * R] = sum.y;
+      om[(size_t)(mr.z * p.d.e_loc + ml.z) * R] = sum.z;
+      om[(size_t)(mr.w * p.d.e_loc + ml.w) * R] = sum.w;
+    }
+  }
+  int4 ds = sum;
+  for (int o = epw; o < 32; o <<= 1) {
+    ds.x += __shfl_xor_sync(0xffffffffu, ds.x, o);
+    ds.y += __shfl_xor_sync(0xffffffffu, ds.y, o);
+    ds.z += __shfl_xor_sync(0xffffffffu, ds.z, o);
+    ds.w += __shfl_xor_sync(0xffffffffu, ds.w, o);
+  }
+  if (g == 0 && e < E && p.ws.demand)
+    *reinterpret_cast<int4*>(p.ws.demand + ((size_t)b * p.d.M + dm) * E + e) = ds;
+}
+
 __global__ void empty_kernel() {}
 
 }  // namespace
@@ -133,6 +188,14 @@ cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t s
 }
 
 cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream) {
+  auto al16 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
+  // large calls only: with few CTAs the four-times-longer per-thread chain costs latency
+  // (one 32-rank plan: 6.7 us -> 8.1 us for histogram + omega; 232 plans: 338 -> 324 us)
+  if ((long long)p.d.R * batch >= 2 * 148 && p.d.E % 4 == 0 && al16(p.src_omega) && al16(p.out_omega) && al16(p.ws.omega) &&
+      al16(p.ws.demand) && al16(p.ws.tile_cnt) && al16(p.ws.main_rank) && al16(p.ws.main_local)) {
+    const dim3 grid((p.d.E / 4 + 4 * p.epw - 1) / (4 * p.epw), p.d.M, batch);
+    return launch_kernel(omega4_kernel, grid, dim3(128), 0, stream, p.pdl != 0, p);
+  }
   const dim3 grid((p.d.E + 4 * p.epw - 1) / (4 * p.epw), p.d.M, batch);
   return launch_kernel(omega_kernel, grid, dim3(128), 0, stream, p.pdl != 0, p);
 }
