@@ -319,8 +319,6 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.d = h->d;
   sp.ws = h->ws;
   sp.pdl = chain_pdl(h, batch);
-  sp.token_bytes = h->cost.token_bytes;
-  sp.expert_bytes = h->cost.expert_bytes;
   sp.max_iters = h->max_iters;
   sp.min_delta = h->min_delta;
   // 2 D S_tok - ||W|| > 0  <=>  D > floor(||W|| / (2 S_tok)); S_tok = 0 admits no candidate

@@ -107,7 +107,6 @@ struct SolveParams {
   Dims d;
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
-  int64_t token_bytes, expert_bytes;
   int max_iters, min_delta;
   int stage1_slots;   // slots of a rank that inter-node placement may fill (N minus the reserve)
   int cand_thr;   // demand D of a stage-1 candidate exceeds this: floor(||W|| / (2 S_tok))
