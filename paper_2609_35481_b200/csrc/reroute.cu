@@ -196,6 +196,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
     i -= n_list4;
     if (i >= 0 && i < n_tp) cp_async16(tbase + 4 * i, rec + rl.tp + tile * kSplitCap + 4 * i);
     // shapes these fixed assignments do not cover: more pieces than threads, or E % 4 != 0
+#pragma unroll 1
     for (int j = tid + nt; j < n_route + n_head + 2 * n_list4 + n_tp; j += nt) {
       int u = j;
       if (u < n_route) { cp_async16(route + 4 * u, g_route + 4 * u); continue; }
@@ -208,10 +209,16 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
       u -= n_list4;
       cp_async16(tbase + 4 * u, rec + rl.tp + tile * kSplitCap + 4 * u);
     }
-    if (E % 4 != 0)
+    if (E % 4 != 0) {
+#pragma unroll 1
       for (int e = tid; e < E; e += nt) cp_async4(route + e, g_route + e);
+    }
   }
-  for (int i = tid; i < kSplitCap * rows; i += nt) cnt4[i] = make_uint4(0u, 0u, 0u, 0u);
+  // rows = blockDim.x / 8, so the kSplitCap * rows counter words are exactly kSplitCap / 8 per
+  // thread: straight-line stores (a counted loop here cost a hundred instructions per warp)
+  static_assert(kSplitCap % 8 == 0, "counter words per thread");
+#pragma unroll
+  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
   cp_async_wait_all();           // hdr[2], the work-list length, arrives as the record's zero
   __syncthreads();
