@@ -185,7 +185,17 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
         const int ex = warp_exclusive_scan(v, lane, &total);
         if (lane < p.tiles) {
           p.ws.tile_pref[trow + (size_t)lane * E + i] = ex;
-          if (i < kSplitCap) rec[rl.tp + lane * kSplitCap + i] = ex;
+          if (i < kSplitCap) {
+            rec[rl.tp + lane * 2 * kSplitCap + i] = ex;
+            // ranks [ex, ex + v) of this tile: inside one instance's quota interval?
+            int lo = 0, res = -1;
+            for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
+              const int hi = rec[rl.cum + k];
+              if (ex >= lo && ex + v <= hi) { res = rec[rl.inst + k]; break; }
+              lo = hi;
+            }
+            rec[rl.tp + lane * 2 * kSplitCap + kSplitCap + i] = res;
+          }
         }
       }
     } else {
@@ -202,7 +212,16 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
           for (int u = 0; u < 8; ++u)
             if (t0 + u < p.tiles) {
               o[(size_t)(t0 + u) * E] = run;
-              if (sidx[e] < kSplitCap) rec[rl.tp + (t0 + u) * kSplitCap + sidx[e]] = run;
+              if (sidx[e] < kSplitCap) {
+                rec[rl.tp + (t0 + u) * 2 * kSplitCap + sidx[e]] = run;
+                int lo = 0, res = -1;
+                for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
+                  const int hi = rec[rl.cum + k];
+                  if (run >= lo && run + v[u] <= hi) { res = rec[rl.inst + k]; break; }
+                  lo = hi;
+                }
+                rec[rl.tp + (t0 + u) * 2 * kSplitCap + kSplitCap + sidx[e]] = res;
+              }
               run += v[u];
             }
         }
