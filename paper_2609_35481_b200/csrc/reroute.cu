@@ -37,7 +37,7 @@ __host__ __device__ inline RerouteLayout reroute_layout(const Dims& d, int tile_
   o.seg = at;   at += sizeof(int) * pad4(d.E + 1 > kSplitCap + 4 ? d.E + 1 : kSplitCap + 4);
   o.cum = at;   at += sizeof(int) * pad4(d.P);
   o.inst = at;  at += sizeof(int) * pad4(d.P);
-  o.tbase = at; at += sizeof(int) * (size_t)2 * kSplitCap;   // tile prefixes, resolved instances
+  o.tbase = at; at += sizeof(int) * (size_t)3 * kSplitCap;   // tile prefixes, resolved instances, experts
   o.work = at;  at += sizeof(unsigned short) * (size_t)tile_ids;
   o.total = at;
   return o;
@@ -184,7 +184,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
     const int n_route = (E % 4 == 0) ? E / 4 : 0;            // 16-byte pieces of the route table
     const int n_head = (4 + min(E, kSplitCap) + 1 + 3) / 4;  // header + segment starts
     const int n_list4 = (min(P, kFastLists) + 3) / 4;
-    const int n_tp = 2 * kSplitCap / 4;   // this tile's prefixes and resolved instances
+    const int n_tp = 3 * kSplitCap / 4;   // this tile's prefixes, resolved instances, experts
     int i = tid;
     if (i < n_route) cp_async16(route + 4 * i, g_route + 4 * i);
     i -= n_route;
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
     i -= n_list4;
     if (i >= 0 && i < n_list4) cp_async16(inst + 4 * i, rec + rl.inst + 4 * i);
     i -= n_list4;
-    if (i >= 0 && i < n_tp) cp_async16(tbase + 4 * i, rec + rl.tp + tile * 2 * kSplitCap + 4 * i);
+    if (i >= 0 && i < n_tp) cp_async16(tbase + 4 * i, rec + rl.tp + tile * 3 * kSplitCap + 4 * i);
     // shapes these fixed assignments do not cover: more pieces than threads, or E % 4 != 0
 #pragma unroll 1
     for (int j = tid + nt; j < n_route + n_head + 2 * n_list4 + n_tp; j += nt) {
@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
       u -= n_list4;
       if (u < n_list4) { cp_async16(inst + 4 * u, rec + rl.inst + 4 * u); continue; }
       u -= n_list4;
-      cp_async16(tbase + 4 * u, rec + rl.tp + tile * 2 * kSplitCap + 4 * u);
+      cp_async16(tbase + 4 * u, rec + rl.tp + tile * 3 * kSplitCap + 4 * u);
     }
     if (E % 4 != 0) {
 #pragma unroll 1
@@ -222,6 +222,17 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
   cp_async_wait_all();           // hdr[2], the work-list length, arrives as the record's zero
   __syncthreads();
+  // A split expert whose ids of THIS tile all fall inside one instance's quota interval (the
+  // route kernel checked the tile's rank interval against the quotas) is not split here: its
+  // table entry becomes that instance and its ids stream like everyone else's.  Only tiles that
+  // straddle a quota boundary -- about one in ten on the benchmark workloads -- rank anything.
+  if (hdr[0] > 0) {   // uniform: the source has split experts at all
+    if (tid < kSplitCap) {
+      const int res = tbase[kSplitCap + tid], e = tbase[2 * kSplitCap + tid];
+      if (tid < hdr[0] && res >= 0 && e >= 0) route[e] = res;
+    }
+    __syncthreads();
+  }
 
   // Stream: look up and store.  An ignored id and a split id both store -1 for now; the split
   // ones are remembered in a 16-bit mask, pushed on the work list afterwards and patched below.
@@ -251,16 +262,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   while (split_mask) {   // ~3% of the ids on the benchmark workloads
     const int k = __ffs(split_mask) - 1;
     split_mask &= split_mask - 1;
-    const int pos = 4 * ((k >> 2) * nt + tid) + (k & 3);
-    // Its expert's ids of this tile may all fall to one instance (the route kernel checked the
-    // tile's rank interval against the quotas): then that instance is the answer and nothing is
-    // ranked.  Only tiles that straddle a quota boundary put work on the list.
-    const int4 xv = (k >> 2) == 0 ? x[0] : (k >> 2) == 1 ? x[1] : (k >> 2) == 2 ? x[2] : x[3];
-    const int id = (k & 3) == 0 ? xv.x : (k & 3) == 1 ? xv.y : (k & 3) == 2 ? xv.z : xv.w;
-    const int si = -2 - route[id];
-    const int res = si < kSplitCap ? tbase[kSplitCap + si] : -1;
-    if (res >= 0) out[pos] = res;
-    else work[atomicAdd(hdr + 2, 1)] = (unsigned short)pos;
+    work[atomicAdd(hdr + 2, 1)] = (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
   }
   __syncthreads();   // also orders the stores above before the patches below
   const int n_work = hdr[2];

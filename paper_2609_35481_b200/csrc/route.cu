@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
         if (lane < p.tiles) {
           p.ws.tile_pref[trow + (size_t)lane * E + i] = ex;
           if (i < kSplitCap) {
-            rec[rl.tp + lane * 2 * kSplitCap + i] = ex;
+            rec[rl.tp + lane * 3 * kSplitCap + i] = ex;
             // ranks [ex, ex + v) of this tile: inside one instance's quota interval?
             int lo = 0, res = -1;
             for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
@@ -194,7 +194,8 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
               if (ex >= lo && ex + v <= hi) { res = rec[rl.inst + k]; break; }
               lo = hi;
             }
-            rec[rl.tp + lane * 2 * kSplitCap + kSplitCap + i] = res;
+            rec[rl.tp + lane * 3 * kSplitCap + kSplitCap + i] = res;
+            rec[rl.tp + lane * 3 * kSplitCap + 2 * kSplitCap + i] = e;
           }
         }
       }
@@ -213,14 +214,15 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
             if (t0 + u < p.tiles) {
               o[(size_t)(t0 + u) * E] = run;
               if (sidx[e] < kSplitCap) {
-                rec[rl.tp + (t0 + u) * 2 * kSplitCap + sidx[e]] = run;
+                rec[rl.tp + (t0 + u) * 3 * kSplitCap + sidx[e]] = run;
                 int lo = 0, res = -1;
                 for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
                   const int hi = rec[rl.cum + k];
                   if (run >= lo && run + v[u] <= hi) { res = rec[rl.inst + k]; break; }
                   lo = hi;
                 }
-                rec[rl.tp + (t0 + u) * 2 * kSplitCap + kSplitCap + sidx[e]] = res;
+                rec[rl.tp + (t0 + u) * 3 * kSplitCap + kSplitCap + sidx[e]] = res;
+                rec[rl.tp + (t0 + u) * 3 * kSplitCap + 2 * kSplitCap + sidx[e]] = e;
               }
               run += v[u];
             }

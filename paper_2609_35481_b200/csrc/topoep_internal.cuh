@@ -58,11 +58,11 @@ struct Workspace {
 //   seg  [E+1]  list i of the source's i-th split expert = [seg[i], seg[i+1])
 //   cum  [P]    cumulative quota along each list (instances in ascending rank order)
 //   inst [P]    physical instance ids along each list
-//   tp   [max_tiles][2][kSplitCap]  per tile, for the first kSplitCap split experts: the tile
+//   tp   [max_tiles][3][kSplitCap]  per tile, for the first kSplitCap split experts: the tile
 //               prefixes (the full table tile_pref is only read when a source has more split
-//               experts than that), then the tile's RESOLVED instance: when all ids of the
-//               expert in this tile fall inside one instance's quota interval, that instance
-//               (no ranking needed in this tile), else -1
+//               experts than that); the tile's RESOLVED instance: when all ids of the expert in
+//               this tile fall inside one instance's quota interval, that instance (no ranking
+//               needed in this tile), else -1; and the expert ids themselves (-1 beyond n_split)
 struct SplitRec {
   int seg, cum, inst, tp, ints;
 };
@@ -72,7 +72,7 @@ __host__ __device__ inline SplitRec split_rec_layout(int E, int P, int max_tiles
   r.cum = r.seg + ((E + 1 + 3) & ~3);
   r.inst = r.cum + ((P + 3) & ~3);
   r.tp = r.inst + ((P + 3) & ~3);
-  r.ints = r.tp + max_tiles * 2 * kSplitCap;
+  r.ints = r.tp + max_tiles * 3 * kSplitCap;
   return r;
 }
 constexpr int kFastLists = 128;     // list entries the reroute kernel fetches before it knows n_list
