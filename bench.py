@@ -40,8 +40,8 @@ KERNELS_PER_PLAN = 5
 # 16-plan call (profiles/reroute_kernel_dsv3_batch16.md, profiles/hist_kernel_dsv3_batch16.md);
 # a launch's traffic is this times its plans (every CTA touches only its own tile and tables).
 NCU_TRAFFIC_PER_PLAN = {
-    "reroute": (136072192 + 87091968) / 16,
-    "hist": (134233600 + 6310912) / 16,
+    "reroute": (137112320 + 85663744) / 16,
+    "hist": (134235136 + 6251776) / 16,
 }
 
 
