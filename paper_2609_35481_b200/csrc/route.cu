@@ -20,7 +20,7 @@ namespace topoep {
 
 namespace {
 
-struct RouteLayout { size_t rm, qrow, mr, ml, nz, single, sidx, seg, crow, split_e, warp_tot, total; };
+struct RouteLayout { size_t rm, qrow, mr, ml, nz, single, sidx, seg, crow, split_e, warp_tot, cum_s, inst_s, total; };
 
 __host__ __device__ inline RouteLayout route_layout(const Dims& d) {
   RouteLayout o;
@@ -36,6 +36,8 @@ __host__ __device__ inline RouteLayout route_layout(const Dims& d) {
   o.crow = at;     at += sizeof(int) * (size_t)d.R;
   o.split_e = at;  at += sizeof(int) * (size_t)d.E;
   o.warp_tot = at; at += sizeof(int) * 2 * (kRouteThreads / 32);
+  o.cum_s = at;    at += sizeof(int) * (size_t)d.P;
+  o.inst_s = at;   at += sizeof(int) * (size_t)d.P;
   o.total = at;
   return o;
 }
@@ -92,6 +94,8 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   int* crow = reinterpret_cast<int*>(smem + lay.crow);     // [R]   counts[s][.]
   int* split_e = reinterpret_cast<int*>(smem + lay.split_e); // [E]   expert of split index i
   int* warp_tot = reinterpret_cast<int*>(smem + lay.warp_tot);
+  int* cum_s = reinterpret_cast<int*>(smem + lay.cum_s);     // [n_list] cumulative quotas
+  int* inst_s = reinterpret_cast<int*>(smem + lay.inst_s);   // [n_list] instances
 
   const size_t row = (size_t)b * R + s;
   const int RN = R * N;
@@ -139,94 +143,105 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     rec[rl.seg + n_split] = n_list;
   }
 
-  // Split lists: position of an instance = number of nonzero instances of e on lower ranks; its
-  // cumulative quota = its own share plus the shares of those.
-  for (int e = tid; e < E; e += nt) {
-    if (nz[e] < 2 || qrow[ml[e]] <= 0) continue;
-    int pos = 0, below = 0;
-    const int lim = mr[e] * N;
-    for (int i = 0, r = 0, j = 0; i < lim; ++i) {
-      const int v = qrow[r * s_phys + e_loc + j];
-      if (rm[i] == e && v > 0) { ++pos; below += v; }
-      if (++j == N) { j = 0; ++r; }
-    }
-    rec[rl.cum + seg[e] + pos] = below + qrow[ml[e]];
-    rec[rl.inst + seg[e] + pos] = ml[e];
-  }
-  for (int i = tid; i < RN; i += nt) {
-    const int e = rm[i];
-    if (e < 0 || nz[e] < 2) continue;
-    const int r = i / N, pi = r * s_phys + e_loc + (i - r * N);
-    if (qrow[pi] <= 0) continue;
-    const int qm = qrow[ml[e]];
-    int pos = 0, below = 0;
-    if (mr[e] < r && qm > 0) { pos = 1; below = qm; }
-    const int lim = r * N;
-    for (int i2 = 0, r2 = 0, j2 = 0; i2 < lim; ++i2) {
-      const int v = qrow[r2 * s_phys + e_loc + j2];
-      if (rm[i2] == e && v > 0) { ++pos; below += v; }
-      if (++j2 == N) { j2 = 0; ++r2; }
-    }
-    rec[rl.cum + seg[e] + pos] = below + qrow[pi];
-    rec[rl.inst + seg[e] + pos] = pi;
-  }
-
   __syncthreads();   // split_e is complete
-  // Cross-tile base of the stable rank, split experts only: exclusive prefix over the row's tiles.
-  // One (split expert, tile) pair per thread-iteration so that all loads of a sweep are in flight.
-  if (p.tiles > 0 && n_split > 0 && s >= p.rank_first && s < p.rank_first + p.rank_count) {
-    const size_t trow = row * (size_t)p.max_tiles * E;
-    if (p.tiles <= 32) {
-      // a warp owns a split expert, a lane owns a tile
-      for (int i = warp; i < n_split; i += nt >> 5) {
-        const int e = split_e[i];
-        const int v = lane < p.tiles ? __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e) : 0;
-        int total;
-        const int ex = warp_exclusive_scan(v, lane, &total);
-        if (lane < p.tiles) {
-          p.ws.tile_pref[trow + (size_t)lane * E + i] = ex;
-          if (i < kSplitCap) {
-            rec[rl.tp + lane * 3 * kSplitCap + i] = ex;
-            // ranks [ex, ex + v) of this tile: inside one instance's quota interval?
-            int lo = 0, res = -1;
-            for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
-              const int hi = rec[rl.cum + k];
-              if (ex >= lo && ex + v <= hi) { res = rec[rl.inst + k]; break; }
-              lo = hi;
-            }
-            rec[rl.tp + lane * 3 * kSplitCap + kSplitCap + i] = res;
-            rec[rl.tp + lane * 3 * kSplitCap + 2 * kSplitCap + i] = e;
+  // Split lists, one warp per split expert: the instances with a share in ascending rank order
+  // (the replica slots are already in rank order; the main instance goes in front of the first
+  // slot on a higher rank) with cumulative quotas.  Lanes take the slots, positions come from a
+  // ballot, quotas from a warp scan.  The same warp then turns the expert's tile counts into
+  // tile prefixes and checks each tile's rank interval against the quotas.
+  const bool in_window = s >= p.rank_first && s < p.rank_first + p.rank_count;
+  const bool warp_tiles = p.tiles > 0 && p.tiles <= 32 && in_window;
+  const size_t trow = row * (size_t)p.max_tiles * E;
+  for (int i = warp; i < n_split; i += nt >> 5) {
+    const int e = split_e[i];
+    const int base = seg[e], qm = qrow[ml[e]], rmain = mr[e];
+    // tile count of (e, tile = lane): in flight while the list is built
+    const int tv = warp_tiles && lane < p.tiles ? __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e) : 0;
+    int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
+    for (int i0 = 0; i0 < RN; i0 += 32) {
+      const int slot = i0 + lane;
+      int v = 0, r = 0, pi = 0;
+      if (slot < RN && rm[slot] == e) {
+        r = slot / N;
+        pi = r * s_phys + e_loc + (slot - r * N);
+        v = max(qrow[pi], 0);
+      }
+      const unsigned m = __ballot_sync(0xffffffffu, v > 0);
+      int tot;
+      const int ex = warp_exclusive_scan(v, lane, &tot);
+      const bool below_main = v > 0 && r < rmain;
+      main_pos += __popc(__ballot_sync(0xffffffffu, below_main));
+      main_below += __reduce_add_sync(0xffffffffu, below_main ? v : 0);
+      if (v > 0) {
+        const bool after_main = qm > 0 && rmain < r;
+        const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
+        cum_s[base + pos] = carry_cum + ex + v + (after_main ? qm : 0);
+        inst_s[base + pos] = pi;
+      }
+      carry_pos += __popc(m);
+      carry_cum += tot;
+    }
+    if (lane == 0 && qm > 0) {
+      cum_s[base + main_pos] = main_below + qm;
+      inst_s[base + main_pos] = ml[e];
+    }
+    __syncwarp();
+    const int n_e = nz[e];
+    for (int k = lane; k < n_e; k += 32) {
+      rec[rl.cum + base + k] = cum_s[base + k];
+      rec[rl.inst + base + k] = inst_s[base + k];
+    }
+    if (warp_tiles) {
+      // exclusive prefix over the row's tiles: the cross-tile base of the stable rank
+      int total;
+      const int ex = warp_exclusive_scan(tv, lane, &total);
+      if (lane < p.tiles) {
+        p.ws.tile_pref[trow + (size_t)lane * E + i] = ex;
+        if (i < kSplitCap) {
+          // ranks [ex, ex + tv) of this tile: inside one instance's quota interval?
+          int lo = 0, res = -1;
+          for (int k = base; k < base + n_e; ++k) {
+            const int hi = cum_s[k];
+            if (ex >= lo && ex + tv <= hi) { res = inst_s[k]; break; }
+            lo = hi;
           }
+          int32_t* t3 = rec + rl.tp + lane * 3 * kSplitCap + i;
+          t3[0] = ex;
+          t3[kSplitCap] = res;
+          t3[2 * kSplitCap] = e;
         }
       }
-    } else {
-      for (int e = tid; e < E; e += nt) {
-        if (nz[e] < 2) continue;
-        const int32_t* c = p.ws.tile_cnt + trow + e;
-        int32_t* o = p.ws.tile_pref + trow + sidx[e];
-        int run = 0;
-        for (int t0 = 0; t0 < p.tiles; t0 += 8) {
-          int v[8];
+    }
+  }
+  if (p.tiles > 32 && n_split > 0 && in_window) {   // long rows: a thread walks an expert's tiles
+    __syncthreads();   // the lists of every split expert are in shared memory
+    for (int e = tid; e < E; e += nt) {
+      if (nz[e] < 2) continue;
+      const int32_t* c = p.ws.tile_cnt + trow + e;
+      int32_t* o = p.ws.tile_pref + trow + sidx[e];
+      int run = 0;
+      for (int t0 = 0; t0 < p.tiles; t0 += 8) {
+        int v[8];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
+        for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
 #pragma unroll
-          for (int u = 0; u < 8; ++u)
-            if (t0 + u < p.tiles) {
-              o[(size_t)(t0 + u) * E] = run;
-              if (sidx[e] < kSplitCap) {
-                rec[rl.tp + (t0 + u) * 3 * kSplitCap + sidx[e]] = run;
-                int lo = 0, res = -1;
-                for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
-                  const int hi = rec[rl.cum + k];
-                  if (run >= lo && run + v[u] <= hi) { res = rec[rl.inst + k]; break; }
-                  lo = hi;
-                }
-                rec[rl.tp + (t0 + u) * 3 * kSplitCap + kSplitCap + sidx[e]] = res;
-                rec[rl.tp + (t0 + u) * 3 * kSplitCap + 2 * kSplitCap + sidx[e]] = e;
+        for (int u = 0; u < 8; ++u)
+          if (t0 + u < p.tiles) {
+            o[(size_t)(t0 + u) * E] = run;
+            if (sidx[e] < kSplitCap) {
+              int lo = 0, res = -1;
+              for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
+                const int hi = cum_s[k];
+                if (run >= lo && run + v[u] <= hi) { res = inst_s[k]; break; }
+                lo = hi;
               }
-              run += v[u];
+              int32_t* t3 = rec + rl.tp + (t0 + u) * 3 * kSplitCap + sidx[e];
+              t3[0] = run;
+              t3[kSplitCap] = res;
+              t3[2 * kSplitCap] = e;
             }
-        }
+            run += v[u];
+          }
       }
     }
   }
