@@ -50,6 +50,7 @@ __device__ void block_scan2(const int* nz, int n, int* out_a, int* out_b, int* w
   const int chunk = (n + nt - 1) / nt;
   const int i0 = min(n, tid * chunk), i1 = min(n, i0 + chunk);
   int a = 0, b = 0;
+#pragma unroll 1
   for (int i = i0; i < i1; ++i) {
     const int f = nz[i] >= 2;
     a += f;
@@ -61,9 +62,11 @@ __device__ void block_scan2(const int* nz, int n, int* out_a, int* out_b, int* w
   if (lane == 0) { warp_tot[warp] = ta; warp_tot[nw + warp] = tb; }
   __syncthreads();
   int ba = 0, bb = 0;
+#pragma unroll 1
   for (int w = 0; w < warp; ++w) { ba += warp_tot[w]; bb += warp_tot[nw + w]; }
   ea += ba;
   eb += bb;
+#pragma unroll 1
   for (int i = i0; i < i1; ++i) {
     const int f = nz[i] >= 2;
     out_a[i] = ea;
@@ -100,27 +103,34 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   const size_t row = (size_t)b * R + s;
   const int RN = R * N;
   // static tables before the solver is known to be done, its results after
+#pragma unroll 4
   for (int e = tid; e < E; e += nt) {
     const int r = p.ws.main_rank[e];
     mr[e] = r;
     ml[e] = r * s_phys + p.ws.main_local[e];
   }
   pdl_wait();
+#pragma unroll 4
   for (int i = tid; i < RN; i += nt) rm[i] = p.ws.replica_map[(size_t)b * RN + i];
+#pragma unroll 4
   for (int i = tid; i < P; i += nt) qrow[i] = p.ws.q[row * P + i];
+#pragma unroll 4
   for (int r = tid; r < R; r += nt) crow[r] = p.ws.counts[row * R + r];
   __syncthreads();
 
+#pragma unroll 1
   for (int e = tid; e < E; e += nt) {
     nz[e] = qrow[ml[e]] > 0 ? 1 : 0;
     single[e] = ml[e];
   }
   __syncthreads();
+#pragma unroll 1
   for (int i = tid; i < RN; i += nt) {
     const int e = rm[i];
     if (e >= 0 && qrow[(i / N) * s_phys + e_loc + i % N] > 0) atomicAdd(&nz[e], 1);
   }
   __syncthreads();
+#pragma unroll 1
   for (int i = tid; i < RN; i += nt) {   // the one instance with a share, when it is a replica
     const int e = rm[i];
     const int pi = (i / N) * s_phys + e_loc + i % N;
@@ -133,6 +143,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
   int32_t* rec = p.ws.split_rec + row * (size_t)rl.ints;
   int32_t* route = p.ws.route + row * E;
+#pragma unroll 1
   for (int e = tid; e < E; e += nt) {
     const bool split = nz[e] >= 2;
     route[e] = split ? -2 - sidx[e] : single[e];
@@ -152,12 +163,14 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   const bool in_window = s >= p.rank_first && s < p.rank_first + p.rank_count;
   const bool warp_tiles = p.tiles > 0 && p.tiles <= 32 && in_window;
   const size_t trow = row * (size_t)p.max_tiles * E;
+#pragma unroll 1
   for (int i = warp; i < n_split; i += nt >> 5) {
     const int e = split_e[i];
     const int base = seg[e], qm = qrow[ml[e]], rmain = mr[e];
     // tile count of (e, tile = lane): in flight while the list is built
     const int tv = warp_tiles && lane < p.tiles ? __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e) : 0;
     int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
+#pragma unroll 1
     for (int i0 = 0; i0 < RN; i0 += 32) {
       const int slot = i0 + lane;
       int v = 0, r = 0, pi = 0;
@@ -187,6 +200,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     }
     __syncwarp();
     const int n_e = nz[e];
+#pragma unroll 1
     for (int k = lane; k < n_e; k += 32) {
       rec[rl.cum + base + k] = cum_s[base + k];
       rec[rl.inst + base + k] = inst_s[base + k];
@@ -200,6 +214,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
         if (i < kSplitCap) {
           // ranks [ex, ex + tv) of this tile: inside one instance's quota interval?
           int lo = 0, res = -1;
+#pragma unroll 1
           for (int k = base; k < base + n_e; ++k) {
             const int hi = cum_s[k];
             if (ex >= lo && ex + tv <= hi) { res = inst_s[k]; break; }
@@ -215,11 +230,13 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
   }
   if (p.tiles > 32 && n_split > 0 && in_window) {   // long rows: a thread walks an expert's tiles
     __syncthreads();   // the lists of every split expert are in shared memory
+#pragma unroll 1
     for (int e = tid; e < E; e += nt) {
       if (nz[e] < 2) continue;
       const int32_t* c = p.ws.tile_cnt + trow + e;
       int32_t* o = p.ws.tile_pref + trow + sidx[e];
       int run = 0;
+#pragma unroll 1
       for (int t0 = 0; t0 < p.tiles; t0 += 8) {
         int v[8];
 #pragma unroll
@@ -230,6 +247,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
             o[(size_t)(t0 + u) * E] = run;
             if (sidx[e] < kSplitCap) {
               int lo = 0, res = -1;
+#pragma unroll 1
               for (int k = seg[e]; k < seg[e] + nz[e]; ++k) {
                 const int hi = cum_s[k];
                 if (run >= lo && run + v[u] <= hi) { res = inst_s[k]; break; }
@@ -252,9 +270,11 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     const int ch = (R + 31) / 32;
     const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
     int sum = 0;
+#pragma unroll 1
     for (int r = i0; r < i1; ++r) sum += crow[r];
     int total;
     int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
     for (int r = i0; r < i1; ++r) { send[r] = pre; pre += crow[r]; }
     if (lane == 0) send[R] = total;
   }

@@ -75,8 +75,10 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
 // n ints global -> shared, 16 bytes at a time when both sides allow it.
 __device__ __forceinline__ void copy_async(int* dst, const int32_t* src, int n, int tid, int nt) {
   if ((n & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+#pragma unroll 1
     for (int i = tid; i < n / 4; i += nt) cp_async16(dst + 4 * i, src + 4 * i);
   } else {
+#pragma unroll 1
     for (int i = tid; i < n; i += nt) cp_async4(dst + i, src + i);
   }
 }
@@ -119,6 +121,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   copy_async(reinterpret_cast<int*>(smem + lay.stat),
              p.ws.solve_static + (size_t)dm * solve_static_ints(d), (int)solve_static_ints(d), tid, nt);
   if (tid < G) used[tid] = 0;
+#pragma unroll 1
   for (int i = tid; i < R * G; i += nt) cnt[i] = 0;
   pdl_wait();
   copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
@@ -137,6 +140,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       // compact the candidates (D > 0) of this domain into cand[]: key = (D, -e)
       unsigned long long* cand = cand_all + (size_t)warp * kRankCap;
       int n_c = 0;
+#pragma unroll 1
       for (int e0 = 0; e0 < E; e0 += 32) {
         const int e = e0 + lane;
         int v = 0;
@@ -175,6 +179,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         }
       } else {
         // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
+#pragma unroll 1
         for (int e = lane; e < E; e += 32) {
           const unsigned hosted = dd < 32 ? host_lo[e] >> dd : host_hi[e] >> (dd - 32);
           if ((hosted & 1u) || Dd[e] <= p.cand_thr) Dd[e] = 0;
@@ -182,6 +187,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         __syncwarp();
         for (int i = 0; i < slots; ++i) {
           int bestD = 0, bestE = INT_MAX;
+#pragma unroll 1
           for (int e = lane; e < E; e += 32) {
             const int x = Dd[e];
             if (x > bestD) { bestD = x; bestE = e; }   // ascending e: first hit is smallest
@@ -208,6 +214,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   __syncthreads();
 
   // ---- round 2 of asynchronous copies: the routing-matrix columns of this domain's replicas ----
+#pragma unroll 1
   for (int i = warp; i < G * N; i += nwarps) {
     const int e = col_expert[(i / N) * s_phys + e_loc + i % N];
     if (e < 0) continue;
@@ -253,6 +260,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           idx[u] = __popcll(hm[u] & ((1ull << dm) - 1ull));
         }
       }
+#pragma unroll 1
       for (int s0 = 0; s0 < R; s0 += 32) {
         const int s = s0 + lane;
         const int ds = s < R ? sdom[s] : 0;
@@ -284,6 +292,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   __syncthreads();
   if (tid < G) {
     int sum = 0;
+#pragma unroll 1
     for (int l = 0; l < s_phys; ++l) sum += U[tid * s_phys + l];
     L[tid] = sum;
   }
@@ -311,6 +320,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         const int half = (Lb - Lt) >> 1;                         // half-gap bound
         const bool has_slot = used[gt] < N;
         if (half >= p.min_delta) {
+#pragma unroll 1
           for (int l = k0; l < s_phys; l += kstep) {
             const int cb = gb * s_phys + l;
             const int e = col_expert[cb];
@@ -354,6 +364,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       const int lo = min(rb, rt), hi = max(rb, rt);
       const int i0 = min(R, lane * chunk), i1 = min(R, i0 + chunk);
       int sum = 0;
+#pragma unroll 1
       for (int i = i0; i < i1; ++i) {
         int s = i == 0 ? rt : (i == R - 1 ? rb : i - 1);
         if (i != 0 && i != R - 1) { if (s >= lo) ++s; if (s >= hi) ++s; }
@@ -361,6 +372,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       }
       int total;
       int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
       for (int i = i0; i < i1; ++i) {
         int s = i == 0 ? rt : (i == R - 1 ? rb : i - 1);
         if (i != 0 && i != R - 1) { if (s >= lo) ++s; if (s >= hi) ++s; }
@@ -384,6 +396,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   __syncthreads();
 
   // ---- results of this domain ----------------------------------------------------------------
+#pragma unroll 1
   for (int idx = tid; idx < G * N; idx += nt) {
     const int g = idx / N, j = idx - g * N;
     const int e = col_expert[g * s_phys + e_loc + j];
@@ -391,6 +404,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     p.ws.replica_map[at] = e;
     if (p.out_replica_map) p.out_replica_map[at] = e;
   }
+#pragma unroll 1
   for (int c = tid; c < C; c += nt) {
     const int u = col_expert[c] >= 0 ? U[c] : 0;
     const size_t at = (size_t)b * d.P + (size_t)dm * C + c;
@@ -399,8 +413,10 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   }
   if (tid < G) p.ws.rank_load[(size_t)b * R + dm * G + tid] = L[tid];
   // q rows of this domain's columns; counts[s][r] accumulated per (source, rank) on the way
+#pragma unroll 1
   for (int s = warp; s < R; s += nwarps) {
     int32_t* qrow = p.ws.q + ((size_t)b * R + s) * d.P + (size_t)dm * C;
+#pragma unroll 1
     for (int c = lane; c < C; c += 32) {
       const int v = qd[s * QS + c];
       qrow[c] = v;
@@ -408,6 +424,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     }
   }
   __syncthreads();
+#pragma unroll 1
   for (int i = tid; i < R * G; i += nt) {
     const int s = i / G, g = i - s * G;
     const size_t at = ((size_t)b * R + s) * R + dm * G + g;
@@ -415,14 +432,17 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     p.out_counts[at] = cnt[i];
   }
   // receive offsets of rank r: exclusive scan over the sources, one warp per rank
+#pragma unroll 1
   for (int g = warp; g < G; g += nwarps) {
     int32_t* recv = p.out_offsets + (((size_t)b * 2 + 1) * R + dm * G + g) * (R + 1);
     const int ch = (R + 31) / 32;
     const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
     int sum = 0;
+#pragma unroll 1
     for (int s = i0; s < i1; ++s) sum += cnt[s * G + g];
     int total;
     int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
     for (int s = i0; s < i1; ++s) { recv[s] = pre; pre += cnt[s * G + g]; }
     if (lane == 0) recv[R] = total;
   }
