@@ -135,6 +135,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   // ties to the lower rank).
   if (M > 1 && p.stage1_slots > 0) {
     const int slots = G * p.stage1_slots;   // all N per rank unless some are reserved
+#pragma unroll 1
     for (int dd = warp; dd < M; dd += nwarps) {
       int* Dd = D + dd * E;
       // compact the candidates (D > 0) of this domain into cand[]: key = (D, -e)
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       __syncwarp();
       if (n_c <= kRankCap) {
         // few candidates: every candidate counts the keys above its own; rank < slots wins
+#pragma unroll 1
         for (int c0 = 0; c0 < n_c; c0 += 32) {
           const int c = c0 + lane;
           const unsigned long long mine = c < n_c ? cand[c] : 0ull;
@@ -185,6 +187,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           if ((hosted & 1u) || Dd[e] <= p.cand_thr) Dd[e] = 0;
         }
         __syncwarp();
+#pragma unroll 1
         for (int i = 0; i < slots; ++i) {
           int bestD = 0, bestE = INT_MAX;
 #pragma unroll 1
@@ -228,6 +231,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   // rank == ascending hosting domain), remainder to `rem` instances starting at (s+e) mod n.
   // A warp takes a column, its lanes the sources; main columns first, replica columns once their
   // copies have landed.
+#pragma unroll 1
   for (int pass = 0; pass < 2; ++pass) {
     if (pass == 1) {
       cp_async_wait_all();
@@ -238,6 +242,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     const int* w_base = pass == 0 ? col_main : col_rep;
     // four columns of a warp at a time, so that their dependent shared-memory reads overlap
     constexpr int kCols = 4;
+#pragma unroll 1
     for (int i0 = warp; i0 < ncols; i0 += kCols * nwarps) {
       int c[kCols], e[kCols], n[kCols], idx[kCols], usum[kCols];
       unsigned long long hm[kCols];
