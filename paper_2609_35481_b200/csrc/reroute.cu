@@ -66,21 +66,26 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
   const int lane = tid & 31, rows = c.rows;
   auto sync = [] { __syncthreads(); };
   if (c.n_split > kSplitCap || c.n_list > kFastLists) {   // rare: fetch the rest of the record
+#pragma unroll 1
     for (int i = tid; i <= c.n_split; i += nt) c.seg[i] = c.rec[c.rl.seg + i];
+#pragma unroll 1
     for (int i = tid; i < c.n_list; i += nt) {
       c.cum[i] = c.rec[c.rl.cum + i];
       c.inst[i] = c.rec[c.rl.inst + i];
     }
   }
   bool broken = false;
+#pragma unroll 1
   for (int p0 = 0; p0 < c.n_split; p0 += kSplitCap) {
     const int n_here = min(kSplitCap, c.n_split - p0);
     if (p0 > 0) {   // later passes: fresh counters and tile bases (the first set came up front)
+#pragma unroll 1
       for (int i = tid; i < n_here * rows; i += nt) c.cnt4[i] = make_uint4(0u, 0u, 0u, 0u);
       if (tid < n_here) c.tbase[tid] = c.g_tp[p0 + tid];
     }
     if (p0 > 0 || c.n_split > kSplitCap || c.n_list > kFastLists) sync();
     // every item bumps the 4-bit counter of its (split expert, row, lane)
+#pragma unroll 1
     for (int w = tid; w < c.n_work; w += nt) {
       const int pos = c.work[w];
       const int i = -2 - c.route[__ldg(c.ids + pos)] - p0;
@@ -91,8 +96,10 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
     }
     sync();
     // base[i][rr] = tile base + ids of split expert i in rows before rr
+#pragma unroll 1
     for (int i = warp; i < n_here; i += nwarps) {
       int carry = c.tbase[i];
+#pragma unroll 1
       for (int r0 = 0; r0 < rows; r0 += 32) {
         const int rr = r0 + lane;
         int tot = 0;
@@ -107,12 +114,14 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
       }
     }
     sync();
+#pragma unroll 1
     for (int w = tid; w < c.n_work; w += nt) {
       const int pos = c.work[w], vec = pos >> 2;
       const int e = __ldg(c.ids + pos);
       const int i = -2 - c.route[e] - p0;
       if (i < 0 || i >= n_here) continue;
       int prev = 0;   // equal ids earlier in the same group of four
+#pragma unroll 1
       for (int u = pos & ~3; u < pos; ++u) prev += __ldg(c.ids + u) == e ? 1 : 0;
       const int rr = vec >> 5, ln = vec & 31, word = ln >> 3, shift = 4 * (ln & 7);
       const uint4 q = c.cnt4[i * rows + rr];
