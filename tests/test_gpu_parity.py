@@ -509,3 +509,37 @@ def test_two_chunk_dispatch_windows_match_the_oracle(name, over, batch, cut):
     # window errors
     assert B.topoep_dispatch_window(pl.handle, out.token_replica, T, batch, T - 1, 2, None, None,
                                     None, None, None, 256, 0, 0) == -6
+
+
+# ---- quota boundaries against tile boundaries ---------------------------------------------------
+@pytest.mark.parametrize("T,pattern", [
+    (4 * 4096, "one_expert"),          # every id the same expert: quotas are multiples of a tile
+    (4 * 4096, "two_experts_blocks"),  # long runs: whole tiles of one expert, boundary mid-run
+    (3 * 4096 + 17, "one_expert"),     # ragged last tile
+    (8192, "alternate"),               # two experts interleaved id by id
+])
+def test_quota_boundaries_on_and_off_tile_edges(T, pattern):
+    """A tile whose ids of a split expert fall inside one instance's quota takes that instance
+    without ranking; a tile that straddles a boundary ranks.  These id patterns put the quota
+    boundaries exactly on tile edges, inside long runs and in a ragged last tile."""
+    w = wl.CONFIGS["tiny"].replace(top_k=1, tokens_per_rank=T, slots_per_rank=3, ffn=16)
+    R, E = w.ranks, w.experts
+    ids = np.empty((2, R, T, 1), np.int32)
+    t = np.arange(T)
+    for b in range(2):
+        for s in range(R):
+            hot, other = (3 * s + b) % E, (3 * s + b + 7) % E
+            if pattern == "one_expert":
+                row = np.full(T, hot)
+            elif pattern == "two_experts_blocks":
+                row = np.where((t // 6000) % 2 == 0, hot, other)
+            else:
+                row = np.where(t % 2 == 0, hot, other)
+            ids[b, s, :, 0] = row
+    gpu, ref, _ = parity(w, 0, ids=ids)
+    # the case is only interesting if assignments really are split across instances
+    assert ref.summaries["replica_served"].sum() > 0
+    for tile_ids in (1024, 8192):
+        pl = make_planner(w, max_batch=2)
+        pl.set_tuning(B.KNOB_TILE_IDS, tile_ids)
+        assert_same(run_gpu(pl, ids), ref)
