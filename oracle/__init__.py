@@ -40,7 +40,7 @@ class _Config(ctypes.Structure):
                 ("top_k", ctypes.c_int32), ("c_intra", ctypes.c_int32),
                 ("c_inter", ctypes.c_int32), ("max_refine_iters", ctypes.c_int32),
                 ("min_delta", ctypes.c_int32), ("stages", ctypes.c_int32),
-                ("reserve_slots", ctypes.c_int32), ("pad_", ctypes.c_int32),
+                ("reserve_slots", ctypes.c_int32), ("stage1_rank", ctypes.c_int32),
                 ("token_bytes", ctypes.c_int64), ("expert_bytes", ctypes.c_int64),
                 ("t_ffn", ctypes.c_int64)]
 
@@ -104,6 +104,7 @@ class OracleConfig:
     main_rank: Optional[np.ndarray] = None   # [E] int32; None = blocked e // (E/R)
     stages: int = 3                          # bit 0 inter-node placement, bit 1 refinement
     reserve_slots: int = 0                   # policy variant: slots stage 1 leaves to refinement
+    stage1_rank: int = 0                     # policy variant: 1 = least estimated load (LPT)
 
     def __post_init__(self):
         R = self.ranks
@@ -122,7 +123,7 @@ class OracleConfig:
     def c_struct(self) -> _Config:
         return _Config(self.nodes, self.gpus_per_node, self.experts, self.slots_per_rank,
                        self.top_k, self.c_intra, self.c_inter, self.max_refine_iters,
-                       self.min_delta, self.stages, self.reserve_slots, 0, self.token_bytes,
+                       self.min_delta, self.stages, self.reserve_slots, self.stage1_rank, self.token_bytes,
                        self.expert_bytes, self.t_ffn)
 
     @property

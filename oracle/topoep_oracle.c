@@ -55,6 +55,9 @@
  *     default it does not (its slot-count experiment reports no gain from refinement with one
  *     slot per rank).  reserve_slots > 0 is a policy variant of ours: stage 1 fills at most
  *     N_slot - reserve_slots slots of a rank.
+ *   - "least occupied" could also be read as least token-loaded; stage1_rank = 1 is that reading
+ *     as a policy variant (LPT), with the load estimated before any routing exists: the demand on
+ *     the rank's main instances plus the domain demand of the replicas it already got.
  *
  * Parity status: O1, O8 are pinned to library routines (bincount, cumsum);
  * O3-O6 are pinned by the paper's worked two-domain example, hand-derived
@@ -80,7 +83,9 @@ typedef struct {
   int32_t stages;           /* bit 0: run inter-node placement; bit 1: run refinement */
   int32_t reserve_slots;    /* non-default policy: slots per rank that inter-node placement
                                must leave free for the refinement (0 = the paper's behaviour) */
-  int32_t pad_;
+  int32_t stage1_rank;      /* non-default policy: 0 = a candidate goes to the rank with the
+                               fewest used slots (the paper's wording), 1 = to the rank with the
+                               smallest estimated token load (LPT) */
   int64_t token_bytes;      /* S_tok */
   int64_t expert_bytes;     /* ||W|| */
   int64_t t_ffn;            /* t_FFN */
@@ -171,6 +176,11 @@ static void inter_node_placement(const oracle_config* c, const int32_t* main_ran
   if (cap < 0) cap = 0;
   if (M == 1) return;
   int8_t* taken = (int8_t*)malloc((size_t)E);
+  /* LPT variant: estimated load of a rank = what its main instances receive from all sources
+     (sum over the domains of D) plus the demand D[d][e] of the replicas placed on it so far */
+  int64_t* est = (int64_t*)calloc((size_t)R, sizeof(int64_t));
+  for (int e = 0; e < E; ++e)
+    for (int d = 0; d < M; ++d) est[main_rank[e]] += D[(size_t)d * E + e];
   for (int d = 0; d < M; ++d) {
     memset(taken, 0, (size_t)E);
     for (;;) {
@@ -184,17 +194,23 @@ static void inter_node_placement(const oracle_config* c, const int32_t* main_ran
         if (best_e < 0 || b > best_b) { best_e = e; best_b = b; }
       }
       if (best_e < 0) break;
-      /* least occupied rank of d that still has a free slot */
+      /* the rank of d that takes it, among those with a free slot: the least occupied one, or
+         (LPT variant) the one with the smallest estimated load; ties to the lowest rank */
       int best_r = -1;
-      for (int r = d * G; r < (d + 1) * G; ++r)
-        if (used[r] < cap && (best_r < 0 || used[r] < used[best_r])) best_r = r;
+      for (int r = d * G; r < (d + 1) * G; ++r) {
+        if (used[r] >= cap) continue;
+        if (best_r < 0) { best_r = r; continue; }
+        if (c->stage1_rank == 1 ? est[r] < est[best_r] : used[r] < used[best_r]) best_r = r;
+      }
       if (best_r < 0) break;
       slotmap[(size_t)best_r * N + used[best_r]] = best_e;
       x[(size_t)best_e * R + best_r] = 1;
       used[best_r] += 1;
+      est[best_r] += D[(size_t)d * E + best_e];
       taken[best_e] = 1;
     }
   }
+  free(est);
   free(taken);
 }
 

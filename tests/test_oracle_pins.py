@@ -682,3 +682,57 @@ def test_reserved_slots_keep_every_constraint(reserve):
                w.token_bytes, w.expert_bytes, ids[0], res.replica_map[0], res.token_replica[0],
                res.dispatch_counts[0], res.dispatch_offsets[0], res.instance_counts[0],
                res.rank_load[0])
+
+
+# ---- policy variant: stage-1 candidates to the least-loaded rank (LPT) ---------------------------
+@pytest.mark.parametrize("seed", range(3))
+def test_lpt_places_the_same_experts_on_the_least_loaded_ranks(seed):
+    """With stage1_rank = 1 inter-node placement alone (stages = 1) must replicate exactly the
+    experts the default policy replicates in each domain, but deal them greedily: the next
+    candidate (benefit down, expert id up) to the rank with a free slot and the smallest estimated
+    load -- main-instance demand plus the demand of replicas already there; ties to the lowest
+    rank.  Re-derived here from the routing matrix with a sort and a loop."""
+    w, ids = _skewed_case(seed, slots=2)
+    M, G, E, N = w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank
+    R = M * G
+    mr = w.main_rank()
+    kw = dict(main_rank=mr, stages=1)
+    base = orc.plan(orc.OracleConfig(M, G, E, N, w.top_k, w.token_bytes, w.expert_bytes, **kw), ids)
+    lpt = orc.plan(orc.OracleConfig(M, G, E, N, w.top_k, w.token_bytes, w.expert_bytes,
+                                    stage1_rank=1, **kw), ids)
+    omega = base.omega[0]
+    D = omega.reshape(M, G, E).sum(axis=1)
+    est = np.zeros(R, np.int64)
+    for e in range(E):
+        est[mr[e]] += D[:, e].sum()
+    differs = False
+    for d in range(M):
+        b = 2 * D[d] * w.token_bytes - w.expert_bytes
+        cands = sorted((e for e in range(E) if mr[e] // G != d and b[e] > 0), key=lambda e: (-b[e], e))
+        want = np.full((G, N), -1, np.int32)
+        used = np.zeros(G, int)
+        for e in cands:
+            free = [g for g in range(G) if used[g] < N]
+            if not free:
+                break
+            g = min(free, key=lambda g: (est[d * G + g], g))
+            want[g, used[g]] = e
+            used[g] += 1
+            est[d * G + g] += D[d, e]
+        got = lpt.replica_map[0, d * G:(d + 1) * G]
+        assert np.array_equal(got, want), d
+        assert sorted(got[got >= 0].tolist()) == sorted(base.replica_map[0, d * G:(d + 1) * G][
+            base.replica_map[0, d * G:(d + 1) * G] >= 0].tolist())
+        differs |= not np.array_equal(got, base.replica_map[0, d * G:(d + 1) * G])
+    assert differs          # the variant is not vacuous on this input
+
+
+def test_lpt_keeps_every_constraint():
+    w, ids = _skewed_case(5)
+    cfg = orc.OracleConfig(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k,
+                           w.token_bytes, w.expert_bytes, main_rank=w.main_rank(), stage1_rank=1)
+    res = orc.plan(cfg, ids)
+    check_plan(w.nodes, w.gpus_per_node, w.experts, w.slots_per_rank, w.top_k, w.main_rank(),
+               w.token_bytes, w.expert_bytes, ids[0], res.replica_map[0], res.token_replica[0],
+               res.dispatch_counts[0], res.dispatch_offsets[0], res.instance_counts[0],
+               res.rank_load[0])
