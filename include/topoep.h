@@ -347,9 +347,15 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value);
  *     most N_slot - r replica slots of a rank, leaving r to the intra-node refinement.  The paper
  *     does not say whether slots are held back; by default none are, and with one slot per rank
  *     the refinement then has nothing to work with (paper, slot-count experiment).
+ *   TOPOEP_POLICY_STAGE1_RANK = 0 | 1 (default 0): which rank of a domain takes the next
+ *     inter-node candidate.  0: the rank with the fewest used slots (the paper's "least occupied
+ *     ranks with free slots", as read here); 1: the rank with a free slot and the smallest
+ *     estimated token load (demand on its main instances plus the domain demand of the replicas
+ *     it already took), ties to the lowest rank -- the other reading of the same words.  The set
+ *     of replicated experts is the same, only their ranks differ.
  * Takes effect from the next topoep_plan / topoep_solve.
  */
-enum { TOPOEP_POLICY_RESERVE_SLOTS = 0 };
+enum { TOPOEP_POLICY_RESERVE_SLOTS = 0, TOPOEP_POLICY_STAGE1_RANK = 1 };
 int topoep_set_policy(topoep_handle_t h, int policy, int value);
 
 /*

@@ -230,7 +230,7 @@ def topoep_set_tuning(h, knob: int, value: int) -> int:
     return lib().topoep_set_tuning(h, knob, value)
 
 
-POLICY_RESERVE_SLOTS = 0
+POLICY_RESERVE_SLOTS, POLICY_STAGE1_RANK = 0, 1
 
 
 def topoep_set_policy(h, policy: int, value: int) -> int:

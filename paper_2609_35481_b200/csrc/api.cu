@@ -17,6 +17,7 @@ struct topoep_ctx {
   int max_iters, min_delta, cost_rank_intra, cost_rank_inter;
   std::vector<int32_t> main_rank, main_local, main_inst_expert;
   int tile_ids, hist_mode, pdl;
+  int stage1_lpt;      // policy: 1 = stage-1 candidates to the least-loaded rank
   int reserve_slots;   // policy: slots per rank left to the refinement by inter-node placement
   int rank_first, rank_count;   // window of source ranks of the histogram / reroute buffers
   size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
@@ -203,6 +204,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->hist_mode = 0;
   h->pdl = 1;
   h->reserve_slots = 0;
+  h->stage1_lpt = 0;
   h->rank_first = 0;
   h->rank_count = (int)R;
   h->dispatch_smem = 0;
@@ -328,6 +330,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
     sp.cand_thr = (int)std::min<long long>(thr, INT_MAX);
   }
   sp.stage1_slots = std::max(0, h->d.N - h->reserve_slots);
+  sp.stage1_lpt = h->stage1_lpt;
   sp.cost_rank_intra = h->cost_rank_intra;
   sp.cost_rank_inter = h->cost_rank_inter;
   sp.out_replica_map = replica_map;
@@ -648,6 +651,10 @@ int topoep_set_policy(topoep_handle_t h, int policy, int value) {
     case TOPOEP_POLICY_RESERVE_SLOTS:
       if (value < 0 || value > h->d.N) return TOPOEP_ERR_ARG;
       h->reserve_slots = value;
+      return TOPOEP_OK;
+    case TOPOEP_POLICY_STAGE1_RANK:
+      if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
+      h->stage1_lpt = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

@@ -31,7 +31,7 @@ constexpr int kRankCap = 128;   // stage 1 ranks up to this many candidates of a
 
 struct SolveLayout {
   size_t cand, col_main, col_rep, stat, mrank, mlocal, host_lo, host_hi, col_expert, col_cr, hostcol,
-      sdom, col_rank, D, qd, U, L, used, cnt, total;
+      sdom, col_rank, D, qd, U, L, used, cnt, win_e, win_v, est, total;
 };
 
 // The static block: everything that depends only on the handle and the domain, laid out in the
@@ -68,6 +68,10 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   o.L = at;          at += sizeof(int) * (size_t)d.G;
   o.used = at;       at += sizeof(int) * (size_t)d.G;
   o.cnt = at;        at += sizeof(int) * (size_t)d.R * d.G;
+  o.win_e = at;      at += sizeof(int) * (size_t)d.G * d.N;   // LPT policy: stage-1 winners in order
+  o.win_v = at;      at += sizeof(int) * (size_t)d.G * d.N;   //             and their demand
+  at = (at + 7) & ~(size_t)7;
+  o.est = at;        at += sizeof(long long) * (size_t)d.G;   //             estimated rank loads
   o.total = (at + 15) & ~(size_t)15;
   return o;
 }
@@ -81,6 +85,43 @@ __device__ __forceinline__ void copy_async(int* dst, const int32_t* src, int n, 
 #pragma unroll 1
     for (int i = tid; i < n; i += nt) cp_async4(dst + i, src + i);
   }
+}
+
+// Policy variant of inter-node placement (kept out of line: it is rarely on, and the solver's
+// straight-line code is fetch-bound): the winners, in candidate order, each to the rank with a
+// free slot and the smallest estimated load (demand on its main instances + demand of the
+// replicas it already took); ties to the lowest rank.  Sequential by nature: one lane deals.
+__device__ __noinline__ void lpt_deal(const int* col_main, long long* est, const int* win_e,
+                                      const int* win_v, int* used, int* col_expert, int* col_cr,
+                                      short* hostcol, int n_win, int G, int R, int E, int e_loc,
+                                      int s_phys, int stage1_slots, int cost_rank_inter, int lane) {
+  const unsigned full = 0xffffffffu;
+  __syncwarp();
+  for (int g = 0; g < G; ++g) {   // main-instance demand of rank g: its columns, all sources
+    long long sum = 0;
+#pragma unroll 1
+    for (int i = lane; i < e_loc * R; i += 32) sum += col_main[(size_t)g * e_loc * R + i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(full, sum, o);
+    if (lane == 0) est[g] = sum;
+  }
+  __syncwarp();
+  if (lane == 0) {
+#pragma unroll 1
+    for (int k = 0; k < n_win; ++k) {
+      int bg = -1;
+#pragma unroll 1
+      for (int g = 0; g < G; ++g)
+        if (used[g] < stage1_slots && (bg < 0 || est[g] < est[bg])) bg = g;
+      const int e = win_e[k], col = bg * s_phys + e_loc + used[bg];   // n_win <= G * slots
+      col_expert[col] = e;
+      col_cr[col] = cost_rank_inter;
+      hostcol[bg * E + e] = (short)col;
+      used[bg] += 1;
+      est[bg] += win_v[k];
+    }
+  }
+  __syncwarp();
 }
 
 __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams p) {
@@ -109,6 +150,9 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   int* L = reinterpret_cast<int*>(smem + lay.L);
   int* used = reinterpret_cast<int*>(smem + lay.used);
   int* cnt = reinterpret_cast<int*>(smem + lay.cnt);
+  int* win_e = reinterpret_cast<int*>(smem + lay.win_e);
+  int* win_v = reinterpret_cast<int*>(smem + lay.win_v);
+  long long* est = reinterpret_cast<long long*>(smem + lay.est);
   short* hostcol = reinterpret_cast<short*>(smem + lay.hostcol);
   const short* sdom = reinterpret_cast<const short*>(smem + lay.sdom);
   const short* col_rank = reinterpret_cast<const short*>(smem + lay.col_rank);   // rank of a column
@@ -159,7 +203,9 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         n_c += __popc(m);
       }
       __syncwarp();
+      int n_win = 0;   // candidates that get a slot
       if (n_c <= kRankCap) {
+        n_win = min(n_c, slots);
         // few candidates: every candidate counts the keys above its own; rank < slots wins
 #pragma unroll 1
         for (int c0 = 0; c0 < n_c; c0 += 32) {
@@ -170,7 +216,10 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           if (c < n_c && rank < slots) {
             const int e = (int)~(unsigned)mine;
             if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
-            if (dd == dm) {
+            if (dd == dm && p.stage1_lpt) {
+              win_e[rank] = e;                   // placed below, in order, by estimated load
+              win_v[rank] = (int)(mine >> 32);
+            } else if (dd == dm) {
               const int g = rank % G, j = rank / G, col = g * s_phys + e_loc + j;
               col_expert[col] = e;
               col_cr[col] = p.cost_rank_inter;   // its main lies in another domain
@@ -197,11 +246,15 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           }
           const int maxD = __reduce_max_sync(full, bestD);
           if (maxD <= 0) break;
+          n_win = i + 1;
           const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
           if (lane == 0) {
             Dd[e] = 0;   // taken
             if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
-            if (dd == dm) {
+            if (dd == dm && p.stage1_lpt) {
+              win_e[i] = e;
+              win_v[i] = maxD;
+            } else if (dd == dm) {
               const int g = i % G, j = i / G, col = g * s_phys + e_loc + j;
               col_expert[col] = e;
               col_cr[col] = p.cost_rank_inter;
@@ -212,6 +265,9 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           __syncwarp();
         }
       }
+      if (dd == dm && p.stage1_lpt)
+        lpt_deal(col_main, est, win_e, win_v, used, col_expert, col_cr, hostcol, n_win, G, R, E, e_loc,
+                 s_phys, p.stage1_slots, p.cost_rank_inter, lane);
     }
   }
   __syncthreads();

@@ -110,6 +110,7 @@ struct SolveParams {
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
   int max_iters, min_delta;
+  int stage1_lpt;     // policy: stage-1 winners go to the least-loaded rank, not round robin
   int stage1_slots;   // slots of a rank that inter-node placement may fill (N minus the reserve)
   int cand_thr;   // demand D of a stage-1 candidate exceeds this: floor(||W|| / (2 S_tok))
   int cost_rank_intra, cost_rank_inter;   // dense ranks of {0, c_intra*W, c_inter*W}

@@ -270,6 +270,27 @@ def test_reserved_slots_policy_matches_the_oracle(name, over, reserve):
     assert_same(run_gpu(pl, ids), orc.plan(oracle_config(w), ids))
 
 
+@pytest.mark.parametrize("name,over,reserve", [
+    ("dsv3", dict(slots_per_rank=2, tokens_per_rank=2048), 0),
+    ("mid", dict(slots_per_rank=3), 1),
+    ("scaleout", dict(slots_per_rank=3, tokens_per_rank=2048, zipf_s=1.0), 0),
+    ("tiny", dict(slots_per_rank=3, ffn=16), 0),
+    ("tiny", dict(slots_per_rank=5, ffn=1, experts=512, tokens_per_rank=4096, top_k=4), 0),  # > 128 candidates
+])
+def test_least_loaded_rank_policy_matches_the_oracle(name, over, reserve):
+    w = wl.CONFIGS[name].replace(**over)
+    ids = wl.make_topk_ids(w, seed=43, batch=2)
+    pl = make_planner(w, max_batch=2)
+    pl.set_policy(B.POLICY_STAGE1_RANK, 1)
+    pl.set_policy(B.POLICY_RESERVE_SLOTS, reserve)
+    ref = orc.plan(oracle_config(w, stage1_rank=1, reserve_slots=reserve), ids)
+    assert_same(run_gpu(pl, ids), ref)
+    assert ref.summaries["replicas_inter"].sum() > 0
+    pl.set_policy(B.POLICY_STAGE1_RANK, 0)
+    pl.set_policy(B.POLICY_RESERVE_SLOTS, 0)
+    assert_same(run_gpu(pl, ids), orc.plan(oracle_config(w), ids))
+
+
 # ---- sharded deployment: every rank plans from the gathered routing matrix -----------------------
 @pytest.mark.parametrize("name,over,batch,window", [
     ("mid", dict(slots_per_rank=3), 2, 1),
