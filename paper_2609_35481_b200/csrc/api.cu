@@ -115,7 +115,7 @@ int chain_pdl(const topoep_ctx* h, int batch) {
   long long tiles = 1;
   if (h->hist_tokens >= 0 && h->hist_tile_ids > 0)
     tiles = std::max(1ll, ((long long)h->hist_tokens * h->d.k + h->hist_tile_ids - 1) / h->hist_tile_ids);
-  return tiles * h->rank_count * batch <= 8ll * 148 ? 2 : 1;
+  return tiles * h->rank_count * batch <= 8ll * (h->sms > 0 ? h->sms : 148) ? 2 : 1;
 }
 
 OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, int tiles, int batch) {

@@ -496,6 +496,7 @@ def test_imbalance_against_slot_count_on_the_slot_experiment_shape():
     ("mid", dict(slots_per_rank=3), 2, 2048),                      # the even split of the paper
     ("tiny", dict(slots_per_rank=2), 1, 511),                      # odd cut: ragged, unaligned rows
     ("dsv3", dict(slots_per_rank=2, tokens_per_rank=1024), 1, 384),
+    ("tiny", dict(slots_per_rank=1), 2, 0),                        # an empty first chunk
 ])
 def test_two_chunk_dispatch_windows_match_the_oracle(name, over, batch, cut):
     """The routed tokens are cut into chunks c1 = tokens [0, cut) and c2 = [cut, T) of every source.
