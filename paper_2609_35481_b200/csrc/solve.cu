@@ -124,6 +124,9 @@ __device__ __noinline__ void lpt_deal(const int* col_main, long long* est, const
   __syncwarp();
 }
 
+// LPT: the least-loaded-rank policy of inter-node placement is compiled in (a separate
+// instantiation: the default kernel is fetch-bound and carries no code it never runs).
+template <bool LPT>
 __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const Dims d = p.d;
@@ -216,7 +219,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           if (c < n_c && rank < slots) {
             const int e = (int)~(unsigned)mine;
             if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
-            if (dd == dm && p.stage1_lpt) {
+            if (LPT && dd == dm) {
               win_e[rank] = e;                   // placed below, in order, by estimated load
               win_v[rank] = (int)(mine >> 32);
             } else if (dd == dm) {
@@ -251,7 +254,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           if (lane == 0) {
             Dd[e] = 0;   // taken
             if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
-            if (dd == dm && p.stage1_lpt) {
+            if (LPT && dd == dm) {
               win_e[i] = e;
               win_v[i] = maxD;
             } else if (dd == dm) {
@@ -265,7 +268,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
           __syncwarp();
         }
       }
-      if (dd == dm && p.stage1_lpt)
+      if (LPT && dd == dm)
         lpt_deal(col_main, est, win_e, win_v, used, col_expert, col_cr, hostcol, n_win, G, R, E, e_loc,
                  s_phys, p.stage1_slots, p.cost_rank_inter, lane);
     }
@@ -552,12 +555,16 @@ cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream) {
   // few CTAs: 512 threads shorten each CTA's phases (33.6 vs 35.1 us per single plan); enough
   // CTAs to fill the GPU twice over: 256 threads fit more CTAs per SM (91 vs 106 us per 232 plans)
   const int threads = (long long)p.d.M * batch >= 2 * 148 ? 256 : kSolveThreads;
-  return launch_kernel(solve_kernel, grid, dim3(threads), solve_smem_bytes(p.d), stream,
-                       p.pdl != 0, p);
+  return p.stage1_lpt ? launch_kernel(solve_kernel<true>, grid, dim3(threads), solve_smem_bytes(p.d),
+                                      stream, p.pdl != 0, p)
+                      : launch_kernel(solve_kernel<false>, grid, dim3(threads), solve_smem_bytes(p.d),
+                                      stream, p.pdl != 0, p);
 }
 
 cudaError_t configure_solve(size_t smem) {
-  return cudaFuncSetAttribute(solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(solve_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(solve_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
 }  // namespace topoep
