@@ -130,6 +130,19 @@ def test_many_domains_wide_nodes_and_many_candidates():
     assert ref.summaries["replicas_inter"][0] > 128
 
 
+@pytest.mark.parametrize("nodes,gpus,experts,slots", [(32, 8, 768, 1), (16, 8, 1024, 2), (32, 8, 512, 2)])
+def test_largest_shapes_the_library_accepts(nodes, gpus, experts, slots):
+    """Shapes at the edge of what fits one SM's shared memory (the next larger ones are refused
+    with TOPOEP_ERR_SMEM): 256 ranks, up to 1024 experts."""
+    w = wl.CONFIGS["scaleout"].replace(nodes=nodes, gpus_per_node=gpus, experts=experts,
+                                       slots_per_rank=slots, top_k=4, tokens_per_rank=1536)
+    gpu, ref, _ = parity(w, 71)
+    assert ref.summaries["replicas_inter"].sum() > 0
+    cost = B.CostParams(w.token_bytes, w.expert_bytes, 1, 8, 0, 0, 0)
+    rc, _ = B.topoep_create(nodes, gpus, 4 * experts, slots, 4, 64, 1, None, cost)
+    assert rc == -9
+
+
 def test_random_small_problems():
     rng = np.random.default_rng(11)
     for trial in range(40):
