@@ -372,17 +372,19 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
     const bool lane_on = lane < G * kstep;
     // Inter-node placement leaves an expert at most one instance per domain, so a move needs a
     // target with a free slot; when every slot of the domain is taken there is nothing to do.
-    const bool any_free = __any_sync(full, lane < G && used[lane] < N);
+    // lane g keeps L_g and the used-slot count of rank g in registers for the whole loop
+    int Lreg = lane < G ? L[lane] : -1;
+    int usedreg = lane < G ? used[lane] : N;
+    const bool any_free = __any_sync(full, usedreg < N);
     for (; any_free;) {
-      const int Lg = lane < G ? L[lane] : -1;
-      const int Lb = __reduce_max_sync(full, Lg);
-      const int gb = __ffs(__ballot_sync(full, Lg == Lb)) - 1;   // busiest, lowest id on ties
+      const int Lb = __reduce_max_sync(full, Lreg);
+      const int gb = __ffs(__ballot_sync(full, Lreg == Lb)) - 1;   // busiest, lowest id on ties
+      const int Lt = __shfl_sync(full, Lreg, gt);
+      const bool has_slot = __shfl_sync(full, usedreg, gt) < N;
       int bd = 0, bl = INT_MAX;
       unsigned bk = 0xffffffffu;
       if (lane_on && gt != gb) {
-        const int Lt = L[gt];
         const int half = (Lb - Lt) >> 1;                         // half-gap bound
-        const bool has_slot = used[gt] < N;
         if (half >= p.min_delta) {
 #pragma unroll 1
           for (int l = k0; l < s_phys; l += kstep) {
@@ -413,14 +415,13 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
       const int cb = hostcol[gb * E + e];
       int ct = hostcol[wt * E + e];
       if (ct < 0) {   // create the replica in the target's next free slot
-        ct = wt * s_phys + e_loc + used[wt];
-        __syncwarp();
+        ct = wt * s_phys + e_loc + __shfl_sync(full, usedreg, wt);
         if (lane == 0) {
           col_expert[ct] = e;
           col_cr[ct] = col_cr[cb];
           hostcol[wt * E + e] = (short)ct;
-          used[wt] += 1;
         }
+        if (lane == wt) usedreg += 1;
       }
       // Move md units of q from column cb to ct; sources in the order: the target rank itself,
       // then the others ascending, the busiest rank last.
@@ -448,13 +449,13 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         }
         pre += v;
       }
-      if (lane == 0) {
-        U[cb] -= md; U[ct] += md;
-        L[gb] -= md; L[wt] += md;
-      }
+      if (lane == 0) { U[cb] -= md; U[ct] += md; }
+      if (lane == gb) Lreg -= md;
+      if (lane == wt) Lreg += md;
       __syncwarp();
       ++it;
     }
+    if (lane < G) { L[lane] = Lreg; used[lane] = usedreg; }
     if (lane == 0) p.ws.refine_iters[(size_t)b * M + dm] = it;
   }
   __syncthreads();
