@@ -458,6 +458,73 @@ def test_plan_is_capturable_in_a_cuda_graph_and_replays_identically():
     assert np.array_equal(out.token_replica.cpu().numpy(), ref.token_replica)
 
 
+def test_plan_dispatch_and_replica_copies_in_one_captured_graph():
+    """What a training step would enqueue per layer -- plan, the two chunks' dispatch layouts, the
+    parameter pull and the gradient return -- captured once (after a warm-up call of each entry
+    point) and replayed: nothing in it may allocate, copy to the host or synchronise."""
+    w = wl.CONFIGS["mid"].replace(slots_per_rank=2)
+    cfg = oracle_config(w)
+    ids = wl.make_topk_ids(w, seed=23)
+    pl = make_planner(w)
+    dev = pl.device
+    R, T, k, N, S, Wb = w.ranks, w.tokens_per_rank, w.top_k, 2, pl.s_phys, 4096
+    dev_ids = torch.from_numpy(ids).to(dev)
+    out = pl.alloc_outputs(1, T)
+    i32 = dict(dtype=torch.int32, device=dev)
+    half = T // 2
+    chunks = []
+    for first, count in ((0, half), (half, T - half)):
+        nb = B.topoep_dispatch_scratch_bytes(pl.handle, count, 1)
+        chunks.append(dict(first=first, count=count, nb=nb,
+                           scratch=torch.empty(nb + 256, dtype=torch.uint8, device=dev),
+                           send=torch.empty((1, R, count, k), **i32), recv=torch.empty((1, R, count, k), **i32),
+                           ioff=torch.empty((1, R, S + 1), **i32), counts=torch.empty((1, R, R), **i32),
+                           offs=torch.empty((1, 2, R, R + 1), **i32)))
+    main = torch.from_numpy(wl.make_param_bytes((R, pl.e_loc, Wb), 5)).to(dev)
+    slots = torch.zeros((R, N, Wb), dtype=torch.uint8, device=dev)
+    acc = torch.zeros((R, R, pl.e_loc, Wb), dtype=torch.uint8, device=dev)
+
+    def step(st):
+        pl.plan(dev_ids, out, stream=st)
+        for c in chunks:
+            ptr = (c["scratch"].data_ptr() + 255) // 256 * 256
+            assert B.topoep_dispatch_window(pl.handle, out.token_replica, T, 1, c["first"], c["count"],
+                                            c["send"], c["recv"], c["ioff"], c["counts"], c["offs"],
+                                            ptr, c["nb"], st.cuda_stream) == 0
+        assert B.topoep_replica_pull(pl.handle, out.replica_map[0], main, slots, Wb, st.cuda_stream) == 0
+        assert B.topoep_replica_grad_return(pl.handle, out.replica_map[0], slots, acc, Wb,
+                                            st.cuda_stream) == 0
+
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        step(stream)                                   # first calls set kernel attributes
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step(stream)
+    slots.zero_()
+    acc.zero_()
+    for c in chunks:
+        c["send"].fill_(-9)
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    ref = orc.plan(cfg, ids)
+    assert np.array_equal(out.token_replica.cpu().numpy(), ref.token_replica)
+    for c in chunks:
+        part = np.ascontiguousarray(ref.token_replica[0][:, c["first"]:c["first"] + c["count"]])
+        want_send, want_recv, want_ioff = orc.dispatch_positions(cfg, part)
+        assert np.array_equal(c["send"][0].cpu().numpy(), want_send)
+        assert np.array_equal(c["recv"][0].cpu().numpy(), want_recv)
+        assert np.array_equal(c["ioff"][0].cpu().numpy(), want_ioff)
+    want_slots = orc.replica_pull(cfg, ref.replica_map[0], main.cpu().numpy(), np.zeros((R, N, Wb), np.uint8))
+    assert np.array_equal(slots.cpu().numpy(), want_slots)
+    want_acc = orc.replica_grad_return(cfg, ref.replica_map[0], want_slots,
+                                       np.zeros((R, R, pl.e_loc, Wb), np.uint8))
+    assert np.array_equal(acc.cpu().numpy(), want_acc)
+    assert pl.status() == 0
+
+
 # ---- boundary errors that need a live workspace ---------------------------------------------
 def test_size_and_pointer_errors():
     w = wl.CONFIGS["tiny"]
