@@ -27,6 +27,9 @@ namespace topoep {
 namespace {
 
 constexpr int kPosThreads = 256;
+// ids per thread of the ranking kernel = steps of a warp's dependent chain (measured per
+// 232-plan call: 16 -> 3.08 ms, 8 -> 2.83 ms, 4 -> 3.73 ms)
+constexpr int kPosIds = 8;
 
 // 2a. CTA = (plan, source): exclusive prefix over tiles of the tile counts, in place, and the
 // totals tot[s][p] = assignments of source s on instance p inside the window.
@@ -148,7 +151,7 @@ __global__ void __launch_bounds__(kPosThreads) pos_base_kernel(const PosParams p
   }
 }
 
-__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(const PosParams p) {
+__global__ void __launch_bounds__(kMaxTileIds / kPosIds) pos_rank_kernel(const PosParams p) {
   extern __shared__ int sm[];   // base_a[P], base_b[P], wh[nwarps][P]
   const Dims d = p.d;
   const int P = d.P;
@@ -163,10 +166,10 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
   const int32_t* tr = p.token_replica + row * (size_t)p.row_stride + p.first_id + begin;
 
   // this warp's 512 assignments: step j covers 32 consecutive ones, so (step, lane) is flat order
-  const int wbase = warp * (32 * kIdsPerThread);
-  int x[kIdsPerThread];
+  const int wbase = warp * (32 * kPosIds);
+  int x[kPosIds];
 #pragma unroll
-  for (int j = 0; j < kIdsPerThread; ++j) {
+  for (int j = 0; j < kPosIds; ++j) {
     const int i = wbase + j * 32 + lane;
     x[j] = i < count ? __ldg(tr + i) : -1;
   }
@@ -185,10 +188,10 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
   // need their lanes ordered, which takes one ballot per such instance -- instead of a
   // __match_any_sync per step, whose cost on B200 grows with every distinct value in the warp.
   int* my = wh + warp * P;
-  int rho[kIdsPerThread];
+  int rho[kPosIds];
   const unsigned lt = lanemask_lt();
 #pragma unroll
-  for (int j = 0; j < kIdsPerThread; ++j) {
+  for (int j = 0; j < kPosIds; ++j) {
     const int v = x[j];
     const bool valid = v >= 0 && v < P;
     const int before = valid ? my[v] : 0;
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
   int32_t* send = p.out_send_pos + row * (size_t)p.n_ids + begin;
   int32_t* recv = p.out_recv_pos + row * (size_t)p.n_ids + begin;
 #pragma unroll
-  for (int j = 0; j < kIdsPerThread; ++j) {
+  for (int j = 0; j < kPosIds; ++j) {
     const int i = wbase + j * 32 + lane;
     const int v = x[j];
     int a = -1, c = -1;
@@ -236,7 +239,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) pos_rank_kernel(c
 }  // namespace
 
 size_t pos_rank_smem_bytes(const Dims& d, int tile_ids) {
-  return sizeof(int) * ((size_t)2 * d.P + (size_t)(tile_ids / 512) * d.P);
+  return sizeof(int) * ((size_t)2 * d.P + (size_t)(tile_ids / (32 * kPosIds)) * d.P);
 }
 
 size_t pos_prefix_smem_bytes(const Dims& d) {
@@ -281,7 +284,7 @@ cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) 
   if (e != cudaSuccess) return e;
   // 3. stable ranks inside the tile
   const dim3 grid(p.tiles, p.d.R, batch);
-  const dim3 block(p.tile_ids / kIdsPerThread);
+  const dim3 block(p.tile_ids / kPosIds);
   pos_rank_kernel<<<grid, block, pos_rank_smem_bytes(p.d, p.tile_ids), stream>>>(p);
   return cudaGetLastError();
 }
