@@ -453,7 +453,7 @@ def main():
         dispatch = {"us_per_call": round(us, 2), "us_per_layer_plan": round(us / w.batch, 3),
                     "bytes_per_assignment": 16,
                     "hbm_frac": round(16 * w.assignments / (us * 1e-6) / 1e9 / measured_peak_gbs()[0], 4),
-                    "note": "send/recv positions of every assignment; off the planning path, issue-bound"}
+                    "note": "send/recv positions of every assignment; off the planning path, bound by the per-warp chain of ranking steps"}
         del scratch, send, recv, ioff
 
     # ---- replica parameter executor driven by plan 0 of the batch (reported, not timed into
