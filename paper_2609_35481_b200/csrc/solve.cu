@@ -100,7 +100,11 @@ __device__ __noinline__ void lpt_deal(const int* col_main, long long* est, const
   for (int g = 0; g < G; ++g) {   // main-instance demand of rank g: its columns, all sources
     long long sum = 0;
 #pragma unroll 1
-    for (int i = lane; i < e_loc * R; i += 32) sum += col_main[(size_t)g * e_loc * R + i];
+    for (int l = 0; l < e_loc; ++l) {
+      if (col_expert[g * s_phys + l] < 0) continue;   // a rank with fewer mains: no such column
+#pragma unroll 1
+      for (int i = lane; i < R; i += 32) sum += col_main[((size_t)g * e_loc + l) * R + i];
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(full, sum, o);
     if (lane == 0) est[g] = sum;

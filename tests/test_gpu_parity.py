@@ -165,6 +165,44 @@ def test_random_small_problems():
         pl.close()
 
 
+def test_random_problems_with_policies_tunings_and_skew():
+    """Random topologies, UNEVEN random main maps, skewed and partly padded ids, random policy
+    variants, tile sizes and launch protocols (a wider net of the same kind found a wrong load
+    estimate for ranks with fewer main experts than E_loc under the least-loaded-rank policy)."""
+    rng = np.random.default_rng(12)
+    for trial in range(60):
+        M, G = int(rng.integers(1, 7)), int(rng.integers(1, 9))
+        R = M * G
+        E = int(rng.integers(1, 120))
+        N = int(rng.integers(0, 6))
+        k = int(rng.integers(1, min(E, 6) + 1))
+        T = int(rng.integers(1, 3000))
+        Bn = int(rng.integers(1, 4))
+        main = rng.integers(0, R, size=E).astype(np.int32)
+        tok, W = int(rng.integers(1, 64)), int(rng.integers(0, 4000))
+        skew = float(rng.uniform(0.5, 3.0))
+        ids = np.minimum((rng.random((Bn, R, T, k)) ** skew * E).astype(np.int32), E - 1)
+        if rng.random() < 0.2:
+            ids[rng.random(ids.shape) < 0.05] = -1
+        w = wl.Workload("rnd", M, G, E, N, k, T)
+        reserve, lpt = int(rng.integers(0, N + 1)), int(rng.integers(0, 2))
+        over = dict(main_rank=main, token_bytes=tok, expert_bytes=W,
+                    c_intra=int(rng.integers(0, 3)), c_inter=int(rng.integers(0, 9)))
+        pl = make_planner(w, max_batch=Bn, **over)
+        pl.set_policy(B.POLICY_RESERVE_SLOTS, reserve)
+        pl.set_policy(B.POLICY_STAGE1_RANK, lpt)
+        pl.set_tuning(B.KNOB_TILE_IDS, int(rng.choice([1024, 2048, 4096, 8192])))
+        pl.set_tuning(B.KNOB_PDL, int(rng.integers(0, 4)))
+        gpu = run_gpu(pl, ids)
+        ref = orc.plan(oracle_config(w, reserve_slots=reserve, stage1_rank=lpt, **over), ids)
+        try:
+            assert_same(gpu, ref)
+        except AssertionError as err:
+            raise AssertionError("trial %d %s: %s" % (trial, (M, G, E, N, k, T, Bn, reserve, lpt), err))
+        assert gpu["flags"] == ref.flags
+        pl.close()
+
+
 def test_invalid_and_padded_ids():
     w = wl.CONFIGS["tiny"].replace(slots_per_rank=2)
     ids = wl.make_topk_ids(w, seed=4, batch=2).copy()
