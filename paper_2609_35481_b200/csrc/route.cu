@@ -180,6 +180,7 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
         v = max(qrow[pi], 0);
       }
       const unsigned m = __ballot_sync(0xffffffffu, v > 0);
+      if (m == 0) continue;   // no instance of e among these 32 slots (the common case)
       int tot;
       const int ex = warp_exclusive_scan(v, lane, &tot);
       const bool below_main = v > 0 && r < rmain;

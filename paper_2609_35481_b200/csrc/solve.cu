@@ -428,25 +428,25 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
         if (lane == wt) usedreg += 1;
       }
       // Move md units of q from column cb to ct; sources in the order: the target rank itself,
-      // then the others ascending, the busiest rank last.
+      // then the others ascending, the busiest rank last.  The lanes walk the sources in natural
+      // order (a plain scan) and correct for the two that are out of place: in the required
+      // order a source s other than those two is preceded by rt and by the lower sources except
+      // rt and rb; rb is preceded by everything else.
       const int rb = dm * G + gb, rt = dm * G + wt;
-      const int lo = min(rb, rt), hi = max(rb, rt);
+      const int qrt = qd[rt * QS + cb], qrb = qd[rb * QS + cb];
       const int i0 = min(R, lane * chunk), i1 = min(R, i0 + chunk);
       int sum = 0;
 #pragma unroll 1
-      for (int i = i0; i < i1; ++i) {
-        int s = i == 0 ? rt : (i == R - 1 ? rb : i - 1);
-        if (i != 0 && i != R - 1) { if (s >= lo) ++s; if (s >= hi) ++s; }
-        sum += qd[s * QS + cb];
-      }
+      for (int s = i0; s < i1; ++s) sum += qd[s * QS + cb];
       int total;
       int pre = warp_exclusive_scan(sum, lane, &total);
 #pragma unroll 1
-      for (int i = i0; i < i1; ++i) {
-        int s = i == 0 ? rt : (i == R - 1 ? rb : i - 1);
-        if (i != 0 && i != R - 1) { if (s >= lo) ++s; if (s >= hi) ++s; }
+      for (int s = i0; s < i1; ++s) {
         const int v = qd[s * QS + cb];
-        const int take = min(max(md - pre, 0), v);
+        int before = qrt + pre - (rt < s ? qrt : 0) - (rb < s ? qrb : 0);
+        if (s == rt) before = 0;
+        if (s == rb) before = total - qrb;
+        const int take = min(max(md - before, 0), v);
         if (take > 0) {
           qd[s * QS + cb] = v - take;
           qd[s * QS + ct] += take;
