@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
 
   const int32_t* om_m = p.ws.omega_m + (size_t)b * R * e_loc * R;   // rows = main instances
 
-  // ---- round 1 of asynchronous copies: the static block of this domain first (main-rank tables,
+  // ---- first batch of asynchronous copies: the static block of this domain first (main-rank tables,
   // hosting masks and column tables as they are before any replica exists), then -- once the
   // omega kernel is done -- the demand and this domain's main columns
   copy_async(reinterpret_cast<int*>(smem + lay.stat),
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   }
   __syncthreads();
 
-  // ---- round 2 of asynchronous copies: the routing-matrix columns of this domain's replicas ----
+  // ---- second batch of asynchronous copies: the routing-matrix columns of this domain's replicas ----
 #pragma unroll 1
   for (int i = warp; i < G * N; i += nwarps) {
     const int e = col_expert[(i / N) * s_phys + e_loc + i % N];
