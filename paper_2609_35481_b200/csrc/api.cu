@@ -245,6 +245,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.omega_m = at<int32_t>(dev_ptr, h->off[W_OMEGA_M]);
   w.demand = at<int32_t>(dev_ptr, h->off[W_DEMAND]);
   w.tile_cnt = at<int32_t>(dev_ptr, h->off[W_TILE_CNT]);
+  w.tile_cnt16 = 1;
   w.tile_pref = at<int32_t>(dev_ptr, h->off[W_TILE_PREF]);
   w.q = at<int32_t>(dev_ptr, h->off[W_Q]);
   w.rank_load = at<int32_t>(dev_ptr, h->off[W_LOAD]);

@@ -261,6 +261,7 @@ cudaError_t launch_dispatch(const PosParams& p, int batch, cudaStream_t stream) 
   hp.d.E = p.d.P;
   hp.ws = p.ws;
   hp.ws.tile_cnt = p.pos_cnt;
+  hp.ws.tile_cnt16 = 0;   // these counts become prefixes over tiles in place: 32 bits
   hp.ids = p.token_replica;
   hp.rank_first = 0;
   hp.rank_count = p.d.R;

@@ -67,8 +67,17 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   pdl_wait();   // the ids are nobody's output; everything written below may still be in use
   if (mx > (unsigned)E) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);
   __syncthreads();
-  int32_t* out = p.ws.tile_cnt + (row * (size_t)p.max_tiles + tile) * E;
-  for (int e = tid; e < E; e += nt) out[e] = cnt[e];
+  const size_t at = (row * (size_t)p.max_tiles + tile) * E;
+  if (!p.ws.tile_cnt16) {
+    int32_t* out = p.ws.tile_cnt + at;
+    for (int e = tid; e < E; e += nt) out[e] = cnt[e];
+  } else if (E % 2 == 0) {   // two 16-bit counts per word (at * 2 bytes is a multiple of 4)
+    unsigned* out = reinterpret_cast<unsigned*>(reinterpret_cast<unsigned short*>(p.ws.tile_cnt) + at);
+    for (int t = tid; t < E / 2; t += nt) out[t] = (unsigned)cnt[2 * t] | ((unsigned)cnt[2 * t + 1] << 16);
+  } else {
+    unsigned short* out = reinterpret_cast<unsigned short*>(p.ws.tile_cnt) + at;
+    for (int e = tid; e < E; e += nt) out[e] = (unsigned short)cnt[e];
+  }
 }
 
 // omega[b][s][e] = sum over the row's tiles (or a routing matrix handed in), written three ways
@@ -94,11 +103,16 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
     if (p.src_omega) {
       sum = __ldg(p.src_omega + row * E + e);
     } else {
-      const int32_t* c = p.ws.tile_cnt + row * (size_t)p.max_tiles * E + e;
+      const size_t at = row * (size_t)p.max_tiles * E + e;
+      const int32_t* c = p.ws.tile_cnt + at;
+      const unsigned short* c16 = reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + at;
+      const bool n16 = p.ws.tile_cnt16 != 0;
       for (int t0 = 0; t0 < p.tiles; t0 += 16) {
         int v[16];
 #pragma unroll
-        for (int u = 0; u < 16; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
+        for (int u = 0; u < 16; ++u)
+          v[u] = t0 + u >= p.tiles ? 0 : n16 ? (int)__ldg(c16 + (size_t)(t0 + u) * E)
+                                              : __ldg(c + (size_t)(t0 + u) * E);
 #pragma unroll
         for (int u = 0; u < 16; ++u) sum += v[u];
       }
@@ -135,15 +149,31 @@ __global__ void __launch_bounds__(128) omega4_kernel(const OmegaParams p) {
     if (p.src_omega) {
       sum = __ldg(reinterpret_cast<const int4*>(p.src_omega + row * E + e));
     } else {
-      const int4* c = reinterpret_cast<const int4*>(p.ws.tile_cnt + row * (size_t)p.max_tiles * E + e);
+      const size_t at = row * (size_t)p.max_tiles * E + e;
       const size_t stride = (size_t)E / 4;
-      for (int t0 = 0; t0 < p.tiles; t0 += 8) {
-        int4 v[8];
+      if (p.ws.tile_cnt16) {   // four 16-bit counts = one 8-byte load
+        const uint2* c = reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + at);
+        for (int t0 = 0; t0 < p.tiles; t0 += 8) {
+          uint2 v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-          v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * stride) : make_int4(0, 0, 0, 0);
+          for (int u = 0; u < 8; ++u)
+            v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * stride) : make_uint2(0u, 0u);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { sum.x += v[u].x; sum.y += v[u].y; sum.z += v[u].z; sum.w += v[u].w; }
+          for (int u = 0; u < 8; ++u) {
+            sum.x += (int)(v[u].x & 0xffffu); sum.y += (int)(v[u].x >> 16);
+            sum.z += (int)(v[u].y & 0xffffu); sum.w += (int)(v[u].y >> 16);
+          }
+        }
+      } else {
+        const int4* c = reinterpret_cast<const int4*>(p.ws.tile_cnt + at);
+        for (int t0 = 0; t0 < p.tiles; t0 += 8) {
+          int4 v[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u)
+            v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * stride) : make_int4(0, 0, 0, 0);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) { sum.x += v[u].x; sum.y += v[u].y; sum.z += v[u].z; sum.w += v[u].w; }
+        }
       }
     }
     if (p.ws.omega) *reinterpret_cast<int4*>(p.ws.omega + row * E + e) = sum;

@@ -168,7 +168,10 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     const int e = split_e[i];
     const int base = seg[e], qm = qrow[ml[e]], rmain = mr[e];
     // tile count of (e, tile = lane): in flight while the list is built
-    const int tv = warp_tiles && lane < p.tiles ? __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e) : 0;
+    int tv = 0;
+    if (warp_tiles && lane < p.tiles)
+      tv = p.ws.tile_cnt16 ? (int)__ldg(reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + trow + (size_t)lane * E + e)
+                           : __ldg(p.ws.tile_cnt + trow + (size_t)lane * E + e);
     int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
 #pragma unroll 1
     for (int i0 = 0; i0 < RN; i0 += 32) {
@@ -235,13 +238,16 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
     for (int e = tid; e < E; e += nt) {
       if (nz[e] < 2) continue;
       const int32_t* c = p.ws.tile_cnt + trow + e;
+      const unsigned short* c16 = reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + trow + e;
       int32_t* o = p.ws.tile_pref + trow + sidx[e];
       int run = 0;
 #pragma unroll 1
       for (int t0 = 0; t0 < p.tiles; t0 += 8) {
         int v[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = t0 + u < p.tiles ? __ldg(c + (size_t)(t0 + u) * E) : 0;
+        for (int u = 0; u < 8; ++u)
+          v[u] = t0 + u >= p.tiles ? 0 : p.ws.tile_cnt16 ? (int)__ldg(c16 + (size_t)(t0 + u) * E)
+                                                         : __ldg(c + (size_t)(t0 + u) * E);
 #pragma unroll
         for (int u = 0; u < 8; ++u)
           if (t0 + u < p.tiles) {

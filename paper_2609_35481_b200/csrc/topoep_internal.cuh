@@ -40,6 +40,8 @@ struct Workspace {
                                     //   instance (row = main_rank(e)*e_loc + main_local(e))
   int32_t* demand;                  // [max_batch][M][E] domain demand D
   int32_t* tile_cnt;                // [max_batch][R][max_tiles][E] per-tile histogram
+  int tile_cnt16;                   // 1: the per-tile counts are 16-bit (a tile has < 65536 ids);
+                                    //   same indexing, half the bytes.  0: 32-bit (dispatch, static)
   int32_t* tile_pref;               // [max_batch][R][max_tiles][E] exclusive prefix over tiles,
                                     //   column i = i-th split expert of the source
   int32_t* q;                       // [max_batch][R][P]
