@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
                    ((unsigned)(t2 + 1) >> 31) << 2 | ((unsigned)(t3 + 1) >> 31) << 3) << (4 * j);
     const int4 r = make_int4(max(t0, -1), max(t1, -1), max(t2, -1), max(t3, -1));
     if (VEC) {
-      if (4 * vec < count) reinterpret_cast<int4*>(out)[vec] = r;
+      if (4 * vec < count) __stcs(reinterpret_cast<int4*>(out) + vec, r);
     } else {
       if (4 * vec + 0 < count) out[4 * vec + 0] = r.x;
       if (4 * vec + 1 < count) out[4 * vec + 1] = r.y;
