@@ -111,6 +111,7 @@ def test_two_stage_example_matches_paper():
 
     r0 = orc.solve(_cfg(g["config"], stages=0), om)
     assert r0.L.tolist() == g["expect_no_placement"]["L"]
+    assert orc.summary(cfg, r0)["replica_served"] == 0        # every assignment on a main instance
     assert _cross(cfg, r0.q) == g["expect_no_placement"]["cross"] == pv["assignments_gpu0_to_E4"]
 
     r1 = orc.solve(_cfg(g["config"], stages=1), om)
@@ -118,6 +119,8 @@ def test_two_stage_example_matches_paper():
     assert r1.L.tolist() == g["expect_stage1"]["L"]
     assert r1.L[:2].tolist() == pv["loads_gpu0_gpu1_after_inter_node"]
     assert _cross(cfg, r1.q) == 0
+    # the eight assignments now execute on the replica E4' (GPU 0)
+    assert orc.summary(cfg, r1)["replica_served"] == pv["E4_assignments_on_replicas"]
 
     r = orc.solve(cfg, om, trace_cap=8)
     ex = g["expect_final"]
@@ -130,6 +133,11 @@ def test_two_stage_example_matches_paper():
         assert row[key] == val
     assert row["delta"] == pv["moved_by_refinement"]
     assert _cross(cfg, r.q) == pv["new_cross_domain_routes"]
+    # four stay on E4', four moved to E4'': all eight are executed by replicas, none by GPU 2
+    sm = orc.summary(cfg, r)
+    assert sm["replica_served"] == pv["E4_assignments_on_replicas"]
+    assert sm["replica_fraction"] == pv["E4_assignments_on_replicas"] / om.sum()
+    assert r.q[0, 4].tolist() == [4, 4, 0, 0]
 
 
 @pytest.mark.parametrize("variant", ["variant_cost_tiebreak", "variant_cost_uses_main_rank"])
@@ -162,6 +170,11 @@ def test_hand_derived_fixture(case):
         assert r.L.tolist() == ex["L"]
     if "cross" in ex:
         assert _cross(cfg, r.q) == ex["cross"]
+    if "replica_served" in ex:
+        # executed by a replica = on a rank other than main(e), whatever its domain
+        summ = orc.summary(cfg, r)
+        assert summ["replica_served"] == ex["replica_served"]
+        assert summ["replica_fraction"] == ex["replica_served"] / om.sum()
     if "trace" in ex:
         assert len(r.trace) == len(ex["trace"])
         for got, want in zip(r.trace, ex["trace"]):
