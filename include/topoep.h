@@ -112,7 +112,9 @@ enum {
   TOPOEP_T_OMEGA = 0,       /* [max_batch][R][E]   routing matrix Omega           */
   TOPOEP_T_Q = 1,           /* [max_batch][R][P]   q(s, instance)                 */
   TOPOEP_T_RANK_LOAD = 2,   /* [max_batch][R]      L_r                            */
-  TOPOEP_T_REFINE_ITERS = 3 /* [max_batch][M]      commits per domain             */
+  TOPOEP_T_REFINE_ITERS = 3,/* [max_batch][M]      commits per domain             */
+  TOPOEP_T_D = 4,           /* [max_batch][M][E]   domain demand D                */
+  TOPOEP_T_U = 5            /* [max_batch][P]      per-instance load U            */
 };
 
 /* Knobs for topoep_set_tuning; no knob may change any output bit. */
@@ -127,9 +129,15 @@ enum {
                                    GPU all at once also lets each kernel start its
                                    dependents early; 2: on, never early; 3: on,
                                    always early                                   */
-  TOPOEP_KNOB_TRANSFER_MODE = 3 /* replica transfers: 0 (default) the bulk
+  TOPOEP_KNOB_TRANSFER_MODE = 3,/* replica transfers: 0 (default) the bulk
                                    asynchronous copy unit through shared memory,
                                    1 plain 16-byte loads and stores               */
+  TOPOEP_KNOB_TRANSFER_SELFTEST = 4 /* tests only (the one knob that does change
+                                   output): 1 makes one block of the bulk engine
+                                   wait for a copy it never issued, so its bounded
+                                   wait runs out: the transfer sets
+                                   TOPOEP_FLAG_INTERNAL, skips that block's chunks
+                                   and returns by itself; 0 (default) off         */
 };
 
 /*
@@ -167,7 +175,8 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes);
  * Plan B batches.  (Paper: routing matrix Omega; "Two-Stage GPU-Native
  * Solver": inter-node placement with b_{d,e}, routing construction, loads
  * U and L, intra-node refinement with the half-gap delta; constraints
- * C1-C5; "derives receive counts on the GPU".)
+ * C1-C5; Implementation, "DeepEP dispatch and combine": receive counts are
+ * computed on the device from the routing.)
  *
  *   dev_topk_ids        in  [B][R][T][k] int32, expert id per assignment; ids
  *                           outside [0,E) are ignored (-1 is the padding value)
@@ -228,7 +237,9 @@ int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_
  *
  * The first call on a device looks up the array's device address (once per
  * device, with that device current); make that first call outside any stream
- * capture.  All calls share the one array, which keeps the previous call's
+ * capture.  The address is remembered per device ordinal, that is, for the
+ * runtime's primary context: a second (driver-API) context on the same device
+ * is not supported.  All calls share the one array, which keeps the previous call's
  * contents: the call clears the only word that must start at zero itself, and
  * two calls that overlap on the GPU (different streams, or graphs replayed
  * concurrently) race on it -- serialise them.

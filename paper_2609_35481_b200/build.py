@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtopoep.so")
 SOURCES = ["api.cu", "hist.cu", "hist_static.cu", "solve.cu", "route.cu", "reroute.cu", "dispatch.cu", "transfer.cu", "summary.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
-              "-Xcompiler", "-fPIC", "-shared", "--use_fast_math"]
+              "-Xcompiler", "-fPIC", "-shared"]
 
 
 def _stale() -> bool:

@@ -22,6 +22,7 @@ struct topoep_ctx {
   int rank_first, rank_count;   // window of source ranks of the histogram / reroute buffers
   size_t dispatch_smem;   // shared memory the dispatch ranking kernel was configured for
   int transfer_ready, transfer_mode, sms;   // replica executor: configured?, copy engine, SM count
+  int transfer_selftest;   // tests only: the bulk engine's bounded wait is made to run out once
   int max_tiles;
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
   // workspace
@@ -115,7 +116,7 @@ int chain_pdl(const topoep_ctx* h, int batch) {
   long long tiles = 1;
   if (h->hist_tokens >= 0 && h->hist_tile_ids > 0)
     tiles = std::max(1ll, ((long long)h->hist_tokens * h->d.k + h->hist_tile_ids - 1) / h->hist_tile_ids);
-  return tiles * h->rank_count * batch <= 8ll * (h->sms > 0 ? h->sms : 148) ? 2 : 1;
+  return tiles * h->rank_count * batch <= 8ll * h->d.sms ? 2 : 1;
 }
 
 OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, int tiles, int batch) {
@@ -150,7 +151,10 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
     return TOPOEP_ERR_CONFIG;
   const long long R = (long long)nodes * gpus_per_node;
   const long long n_ids = (long long)max_tokens_per_rank * top_k;
-  if (n_ids * gpus_per_node >= (1ll << 31)) return TOPOEP_ERR_CONFIG;   // D and L stay in int32
+  // every count the plan derives is at most the R * T * k assignments of one plan (the rank load
+  // L_r, the receive offsets and the column sums of the dispatch counts can reach it under
+  // skewed routing): it must fit an int32
+  if (R * n_ids >= (1ll << 31)) return TOPOEP_ERR_CONFIG;
   if (cost->token_bytes < 0 || cost->expert_bytes < 0 || cost->c_intra < 0 || cost->c_inter < 0 ||
       cost->t_ffn < 0)
     return TOPOEP_ERR_COST;
@@ -175,6 +179,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   d.P = d.R * d.s_phys;
   d.C = d.G * d.s_phys;
   d.qstride = d.C | 1;
+  d.sms = 0;   // read from the device in topoep_set_workspace
   if (d.s_phys < 1 || (long long)d.C > 32767) { delete h; return TOPOEP_ERR_CONFIG; }
   h->main_inst_expert.assign((size_t)R * std::max(d.e_loc, 1), -1);
   for (int e = 0; e < experts; ++e)
@@ -210,6 +215,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->dispatch_smem = 0;
   h->transfer_ready = 0;
   h->transfer_mode = 0;
+  h->transfer_selftest = 0;
   h->sms = 0;
   h->max_tiles = (int)std::max(1ll, (n_ids + kMinTileIds - 1) / kMinTileIds);
   h->have_ws = false;
@@ -258,6 +264,12 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
 
   cudaError_t e;
   const size_t E = h->d.E;
+  {
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) goto fail;
+    if ((e = cudaDeviceGetAttribute(&h->d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) goto fail;
+    h->sms = h->d.sms;
+  }
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_rank), h->main_rank.data(), 4 * E,
                       cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_local), h->main_local.data(), 4 * E,
@@ -539,11 +551,8 @@ int enqueue_transfer(topoep_handle_t h, int direction, const int32_t* dev_replic
   if (transfer_smem_bytes(h->d, h->transfer_mode) > 113 * 1024) return TOPOEP_ERR_SMEM;
   cudaError_t e = cudaSuccess;
   if (!h->transfer_ready) {
-    // first use: host-side attributes only (shared-memory opt-in, SM count)
-    int dev = 0;
-    e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess) e = configure_transfer(h->d);
+    // first use: host-side attributes only (shared-memory opt-in)
+    e = configure_transfer(h->d);
     if (e == cudaSuccess) h->transfer_ready = 1;
   }
   if (e == cudaSuccess) {
@@ -554,6 +563,7 @@ int enqueue_transfer(topoep_handle_t h, int direction, const int32_t* dev_replic
     p.src = src;
     p.dst = dst;
     p.param_bytes = param_bytes;
+    p.selftest = h->transfer_selftest;
     e = launch_transfer(p, direction, h->transfer_mode, h->sms, stream);
   }
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
@@ -617,6 +627,8 @@ int topoep_debug_tensor(topoep_handle_t h, int which, const void** dev_ptr, size
     case TOPOEP_T_Q: *dev_ptr = h->ws.q; *bytes = 4 * B * d.R * d.P; break;
     case TOPOEP_T_RANK_LOAD: *dev_ptr = h->ws.rank_load; *bytes = 4 * B * d.R; break;
     case TOPOEP_T_REFINE_ITERS: *dev_ptr = h->ws.refine_iters; *bytes = 4 * B * d.M; break;
+    case TOPOEP_T_D: *dev_ptr = h->ws.demand; *bytes = 4 * B * d.M * d.E; break;
+    case TOPOEP_T_U: *dev_ptr = h->ws.inst_counts; *bytes = 4 * B * d.P; break;
     default: return TOPOEP_ERR_ARG;
   }
   return TOPOEP_OK;
@@ -640,6 +652,10 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_TRANSFER_MODE:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->transfer_mode = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_TRANSFER_SELFTEST:
+      if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
+      h->transfer_selftest = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

@@ -221,7 +221,7 @@ cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream) {
   auto al16 = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15u) == 0; };
   // large calls only: with few CTAs the four-times-longer per-thread chain costs latency
   // (one 32-rank plan: 6.7 us -> 8.1 us for histogram + omega; 232 plans: 338 -> 324 us)
-  if ((long long)p.d.R * batch >= 2 * 148 && p.d.E % 4 == 0 && al16(p.src_omega) && al16(p.out_omega) && al16(p.ws.omega) &&
+  if ((long long)p.d.R * batch >= 2ll * p.d.sms && p.d.E % 4 == 0 && al16(p.src_omega) && al16(p.out_omega) && al16(p.ws.omega) &&
       al16(p.ws.demand) && al16(p.ws.tile_cnt) && al16(p.ws.main_rank) && al16(p.ws.main_local)) {
     const dim3 grid((p.d.E / 4 + 4 * p.epw - 1) / (4 * p.epw), p.d.M, batch);
     return launch_kernel(omega4_kernel, grid, dim3(128), 0, stream, p.pdl != 0, p);

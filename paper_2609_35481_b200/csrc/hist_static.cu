@@ -26,9 +26,13 @@ static __device__ __align__(256) unsigned char g_hist_scratch[kScratchBytes];
 
 std::mutex g_setup_mutex;
 void* g_scratch_addr[kMaxDevices];   // device address of g_hist_scratch, per device ordinal
+int g_sms[kMaxDevices];              // SM count of the device (launch shapes)
 
 // Device address of the scratch array on the current device; resolved on the first call there.
-cudaError_t scratch_address(void** out) {
+// The cache is keyed by the device ordinal, i.e. it assumes the runtime's primary context: a
+// program that drives the same device through a second, driver-API context would be handed the
+// primary context's address there.
+cudaError_t scratch_address(void** out, int* sms) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -38,9 +42,12 @@ cudaError_t scratch_address(void** out) {
     void* ptr = nullptr;
     e = cudaGetSymbolAddress(&ptr, g_hist_scratch);
     if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&g_sms[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
     g_scratch_addr[dev] = ptr;
   }
   *out = g_scratch_addr[dev];
+  *sms = g_sms[dev];
   return cudaSuccess;
 }
 
@@ -63,12 +70,20 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   const long long n_ids = (long long)tokens_per_rank * top_k;
   if (n_ids >= (1ll << 31)) return TOPOEP_ERR_CONFIG;
   const long long tiles = std::max(1ll, (n_ids + kStaticTileIds - 1) / kStaticTileIds);
-  const unsigned long long need =
-      kFlagsBytes + 4ull * (unsigned long long)batch * ranks * tiles * experts;
-  if (need > kScratchBytes) return TOPOEP_ERR_SCRATCH;   // beyond the built-in array: no fallback
+  // 4 * batch * ranks * tiles * experts bytes of tile counts must fit behind the flag word.
+  // Checked by division, one factor at a time: the product itself can exceed 64 bits for sizes
+  // the range checks above let through.
+  {
+    unsigned long long cells = (kScratchBytes - kFlagsBytes) / 4;   // 32-bit counts that fit
+    cells /= (unsigned long long)experts;
+    cells /= (unsigned long long)tiles;
+    cells /= (unsigned long long)ranks;
+    if ((unsigned long long)batch > cells) return TOPOEP_ERR_SCRATCH;   // no fallback
+  }
 
   void* base = nullptr;
-  cudaError_t e = scratch_address(&base);
+  int sms = 0;
+  cudaError_t e = scratch_address(&base, &sms);
   if (e != cudaSuccess) return TOPOEP_ERR_CUDA;
   uint32_t* flags = dev_flags ? dev_flags : static_cast<uint32_t*>(base);
   // the status word only ever gets bits OR-ed in, so it must start at zero for this call; the
@@ -80,6 +95,7 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   hp.d.R = ranks;
   hp.d.E = experts;
   hp.d.k = top_k;
+  hp.d.sms = sms;
   hp.rank_first = 0;
   hp.rank_count = ranks;
   hp.ws.status = flags;
@@ -100,6 +116,7 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
     op.d.M = ranks;
     op.d.G = 1;
     op.d.E = experts;
+    op.d.sms = sms;
     op.ws.tile_cnt = hp.ws.tile_cnt;
     op.out_omega = dev_omega;
     op.tiles = hp.tiles;

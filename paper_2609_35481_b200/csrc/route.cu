@@ -1,5 +1,6 @@
 // Per-source routing tables and send offsets (paper, "System Design": the token-routing
-// decisions q drive dispatch; "derives receive counts on the GPU").
+// decisions q drive dispatch; Implementation, "DeepEP dispatch and combine" paragraph: the counts
+// a rank will receive are computed on the device from the routing, with no host round trip).
 //
 // One CTA per (plan, source rank s).  For every expert e it looks at the instances that got a
 // nonzero share q(s,e,.) of the source's assignments:
@@ -296,7 +297,7 @@ cudaError_t launch_route(const RouteParams& p, int batch, cudaStream_t stream) {
   // few CTAs: 256 threads shorten each CTA's phases (latency); enough CTAs to fill the GPU twice
   // over: two warps per CTA spend far fewer issue slots on barriers, scans and idle lanes
   // (232 plans: solver + route stage 83.7 us with 256 threads, 62.9 with 128, 57.3 with 64)
-  const int thr = (long long)p.d.R * batch >= 2 * 148 ? 64 : kRouteThreads;
+  const int thr = (long long)p.d.R * batch >= 2ll * p.d.sms ? 64 : kRouteThreads;
   return launch_kernel(route_kernel, grid, dim3(thr), route_smem_bytes(p.d), stream,
                        p.pdl != 0, p);
 }

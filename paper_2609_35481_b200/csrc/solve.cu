@@ -559,7 +559,7 @@ cudaError_t launch_solve(const SolveParams& p, int batch, cudaStream_t stream) {
   const dim3 grid(p.d.M, batch);
   // few CTAs: 512 threads shorten each CTA's phases (33.6 vs 35.1 us per single plan); enough
   // CTAs to fill the GPU twice over: 256 threads fit more CTAs per SM (91 vs 106 us per 232 plans)
-  const int threads = (long long)p.d.M * batch >= 2 * 148 ? 256 : kSolveThreads;
+  const int threads = (long long)p.d.M * batch >= 2ll * p.d.sms ? 256 : kSolveThreads;
   return p.stage1_lpt ? launch_kernel(solve_kernel<true>, grid, dim3(threads), solve_smem_bytes(p.d),
                                       stream, p.pdl != 0, p)
                       : launch_kernel(solve_kernel<false>, grid, dim3(threads), solve_smem_bytes(p.d),

@@ -26,6 +26,7 @@ struct Dims {
   int e_loc, s_phys, P;
   int C;        // G * s_phys: instance columns of one domain
   int qstride;  // padded row stride of the shared q block (odd, avoids bank conflicts)
+  int sms;      // streaming multiprocessors of the device the workspace lives on (launch shapes)
 };
 
 // Device pointers into the caller's workspace.
@@ -167,6 +168,7 @@ struct TransferParams {
   const void* src;              // pull: main_params [R][e_loc][W]; return: replica_buf [R][N][W]
   void* dst;                    // pull: replica_buf;  return: grad_acc [R][R][e_loc][W]
   unsigned long long param_bytes;   // W, a multiple of 16
+  int selftest;                 // tests only: CTA 0 of the bulk engine runs its give-up path once
 };
 
 struct SummaryParams {

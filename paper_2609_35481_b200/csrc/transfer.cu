@@ -33,6 +33,7 @@ constexpr int kBulkCtasPerSm = 2;
 constexpr int kBulkThreads = 32;
 constexpr int kPlainThreads = 256;
 constexpr unsigned kWaitLimit = 1u << 22;   // polls (about 0.1 s) before a wait is given up
+constexpr unsigned kSelfTestWaitLimit = 1u << 12;   // the self test's wait, which cannot succeed
 
 struct CopyPair { uint32_t src, dst; };   // block indices, in units of |W| bytes
 
@@ -92,9 +93,9 @@ __device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-// Bounded wait for the phase with the given parity; false if it ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (unsigned i = 0; i < kWaitLimit; ++i) {
+// Bounded wait for the phase with the given parity; false if it ran out after `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned limit) {
+  for (unsigned i = 0; i < limit; ++i) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -146,16 +147,34 @@ __global__ void __launch_bounds__(kBulkThreads) transfer_bulk_kernel(const Trans
     *d = dst_base + (unsigned long long)cp.dst * W + off;
   };
 
+  // Self test of the give-up path (host knob, tests only): CTA 0 announces the bytes of its first
+  // chunk on the stage's barrier but never issues the copy, so nothing is in flight for that
+  // stage, its wait runs out after a short limit, and the CTA must flag, drain and return.
+  const bool selftest = p.selftest != 0 && blockIdx.x == 0;
+  const unsigned limit = selftest ? kSelfTestWaitLimit : kWaitLimit;
   const unsigned long long lead = min((unsigned long long)(kStages - 1), mine);
+  unsigned long long issued = 0;   // items whose load has been handed to the copy unit
   for (unsigned long long n = 0; n < lead; ++n) {
     const unsigned char* s; unsigned char* d; uint32_t bytes;
     locate(n, &s, &d, &bytes);
-    bulk_load(smem_u32(ring + (n % kStages) * kStageBytes), s, bytes, smem_u32(&bars[n % kStages]));
+    if (selftest && n == 0) {
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&bars[0])),
+                   "r"(bytes)
+                   : "memory");
+    } else {
+      bulk_load(smem_u32(ring + (n % kStages) * kStageBytes), s, bytes, smem_u32(&bars[n % kStages]));
+    }
+    issued = n + 1;
   }
   for (unsigned long long n = 0; n < mine; ++n) {
     const int st = (int)(n % kStages);
-    if (!mbar_wait(smem_u32(&bars[st]), (uint32_t)((n / kStages) & 1))) {
+    if (!mbar_wait(smem_u32(&bars[st]), (uint32_t)((n / kStages) & 1), limit)) {
+      // Gave up on item n: report it, issue nothing more, and let the loads already handed to the
+      // copy unit land (bounded waits again) so that none is still writing this CTA's shared
+      // memory when it exits; the stores are drained below.
       atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
+      for (unsigned long long m = n + 1; m < issued; ++m)
+        mbar_wait(smem_u32(&bars[m % kStages]), (uint32_t)((m / kStages) & 1), kWaitLimit);
       break;
     }
     const unsigned char* s; unsigned char* d; uint32_t bytes;
@@ -170,6 +189,7 @@ __global__ void __launch_bounds__(kBulkThreads) transfer_bulk_kernel(const Trans
       locate(nx, &s, &d, &bytes);
       bulk_load(smem_u32(ring + (nx % kStages) * kStageBytes), s, bytes,
                 smem_u32(&bars[nx % kStages]));
+      issued = nx + 1;
     }
   }
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");

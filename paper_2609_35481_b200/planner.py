@@ -254,7 +254,7 @@ class Planner:
         if rc != B.OK:
             raise B.TopoEPError(rc)
         shape = {B.T_OMEGA: (self.R, self.E), B.T_Q: (self.R, self.P), B.T_RANK_LOAD: (self.R,),
-                 B.T_REFINE_ITERS: (self.M,)}[which]
+                 B.T_REFINE_ITERS: (self.M,), B.T_D: (self.M, self.E), B.T_U: (self.P,)}[which]
         off = (ptr - self.workspace.data_ptr())
         per = int(np.prod(shape)) * 4
         torch.cuda.synchronize(self.device)

@@ -46,6 +46,9 @@ def run_gpu(pl: Planner, ids: np.ndarray):
     res["q_instances"] = pl.debug_tensor(B.T_Q, Bn).numpy()
     res["rank_load"] = pl.debug_tensor(B.T_RANK_LOAD, Bn).numpy()
     res["refine_iters"] = pl.debug_tensor(B.T_REFINE_ITERS, Bn).numpy()
+    res["demand"] = pl.debug_tensor(B.T_D, Bn).numpy()
+    res["inst_load"] = pl.debug_tensor(B.T_U, Bn).numpy()
+    res["dims"] = (pl.M, pl.G)
     res["summaries"] = pl.summary(Bn)
     res["flags"] = pl.status()
     return res
@@ -67,6 +70,15 @@ def assert_same(gpu: dict, ref: orc.PlanResult, plans=None):
             bad = np.argwhere(g != r)
             raise AssertionError("%s differs at %d places, first %s: gpu %s oracle %s"
                                  % (name, len(bad), bad[0].tolist(), g[tuple(bad[0])], r[tuple(bad[0])]))
+    # the two remaining intermediates: domain demand D = the routing matrix summed over the ranks
+    # of a domain (the solver reads it when it runs inter-node placement), per-instance load U
+    M, G = gpu["dims"]
+    D, U = gpu["demand"], gpu["inst_load"]
+    if plans is not None:
+        D, U = D[plans], U[plans]
+    om = ref.omega.astype(np.int64)
+    assert np.array_equal(D, om.reshape(om.shape[0], M, G, -1).sum(axis=2)), "demand"
+    assert np.array_equal(U, ref.instance_counts), "instance load"
     gs = gpu["summaries"] if plans is None else gpu["summaries"][plans]
     for name in orc.SUMMARY_INT_FIELDS:
         assert np.array_equal(gs[name], ref.summaries[name]), name

@@ -57,6 +57,17 @@ def test_create_rejects_bad_arguments():
     assert rc(cost=B.CostParams(1, 1, -1, 8, 0, 0, 0)) == -4
     assert rc(cost=None) == -1
     assert rc(experts=1 << 14, main_rank_host=(np.arange(1 << 14) % 8).astype(np.int32)) == -9  # shared memory
+    # every count of a plan (rank loads, receive offsets) is bounded by R * T * k: it must fit int32
+    assert rc(nodes=64, gpus_per_node=32, experts=2048, top_k=1, max_tokens_per_rank=1 << 20) == -2
+    assert rc(nodes=64, gpus_per_node=32, experts=2048, top_k=1, max_tokens_per_rank=(1 << 20) - 1) != -2
+
+
+def test_static_histogram_size_rule_cannot_be_wrapped_around():
+    # 4 * batch * ranks * tiles * experts = 2^66 here: the product wraps to 0 in 64 bits, the
+    # stepwise check must still refuse it (the pointers are never dereferenced: nothing is enqueued)
+    rc = B.topoep_histogram_static(256, 32768, 32768, 2**31 - 1, 1, 8192, 256, None, 0)
+    assert rc == -11
+    assert B.topoep_histogram_static(256, 1, 1, 2**31 - 1, 2, 8, 256, None, 0) == -2   # T*k >= 2^31
 
 
 def test_calls_without_workspace_or_handle_fail_cleanly():

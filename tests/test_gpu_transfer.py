@@ -103,3 +103,43 @@ def test_transfer_argument_errors_and_bad_entries():
     assert np.array_equal(got[1, 1], main[m, l].cpu().numpy())
     got[1, 1] = 7
     assert (got == 7).all()
+
+
+def test_bounded_wait_that_runs_out_flags_drains_and_returns():
+    """The bulk engine waits on its ring's barriers with a poll limit.  The self-test knob makes
+    block 0 wait for a copy it never issued: that wait runs out, the block must set
+    TOPOEP_FLAG_INTERNAL, let its other copies land and return by itself (the context stays
+    usable).  Every other block completes, so exactly block 0's chunks keep their old bytes."""
+    w = wl.CONFIGS["mid"].replace(slots_per_rank=2)
+    pl = make_planner(w)
+    cfg = oracle_config(w)
+    R, N, e_loc, W = w.ranks, 2, pl.e_loc, 96 * 1024
+    rng = np.random.default_rng(8)
+    rmap = np.stack([rng.choice([e for e in range(w.experts) if w.main_rank()[e] != r], N,
+                                replace=False) for r in range(R)]).astype(np.int32)
+    main = wl.make_param_bytes((R, e_loc, W), 3)
+    slots0 = np.full((R, N, W), 0xEE, np.uint8)
+    d_map = torch.from_numpy(rmap).to(pl.device)
+    d_main = torch.from_numpy(main).to(pl.device)
+    d_slots = torch.from_numpy(slots0).to(pl.device)
+    pl.set_tuning(B.KNOB_TRANSFER_SELFTEST, 1)
+    pl.replica_pull(d_map, d_main, d_slots)
+    torch.cuda.synchronize()                      # returns: the kernel ended on its own
+    assert pl.status() == B.FLAG_INTERNAL
+    want = orc.replica_pull(cfg, rmap, main, slots0)
+    got = d_slots.cpu().numpy()
+    sms = torch.cuda.get_device_properties(pl.device).multi_processor_count
+    chunk, grid = 32 * 1024, 2 * sms
+    per_block = W // chunk
+    skipped = np.zeros((R * N, per_block), bool)  # block 0 owns items 0, grid, 2*grid, ...
+    skipped.ravel()[0::grid] = True
+    g = got.reshape(R * N, per_block, chunk)
+    wv = want.reshape(R * N, per_block, chunk)
+    assert np.array_equal(g[~skipped], wv[~skipped])
+    assert (g[skipped] == 0xEE).all()
+    # switched off again: a normal transfer, no flag
+    pl.set_tuning(B.KNOB_TRANSFER_SELFTEST, 0)
+    pl.replica_pull(d_map, d_main, d_slots)
+    torch.cuda.synchronize()
+    assert pl.status() == 0
+    assert np.array_equal(d_slots.cpu().numpy(), want)
