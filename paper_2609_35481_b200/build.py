@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtopoep.so")
-SOURCES = ["api.cu", "hist.cu", "hist_static.cu", "solve.cu", "route.cu", "reroute.cu", "dispatch.cu", "transfer.cu", "summary.cu"]
+SOURCES = ["api.cu", "hist.cu", "hist_static.cu", "solve.cu", "route.cu", "reroute.cu", "plan_tail.cu", "dispatch.cu", "transfer.cu", "summary.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -24,11 +24,15 @@ struct topoep_ctx {
   int transfer_ready, transfer_mode, sms;   // replica executor: configured?, copy engine, SM count
   int transfer_selftest;   // tests only: the bulk engine's bounded wait is made to run out once
   int max_tiles;
+  int chain;           // knob: 0 choose by size, 1 always five kernels, 2 three kernels when they fit
+  size_t tail_smem;    // shared memory the per-token kernel of the three-kernel chain may use
+  bool aux_valid;      // omega_m and demand in the workspace belong to the omega now there
+  bool routes_valid;   // route tables in the workspace belong to the tile counts now there
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
   // workspace
   bool have_ws;
   Workspace ws;
-  size_t off[24];
+  size_t off[32];
   size_t ws_bytes;
   cudaError_t last_cuda;
 };
@@ -40,9 +44,10 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 enum WsSlot {
   W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
-  W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC, W_SLOTS
+  W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC,
+  W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_SLOTS
 };
-static_assert(W_SLOTS <= 24, "offset table size");
+static_assert(W_SLOTS <= 32, "offset table size");
 
 void carve(topoep_ctx* h) {
   const Dims& d = h->d;
@@ -66,6 +71,9 @@ void carve(topoep_ctx* h) {
   sz[W_COUNTS] = 4 * B * R * R;
   sz[W_ROUTE] = 4 * B * R * E;
   sz[W_SPLIT_REC] = 4 * B * R * (size_t)split_rec_layout(d.E, d.P, h->max_tiles).ints;
+  sz[W_ACC_OMEGA0] = sz[W_ACC_OMEGA1] = 4 * B * R * E;
+  sz[W_ACC_DEMAND0] = sz[W_ACC_DEMAND1] = 4 * B * (size_t)d.M * E;
+  sz[W_EPOCH] = 16;
   size_t at = 0;
   for (int i = 0; i < W_SLOTS; ++i) { h->off[i] = at; at += align_up(sz[i]); }
   h->ws_bytes = at;
@@ -102,6 +110,8 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   p.pdl = 0;
   p.rank_first = h->rank_first;
   p.rank_count = h->rank_count;
+  p.acc = 0;
+  p.max_batch = h->max_batch;
   return p;
 }
 
@@ -206,6 +216,10 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->max_tokens = max_tokens_per_rank;
   h->max_batch = max_batch;
   h->tile_ids = 4096;
+  h->chain = 0;
+  h->tail_smem = 0;
+  h->aux_valid = false;
+  h->routes_valid = false;
   h->hist_mode = 0;
   h->pdl = 1;
   h->reserve_slots = 0;
@@ -261,6 +275,11 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.counts = at<int32_t>(dev_ptr, h->off[W_COUNTS]);
   w.route = at<int32_t>(dev_ptr, h->off[W_ROUTE]);
   w.split_rec = at<int32_t>(dev_ptr, h->off[W_SPLIT_REC]);
+  w.acc_omega[0] = at<int32_t>(dev_ptr, h->off[W_ACC_OMEGA0]);
+  w.acc_omega[1] = at<int32_t>(dev_ptr, h->off[W_ACC_OMEGA1]);
+  w.acc_demand[0] = at<int32_t>(dev_ptr, h->off[W_ACC_DEMAND0]);
+  w.acc_demand[1] = at<int32_t>(dev_ptr, h->off[W_ACC_DEMAND1]);
+  w.epoch = at<unsigned>(dev_ptr, h->off[W_EPOCH]);
 
   cudaError_t e;
   const size_t E = h->d.E;
@@ -287,6 +306,11 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
     if (e != cudaSuccess) goto fail;
   }
   if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
+  // accumulators of the three-kernel chain start clean (each call leaves them clean for the next)
+  if ((e = cudaMemset(w.acc_omega[0], 0, h->off[W_EPOCH] + 16 - h->off[W_ACC_OMEGA0])) != cudaSuccess) goto fail;
+  h->tail_smem = std::min<size_t>(tail_smem_bytes(h->d, kMaxTileIds, h->max_tiles), 227 * 1024);
+  if ((e = configure_tail(h->tail_smem)) != cudaSuccess) goto fail;
+  h->aux_valid = false;
   if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_reroute(reroute_smem_bytes(h->d, kMaxTileIds))) != cudaSuccess) goto fail;
@@ -301,13 +325,16 @@ fail:
 namespace {
 
 int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* out_omega,
-                 cudaStream_t stream) {
-  const HistParams hp = make_hist(h, ids, T, out_omega);
+                 cudaStream_t stream, bool three = false) {
+  HistParams hp = make_hist(h, ids, T, out_omega);
   h->hist_tile_ids = hp.tile_ids;
   h->hist_tokens = T;
   h->hist_batch = batch;
+  h->routes_valid = false;
+  h->aux_valid = !three && h->rank_count == h->d.R;
+  hp.acc = three ? 1 : 0;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && !three) {
     OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles, batch);
     if (h->rank_count != h->d.R) {
       // a window of ranks: plain tile sums, rank by rank; the demand and the transposed copy need
@@ -329,11 +356,16 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
 // Solver, then the per-source routing tables.  The tile prefixes are (re)built only when the tile
 // counts in the workspace belong to this batch size.
 int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* replica_map,
-                  int32_t* counts, int32_t* offsets, int32_t* inst_counts, cudaStream_t stream) {
+                  int32_t* counts, int32_t* offsets, int32_t* inst_counts, cudaStream_t stream,
+                  bool three = false) {
   SolveParams sp;
   sp.d = h->d;
   sp.ws = h->ws;
-  sp.pdl = chain_pdl(h, batch);
+  // three-kernel chain: programmatic launch without the trigger at kernel start (the solver
+  // releases the per-token kernel itself, once it has seen the histogram complete)
+  sp.pdl = three ? (h->pdl != 0 ? 1 : 0) : chain_pdl(h, batch);
+  sp.acc = three ? 1 : 0;
+  sp.batch = batch;
   sp.max_iters = h->max_iters;
   sp.min_delta = h->min_delta;
   // 2 D S_tok - ||W|| > 0  <=>  D > floor(||W|| / (2 S_tok)); S_tok = 0 admits no candidate
@@ -351,10 +383,15 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.out_offsets = offsets;
   sp.out_inst_counts = inst_counts;
   cudaError_t e = cudaSuccess;
-  // a routing matrix handed in from outside: derive the demand and the transposed copy from it
+  // a routing matrix handed in from outside: derive the demand and the transposed copy from it;
+  // likewise when the matrix in the workspace was left by the three-kernel chain, which does
+  // not keep those two layouts
   if (omega) e = launch_omega(make_omega(h, omega, nullptr, 0, batch), batch, stream);
+  else if (!three && !h->aux_valid)
+    e = launch_omega(make_omega(h, h->ws.omega, nullptr, 0, batch), batch, stream);
+  if (!three) h->aux_valid = true;
   if (e == cudaSuccess) e = launch_solve(sp, batch, stream);
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && !three) {
     RouteParams rp;
     rp.d = h->d;
     rp.ws = h->ws;
@@ -369,6 +406,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
       rp.tiles = std::max(1, (n_ids + h->hist_tile_ids - 1) / h->hist_tile_ids);
     }
     e = launch_route(rp, batch, stream);
+    h->routes_valid = rp.tiles > 0;
   }
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
@@ -394,6 +432,47 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   const cudaError_t e = launch_reroute(rp, batch, stream);
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
+}
+
+// Per-token kernel of the three-kernel chain (builds the routing table of its source itself).
+int enqueue_tail(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* token_replica,
+                 int32_t* offsets, cudaStream_t stream) {
+  TailParams tp;
+  tp.d = h->d;
+  tp.ws = h->ws;
+  tp.pdl = h->pdl != 0;
+  tp.stage1_lpt = h->stage1_lpt;
+  tp.stage1_slots = std::max(0, h->d.N - h->reserve_slots);
+  {
+    const long long st = h->cost.token_bytes, wb = h->cost.expert_bytes;
+    const long long thr = st > 0 ? wb / (2 * st) : (long long)INT_MAX;
+    tp.cand_thr = (int)std::min<long long>(thr, INT_MAX);
+  }
+  tp.ids = ids;
+  tp.out_token_replica = token_replica;
+  tp.out_offsets = offsets;
+  tp.n_ids = T * h->d.k;
+  tp.tile_ids = h->hist_tile_ids;
+  tp.tiles = std::max(1, (tp.n_ids + tp.tile_ids - 1) / tp.tile_ids);
+  tp.max_tiles = h->max_tiles;
+  tp.vec_ok = (tp.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0) &&
+              ((reinterpret_cast<uintptr_t>(token_replica) & 15u) == 0);
+  const cudaError_t e = launch_tail(tp, batch, stream);
+  if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  return TOPOEP_OK;
+}
+
+// Which chain plans this call: three kernels when the per-token kernel's tables fit its shared
+// memory and (unless forced) the whole call is resident on the GPU at once.
+bool use_three_kernels(const topoep_ctx* h, int T, int batch) {
+  if (h->chain == 1 || T <= 0 || h->rank_count != h->d.R) return false;
+  const long long n_ids = (long long)T * h->d.k;
+  const long long tiles = std::max(1ll, (n_ids + h->tile_ids - 1) / h->tile_ids);
+  const size_t smem = tail_smem_bytes(h->d, h->tile_ids, (int)tiles);
+  if (smem > h->tail_smem) return false;
+  if (h->chain == 2) return true;
+  const long long per_sm = std::max<long long>(1, std::min<long long>(8, (227 * 1024) / (long long)smem));
+  return tiles * h->d.R * batch <= per_sm * h->d.sms;
 }
 
 }  // namespace
@@ -430,7 +509,8 @@ int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_pe
   int rc = check_sizes(h, tokens_per_rank, batch);
   if (rc != TOPOEP_OK) return rc;
   if (batch == 0) return TOPOEP_OK;
-  if (tokens_per_rank != h->hist_tokens || batch != h->hist_batch) return TOPOEP_ERR_SIZE;
+  if (tokens_per_rank != h->hist_tokens || batch != h->hist_batch || !h->routes_valid)
+    return TOPOEP_ERR_SIZE;
   if (tokens_per_rank > 0 && (!dev_topk_ids || !dev_token_replica)) return TOPOEP_ERR_NULL;
   if (!aligned4(dev_topk_ids) || !aligned4(dev_token_replica)) return TOPOEP_ERR_ALIGN;
   return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
@@ -451,11 +531,15 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
       !aligned4(dev_instance_counts))
     return TOPOEP_ERR_ALIGN;
   if (h->rank_count != h->d.R) return TOPOEP_ERR_ARG;   // a whole plan needs every rank's ids
-  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream);
+  const bool three = use_three_kernels(h, tokens_per_rank, batch);
+  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, three);
   if (rc != TOPOEP_OK) return rc;
   rc = enqueue_solve(h, nullptr, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
-                     dev_instance_counts, stream);
+                     dev_instance_counts, stream, three);
   if (rc != TOPOEP_OK) return rc;
+  if (three)
+    return enqueue_tail(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica,
+                        dev_dispatch_offsets, stream);
   return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
 }
 
@@ -652,6 +736,10 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_TRANSFER_MODE:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->transfer_mode = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_CHAIN:
+      if (value < 0 || value > 2) return TOPOEP_ERR_ARG;
+      h->chain = value;
       return TOPOEP_OK;
     case TOPOEP_KNOB_TRANSFER_SELFTEST:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;

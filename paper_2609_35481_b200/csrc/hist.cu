@@ -37,13 +37,23 @@ __device__ __forceinline__ void count_one(int* cnt, int e, unsigned E, unsigned 
 }
 
 // IPT ids per thread (IPT/4 int4 loads in flight per thread); blockDim.x = tile_ids / IPT.
-template <int MODE, int IPT>
+// ACC: first kernel of the three-kernel chain for small calls.  The tile's counts are also added
+// into the routing-matrix and demand accumulators (see Workspace), which replaces the omega
+// kernel, and the kernel lets its dependents become resident from the start.
+template <int MODE, int IPT, bool ACC>
 __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const HistParams p) {
   extern __shared__ int cnt[];   // [E + 1]: the last bin collects ignored ids
   const int E = p.d.E;
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int nt = blockDim.x, tid = threadIdx.x;
   const unsigned lane = tid & 31;
+  unsigned epoch = 0, dirty0 = 0, dirty1 = 0;
+  if (ACC) {
+    pdl_trigger();
+    epoch = __ldcg(p.ws.epoch);        // in flight together with the ids
+    dirty0 = __ldcg(p.ws.epoch + 1);
+    dirty1 = __ldcg(p.ws.epoch + 2);
+  }
 
   // workspace rows are indexed by the global source rank, the caller's buffer by its window
   const size_t row = (size_t)b * p.d.R + p.rank_first + s;
@@ -77,6 +87,26 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   } else {
     unsigned short* out = reinterpret_cast<unsigned short*>(p.ws.tile_cnt) + at;
     for (int e = tid; e < E; e += nt) out[e] = (unsigned short)cnt[e];
+  }
+  if (ACC) {
+    // omega[s][e] and D[dom(s)][e] (paper, "System Model", Eq. Omega and Eq. D) by integer adds
+    const unsigned cur = epoch & 1u;
+    int32_t* om = p.ws.acc_omega[cur] + row * E;
+    int32_t* dem = p.ws.acc_demand[cur] + ((size_t)b * p.d.M + (p.rank_first + s) / p.d.G) * E;
+    for (int e = tid; e < E; e += nt) {
+      const int c = cnt[e];
+      if (c != 0) { atomicAdd(om + e, c); atomicAdd(dem + e, c); }
+    }
+    // clear the sums the previous call left in the other pair (nobody reads them any more: this
+    // kernel is launched in plain stream order, after everything of the previous call)
+    const size_t dirty = min((size_t)(cur ? dirty0 : dirty1), (size_t)p.max_batch);
+    const size_t n_om = dirty * p.d.R * E, n_dem = dirty * p.d.M * E;
+    const size_t ctas = (size_t)gridDim.x * gridDim.y * gridDim.z;
+    const size_t cta = ((size_t)b * gridDim.y + s) * gridDim.x + tile;
+    int32_t* zo = p.ws.acc_omega[cur ^ 1u];
+    int32_t* zd = p.ws.acc_demand[cur ^ 1u];
+    for (size_t i = cta * nt + tid; i < n_om; i += ctas * nt) zo[i] = 0;
+    for (size_t i = cta * nt + tid; i < n_dem; i += ctas * nt) zd[i] = 0;
   }
 }
 
@@ -209,12 +239,20 @@ cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t s
   const bool wide = p.tile_ids >= 2048;   // 32 ids per thread once the CTA still has 2+ warps
   const dim3 block(p.tile_ids / (wide ? 32 : 16));
   const bool pdl = p.pdl != 0;
-  if (mode == 1) {
-    return wide ? launch_kernel(hist_kernel<1, 32>, grid, block, smem, stream, pdl, p)
-                : launch_kernel(hist_kernel<1, 16>, grid, block, smem, stream, pdl, p);
+  if (p.acc) {
+    if (mode == 1) {
+      return wide ? launch_kernel(hist_kernel<1, 32, true>, grid, block, smem, stream, pdl, p)
+                  : launch_kernel(hist_kernel<1, 16, true>, grid, block, smem, stream, pdl, p);
+    }
+    return wide ? launch_kernel(hist_kernel<0, 32, true>, grid, block, smem, stream, pdl, p)
+                : launch_kernel(hist_kernel<0, 16, true>, grid, block, smem, stream, pdl, p);
   }
-  return wide ? launch_kernel(hist_kernel<0, 32>, grid, block, smem, stream, pdl, p)
-              : launch_kernel(hist_kernel<0, 16>, grid, block, smem, stream, pdl, p);
+  if (mode == 1) {
+    return wide ? launch_kernel(hist_kernel<1, 32, false>, grid, block, smem, stream, pdl, p)
+                : launch_kernel(hist_kernel<1, 16, false>, grid, block, smem, stream, pdl, p);
+  }
+  return wide ? launch_kernel(hist_kernel<0, 32, false>, grid, block, smem, stream, pdl, p)
+              : launch_kernel(hist_kernel<0, 16, false>, grid, block, smem, stream, pdl, p);
 }
 
 cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream) {

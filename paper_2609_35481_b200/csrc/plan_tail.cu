@@ -1,0 +1,538 @@
+// Per-token kernel of the three-kernel chain for small calls (paper, "Planning on the Critical
+// Path": one (layer, microbatch) plan at a time sits in front of every MoE layer, so its latency,
+// not its throughput, is what counts).
+//
+// Chain: accumulating histogram -> solver -> this kernel.  A CTA owns one tile of one source
+// rank s.  It builds the routing table of s ITSELF instead of waiting for a route kernel:
+//
+//   * inter-node placement of every domain is recomputed in the CTA from the demand D (the
+//     paper's "every rank recomputes, no broadcast" idea, applied per CTA);
+//   * if that placement used every replica slot, intra-node refinement cannot act (a move needs
+//     a target with a free slot, because an expert has at most one instance per domain after
+//     inter-node placement): then row s of q follows in closed form from row s of the routing
+//     matrix and the placement (paper, "Inter-node placement", routing construction), and the
+//     CTA never waits for the solver: histogram -> per-token assignment is the critical path,
+//     the solver runs beside it and only produces the placement, loads and dispatch layout;
+//   * otherwise the CTA waits for the solver and reads row s of q and the replica map.
+//
+// From the q row on, the steps are those of the route and reroute kernels: instances with a
+// share per expert, split lists with cumulative quotas, tile prefixes, resolved tiles, stream,
+// ranking tail.  The tile with index 0 of a row also writes the row's send offsets.
+//
+// Stream order is kept transitive: every CTA executes griddepcontrol.wait before it exits, so
+// the kernel completes only after the solver has.
+#include <limits.h>
+
+#include "topoep_internal.cuh"
+#include "reroute_tail.cuh"
+
+namespace topoep {
+
+namespace {
+
+constexpr int kTailRankCap = 128;   // candidates of a domain ranked all-pairs (as in the solver)
+constexpr int kTailMaxWarps = kMaxTileIds / kIdsPerThread / 32;
+
+struct TailLayout {
+  // scratch with two lives: inter-node placement first, the ranking tail afterwards
+  size_t D, cand;              // life 1
+  size_t cnt, base, work;      // life 2
+  // tables that live from their construction to the end
+  size_t route, hdr, seg, cum, inst, tbase, tpre;
+  size_t rm, qrow, mr, ml, mie, orow, hm_lo, hm_hi, win, nwin, nz, single, sidx, seg_e, crow, split_e,
+      warp_tot, tc;
+  size_t total;
+};
+
+__host__ __device__ inline TailLayout tail_layout(const Dims& d, int tile_ids, int tiles) {
+  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
+  const int nwarps = tile_ids / kIdsPerThread / 32 > 0 ? tile_ids / kIdsPerThread / 32 : 1;
+  const int rows = 4 * nwarps;
+  const size_t RN = (size_t)d.R * d.N, GN = (size_t)d.G * d.N;
+  TailLayout o;
+  size_t at = 0;
+  // life 1
+  o.D = at;
+  size_t l1 = sizeof(int) * pad4((size_t)d.M * d.E);
+  l1 = (l1 + 15) & ~(size_t)15;
+  o.cand = o.D + l1;
+  l1 += sizeof(unsigned long long) * (size_t)kTailRankCap * nwarps;
+  // life 2
+  o.cnt = at;
+  size_t l2 = sizeof(uint4) * (size_t)kSplitCap * rows;
+  o.base = at + l2;
+  l2 += sizeof(int) * (size_t)kSplitCap * rows;
+  o.work = at + l2;
+  l2 += sizeof(unsigned short) * (size_t)tile_ids;
+  at += ((l1 > l2 ? l1 : l2) + 15) & ~(size_t)15;
+  auto ints = [&](size_t n) { const size_t r = at; at += sizeof(int) * pad4(n); return r; };
+  o.route = ints(d.E + 1);
+  o.hdr = ints(4);
+  o.seg = ints(d.E + 1);
+  o.cum = ints(d.P);
+  o.inst = ints(d.P);
+  o.tbase = ints(kSplitCap);
+  o.tpre = ints(d.E);
+  o.rm = ints(RN + 1);
+  o.qrow = ints(d.P);
+  o.mr = ints(d.E);
+  o.ml = ints(d.E);
+  o.mie = ints((size_t)d.R * (d.e_loc > 0 ? d.e_loc : 1));
+  o.orow = ints(d.E);
+  o.hm_lo = ints(d.E);
+  o.hm_hi = ints(d.E);
+  o.win = ints((size_t)d.M * GN + 1);
+  o.nwin = ints(d.M);
+  o.nz = ints(d.E);
+  o.single = ints(d.E);
+  o.sidx = ints(d.E + 1);
+  o.seg_e = ints(d.E + 1);
+  o.crow = ints(d.R);
+  o.split_e = ints(d.E);
+  o.warp_tot = ints(2 * kTailMaxWarps);
+  o.tc = at;   // per-tile counts of the row, 16 bits each: [tiles][E]
+  at += (sizeof(unsigned short) * (size_t)tiles * d.E + 15) & ~(size_t)15;
+  o.total = at;
+  return o;
+}
+
+__device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gmem_src) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+
+// Exclusive scan of (flag[e], flag[e] * nz[e]) with flag = nz >= 2 over e < n by the whole CTA;
+// results in out_a / out_b (entry n = totals).  Each thread owns a contiguous chunk.
+__device__ __forceinline__ void tail_scan2(const int* nz, int n, int* out_a, int* out_b,
+                                           int* warp_tot, int tid, int nt) {
+  const int lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+  const int chunk = (n + nt - 1) / nt;
+  const int i0 = min(n, tid * chunk), i1 = min(n, i0 + chunk);
+  int a = 0, b = 0;
+#pragma unroll 1
+  for (int i = i0; i < i1; ++i) {
+    const int f = nz[i] >= 2;
+    a += f;
+    b += f ? nz[i] : 0;
+  }
+  int ta, tb;
+  int ea = warp_exclusive_scan(a, lane, &ta);
+  int eb = warp_exclusive_scan(b, lane, &tb);
+  if (lane == 0) { warp_tot[warp] = ta; warp_tot[nw + warp] = tb; }
+  __syncthreads();
+  int ba = 0, bb = 0;
+#pragma unroll 1
+  for (int w = 0; w < warp; ++w) { ba += warp_tot[w]; bb += warp_tot[nw + w]; }
+  ea += ba;
+  eb += bb;
+#pragma unroll 1
+  for (int i = i0; i < i1; ++i) {
+    const int f = nz[i] >= 2;
+    out_a[i] = ea;
+    out_b[i] = eb;
+    ea += f;
+    eb += f ? nz[i] : 0;
+  }
+  if (tid == nt - 1) { out_a[n] = ea; out_b[n] = eb; }
+  __syncthreads();
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) tail_kernel(const TailParams p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const Dims d = p.d;
+  const int M = d.M, G = d.G, R = d.R, E = d.E, N = d.N, P = d.P, s_phys = d.s_phys, e_loc = d.e_loc;
+  const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+  const int rows = 4 * nwarps;   // 128-id rows of the tile, in flat order
+  const unsigned full = 0xffffffffu;
+  const TailLayout lay = tail_layout(d, p.tile_ids, p.tiles);
+  int* Dsm = reinterpret_cast<int*>(smem + lay.D);
+  unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);
+  uint4* cnt4 = reinterpret_cast<uint4*>(smem + lay.cnt);
+  unsigned* cntw = reinterpret_cast<unsigned*>(smem + lay.cnt);
+  int* base = reinterpret_cast<int*>(smem + lay.base);
+  unsigned short* work = reinterpret_cast<unsigned short*>(smem + lay.work);
+  int* route = reinterpret_cast<int*>(smem + lay.route);
+  int* hdr = reinterpret_cast<int*>(smem + lay.hdr);
+  int* seg = reinterpret_cast<int*>(smem + lay.seg);         // [n_split+1] list start of split i
+  int* cum = reinterpret_cast<int*>(smem + lay.cum);
+  int* inst = reinterpret_cast<int*>(smem + lay.inst);
+  int* tbase = reinterpret_cast<int*>(smem + lay.tbase);
+  int* tpre = reinterpret_cast<int*>(smem + lay.tpre);       // [n_split] prefix over earlier tiles
+  int* rm = reinterpret_cast<int*>(smem + lay.rm);           // [R*N] expert in replica slot
+  int* qrow = reinterpret_cast<int*>(smem + lay.qrow);       // [P]   q(s, instance)
+  int* mr = reinterpret_cast<int*>(smem + lay.mr);           // [E]   main rank
+  int* ml = reinterpret_cast<int*>(smem + lay.ml);           // [E]   main instance id
+  int* mie = reinterpret_cast<int*>(smem + lay.mie);         // [R*e_loc] expert of a main instance
+  int* orow = reinterpret_cast<int*>(smem + lay.orow);       // [E]   omega[s][.]
+  unsigned* hm_lo = reinterpret_cast<unsigned*>(smem + lay.hm_lo);   // hosting domains 0..31
+  unsigned* hm_hi = reinterpret_cast<unsigned*>(smem + lay.hm_hi);   // hosting domains 32..63
+  int* win = reinterpret_cast<int*>(smem + lay.win);         // [M][G*N] stage-1 winners in order
+  int* nwin = reinterpret_cast<int*>(smem + lay.nwin);       // [M]
+  int* nz = reinterpret_cast<int*>(smem + lay.nz);           // [E]   instances with q > 0
+  int* single = reinterpret_cast<int*>(smem + lay.single);   // [E]
+  int* sidx = reinterpret_cast<int*>(smem + lay.sidx);       // [E+1] split index of e
+  int* seg_e = reinterpret_cast<int*>(smem + lay.seg_e);     // [E+1] list start of e (split only)
+  int* crow = reinterpret_cast<int*>(smem + lay.crow);       // [R]   counts[s][.]
+  int* split_e = reinterpret_cast<int*>(smem + lay.split_e); // [n_split] expert of split index i
+  int* warp_tot = reinterpret_cast<int*>(smem + lay.warp_tot);
+  unsigned short* tc = reinterpret_cast<unsigned short*>(smem + lay.tc);   // [tiles][E]
+
+  const size_t row = (size_t)b * R + s;
+  const int begin = tile * p.tile_ids;
+  const int count = min(p.tile_ids, p.n_ids - begin);
+  const int32_t* ids = p.ids + row * (size_t)p.n_ids + begin;
+  int32_t* out = p.out_token_replica + row * (size_t)p.n_ids + begin;
+  const int RN = R * N, GN = G * N, ds = s / G;
+
+  // ---- one round of loads.  This kernel starts once the solver's blocks have seen the histogram
+  // kernel complete (they trigger right after their own wait), so everything the histogram wrote
+  // may be read here without a wait; accumulators and tile counts are read past L1.
+  int4 x[kIdsPerThread / 4];
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+  {
+    const unsigned short* src =
+        reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + row * (size_t)p.max_tiles * E;
+    const int n16 = (tile + 1) * E;   // the row's tiles up to and including this one
+    if (E % 8 == 0) {
+#pragma unroll 4
+      for (int i = tid; i < n16 / 8; i += nt) cp_async16_cg(tc + 8 * i, src + 8 * i);
+    } else {
+#pragma unroll 4
+      for (int i = tid; i < n16; i += nt) tc[i] = __ldcg(src + i);
+    }
+  }
+  {
+    const int32_t* oA = p.ws.acc_omega[0] + row * E;
+    const int32_t* oB = p.ws.acc_omega[1] + row * E;
+#pragma unroll 2
+    for (int e = tid; e < E; e += nt) {
+      const int r = __ldg(p.ws.main_rank + e);
+      mr[e] = r;
+      ml[e] = r * s_phys + __ldg(p.ws.main_local + e);
+      const int md = r / G;   // the expert's main domain hosts it from the start
+      hm_lo[e] = md < 32 ? 1u << md : 0u;
+      hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
+      orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
+    }
+    const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
+    const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
+#pragma unroll 4
+    for (int i = tid; i < M * E; i += nt) Dsm[i] = __ldcg(dA + i) + __ldcg(dB + i);
+#pragma unroll 2
+    for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
+  }
+#pragma unroll 1
+  for (int i = tid; i < M * GN; i += nt) win[i] = -1;
+  if (tid < M) nwin[tid] = 0;
+  if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
+  cp_async_wait_all();
+  __syncthreads();
+
+  // ---- inter-node placement of every domain, one warp each (paper, "Inter-node placement":
+  // candidates with positive benefit in descending order, i-th winner to rank i mod G, slot i / G)
+  const int slots = G * p.stage1_slots;
+  if (M > 1 && p.stage1_slots > 0) {
+#pragma unroll 1
+    for (int dd = warp; dd < M; dd += nwarps) {
+      int* Dd = Dsm + dd * E;
+      unsigned long long* cand = cand_all + (size_t)warp * kTailRankCap;
+      int n_c = 0;
+#pragma unroll 1
+      for (int e0 = 0; e0 < E; e0 += 32) {
+        const int e = e0 + lane;
+        int v = 0;
+        if (e < E) {
+          // bit dd is still the main-domain bit here: only this warp sets it, further down
+          const unsigned hosted = dd < 32 ? hm_lo[e] >> dd : hm_hi[e] >> (dd - 32);
+          v = (hosted & 1u) ? 0 : Dd[e];
+          v = v > p.cand_thr ? v : 0;
+        }
+        const unsigned m = __ballot_sync(full, v > 0);
+        const int at = n_c + __popc(m & lanemask_lt());
+        if (v > 0 && at < kTailRankCap)
+          cand[at] = ((unsigned long long)(unsigned)v << 32) | (unsigned)~(unsigned)e;
+        n_c += __popc(m);
+      }
+      __syncwarp();
+      int n_win = 0;
+      if (n_c <= kTailRankCap) {
+        n_win = min(n_c, slots);
+#pragma unroll 1
+        for (int c0 = 0; c0 < n_c; c0 += 32) {
+          const int c = c0 + lane;
+          const unsigned long long mine = c < n_c ? cand[c] : 0ull;
+          int rank = 0;
+#pragma unroll 4
+          for (int o = 0; o < n_c; ++o) rank += cand[o] > mine ? 1 : 0;
+          if (c < n_c && rank < slots) {
+            const int e = (int)~(unsigned)mine;
+            if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
+            win[dd * GN + rank] = e;
+          }
+        }
+      } else {
+        // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
+#pragma unroll 1
+        for (int e = lane; e < E; e += 32) {
+          const unsigned hosted = dd < 32 ? hm_lo[e] >> dd : hm_hi[e] >> (dd - 32);
+          if ((hosted & 1u) || Dd[e] <= p.cand_thr) Dd[e] = 0;
+        }
+        __syncwarp();
+#pragma unroll 1
+        for (int i = 0; i < slots; ++i) {
+          int bestD = 0, bestE = INT_MAX;
+#pragma unroll 1
+          for (int e = lane; e < E; e += 32) {
+            const int v = Dd[e];
+            if (v > bestD) { bestD = v; bestE = e; }   // ascending e: first hit is smallest
+          }
+          const int maxD = __reduce_max_sync(full, bestD);
+          if (maxD <= 0) break;
+          n_win = i + 1;
+          const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
+          if (lane == 0) {
+            Dd[e] = 0;   // taken
+            if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
+            win[dd * GN + i] = e;
+          }
+          __syncwarp();
+        }
+      }
+      if (lane == 0) nwin[dd] = n_win;
+    }
+  }
+  __syncthreads();
+
+  // ---- can the refinement act at all?  Only a target with a free slot can take a move.
+  bool closed_form = p.stage1_lpt == 0;
+  if (N > 0) {
+    if (M == 1 || p.stage1_slots != N) closed_form = false;
+#pragma unroll 1
+    for (int dd = 0; dd < M; ++dd) closed_form = closed_form && nwin[dd] == GN;
+  }
+
+  // ---- row s of q and the replica map
+  if (closed_form) {
+#pragma unroll 1
+    for (int i = tid; i < RN; i += nt) {
+      const int r = i / N, j = i - r * N, dd = r / G, g = r - dd * G;
+      rm[i] = win[dd * GN + j * G + g];
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int pi = tid; pi < P; pi += nt) {
+      const int r = pi / s_phys, l = pi - r * s_phys;
+      const int e = l < e_loc ? mie[r * e_loc + l] : rm[r * N + l - e_loc];
+      int v = 0;
+      if (e >= 0) {
+        const int w = orow[e];
+        const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
+        const int n = __popcll(hm), dd = r / G;
+        if (ds == dd || n == 1) {   // own domain, or the only instance anywhere
+          v = w;
+        } else if (!((hm >> ds) & 1ull)) {
+          const int bs = w / n, rem = w - bs * n;
+          int sh = __popcll(hm & ((1ull << dd) - 1ull)) - (s + e) % n;
+          if (sh < 0) sh += n;
+          v = bs + (sh < rem ? 1 : 0);
+        }
+      }
+      qrow[pi] = v;
+    }
+  } else {
+    pdl_wait();   // the solver's refinement decides q: wait for it
+#pragma unroll 4
+    for (int i = tid; i < RN; i += nt) rm[i] = __ldcg(p.ws.replica_map + (size_t)b * RN + i);
+#pragma unroll 4
+    for (int i = tid; i < P; i += nt) qrow[i] = __ldcg(p.ws.q + row * P + i);
+  }
+  __syncthreads();
+
+  // ---- instances with a share, per expert; split experts and their lists
+#pragma unroll 1
+  for (int e = tid; e < E; e += nt) {
+    nz[e] = qrow[ml[e]] > 0 ? 1 : 0;
+    single[e] = ml[e];
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i < RN; i += nt) {
+    const int e = rm[i];
+    if (e >= 0 && qrow[(i / N) * s_phys + e_loc + i % N] > 0) atomicAdd(&nz[e], 1);
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i < RN; i += nt) {   // the one instance with a share, when it is a replica
+    const int e = rm[i];
+    const int pi = (i / N) * s_phys + e_loc + i % N;
+    if (e >= 0 && nz[e] == 1 && qrow[pi] > 0) single[e] = pi;
+  }
+  tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
+  const int n_split = sidx[E], n_list = seg_e[E];
+#pragma unroll 1
+  for (int e = tid; e < E; e += nt) {
+    const bool split = nz[e] >= 2;
+    route[e] = split ? -2 - sidx[e] : single[e];
+    if (split) { seg[sidx[e]] = seg_e[e]; split_e[sidx[e]] = e; }
+  }
+  if (tid == 0) {
+    hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
+    seg[n_split] = n_list;
+  }
+  if (tile == 0) {   // dispatch counts of row s, for the send offsets below
+#pragma unroll 1
+    for (int r = tid; r < R; r += nt) {
+      int sum = 0;
+#pragma unroll 1
+      for (int l = 0; l < s_phys; ++l) sum += qrow[r * s_phys + l];
+      crow[r] = sum;
+    }
+  }
+  __syncthreads();
+  // Split lists, one warp per split expert: the instances with a share in ascending rank order
+  // (the replica slots are in rank order; the main instance goes in front of the first slot on a
+  // higher rank) with cumulative quotas.
+#pragma unroll 1
+  for (int i = warp; i < n_split; i += nwarps) {
+    const int e = split_e[i];
+    const int lb = seg_e[e], qm = qrow[ml[e]], rmain = mr[e];
+    int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
+#pragma unroll 1
+    for (int i0 = 0; i0 < RN; i0 += 32) {
+      const int slot = i0 + lane;
+      int v = 0, r = 0, pi = 0;
+      if (slot < RN && rm[slot] == e) {
+        r = slot / N;
+        pi = r * s_phys + e_loc + (slot - r * N);
+        v = max(qrow[pi], 0);
+      }
+      const unsigned m = __ballot_sync(full, v > 0);
+      if (m == 0) continue;
+      int tot;
+      const int ex = warp_exclusive_scan(v, lane, &tot);
+      const bool below_main = v > 0 && r < rmain;
+      main_pos += __popc(__ballot_sync(full, below_main));
+      main_below += __reduce_add_sync(full, below_main ? v : 0);
+      if (v > 0) {
+        const bool after_main = qm > 0 && rmain < r;
+        const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
+        cum[lb + pos] = carry_cum + ex + v + (after_main ? qm : 0);
+        inst[lb + pos] = pi;
+      }
+      carry_pos += __popc(m);
+      carry_cum += tot;
+    }
+    if (lane == 0 && qm > 0) {
+      cum[lb + main_pos] = main_below + qm;
+      inst[lb + main_pos] = ml[e];
+    }
+  }
+  __syncthreads();
+  // Cross-tile base of every split expert's stable rank, and the resolved tiles: when the ids of
+  // the expert in this tile occupy ranks [ex, ex + tv) inside ONE instance's quota interval, they
+  // all go to that instance and the tile ranks nothing for it.
+#pragma unroll 1
+  for (int i = tid; i < n_split; i += nt) {
+    const int e = split_e[i];
+    int ex = 0;
+#pragma unroll 4
+    for (int t = 0; t < tile; ++t) ex += tc[(size_t)t * E + e];
+    const int tv = tc[(size_t)tile * E + e];
+    int lo = 0, res = -1;
+#pragma unroll 1
+    for (int k = seg[i]; k < seg[i + 1]; ++k) {
+      const int hi = cum[k];
+      if (ex >= lo && ex + tv <= hi) { res = inst[k]; break; }
+      lo = hi;
+    }
+    tpre[i] = ex;
+    if (i < kSplitCap) tbase[i] = ex;
+    if (res >= 0) route[e] = res;
+  }
+  if (tile == 0) {
+    // row s of the routing matrix, kept for inspection and the summaries
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) p.ws.omega[row * E + e] = orow[e];
+    // send offsets of source s: exclusive scan over the destination ranks, total appended
+    if (warp == 0) {
+      int32_t* send = p.out_offsets + (((size_t)b * 2 + 0) * R + s) * (R + 1);
+      const int ch = (R + 31) / 32;
+      const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
+      int sum = 0;
+#pragma unroll 1
+      for (int r = i0; r < i1; ++r) sum += crow[r];
+      int total;
+      int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
+      for (int r = i0; r < i1; ++r) { send[r] = pre; pre += crow[r]; }
+      if (lane == 0) send[R] = total;
+    }
+  }
+  // second life of the scratch region: the ranking counters (the placement is done with it)
+  static_assert(kSplitCap % 8 == 0, "counter words per thread");
+#pragma unroll
+  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+
+  // ---- stream: look up and store; split ids are remembered, pushed and patched below
+  const unsigned uE = (unsigned)E;
+  unsigned split_mask = 0;
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread / 4; ++j) {
+    const int vec = j * nt + tid;
+    const int t0 = route[min((unsigned)x[j].x, uE)];
+    const int t1 = route[min((unsigned)x[j].y, uE)];
+    const int t2 = route[min((unsigned)x[j].z, uE)];
+    const int t3 = route[min((unsigned)x[j].w, uE)];
+    split_mask |= (((unsigned)(t0 + 1) >> 31) | ((unsigned)(t1 + 1) >> 31) << 1 |
+                   ((unsigned)(t2 + 1) >> 31) << 2 | ((unsigned)(t3 + 1) >> 31) << 3) << (4 * j);
+    const int4 r = make_int4(max(t0, -1), max(t1, -1), max(t2, -1), max(t3, -1));
+    if (VEC) {
+      if (4 * vec < count) __stcs(reinterpret_cast<int4*>(out) + vec, r);
+    } else {
+      if (4 * vec + 0 < count) out[4 * vec + 0] = r.x;
+      if (4 * vec + 1 < count) out[4 * vec + 1] = r.y;
+      if (4 * vec + 2 < count) out[4 * vec + 2] = r.z;
+      if (4 * vec + 3 < count) out[4 * vec + 3] = r.w;
+    }
+  }
+  while (split_mask) {
+    const int k = __ffs(split_mask) - 1;
+    split_mask &= split_mask - 1;
+    work[atomicAdd(hdr + 2, 1)] = (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
+  }
+  __syncthreads();   // also orders the stores above before the patches below
+  const int n_work = hdr[2];
+  if (n_work > 0) {
+    const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
+    const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, nullptr, tpre, ids, out,
+                        rl, rows, n_split, n_list, n_work, p.ws.status, true};
+    rank_and_patch(c, tid, nt, warp, nwarps);
+  }
+  pdl_wait();   // completion stays transitive: this kernel ends only after the solver has
+}
+
+}  // namespace
+
+size_t tail_smem_bytes(const Dims& d, int tile_ids, int tiles) {
+  return tail_layout(d, tile_ids, tiles).total;
+}
+
+cudaError_t launch_tail(const TailParams& p, int batch, cudaStream_t stream) {
+  const dim3 grid(p.tiles, p.d.R, batch);
+  const dim3 block(p.tile_ids / kIdsPerThread);
+  const size_t smem = tail_smem_bytes(p.d, p.tile_ids, p.tiles);
+  return p.vec_ok ? launch_kernel(tail_kernel<true>, grid, block, smem, stream, p.pdl != 0, p)
+                  : launch_kernel(tail_kernel<false>, grid, block, smem, stream, p.pdl != 0, p);
+}
+
+cudaError_t configure_tail(size_t smem) {
+  cudaError_t e = cudaFuncSetAttribute(tail_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(tail_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+
+}  // namespace topoep

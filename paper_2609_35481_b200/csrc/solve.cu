@@ -174,11 +174,44 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   if (tid < G) used[tid] = 0;
 #pragma unroll 1
   for (int i = tid; i < R * G; i += nt) cnt[i] = 0;
-  pdl_wait();
-  copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
-  copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
-  cp_async_wait_all();
-  __syncthreads();
+  if (!p.acc) {
+    pdl_wait();
+    copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
+    copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
+    cp_async_wait_all();
+    __syncthreads();
+  } else {
+    // Three-kernel chain: the histogram kernel summed the routing matrix and the demand into the
+    // accumulators (one pair holds the sums, the other zeros: add them).  The static block must
+    // be in first, it names the experts of the columns.
+    cp_async_wait_all();
+    __syncthreads();
+    pdl_wait();
+    pdl_trigger();   // the histogram is complete: the per-token kernel may read the accumulators
+    const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
+    const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
+#pragma unroll 4
+    for (int i = tid; i < M * E; i += nt) D[i] = __ldcg(dA + i) + __ldcg(dB + i);
+    // main columns: a warp step covers 8 columns x 4 sources (blocked main maps: one sector each)
+    const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E;
+    const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E;
+    const int ncols = G * e_loc, nc8 = (ncols + 7) / 8, ns4 = (R + 3) / 4;
+#pragma unroll 2
+    for (int task = warp; task < nc8 * ns4; task += nwarps) {
+      const int cb = task % nc8, sb = task / nc8;
+      const int c = cb * 8 + (lane & 7), s = sb * 4 + (lane >> 3);
+      if (c < ncols && s < R) {
+        const int g = c / e_loc, l = c - g * e_loc;
+        const int e = col_expert[g * s_phys + l];
+        col_main[c * R + s] = e < 0 ? 0 : __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
+      }
+    }
+    __syncthreads();
+    if (p.ws.demand) {   // kept for inspection (debug tensor); row dm by this CTA
+#pragma unroll 1
+      for (int e = tid; e < E; e += nt) p.ws.demand[((size_t)b * M + dm) * E + e] = D[dm * E + e];
+    }
+  }
 
   // ---- inter-node placement, every domain, one warp each ------------------------------------
   // Candidates in descending (b, then ascending e) order == descending (D, ascending e) for a
@@ -284,6 +317,14 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
   for (int i = warp; i < G * N; i += nwarps) {
     const int e = col_expert[(i / N) * s_phys + e_loc + i % N];
     if (e < 0) continue;
+    if (p.acc) {
+      const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E + e;
+      const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E + e;
+#pragma unroll 1
+      for (int s = lane; s < R; s += 32)
+        col_rep[i * R + s] = __ldcg(oA + (size_t)s * E) + __ldcg(oB + (size_t)s * E);
+      continue;
+    }
     const int32_t* src = om_m + (size_t)(mrank[e] * e_loc + mlocal[e]) * R;
     copy_async(col_rep + i * R, src, R, lane, 32);
   }
@@ -514,6 +555,15 @@ __global__ void __launch_bounds__(kSolveThreads) solve_kernel(const SolveParams 
 #pragma unroll 1
     for (int s = i0; s < i1; ++s) { recv[s] = pre; pre += cnt[s * G + g]; }
     if (lane == 0) recv[R] = total;
+  }
+  // Three-kernel chain: one thread closes the call's bookkeeping -- this call's sums are in pair
+  // (epoch & 1), the other pair is clean; the next call takes the other pair.  Nothing of this
+  // call reads these words (the readers of the accumulators add both pairs).
+  if (p.acc && dm == 0 && b == 0 && tid == 0) {
+    const unsigned ep = __ldcg(p.ws.epoch);
+    p.ws.epoch[1 + (ep & 1u)] = (unsigned)p.batch;
+    p.ws.epoch[1 + ((ep & 1u) ^ 1u)] = 0u;
+    p.ws.epoch[0] = ep + 1u;
   }
 }
 
