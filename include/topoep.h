@@ -134,13 +134,15 @@ enum {
                                    1 plain 16-byte loads and stores               */
   TOPOEP_KNOB_CHAIN = 5,        /* kernels of a topoep_plan call.  1: five (tile
                                    histogram, omega, solver, route tables, reroute);
-                                   2: three whenever the tables fit shared memory
-                                   (accumulating histogram, solver, and a per-token
-                                   kernel that builds its source's route table
-                                   itself and, when inter-node placement used every
-                                   slot, does not wait for the solver); 0 (default):
-                                   three for calls small enough to be resident on
-                                   the GPU at once, where latency counts, else five */
+                                   2: two whenever the tables fit shared memory (a
+                                   histogram that also sums the routing matrix, then
+                                   one grid of solver blocks and per-token blocks;
+                                   a per-token block builds its source's route
+                                   table itself and, when inter-node placement used
+                                   every slot, does not wait for the solver); 0
+                                   (default): two for calls small enough to be
+                                   resident on the GPU at once, where latency
+                                   counts, else five                              */
   TOPOEP_KNOB_TRANSFER_SELFTEST = 4 /* tests only (the one knob that does change
                                    output): 1 makes one block of the bulk engine
                                    wait for a copy it never issued, so its bounded
@@ -206,7 +208,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes);
  * Within a (plan, source, expert) group, assignments are ranked by flat index
  * t*k+j and dealt to the expert's instances in ascending rank order, each
  * taking q(s,e,r) of them.  Equivalent to topoep_histogram, topoep_solve and
- * topoep_reroute in a row: enqueues five kernels on `stream` (three for small
+ * topoep_reroute in a row: enqueues five kernels on `stream` (two for small
  * calls, see TOPOEP_KNOB_CHAIN); capturable in a CUDA graph.  Two plans on one
  * handle must not overlap on the device.  The stage calls below continue from
  * stage calls: topoep_reroute after a topoep_plan returns TOPOEP_ERR_SIZE.

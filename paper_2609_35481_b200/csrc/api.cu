@@ -24,8 +24,8 @@ struct topoep_ctx {
   int transfer_ready, transfer_mode, sms;   // replica executor: configured?, copy engine, SM count
   int transfer_selftest;   // tests only: the bulk engine's bounded wait is made to run out once
   int max_tiles;
-  int chain;           // knob: 0 choose by size, 1 always five kernels, 2 three kernels when they fit
-  size_t tail_smem;    // shared memory the per-token kernel of the three-kernel chain may use
+  int chain;           // knob: 0 choose by size, 1 always five kernels, 2 two kernels when they fit
+  size_t plan2_smem;   // shared memory the second kernel of the two-kernel chain may use
   bool aux_valid;      // omega_m and demand in the workspace belong to the omega now there
   bool routes_valid;   // route tables in the workspace belong to the tile counts now there
   int hist_tile_ids, hist_tokens, hist_batch;   // shape of the tile prefixes now in the workspace
@@ -45,7 +45,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 enum WsSlot {
   W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
   W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC,
-  W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_SLOTS
+  W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_DONE, W_SLOTS
 };
 static_assert(W_SLOTS <= 32, "offset table size");
 
@@ -74,6 +74,7 @@ void carve(topoep_ctx* h) {
   sz[W_ACC_OMEGA0] = sz[W_ACC_OMEGA1] = 4 * B * R * E;
   sz[W_ACC_DEMAND0] = sz[W_ACC_DEMAND1] = 4 * B * (size_t)d.M * E;
   sz[W_EPOCH] = 16;
+  sz[W_DONE] = 4 * B * (size_t)d.M;
   size_t at = 0;
   for (int i = 0; i < W_SLOTS; ++i) { h->off[i] = at; at += align_up(sz[i]); }
   h->ws_bytes = at;
@@ -217,7 +218,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->max_batch = max_batch;
   h->tile_ids = 4096;
   h->chain = 0;
-  h->tail_smem = 0;
+  h->plan2_smem = 0;
   h->aux_valid = false;
   h->routes_valid = false;
   h->hist_mode = 0;
@@ -280,6 +281,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.acc_demand[0] = at<int32_t>(dev_ptr, h->off[W_ACC_DEMAND0]);
   w.acc_demand[1] = at<int32_t>(dev_ptr, h->off[W_ACC_DEMAND1]);
   w.epoch = at<unsigned>(dev_ptr, h->off[W_EPOCH]);
+  w.done_flags = at<unsigned>(dev_ptr, h->off[W_DONE]);
 
   cudaError_t e;
   const size_t E = h->d.E;
@@ -306,10 +308,11 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
     if (e != cudaSuccess) goto fail;
   }
   if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
-  // accumulators of the three-kernel chain start clean (each call leaves them clean for the next)
-  if ((e = cudaMemset(w.acc_omega[0], 0, h->off[W_EPOCH] + 16 - h->off[W_ACC_OMEGA0])) != cudaSuccess) goto fail;
-  h->tail_smem = std::min<size_t>(tail_smem_bytes(h->d, kMaxTileIds, h->max_tiles), 227 * 1024);
-  if ((e = configure_tail(h->tail_smem)) != cudaSuccess) goto fail;
+  // accumulators, serial number and flags of the two-kernel chain start at zero (each call
+  // leaves the accumulators clean for the next)
+  if ((e = cudaMemset(w.acc_omega[0], 0, h->ws_bytes - h->off[W_ACC_OMEGA0])) != cudaSuccess) goto fail;
+  h->plan2_smem = std::min<size_t>(plan2_smem_bytes(h->d, h->max_tiles), 227 * 1024);
+  if ((e = configure_plan2(h->plan2_smem)) != cudaSuccess) goto fail;
   h->aux_valid = false;
   if ((e = configure_solve(solve_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
@@ -325,16 +328,20 @@ fail:
 namespace {
 
 int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* out_omega,
-                 cudaStream_t stream, bool three = false) {
+                 cudaStream_t stream, bool two = false) {
   HistParams hp = make_hist(h, ids, T, out_omega);
+  if (two) {   // the second kernel of the two-kernel chain has one block shape: its tile size
+    hp.tile_ids = kPlan2TileIds;
+    hp.tiles = std::max(1, (hp.n_ids + hp.tile_ids - 1) / hp.tile_ids);
+  }
   h->hist_tile_ids = hp.tile_ids;
   h->hist_tokens = T;
   h->hist_batch = batch;
   h->routes_valid = false;
-  h->aux_valid = !three && h->rank_count == h->d.R;
-  hp.acc = three ? 1 : 0;
+  h->aux_valid = !two && h->rank_count == h->d.R;
+  hp.acc = two ? 1 : 0;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
-  if (e == cudaSuccess && !three) {
+  if (e == cudaSuccess && !two) {
     OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles, batch);
     if (h->rank_count != h->d.R) {
       // a window of ranks: plain tile sums, rank by rank; the demand and the transposed copy need
@@ -355,17 +362,13 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
 
 // Solver, then the per-source routing tables.  The tile prefixes are (re)built only when the tile
 // counts in the workspace belong to this batch size.
-int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* replica_map,
-                  int32_t* counts, int32_t* offsets, int32_t* inst_counts, cudaStream_t stream,
-                  bool three = false) {
+SolveParams make_solve(topoep_ctx* h, int batch, int32_t* replica_map, int32_t* counts,
+                       int32_t* offsets, int32_t* inst_counts) {
   SolveParams sp;
   sp.d = h->d;
   sp.ws = h->ws;
-  // three-kernel chain: programmatic launch without the trigger at kernel start (the solver
-  // releases the per-token kernel itself, once it has seen the histogram complete)
-  sp.pdl = three ? (h->pdl != 0 ? 1 : 0) : chain_pdl(h, batch);
-  sp.acc = three ? 1 : 0;
-  sp.batch = batch;
+  sp.pdl = chain_pdl(h, batch);
+  sp.acc = 0;
   sp.max_iters = h->max_iters;
   sp.min_delta = h->min_delta;
   // 2 D S_tok - ||W|| > 0  <=>  D > floor(||W|| / (2 S_tok)); S_tok = 0 admits no candidate
@@ -382,16 +385,22 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
   sp.out_counts = counts;
   sp.out_offsets = offsets;
   sp.out_inst_counts = inst_counts;
+  return sp;
+}
+
+int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* replica_map,
+                  int32_t* counts, int32_t* offsets, int32_t* inst_counts, cudaStream_t stream) {
+  const SolveParams sp = make_solve(h, batch, replica_map, counts, offsets, inst_counts);
   cudaError_t e = cudaSuccess;
   // a routing matrix handed in from outside: derive the demand and the transposed copy from it;
-  // likewise when the matrix in the workspace was left by the three-kernel chain, which does
-  // not keep those two layouts
+  // likewise when the matrix in the workspace was left by the two-kernel chain, which does not
+  // keep those two layouts
   if (omega) e = launch_omega(make_omega(h, omega, nullptr, 0, batch), batch, stream);
-  else if (!three && !h->aux_valid)
+  else if (!h->aux_valid)
     e = launch_omega(make_omega(h, h->ws.omega, nullptr, 0, batch), batch, stream);
-  if (!three) h->aux_valid = true;
+  h->aux_valid = true;
   if (e == cudaSuccess) e = launch_solve(sp, batch, stream);
-  if (e == cudaSuccess && !three) {
+  if (e == cudaSuccess) {
     RouteParams rp;
     rp.d = h->d;
     rp.ws = h->ws;
@@ -434,45 +443,46 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   return TOPOEP_OK;
 }
 
-// Per-token kernel of the three-kernel chain (builds the routing table of its source itself).
-int enqueue_tail(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* token_replica,
-                 int32_t* offsets, cudaStream_t stream) {
+// Second kernel of the two-kernel chain: solver blocks and per-token blocks in one grid.
+int enqueue_plan2(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* replica_map,
+                  int32_t* token_replica, int32_t* counts, int32_t* offsets, int32_t* inst_counts,
+                  cudaStream_t stream) {
+  SolveParams sp = make_solve(h, batch, replica_map, counts, offsets, inst_counts);
+  sp.pdl = h->pdl != 0;
+  sp.acc = 1;
   TailParams tp;
   tp.d = h->d;
   tp.ws = h->ws;
   tp.pdl = h->pdl != 0;
-  tp.stage1_lpt = h->stage1_lpt;
-  tp.stage1_slots = std::max(0, h->d.N - h->reserve_slots);
-  {
-    const long long st = h->cost.token_bytes, wb = h->cost.expert_bytes;
-    const long long thr = st > 0 ? wb / (2 * st) : (long long)INT_MAX;
-    tp.cand_thr = (int)std::min<long long>(thr, INT_MAX);
-  }
+  tp.stage1_lpt = sp.stage1_lpt;
+  tp.stage1_slots = sp.stage1_slots;
+  tp.cand_thr = sp.cand_thr;
   tp.ids = ids;
   tp.out_token_replica = token_replica;
   tp.out_offsets = offsets;
   tp.n_ids = T * h->d.k;
-  tp.tile_ids = h->hist_tile_ids;
+  tp.tile_ids = kPlan2TileIds;
   tp.tiles = std::max(1, (tp.n_ids + tp.tile_ids - 1) / tp.tile_ids);
   tp.max_tiles = h->max_tiles;
   tp.vec_ok = (tp.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0) &&
               ((reinterpret_cast<uintptr_t>(token_replica) & 15u) == 0);
-  const cudaError_t e = launch_tail(tp, batch, stream);
+  const cudaError_t e = launch_plan2(sp, tp, batch, stream);
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
 }
 
-// Which chain plans this call: three kernels when the per-token kernel's tables fit its shared
+// Which chain plans this call: two kernels when the per-token blocks' tables fit their shared
 // memory and (unless forced) the whole call is resident on the GPU at once.
-bool use_three_kernels(const topoep_ctx* h, int T, int batch) {
+bool use_two_kernels(const topoep_ctx* h, int T, int batch) {
   if (h->chain == 1 || T <= 0 || h->rank_count != h->d.R) return false;
   const long long n_ids = (long long)T * h->d.k;
-  const long long tiles = std::max(1ll, (n_ids + h->tile_ids - 1) / h->tile_ids);
-  const size_t smem = tail_smem_bytes(h->d, h->tile_ids, (int)tiles);
-  if (smem > h->tail_smem) return false;
+  const long long tiles = std::max(1ll, (n_ids + kPlan2TileIds - 1) / kPlan2TileIds);
+  if (tiles > h->max_tiles) return false;
+  const size_t smem = plan2_smem_bytes(h->d, (int)tiles);
+  if (smem > h->plan2_smem) return false;
   if (h->chain == 2) return true;
-  const long long per_sm = std::max<long long>(1, std::min<long long>(8, (227 * 1024) / (long long)smem));
-  return tiles * h->d.R * batch <= per_sm * h->d.sms;
+  const long long per_sm = std::max<long long>(1, std::min<long long>(2, (227 * 1024) / (long long)smem));
+  return (tiles * h->d.R + h->d.M) * batch <= per_sm * h->d.sms;
 }
 
 }  // namespace
@@ -531,15 +541,17 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
       !aligned4(dev_instance_counts))
     return TOPOEP_ERR_ALIGN;
   if (h->rank_count != h->d.R) return TOPOEP_ERR_ARG;   // a whole plan needs every rank's ids
-  const bool three = use_three_kernels(h, tokens_per_rank, batch);
-  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, three);
+  if (use_two_kernels(h, tokens_per_rank, batch)) {
+    rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, true);
+    if (rc != TOPOEP_OK) return rc;
+    return enqueue_plan2(h, dev_topk_ids, tokens_per_rank, batch, dev_replica_map, dev_token_replica,
+                         dev_dispatch_counts, dev_dispatch_offsets, dev_instance_counts, stream);
+  }
+  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream);
   if (rc != TOPOEP_OK) return rc;
   rc = enqueue_solve(h, nullptr, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
-                     dev_instance_counts, stream, three);
+                     dev_instance_counts, stream);
   if (rc != TOPOEP_OK) return rc;
-  if (three)
-    return enqueue_tail(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica,
-                        dev_dispatch_offsets, stream);
   return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
 }
 

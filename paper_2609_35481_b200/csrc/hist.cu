@@ -47,13 +47,8 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int nt = blockDim.x, tid = threadIdx.x;
   const unsigned lane = tid & 31;
-  unsigned epoch = 0, dirty0 = 0, dirty1 = 0;
-  if (ACC) {
-    pdl_trigger();
-    epoch = __ldcg(p.ws.epoch);        // in flight together with the ids
-    dirty0 = __ldcg(p.ws.epoch + 1);
-    dirty1 = __ldcg(p.ws.epoch + 2);
-  }
+  __shared__ unsigned call_state[3];   // ACC: serial of the previous call, plans in pair 0 / 1
+  if (ACC) pdl_trigger();
 
   // workspace rows are indexed by the global source rank, the caller's buffer by its window
   const size_t row = (size_t)b * p.d.R + p.rank_first + s;
@@ -63,6 +58,18 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   int4 x[IPT / 4];
 #pragma unroll
   for (int j = 0; j < IPT / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, p.vec_ok);
+  unsigned checked_in = 0;
+  if (ACC && tid == 0) {
+    // One thread per block reads the bookkeeping words (in flight together with the ids) and
+    // then checks in.  The block that checks in last knows that every block has read them, and
+    // moves them on at its end: this call's sums go to pair (serial & 1), the other pair gets
+    // cleared below, the serial number advances.  Whoever runs after this kernel sees the new
+    // values.
+    const unsigned ep = __ldcg(p.ws.epoch), d0 = __ldcg(p.ws.epoch + 1), d1 = __ldcg(p.ws.epoch + 2);
+    call_state[0] = ep; call_state[1] = d0; call_state[2] = d1;
+    __threadfence();
+    checked_in = atomicAdd(p.ws.epoch + 3, 1u);
+  }
 
   for (int e = tid; e <= E; e += nt) cnt[e] = 0;
   __syncthreads();
@@ -90,7 +97,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   }
   if (ACC) {
     // omega[s][e] and D[dom(s)][e] (paper, "System Model", Eq. Omega and Eq. D) by integer adds
-    const unsigned cur = epoch & 1u;
+    const unsigned cur = call_state[0] & 1u, dirty0 = call_state[1], dirty1 = call_state[2];
     int32_t* om = p.ws.acc_omega[cur] + row * E;
     int32_t* dem = p.ws.acc_demand[cur] + ((size_t)b * p.d.M + (p.rank_first + s) / p.d.G) * E;
     for (int e = tid; e < E; e += nt) {
@@ -107,6 +114,14 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
     int32_t* zd = p.ws.acc_demand[cur ^ 1u];
     for (size_t i = cta * nt + tid; i < n_om; i += ctas * nt) zo[i] = 0;
     for (size_t i = cta * nt + tid; i < n_dem; i += ctas * nt) zd[i] = 0;
+    if (tid == 0 && checked_in == (unsigned)ctas - 1u) {
+      const unsigned ep = call_state[0];
+      p.ws.epoch[3] = 0u;
+      p.ws.epoch[1 + (ep & 1u)] = gridDim.z;
+      p.ws.epoch[1 + ((ep & 1u) ^ 1u)] = 0u;
+      __threadfence();
+      p.ws.epoch[0] = ep + 1u;
+    }
   }
 }
 

@@ -1,30 +1,35 @@
-// Per-token kernel of the three-kernel chain for small calls (paper, "Planning on the Critical
-// Path": one (layer, microbatch) plan at a time sits in front of every MoE layer, so its latency,
-// not its throughput, is what counts).
+// Second kernel of the two-kernel chain for small calls (paper, "Planning on the Critical Path":
+// one (layer, microbatch) plan at a time sits in front of every MoE layer, so its latency, not
+// its throughput, is what counts).
 //
-// Chain: accumulating histogram -> solver -> this kernel.  A CTA owns one tile of one source
-// rank s.  It builds the routing table of s ITSELF instead of waiting for a route kernel:
+// Chain: accumulating histogram -> this kernel.  Its first M * B blocks are the solver blocks
+// (one per plan and domain, the body of the solver kernel); the others are per-token blocks, one
+// per tile of one source rank s.  A per-token block builds the routing table of s ITSELF instead
+// of waiting for a route kernel:
 //
-//   * inter-node placement of every domain is recomputed in the CTA from the demand D (the
-//     paper's "every rank recomputes, no broadcast" idea, applied per CTA);
+//   * inter-node placement of every domain is recomputed in the block from the demand D (the
+//     paper's "every rank recomputes, no broadcast" idea, applied per block);
 //   * if that placement used every replica slot, intra-node refinement cannot act (a move needs
 //     a target with a free slot, because an expert has at most one instance per domain after
 //     inter-node placement): then row s of q follows in closed form from row s of the routing
 //     matrix and the placement (paper, "Inter-node placement", routing construction), and the
-//     CTA never waits for the solver: histogram -> per-token assignment is the critical path,
-//     the solver runs beside it and only produces the placement, loads and dispatch layout;
-//   * otherwise the CTA waits for the solver and reads row s of q and the replica map.
+//     block never waits for the solver: histogram -> per-token assignment is the critical path,
+//     the solver blocks run beside it and only produce the placement, loads and dispatch layout;
+//   * otherwise the block waits until the solver blocks of its plan have published their results
+//     (a flag per solver block, polled with a limit) and reads row s of q and the replica map.
+//     The solver blocks have the lowest block indices, so they are scheduled first, and they wait
+//     for nobody: the wait cannot starve them.
 //
 // From the q row on, the steps are those of the route and reroute kernels: instances with a
 // share per expert, split lists with cumulative quotas, tile prefixes, resolved tiles, stream,
 // ranking tail.  The tile with index 0 of a row also writes the row's send offsets.
-//
-// Stream order is kept transitive: every CTA executes griddepcontrol.wait before it exits, so
-// the kernel completes only after the solver has.
 #include <limits.h>
+
+#include <algorithm>
 
 #include "topoep_internal.cuh"
 #include "reroute_tail.cuh"
+#include "solve_body.cuh"
 
 namespace topoep {
 
@@ -137,12 +142,13 @@ __device__ __forceinline__ void tail_scan2(const int* nz, int n, int* out_a, int
   __syncthreads();
 }
 
+constexpr unsigned kFlagWaitLimit = 1u << 20;   // polls (roughly a second) for a solver block
+
 template <bool VEC>
-__global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) tail_kernel(const TailParams p) {
-  extern __shared__ __align__(16) unsigned char smem[];
+__device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* smem, int tile, int s,
+                                          int b) {
   const Dims d = p.d;
   const int M = d.M, G = d.G, R = d.R, E = d.E, N = d.N, P = d.P, s_phys = d.s_phys, e_loc = d.e_loc;
-  const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
   const int rows = 4 * nwarps;   // 128-id rows of the tile, in flat order
   const unsigned full = 0xffffffffu;
@@ -186,12 +192,31 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) tail_kernel(const
   int32_t* out = p.out_token_replica + row * (size_t)p.n_ids + begin;
   const int RN = R * N, GN = G * N, ds = s / G;
 
-  // ---- one round of loads.  This kernel starts once the solver's blocks have seen the histogram
-  // kernel complete (they trigger right after their own wait), so everything the histogram wrote
-  // may be read here without a wait; accumulators and tile counts are read past L1.
+  // ---- before the histogram kernel is known to be complete: the ids (nobody's output) and the
+  // handle's static tables
   int4 x[kIdsPerThread / 4];
 #pragma unroll
   for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+#pragma unroll 2
+  for (int e = tid; e < E; e += nt) {
+    const int r = __ldg(p.ws.main_rank + e);
+    mr[e] = r;
+    ml[e] = r * s_phys + __ldg(p.ws.main_local + e);
+    const int md = r / G;   // the expert's main domain hosts it from the start
+    hm_lo[e] = md < 32 ? 1u << md : 0u;
+    hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
+  }
+#pragma unroll 2
+  for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
+#pragma unroll 1
+  for (int i = tid; i < M * GN; i += nt) win[i] = -1;
+  if (tid < M) nwin[tid] = 0;
+  if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
+  pdl_wait();
+  // ---- one round of loads of what the histogram kernel wrote (read past L1): the row's tile
+  // counts, row s of the routing matrix and the demand -- one accumulator pair holds the sums, the
+  // other zeros, so the two are added
+  const unsigned serial = __ldcg(p.ws.epoch);   // of this call: the histogram kernel advanced it
   {
     const unsigned short* src =
         reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + row * (size_t)p.max_tiles * E;
@@ -203,31 +228,15 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) tail_kernel(const
 #pragma unroll 4
       for (int i = tid; i < n16; i += nt) tc[i] = __ldcg(src + i);
     }
-  }
-  {
     const int32_t* oA = p.ws.acc_omega[0] + row * E;
     const int32_t* oB = p.ws.acc_omega[1] + row * E;
 #pragma unroll 2
-    for (int e = tid; e < E; e += nt) {
-      const int r = __ldg(p.ws.main_rank + e);
-      mr[e] = r;
-      ml[e] = r * s_phys + __ldg(p.ws.main_local + e);
-      const int md = r / G;   // the expert's main domain hosts it from the start
-      hm_lo[e] = md < 32 ? 1u << md : 0u;
-      hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
-      orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
-    }
+    for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
     const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
     const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
 #pragma unroll 4
     for (int i = tid; i < M * E; i += nt) Dsm[i] = __ldcg(dA + i) + __ldcg(dB + i);
-#pragma unroll 2
-    for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
   }
-#pragma unroll 1
-  for (int i = tid; i < M * GN; i += nt) win[i] = -1;
-  if (tid < M) nwin[tid] = 0;
-  if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
   cp_async_wait_all();
   __syncthreads();
 
@@ -343,7 +352,24 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) tail_kernel(const
       qrow[pi] = v;
     }
   } else {
-    pdl_wait();   // the solver's refinement decides q: wait for it
+    // the refinement decides q: wait for the solver blocks of this plan (bounded polls)
+    if (warp == 0) {
+      const unsigned* flags = p.ws.done_flags + (size_t)b * M;
+      bool done = false;
+#pragma unroll 1
+      for (unsigned it = 0; it < kFlagWaitLimit && !done; ++it) {
+        bool mine = true;
+#pragma unroll 1
+        for (int dd = lane; dd < M; dd += 32) {
+          unsigned v;
+          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flags + dd) : "memory");
+          mine = mine && v == serial;
+        }
+        done = __all_sync(full, mine);
+      }
+      if (!done && lane == 0) atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
+    }
+    __syncthreads();
 #pragma unroll 4
     for (int i = tid; i < RN; i += nt) rm[i] = __ldcg(p.ws.replica_map + (size_t)b * RN + i);
 #pragma unroll 4
@@ -512,27 +538,54 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) tail_kernel(const
                         rl, rows, n_split, n_list, n_work, p.ws.status, true};
     rank_and_patch(c, tid, nt, warp, nwarps);
   }
-  pdl_wait();   // completion stays transitive: this kernel ends only after the solver has
+}
+
+struct Plan2Params {
+  SolveParams sp;
+  TailParams tp;
+  int n_solve;   // solver blocks come first: block i < n_solve is (plan i / M, domain i % M)
+};
+
+template <bool LPT, bool VEC>
+__global__ void __launch_bounds__(kSolveThreads) plan2_kernel(const Plan2Params p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int i = blockIdx.x;
+  if (i < p.n_solve) {
+    solve_body<LPT>(p.sp, smem, i % p.sp.d.M, i / p.sp.d.M);
+  } else {
+    const int t = i - p.n_solve, tiles = p.tp.tiles, R = p.tp.d.R;
+    tail_body<VEC>(p.tp, smem, t % tiles, (t / tiles) % R, t / (tiles * R));
+  }
 }
 
 }  // namespace
 
-size_t tail_smem_bytes(const Dims& d, int tile_ids, int tiles) {
-  return tail_layout(d, tile_ids, tiles).total;
+size_t plan2_smem_bytes(const Dims& d, int tiles) {
+  return std::max(tail_layout(d, kPlan2TileIds, tiles).total, solve_smem_bytes(d));
 }
 
-cudaError_t launch_tail(const TailParams& p, int batch, cudaStream_t stream) {
-  const dim3 grid(p.tiles, p.d.R, batch);
-  const dim3 block(p.tile_ids / kIdsPerThread);
-  const size_t smem = tail_smem_bytes(p.d, p.tile_ids, p.tiles);
-  return p.vec_ok ? launch_kernel(tail_kernel<true>, grid, block, smem, stream, p.pdl != 0, p)
-                  : launch_kernel(tail_kernel<false>, grid, block, smem, stream, p.pdl != 0, p);
+cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream) {
+  Plan2Params p;
+  p.sp = sp;
+  p.tp = tp;
+  p.n_solve = sp.d.M * batch;
+  const dim3 grid(p.n_solve + tp.tiles * tp.d.R * batch), block(kSolveThreads);
+  const size_t smem = plan2_smem_bytes(tp.d, tp.tiles);
+  const bool pdl = tp.pdl != 0;
+  if (sp.stage1_lpt)
+    return tp.vec_ok ? launch_kernel(plan2_kernel<true, true>, grid, block, smem, stream, pdl, p)
+                     : launch_kernel(plan2_kernel<true, false>, grid, block, smem, stream, pdl, p);
+  return tp.vec_ok ? launch_kernel(plan2_kernel<false, true>, grid, block, smem, stream, pdl, p)
+                   : launch_kernel(plan2_kernel<false, false>, grid, block, smem, stream, pdl, p);
 }
 
-cudaError_t configure_tail(size_t smem) {
-  cudaError_t e = cudaFuncSetAttribute(tail_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(tail_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+cudaError_t configure_plan2(size_t smem) {
+  cudaError_t e;
+  const int n = (int)smem;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, n)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, n)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(plan2_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
 }
 
 }  // namespace topoep

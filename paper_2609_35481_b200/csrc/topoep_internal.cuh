@@ -54,7 +54,7 @@ struct Workspace {
   // per (plan, source) routing tables written by the route kernel
   int32_t* route;                   // [max_batch][R][E]  >= 0: the one instance; <= -2: -2 - split index
   int32_t* split_rec;               // [max_batch][R][split_rec_ints(d)]: see SplitRec
-  // Three-kernel chain for small calls: the histogram CTAs add their tile counts straight into
+  // Two-kernel chain for small calls: the histogram CTAs add their tile counts straight into
   // accumulators (integer adds commute, so the sums do not depend on arrival order).  There are
   // two pairs; a call adds into pair (epoch & 1) and clears what the call before it left in the
   // other pair, so that nothing has to be zeroed between the kernels of one call and a captured
@@ -62,7 +62,11 @@ struct Workspace {
   // the other only zeros: readers add the two and need not know which is which.
   int32_t* acc_omega[2];            // [max_batch][R][E] each
   int32_t* acc_demand[2];           // [max_batch][M][E] each
-  unsigned* epoch;                  // [0] calls so far; [1], [2] plans with sums in pair 0, 1
+  unsigned* epoch;                  // [0] calls so far (the serial number of the running call once
+                                    //   its histogram kernel is complete); [1], [2] plans with
+                                    //   sums in pair 0, 1; [3] histogram blocks that have started
+  unsigned* done_flags;             // [max_batch][M] serial of the last call whose solver block
+                                    //   (plan, domain) has finished
 };
 
 // Record of one (plan, source) written by the route kernel, read by the reroute kernel:
@@ -104,7 +108,7 @@ struct HistParams {
   int max_tiles;        // stride of tile_cnt / tile_pref
   int tile_ids;
   int vec_ok;           // rows are 16-byte aligned and n_ids % 4 == 0
-  int acc;              // three-kernel chain: also add the tile counts into the accumulators
+  int acc;              // two-kernel chain: also add the tile counts into the accumulators
   int max_batch;        // plans the accumulators are sized for
 };
 
@@ -132,12 +136,11 @@ struct SolveParams {
   int32_t* out_counts;        // [B][R][R]
   int32_t* out_offsets;       // [B][2][R][R+1]
   int32_t* out_inst_counts;   // [B][P] or NULL
-  int acc;            // three-kernel chain: demand and columns come from the accumulators
-  int batch;          // plans of this call (recorded with the epoch at the end)
+  int acc;            // two-kernel chain: demand and columns come from the accumulators
 };
 
-// Third kernel of the three-kernel chain: per tile, the source's routing table (built in the CTA)
-// and the per-token assignment.
+// Per-token blocks of the second kernel of the two-kernel chain: per tile, the source's routing
+// table (built in the block) and the per-token assignment.
 struct TailParams {
   Dims d;
   Workspace ws;
@@ -214,9 +217,11 @@ void solve_static_fill(const Dims& d, int dm, const int32_t* main_rank, const in
                        const int32_t* main_inst_expert, int cost_rank_intra, int32_t* out);
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
-size_t tail_smem_bytes(const Dims& d, int tile_ids, int tiles);
-cudaError_t configure_tail(size_t smem);
-cudaError_t launch_tail(const TailParams& p, int batch, cudaStream_t stream);
+// second kernel of the two-kernel chain: solver blocks first, per-token blocks after them
+constexpr int kPlan2TileIds = kSolveThreads * kIdsPerThread;   // one block shape for both roles
+size_t plan2_smem_bytes(const Dims& d, int tiles);
+cudaError_t configure_plan2(size_t smem);
+cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream);
 size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
 size_t pos_prefix_smem_bytes(const Dims& d);
 
