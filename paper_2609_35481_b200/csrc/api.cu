@@ -482,7 +482,7 @@ bool use_two_kernels(const topoep_ctx* h, int T, int batch) {
   if (smem > h->plan2_smem) return false;
   if (h->chain == 2) return true;
   const long long per_sm = std::max<long long>(1, std::min<long long>(2, (227 * 1024) / (long long)smem));
-  return (tiles * h->d.R + h->d.M) * batch <= per_sm * h->d.sms;
+  return plan2_blocks(h->d, (int)tiles, batch) <= per_sm * h->d.sms;
 }
 
 }  // namespace

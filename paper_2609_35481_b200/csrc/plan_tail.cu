@@ -2,27 +2,33 @@
 // one (layer, microbatch) plan at a time sits in front of every MoE layer, so its latency, not
 // its throughput, is what counts).
 //
-// Chain: accumulating histogram -> this kernel.  Its first M * B blocks are the solver blocks
-// (one per plan and domain, the body of the solver kernel); the others are per-token blocks, one
-// per tile of one source rank s.  A per-token block builds the routing table of s ITSELF instead
-// of waiting for a route kernel:
+// Chain: accumulating histogram -> this kernel.  One grid, three kinds of blocks:
 //
-//   * inter-node placement of every domain is recomputed in the block from the demand D (the
-//     paper's "every rank recomputes, no broadcast" idea, applied per block);
-//   * if that placement used every replica slot, intra-node refinement cannot act (a move needs
-//     a target with a free slot, because an expert has at most one instance per domain after
-//     inter-node placement): then row s of q follows in closed form from row s of the routing
-//     matrix and the placement (paper, "Inter-node placement", routing construction), and the
-//     block never waits for the solver: histogram -> per-token assignment is the critical path,
-//     the solver blocks run beside it and only produce the placement, loads and dispatch layout;
-//   * otherwise the block waits until the solver blocks of its plan have published their results
-//     (a flag per solver block, polled with a limit) and reads row s of q and the replica map.
-//     The solver blocks have the lowest block indices, so they are scheduled first, and they wait
-//     for nobody: the wait cannot starve them.
+//   solver blocks    (plan, domain)        the body of the solver kernel;
+//   rank blocks      (plan, rank)          the plan in closed form, one rank's share of it;
+//   per-token blocks (plan, source, tile)  the per-token assignment of one tile.
 //
-// From the q row on, the steps are those of the route and reroute kernels: instances with a
-// share per expert, split lists with cumulative quotas, tile prefixes, resolved tiles, stream,
-// ranking tail.  The tile with index 0 of a row also writes the row's send offsets.
+// Every block recomputes the inter-node placement of every domain from the demand D (the
+// paper's "every rank recomputes, no broadcast" idea, applied per block).  If that placement
+// used every replica slot, intra-node refinement cannot act: a move needs a target with a free
+// slot, because an expert has at most one instance per domain after inter-node placement.  Then
+// the plan is a closed form of the routing matrix and the placement (paper, "Inter-node
+// placement": routing construction, loads), and
+//   * a per-token block derives the routing table of its source from row s of the routing matrix
+//     and streams its tile without waiting for anybody: histogram -> per-token assignment is
+//     the critical path;
+//   * a rank block writes what belongs to rank r: row r of q and of the dispatch counts, its
+//     instance loads U, its rank load L, its receive offsets, its replica slots;
+//   * the solver blocks return at once.
+// Otherwise (some slot is free) the rank blocks return at once, the solver blocks run placement,
+// routing and refinement as in the solver kernel and publish a flag each, and a per-token block
+// waits for the flags of its plan (polled with a limit) and reads row s of q and the replica
+// map.  The solver blocks have the lowest block indices, so they are scheduled first, and they
+// wait for nobody: the wait cannot starve them.
+//
+// From the routing table on, a per-token block does what the reroute kernel does: tile prefixes,
+// resolved tiles, stream, ranking tail.  The tile with index 0 of a row also writes the row's
+// send offsets.
 #include <limits.h>
 
 #include <algorithm>
@@ -35,71 +41,9 @@ namespace topoep {
 
 namespace {
 
-constexpr int kTailRankCap = 128;   // candidates of a domain ranked all-pairs (as in the solver)
-constexpr int kTailMaxWarps = kMaxTileIds / kIdsPerThread / 32;
-
-struct TailLayout {
-  // scratch with two lives: inter-node placement first, the ranking tail afterwards
-  size_t D, cand;              // life 1
-  size_t cnt, base, work;      // life 2
-  // tables that live from their construction to the end
-  size_t route, hdr, seg, cum, inst, tbase, tpre;
-  size_t rm, qrow, mr, ml, mie, orow, hm_lo, hm_hi, win, nwin, nz, single, sidx, seg_e, crow, split_e,
-      warp_tot, tc;
-  size_t total;
-};
-
-__host__ __device__ inline TailLayout tail_layout(const Dims& d, int tile_ids, int tiles) {
-  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
-  const int nwarps = tile_ids / kIdsPerThread / 32 > 0 ? tile_ids / kIdsPerThread / 32 : 1;
-  const int rows = 4 * nwarps;
-  const size_t RN = (size_t)d.R * d.N, GN = (size_t)d.G * d.N;
-  TailLayout o;
-  size_t at = 0;
-  // life 1
-  o.D = at;
-  size_t l1 = sizeof(int) * pad4((size_t)d.M * d.E);
-  l1 = (l1 + 15) & ~(size_t)15;
-  o.cand = o.D + l1;
-  l1 += sizeof(unsigned long long) * (size_t)kTailRankCap * nwarps;
-  // life 2
-  o.cnt = at;
-  size_t l2 = sizeof(uint4) * (size_t)kSplitCap * rows;
-  o.base = at + l2;
-  l2 += sizeof(int) * (size_t)kSplitCap * rows;
-  o.work = at + l2;
-  l2 += sizeof(unsigned short) * (size_t)tile_ids;
-  at += ((l1 > l2 ? l1 : l2) + 15) & ~(size_t)15;
-  auto ints = [&](size_t n) { const size_t r = at; at += sizeof(int) * pad4(n); return r; };
-  o.route = ints(d.E + 1);
-  o.hdr = ints(4);
-  o.seg = ints(d.E + 1);
-  o.cum = ints(d.P);
-  o.inst = ints(d.P);
-  o.tbase = ints(kSplitCap);
-  o.tpre = ints(d.E);
-  o.rm = ints(RN + 1);
-  o.qrow = ints(d.P);
-  o.mr = ints(d.E);
-  o.ml = ints(d.E);
-  o.mie = ints((size_t)d.R * (d.e_loc > 0 ? d.e_loc : 1));
-  o.orow = ints(d.E);
-  o.hm_lo = ints(d.E);
-  o.hm_hi = ints(d.E);
-  o.win = ints((size_t)d.M * GN + 1);
-  o.nwin = ints(d.M);
-  o.nz = ints(d.E);
-  o.single = ints(d.E);
-  o.sidx = ints(d.E + 1);
-  o.seg_e = ints(d.E + 1);
-  o.crow = ints(d.R);
-  o.split_e = ints(d.E);
-  o.warp_tot = ints(2 * kTailMaxWarps);
-  o.tc = at;   // per-tile counts of the row, 16 bits each: [tiles][E]
-  at += (sizeof(unsigned short) * (size_t)tiles * d.E + 15) & ~(size_t)15;
-  o.total = at;
-  return o;
-}
+constexpr int kP2RankCap = 128;                  // candidates of a domain ranked all-pairs
+constexpr int kP2Warps = kSolveThreads / 32;     // every block of this kernel has this shape
+constexpr unsigned kFlagWaitLimit = 1u << 20;    // polls (roughly a second) for a solver block
 
 __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gmem_src) {
   const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -142,7 +86,216 @@ __device__ __forceinline__ void tail_scan2(const int* nz, int n, int* out_a, int
   __syncthreads();
 }
 
-constexpr unsigned kFlagWaitLimit = 1u << 20;   // polls (roughly a second) for a solver block
+// ---- inter-node placement of every domain, by the whole block --------------------------------
+// (Paper, "Inter-node placement": the candidates of a domain -- main instance elsewhere, positive
+// benefit, i.e. demand above the threshold -- in descending order (D, then ascending e); the i-th
+// winner goes to rank i mod G, slot i / G.)  In: D[M][E] in shared memory, the hosting masks with
+// the main-domain bits set.  Out: the masks with the winners' bits added, win[dd * GN + i] = the
+// i-th winner of domain dd, nwin[dd] = their number.  A domain is handled by a team of
+// nwarps / M warps when there are that many: each warp compacts the candidates of its share of
+// the experts, then ranks its own candidates against all of the domain's.
+struct Placement {
+  int* D;                       // [M][E]  (the slot-by-slot path zeroes entries)
+  unsigned long long* cand;     // [nwarps][kP2RankCap]
+  int* subcnt;                  // [nwarps]
+  unsigned* hm_lo;              // [E] hosting domains 0..31
+  unsigned* hm_hi;              // [E] hosting domains 32..63
+  int* win;                     // [M][GN], -1 where no winner
+  int* nwin;                    // [M]
+};
+
+__device__ __forceinline__ void place_all_domains(const Placement& pl, int M, int E, int GN, int slots,
+                                                  int thr, int tid, int nt) {
+  const unsigned full = 0xffffffffu;
+  const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+  if (M > 1 && slots > 0) {
+    const int wpd = M <= nwarps ? nwarps / M : 1;   // warps per domain
+    const int nteams = nwarps / wpd, team = warp / wpd, j = warp - team * wpd;
+#pragma unroll 1
+    for (int dd0 = 0; dd0 < M; dd0 += nteams) {   // one trip when a domain has several warps
+      const int dd = dd0 + team;
+      const bool on = dd < M && team < nteams;
+      unsigned long long* cand = pl.cand + (size_t)warp * kP2RankCap;
+      int* Dd = pl.D + (on ? dd : 0) * E;
+      int n_c = 0;
+      if (on) {
+#pragma unroll 1
+        for (int e0 = j * 32; e0 < E; e0 += wpd * 32) {
+          const int e = e0 + lane;
+          int v = 0;
+          if (e < E) {
+            // bit dd is still the main-domain bit here: it is only set below, after the barrier
+            const unsigned hosted = dd < 32 ? pl.hm_lo[e] >> dd : pl.hm_hi[e] >> (dd - 32);
+            v = (hosted & 1u) ? 0 : Dd[e];
+            v = v > thr ? v : 0;
+          }
+          const unsigned m = __ballot_sync(full, v > 0);
+          const int at = n_c + __popc(m & lanemask_lt());
+          if (v > 0 && at < kP2RankCap)
+            cand[at] = ((unsigned long long)(unsigned)v << 32) | (unsigned)~(unsigned)e;
+          n_c += __popc(m);
+        }
+        if (lane == 0) pl.subcnt[warp] = n_c;
+      }
+      if (wpd > 1) __syncthreads(); else __syncwarp();
+      if (on) {
+        int total = 0;
+#pragma unroll 1
+        for (int u = 0; u < wpd; ++u) total += pl.subcnt[team * wpd + u];
+        if (total <= kP2RankCap) {
+          // every candidate counts the keys of its domain above its own; rank < slots wins
+#pragma unroll 1
+          for (int c0 = 0; c0 < n_c; c0 += 32) {
+            const int c = c0 + lane;
+            const unsigned long long mine = c < n_c ? cand[c] : 0ull;
+            int rank = 0;
+#pragma unroll 1
+            for (int u = 0; u < wpd; ++u) {
+              const unsigned long long* sub = pl.cand + (size_t)(team * wpd + u) * kP2RankCap;
+              const int n_u = pl.subcnt[team * wpd + u];
+#pragma unroll 4
+              for (int o = 0; o < n_u; ++o) rank += sub[o] > mine ? 1 : 0;
+            }
+            if (c < n_c && rank < slots) {
+              const int e = (int)~(unsigned)mine;
+              if (dd < 32) atomicOr(&pl.hm_lo[e], 1u << dd); else atomicOr(&pl.hm_hi[e], 1u << (dd - 32));
+              pl.win[dd * GN + rank] = e;
+            }
+          }
+          if (j == 0 && lane == 0) pl.nwin[dd] = min(total, slots);
+        } else if (j == 0) {
+          // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
+#pragma unroll 1
+          for (int e = lane; e < E; e += 32) {
+            const unsigned hosted = dd < 32 ? pl.hm_lo[e] >> dd : pl.hm_hi[e] >> (dd - 32);
+            if ((hosted & 1u) || Dd[e] <= thr) Dd[e] = 0;
+          }
+          __syncwarp();
+          int n_win = 0;
+#pragma unroll 1
+          for (int i = 0; i < slots; ++i) {
+            int bestD = 0, bestE = INT_MAX;
+#pragma unroll 1
+            for (int e = lane; e < E; e += 32) {
+              const int v = Dd[e];
+              if (v > bestD) { bestD = v; bestE = e; }   // ascending e: first hit is smallest
+            }
+            const int maxD = __reduce_max_sync(full, bestD);
+            if (maxD <= 0) break;
+            n_win = i + 1;
+            const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
+            if (lane == 0) {
+              Dd[e] = 0;   // taken
+              if (dd < 32) atomicOr(&pl.hm_lo[e], 1u << dd); else atomicOr(&pl.hm_hi[e], 1u << (dd - 32));
+              pl.win[dd * GN + i] = e;
+            }
+            __syncwarp();
+          }
+          if (lane == 0) pl.nwin[dd] = n_win;
+        }
+      }
+      if (wpd == 1) __syncwarp();
+    }
+  }
+  __syncthreads();
+}
+
+// Can the refinement act at all?  Only a target with a free slot can take a move.
+__device__ __forceinline__ bool plan_is_closed_form(const int* nwin, int M, int GN, int N,
+                                                    int stage1_slots, int lpt) {
+  bool closed = lpt == 0;
+  if (N > 0) {
+    if (M == 1 || stage1_slots != N) closed = false;
+#pragma unroll 1
+    for (int dd = 0; dd < M; ++dd) closed = closed && nwin[dd] == GN;
+  }
+  return closed;
+}
+
+// q(s, instance of e in domain dd) after inter-node placement (paper, "Inter-node placement",
+// routing construction): a source keeps everything in its own domain when an instance is there;
+// otherwise omega(s,e) = w is split over all n instances (ascending hosting domain), remainder to
+// `rem` instances starting at (s+e) mod n.
+__device__ __forceinline__ int closed_q(int w, unsigned long long hm, int dd, int ds, int s, int e) {
+  const int n = __popcll(hm);
+  if (ds == dd || n == 1) return w;   // own domain, or the only instance anywhere
+  if ((hm >> ds) & 1ull) return 0;    // the source's own domain hosts e: nothing leaves it
+  const int bs = w / n, rem = w - bs * n;
+  int sh = __popcll(hm & ((1ull << dd) - 1ull)) - (s + e) % n;
+  if (sh < 0) sh += n;
+  return bs + (sh < rem ? 1 : 0);
+}
+
+// Instance of the replica of e that inter-node placement put into domain dd.
+__device__ __forceinline__ int replica_instance(const int* win, const int* nwin, int dd, int e, int G,
+                                                int GN, int s_phys, int e_loc) {
+  const int* w = win + dd * GN;
+  const int n = nwin[dd];
+  int i = 0;
+#pragma unroll 1
+  while (i < n - 1 && w[i] != e) ++i;
+  return (dd * G + i % G) * s_phys + e_loc + i / G;
+}
+
+// ---- per-token blocks -------------------------------------------------------------------------
+struct TailLayout {
+  // scratch with two lives: inter-node placement first, the ranking tail afterwards
+  size_t D, cand;              // life 1
+  size_t cnt, base, work;      // life 2
+  // tables that live from their construction to the end
+  size_t route, hdr, seg, cum, inst, tbase, tpre;
+  size_t rm, qrow, mr, ml, orow, hm_lo, hm_hi, win, nwin, subcnt, nz, single, sidx, seg_e, crow,
+      split_e, warp_tot, tc;
+  size_t total;
+};
+
+__host__ __device__ inline TailLayout tail_layout(const Dims& d, int tiles) {
+  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
+  const int rows = 4 * kP2Warps;
+  const size_t RN = (size_t)d.R * d.N, GN = (size_t)d.G * d.N;
+  TailLayout o;
+  size_t at = 0;
+  o.D = at;
+  size_t l1 = (sizeof(int) * pad4((size_t)d.M * d.E) + 15) & ~(size_t)15;
+  o.cand = o.D + l1;
+  l1 += sizeof(unsigned long long) * (size_t)kP2RankCap * kP2Warps;
+  o.cnt = at;
+  size_t l2 = sizeof(uint4) * (size_t)kSplitCap * rows;
+  o.base = at + l2;
+  l2 += sizeof(int) * (size_t)kSplitCap * rows;
+  o.work = at + l2;
+  l2 += sizeof(unsigned short) * (size_t)kPlan2TileIds;
+  at += ((l1 > l2 ? l1 : l2) + 15) & ~(size_t)15;
+  auto ints = [&](size_t n) { const size_t r = at; at += sizeof(int) * pad4(n); return r; };
+  o.route = ints(d.E + 1);
+  o.hdr = ints(4);
+  o.seg = ints(d.E + 1);
+  o.cum = ints(d.P);
+  o.inst = ints(d.P);
+  o.tbase = ints(kSplitCap);
+  o.tpre = ints(d.E);
+  o.rm = ints(RN + 1);
+  o.qrow = ints(d.P);
+  o.mr = ints(d.E);
+  o.ml = ints(d.E);
+  o.orow = ints(d.E);
+  o.hm_lo = ints(d.E);
+  o.hm_hi = ints(d.E);
+  o.win = ints((size_t)d.M * GN + 1);
+  o.nwin = ints(d.M);
+  o.subcnt = ints(kP2Warps);
+  o.nz = ints(d.E);
+  o.single = ints(d.E);
+  o.sidx = ints(d.E + 1);
+  o.seg_e = ints(d.E + 1);
+  o.crow = ints(d.R);
+  o.split_e = ints(d.E);
+  o.warp_tot = ints(2 * kP2Warps);
+  o.tc = at;   // per-tile counts of the row, 16 bits each: [tiles][E]
+  at += (sizeof(unsigned short) * (size_t)tiles * d.E + 15) & ~(size_t)15;
+  o.total = at;
+  return o;
+}
 
 template <bool VEC>
 __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* smem, int tile, int s,
@@ -152,7 +305,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
   const int rows = 4 * nwarps;   // 128-id rows of the tile, in flat order
   const unsigned full = 0xffffffffu;
-  const TailLayout lay = tail_layout(d, p.tile_ids, p.tiles);
+  const TailLayout lay = tail_layout(d, p.tiles);
   int* Dsm = reinterpret_cast<int*>(smem + lay.D);
   unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);
   uint4* cnt4 = reinterpret_cast<uint4*>(smem + lay.cnt);
@@ -170,12 +323,12 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   int* qrow = reinterpret_cast<int*>(smem + lay.qrow);       // [P]   q(s, instance)
   int* mr = reinterpret_cast<int*>(smem + lay.mr);           // [E]   main rank
   int* ml = reinterpret_cast<int*>(smem + lay.ml);           // [E]   main instance id
-  int* mie = reinterpret_cast<int*>(smem + lay.mie);         // [R*e_loc] expert of a main instance
   int* orow = reinterpret_cast<int*>(smem + lay.orow);       // [E]   omega[s][.]
-  unsigned* hm_lo = reinterpret_cast<unsigned*>(smem + lay.hm_lo);   // hosting domains 0..31
-  unsigned* hm_hi = reinterpret_cast<unsigned*>(smem + lay.hm_hi);   // hosting domains 32..63
+  unsigned* hm_lo = reinterpret_cast<unsigned*>(smem + lay.hm_lo);
+  unsigned* hm_hi = reinterpret_cast<unsigned*>(smem + lay.hm_hi);
   int* win = reinterpret_cast<int*>(smem + lay.win);         // [M][G*N] stage-1 winners in order
   int* nwin = reinterpret_cast<int*>(smem + lay.nwin);       // [M]
+  int* subcnt = reinterpret_cast<int*>(smem + lay.subcnt);
   int* nz = reinterpret_cast<int*>(smem + lay.nz);           // [E]   instances with q > 0
   int* single = reinterpret_cast<int*>(smem + lay.single);   // [E]
   int* sidx = reinterpret_cast<int*>(smem + lay.sidx);       // [E+1] split index of e
@@ -206,10 +359,10 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     hm_lo[e] = md < 32 ? 1u << md : 0u;
     hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
   }
-#pragma unroll 2
-  for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
 #pragma unroll 1
   for (int i = tid; i < M * GN; i += nt) win[i] = -1;
+#pragma unroll 1
+  for (int r = tid; r < R; r += nt) crow[r] = 0;
   if (tid < M) nwin[tid] = 0;
   if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
   pdl_wait();
@@ -240,119 +393,81 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   cp_async_wait_all();
   __syncthreads();
 
-  // ---- inter-node placement of every domain, one warp each (paper, "Inter-node placement":
-  // candidates with positive benefit in descending order, i-th winner to rank i mod G, slot i / G)
-  const int slots = G * p.stage1_slots;
-  if (M > 1 && p.stage1_slots > 0) {
+  const Placement pl = {Dsm, cand_all, subcnt, hm_lo, hm_hi, win, nwin};
+  place_all_domains(pl, M, E, GN, G * p.stage1_slots, p.cand_thr, tid, nt);
+  int n_split, n_list;
+
+  if (plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) {
+    // ---- the routing table of source s straight from omega[s][.] and the placement: a thread
+    // takes an expert.  An expert hosted in the source's domain, or hosted once, has one instance
+    // with a share; otherwise its share is split over its instances, ascending domain.
 #pragma unroll 1
-    for (int dd = warp; dd < M; dd += nwarps) {
-      int* Dd = Dsm + dd * E;
-      unsigned long long* cand = cand_all + (size_t)warp * kTailRankCap;
-      int n_c = 0;
-#pragma unroll 1
-      for (int e0 = 0; e0 < E; e0 += 32) {
-        const int e = e0 + lane;
-        int v = 0;
-        if (e < E) {
-          // bit dd is still the main-domain bit here: only this warp sets it, further down
-          const unsigned hosted = dd < 32 ? hm_lo[e] >> dd : hm_hi[e] >> (dd - 32);
-          v = (hosted & 1u) ? 0 : Dd[e];
-          v = v > p.cand_thr ? v : 0;
-        }
-        const unsigned m = __ballot_sync(full, v > 0);
-        const int at = n_c + __popc(m & lanemask_lt());
-        if (v > 0 && at < kTailRankCap)
-          cand[at] = ((unsigned long long)(unsigned)v << 32) | (unsigned)~(unsigned)e;
-        n_c += __popc(m);
-      }
-      __syncwarp();
-      int n_win = 0;
-      if (n_c <= kTailRankCap) {
-        n_win = min(n_c, slots);
-#pragma unroll 1
-        for (int c0 = 0; c0 < n_c; c0 += 32) {
-          const int c = c0 + lane;
-          const unsigned long long mine = c < n_c ? cand[c] : 0ull;
-          int rank = 0;
-#pragma unroll 4
-          for (int o = 0; o < n_c; ++o) rank += cand[o] > mine ? 1 : 0;
-          if (c < n_c && rank < slots) {
-            const int e = (int)~(unsigned)mine;
-            if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
-            win[dd * GN + rank] = e;
-          }
-        }
+    for (int e = tid; e < E; e += nt) {
+      const int w = orow[e], md = mr[e] / G;
+      const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
+      const int n = __popcll(hm);
+      int nzv, sg = ml[e];
+      if (((hm >> ds) & 1ull) || n == 1) {
+        nzv = w > 0 ? 1 : 0;
+        if (md != ds && ((hm >> ds) & 1ull)) sg = replica_instance(win, nwin, ds, e, G, GN, s_phys, e_loc);
       } else {
-        // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
+        const int bs = w / n, rem = w - bs * n;
+        nzv = bs > 0 ? n : rem;
+        if (nzv == 1) {   // one unit: it goes to the instance at index (s+e) mod n
+          unsigned long long m = hm;
 #pragma unroll 1
-        for (int e = lane; e < E; e += 32) {
-          const unsigned hosted = dd < 32 ? hm_lo[e] >> dd : hm_hi[e] >> (dd - 32);
-          if ((hosted & 1u) || Dd[e] <= p.cand_thr) Dd[e] = 0;
-        }
-        __syncwarp();
-#pragma unroll 1
-        for (int i = 0; i < slots; ++i) {
-          int bestD = 0, bestE = INT_MAX;
-#pragma unroll 1
-          for (int e = lane; e < E; e += 32) {
-            const int v = Dd[e];
-            if (v > bestD) { bestD = v; bestE = e; }   // ascending e: first hit is smallest
-          }
-          const int maxD = __reduce_max_sync(full, bestD);
-          if (maxD <= 0) break;
-          n_win = i + 1;
-          const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
-          if (lane == 0) {
-            Dd[e] = 0;   // taken
-            if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
-            win[dd * GN + i] = e;
-          }
-          __syncwarp();
+          for (int t = (s + e) % n; t > 0; --t) m &= m - 1;
+          const int dd = __ffsll((long long)m) - 1;
+          if (dd != md) sg = replica_instance(win, nwin, dd, e, G, GN, s_phys, e_loc);
         }
       }
-      if (lane == 0) nwin[dd] = n_win;
-    }
-  }
-  __syncthreads();
-
-  // ---- can the refinement act at all?  Only a target with a free slot can take a move.
-  bool closed_form = p.stage1_lpt == 0;
-  if (N > 0) {
-    if (M == 1 || p.stage1_slots != N) closed_form = false;
-#pragma unroll 1
-    for (int dd = 0; dd < M; ++dd) closed_form = closed_form && nwin[dd] == GN;
-  }
-
-  // ---- row s of q and the replica map
-  if (closed_form) {
-#pragma unroll 1
-    for (int i = tid; i < RN; i += nt) {
-      const int r = i / N, j = i - r * N, dd = r / G, g = r - dd * G;
-      rm[i] = win[dd * GN + j * G + g];
+      nz[e] = nzv;
+      single[e] = sg;
     }
     __syncthreads();
+    tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
+    n_split = sidx[E];
+    n_list = seg_e[E];
 #pragma unroll 1
-    for (int pi = tid; pi < P; pi += nt) {
-      const int r = pi / s_phys, l = pi - r * s_phys;
-      const int e = l < e_loc ? mie[r * e_loc + l] : rm[r * N + l - e_loc];
-      int v = 0;
-      if (e >= 0) {
-        const int w = orow[e];
-        const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
-        const int n = __popcll(hm), dd = r / G;
-        if (ds == dd || n == 1) {   // own domain, or the only instance anywhere
-          v = w;
-        } else if (!((hm >> ds) & 1ull)) {
-          const int bs = w / n, rem = w - bs * n;
-          int sh = __popcll(hm & ((1ull << dd) - 1ull)) - (s + e) % n;
+    for (int e = tid; e < E; e += nt) {
+      const bool split = nz[e] >= 2;
+      route[e] = split ? -2 - sidx[e] : single[e];
+      const int w = orow[e];
+      if (split) {
+        const int i = sidx[e], md = mr[e] / G;
+        seg[i] = seg_e[e];
+        split_e[i] = e;
+        unsigned long long m = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
+        const int n = __popcll(m), bs = w / n, rem = w - bs * n, start = (s + e) % n;
+        int k = seg_e[e], acc = 0;
+#pragma unroll 1
+        for (int idx = 0; idx < n; ++idx) {
+          const int dd = __ffsll((long long)m) - 1;
+          m &= m - 1;
+          int sh = idx - start;
           if (sh < 0) sh += n;
-          v = bs + (sh < rem ? 1 : 0);
+          const int v = bs + (sh < rem ? 1 : 0);
+          if (v > 0) {
+            const int pi = dd == md ? ml[e] : replica_instance(win, nwin, dd, e, G, GN, s_phys, e_loc);
+            acc += v;
+            cum[k] = acc;
+            inst[k] = pi;
+            ++k;
+            if (tile == 0) atomicAdd(&crow[pi / s_phys], v);
+          }
         }
+      } else if (tile == 0 && w > 0) {
+        atomicAdd(&crow[single[e] / s_phys], w);
       }
-      qrow[pi] = v;
     }
+    if (tid == 0) {
+      hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
+      seg[n_split] = n_list;
+    }
+    __syncthreads();
   } else {
-    // the refinement decides q: wait for the solver blocks of this plan (bounded polls)
+    // ---- the refinement decides q: wait for the solver blocks of this plan (bounded polls),
+    // then row s of q and the replica map come from memory
     if (warp == 0) {
       const unsigned* flags = p.ws.done_flags + (size_t)b * M;
       bool done = false;
@@ -374,89 +489,90 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     for (int i = tid; i < RN; i += nt) rm[i] = __ldcg(p.ws.replica_map + (size_t)b * RN + i);
 #pragma unroll 4
     for (int i = tid; i < P; i += nt) qrow[i] = __ldcg(p.ws.q + row * P + i);
+    __syncthreads();
+    // instances with a share, per expert; split experts and their lists
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) {
+      nz[e] = qrow[ml[e]] > 0 ? 1 : 0;
+      single[e] = ml[e];
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int i = tid; i < RN; i += nt) {
+      const int e = rm[i];
+      if (e >= 0 && qrow[(i / N) * s_phys + e_loc + i % N] > 0) atomicAdd(&nz[e], 1);
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int i = tid; i < RN; i += nt) {   // the one instance with a share, when it is a replica
+      const int e = rm[i];
+      const int pi = (i / N) * s_phys + e_loc + i % N;
+      if (e >= 0 && nz[e] == 1 && qrow[pi] > 0) single[e] = pi;
+    }
+    tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
+    n_split = sidx[E];
+    n_list = seg_e[E];
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) {
+      const bool split = nz[e] >= 2;
+      route[e] = split ? -2 - sidx[e] : single[e];
+      if (split) { seg[sidx[e]] = seg_e[e]; split_e[sidx[e]] = e; }
+    }
+    if (tid == 0) {
+      hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
+      seg[n_split] = n_list;
+    }
+    if (tile == 0) {   // dispatch counts of row s, for the send offsets below
+#pragma unroll 1
+      for (int r = tid; r < R; r += nt) {
+        int sum = 0;
+#pragma unroll 1
+        for (int l = 0; l < s_phys; ++l) sum += qrow[r * s_phys + l];
+        crow[r] = sum;
+      }
+    }
+    __syncthreads();
+    // Split lists, one warp per split expert: the instances with a share in ascending rank order
+    // (the replica slots are in rank order; the main instance goes in front of the first slot on
+    // a higher rank) with cumulative quotas.
+#pragma unroll 1
+    for (int i = warp; i < n_split; i += nwarps) {
+      const int e = split_e[i];
+      const int lb = seg_e[e], qm = qrow[ml[e]], rmain = mr[e];
+      int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
+#pragma unroll 1
+      for (int i0 = 0; i0 < RN; i0 += 32) {
+        const int slot = i0 + lane;
+        int v = 0, r = 0, pi = 0;
+        if (slot < RN && rm[slot] == e) {
+          r = slot / N;
+          pi = r * s_phys + e_loc + (slot - r * N);
+          v = max(qrow[pi], 0);
+        }
+        const unsigned m = __ballot_sync(full, v > 0);
+        if (m == 0) continue;
+        int tot;
+        const int ex = warp_exclusive_scan(v, lane, &tot);
+        const bool below_main = v > 0 && r < rmain;
+        main_pos += __popc(__ballot_sync(full, below_main));
+        main_below += __reduce_add_sync(full, below_main ? v : 0);
+        if (v > 0) {
+          const bool after_main = qm > 0 && rmain < r;
+          const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
+          cum[lb + pos] = carry_cum + ex + v + (after_main ? qm : 0);
+          inst[lb + pos] = pi;
+        }
+        carry_pos += __popc(m);
+        carry_cum += tot;
+      }
+      if (lane == 0 && qm > 0) {
+        cum[lb + main_pos] = main_below + qm;
+        inst[lb + main_pos] = ml[e];
+      }
+    }
+    __syncthreads();
   }
-  __syncthreads();
 
-  // ---- instances with a share, per expert; split experts and their lists
-#pragma unroll 1
-  for (int e = tid; e < E; e += nt) {
-    nz[e] = qrow[ml[e]] > 0 ? 1 : 0;
-    single[e] = ml[e];
-  }
-  __syncthreads();
-#pragma unroll 1
-  for (int i = tid; i < RN; i += nt) {
-    const int e = rm[i];
-    if (e >= 0 && qrow[(i / N) * s_phys + e_loc + i % N] > 0) atomicAdd(&nz[e], 1);
-  }
-  __syncthreads();
-#pragma unroll 1
-  for (int i = tid; i < RN; i += nt) {   // the one instance with a share, when it is a replica
-    const int e = rm[i];
-    const int pi = (i / N) * s_phys + e_loc + i % N;
-    if (e >= 0 && nz[e] == 1 && qrow[pi] > 0) single[e] = pi;
-  }
-  tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
-  const int n_split = sidx[E], n_list = seg_e[E];
-#pragma unroll 1
-  for (int e = tid; e < E; e += nt) {
-    const bool split = nz[e] >= 2;
-    route[e] = split ? -2 - sidx[e] : single[e];
-    if (split) { seg[sidx[e]] = seg_e[e]; split_e[sidx[e]] = e; }
-  }
-  if (tid == 0) {
-    hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
-    seg[n_split] = n_list;
-  }
-  if (tile == 0) {   // dispatch counts of row s, for the send offsets below
-#pragma unroll 1
-    for (int r = tid; r < R; r += nt) {
-      int sum = 0;
-#pragma unroll 1
-      for (int l = 0; l < s_phys; ++l) sum += qrow[r * s_phys + l];
-      crow[r] = sum;
-    }
-  }
-  __syncthreads();
-  // Split lists, one warp per split expert: the instances with a share in ascending rank order
-  // (the replica slots are in rank order; the main instance goes in front of the first slot on a
-  // higher rank) with cumulative quotas.
-#pragma unroll 1
-  for (int i = warp; i < n_split; i += nwarps) {
-    const int e = split_e[i];
-    const int lb = seg_e[e], qm = qrow[ml[e]], rmain = mr[e];
-    int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
-#pragma unroll 1
-    for (int i0 = 0; i0 < RN; i0 += 32) {
-      const int slot = i0 + lane;
-      int v = 0, r = 0, pi = 0;
-      if (slot < RN && rm[slot] == e) {
-        r = slot / N;
-        pi = r * s_phys + e_loc + (slot - r * N);
-        v = max(qrow[pi], 0);
-      }
-      const unsigned m = __ballot_sync(full, v > 0);
-      if (m == 0) continue;
-      int tot;
-      const int ex = warp_exclusive_scan(v, lane, &tot);
-      const bool below_main = v > 0 && r < rmain;
-      main_pos += __popc(__ballot_sync(full, below_main));
-      main_below += __reduce_add_sync(full, below_main ? v : 0);
-      if (v > 0) {
-        const bool after_main = qm > 0 && rmain < r;
-        const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
-        cum[lb + pos] = carry_cum + ex + v + (after_main ? qm : 0);
-        inst[lb + pos] = pi;
-      }
-      carry_pos += __popc(m);
-      carry_cum += tot;
-    }
-    if (lane == 0 && qm > 0) {
-      cum[lb + main_pos] = main_below + qm;
-      inst[lb + main_pos] = ml[e];
-    }
-  }
-  __syncthreads();
   // Cross-tile base of every split expert's stable rank, and the resolved tiles: when the ids of
   // the expert in this tile occupy ranks [ex, ex + tv) inside ONE instance's quota interval, they
   // all go to that instance and the tile ranks nothing for it.
@@ -540,28 +656,205 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   }
 }
 
+// ---- rank blocks: the plan in closed form, rank r's share ---------------------------------------
+struct RankLayout {
+  size_t D, cand, subcnt, hm_lo, hm_hi, win, nwin, mr, mie, orow, colv, qrow, crow, ccol, U, total;
+};
+
+__host__ __device__ inline RankLayout rank_layout(const Dims& d) {
+  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
+  RankLayout o;
+  size_t at = 0;
+  o.cand = at;
+  at += sizeof(unsigned long long) * (size_t)kP2RankCap * kP2Warps;
+  auto ints = [&](size_t n) { const size_t r = at; at += sizeof(int) * pad4(n); return r; };
+  o.D = ints((size_t)d.M * d.E);
+  o.subcnt = ints(kP2Warps);
+  o.hm_lo = ints(d.E);
+  o.hm_hi = ints(d.E);
+  o.win = ints((size_t)d.M * d.G * d.N + 1);
+  o.nwin = ints(d.M);
+  o.mr = ints(d.E);
+  o.mie = ints((size_t)d.R * (d.e_loc > 0 ? d.e_loc : 1));
+  o.orow = ints(d.E);
+  o.colv = ints((size_t)d.s_phys * d.R);
+  o.qrow = ints(d.P);
+  o.crow = ints(d.R);
+  o.ccol = ints(d.R);
+  o.U = ints(d.s_phys);
+  o.total = at;
+  return o;
+}
+
+__device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* smem, int r, int b) {
+  const Dims d = p.d;
+  const int M = d.M, G = d.G, R = d.R, E = d.E, N = d.N, P = d.P, s_phys = d.s_phys, e_loc = d.e_loc;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
+  const RankLayout lay = rank_layout(d);
+  int* Dsm = reinterpret_cast<int*>(smem + lay.D);
+  unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);
+  int* subcnt = reinterpret_cast<int*>(smem + lay.subcnt);
+  unsigned* hm_lo = reinterpret_cast<unsigned*>(smem + lay.hm_lo);
+  unsigned* hm_hi = reinterpret_cast<unsigned*>(smem + lay.hm_hi);
+  int* win = reinterpret_cast<int*>(smem + lay.win);
+  int* nwin = reinterpret_cast<int*>(smem + lay.nwin);
+  int* mr = reinterpret_cast<int*>(smem + lay.mr);
+  int* mie = reinterpret_cast<int*>(smem + lay.mie);       // [R][e_loc] expert of a main instance
+  int* orow = reinterpret_cast<int*>(smem + lay.orow);     // [E]   omega[r][.]  (r as a source)
+  int* colv = reinterpret_cast<int*>(smem + lay.colv);     // [s_phys][R] omega[.][e] of my columns
+  int* qrow = reinterpret_cast<int*>(smem + lay.qrow);     // [P]   q(r, instance) (r as a source)
+  int* ccol = reinterpret_cast<int*>(smem + lay.ccol);     // [R]   counts[.][r]
+  int* U = reinterpret_cast<int*>(smem + lay.U);           // [s_phys] loads of my instances
+  const int GN = G * N, dm = r / G, g = r - dm * G;
+  const size_t row = (size_t)b * R + r;
+
+  // static tables first: they name the experts of this rank's main columns
+#pragma unroll 2
+  for (int e = tid; e < E; e += nt) {
+    const int m = __ldg(p.ws.main_rank + e);
+    mr[e] = m;
+    const int md = m / G;
+    hm_lo[e] = md < 32 ? 1u << md : 0u;
+    hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
+  }
+#pragma unroll 2
+  for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
+#pragma unroll 1
+  for (int i = tid; i < M * GN; i += nt) win[i] = -1;
+#pragma unroll 1
+  for (int i = tid; i < R; i += nt) ccol[i] = 0;
+  if (tid < s_phys) U[tid] = 0;
+  if (tid < M) nwin[tid] = 0;
+  __syncthreads();
+  pdl_wait();
+  const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E;
+  const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E;
+  {
+    const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
+    const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
+#pragma unroll 4
+    for (int i = tid; i < M * E; i += nt) Dsm[i] = __ldcg(dA + i) + __ldcg(dB + i);
+#pragma unroll 2
+    for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + (size_t)r * E + e) + __ldcg(oB + (size_t)r * E + e);
+    // my main columns: omega[s][e] for every source s
+#pragma unroll 2
+    for (int i = tid; i < e_loc * R; i += nt) {
+      const int l = i / R, s = i - l * R, e = mie[r * e_loc + l];
+      colv[i] = e < 0 ? 0 : __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
+    }
+  }
+  __syncthreads();
+  if (g == 0 && p.ws.demand) {   // domain demand, kept for inspection (debug tensor)
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) p.ws.demand[((size_t)b * M + dm) * E + e] = Dsm[dm * E + e];
+  }
+  __syncthreads();   // the placement may zero entries of D
+  const Placement pl = {Dsm, cand_all, subcnt, hm_lo, hm_hi, win, nwin};
+  place_all_domains(pl, M, E, GN, G * p.stage1_slots, p.cand_thr, tid, nt);
+  if (!plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) return;   // solver's job
+
+  // my replica columns (every slot is taken): a second, short round of loads
+#pragma unroll 2
+  for (int i = tid; i < N * R; i += nt) {
+    const int j = i / R, s = i - j * R, e = win[dm * GN + j * G + g];
+    colv[(e_loc + j) * R + s] = __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
+  }
+  // meanwhile: row r of q (r as a source) and of the dispatch counts
+#pragma unroll 1
+  for (int pi = tid; pi < P; pi += nt) {
+    const int rr = pi / s_phys, l = pi - rr * s_phys, dd = rr / G;
+    const int e = l < e_loc ? mie[rr * e_loc + l] : win[dd * GN + (l - e_loc) * G + (rr - dd * G)];
+    int v = 0;
+    if (e >= 0) v = closed_q(orow[e], ((unsigned long long)hm_hi[e] << 32) | hm_lo[e], dd, dm, r, e);
+    qrow[pi] = v;
+    p.ws.q[row * P + pi] = v;
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int rr = tid; rr < R; rr += nt) {
+    int sum = 0;
+#pragma unroll 1
+    for (int l = 0; l < s_phys; ++l) sum += qrow[rr * s_phys + l];
+    p.ws.counts[row * R + rr] = sum;
+    p.out_counts[row * R + rr] = sum;
+  }
+  // my columns: q(s, my instance l) for every source s; instance loads U and counts[s][r]
+#pragma unroll 1
+  for (int i = tid; i < s_phys * R; i += nt) {
+    const int l = i / R, s = i - l * R;
+    const int e = l < e_loc ? mie[r * e_loc + l] : win[dm * GN + (l - e_loc) * G + g];
+    if (e < 0) continue;
+    const int v = closed_q(colv[i], ((unsigned long long)hm_hi[e] << 32) | hm_lo[e], dm, s / G, s, e);
+    if (v != 0) { atomicAdd(&U[l], v); atomicAdd(&ccol[s], v); }
+  }
+  __syncthreads();
+  if (tid < s_phys) {
+    const size_t at = (size_t)b * P + (size_t)r * s_phys + tid;
+    p.ws.inst_counts[at] = U[tid];
+    if (p.out_inst_counts) p.out_inst_counts[at] = U[tid];
+  }
+  if (tid < N) {
+    const size_t at = ((size_t)b * R + r) * N + tid;
+    const int e = win[dm * GN + tid * G + g];
+    p.ws.replica_map[at] = e;
+    if (p.out_replica_map) p.out_replica_map[at] = e;
+  }
+  if (tid == 0) {
+    int load = 0;
+#pragma unroll 1
+    for (int l = 0; l < s_phys; ++l) load += U[l];
+    p.ws.rank_load[row] = load;
+    if (g == 0) p.ws.refine_iters[(size_t)b * M + dm] = 0;
+  }
+  // receive offsets of rank r: exclusive scan over the sources, total appended
+  if (warp == 0) {
+    int32_t* recv = p.out_offsets + (((size_t)b * 2 + 1) * R + r) * (R + 1);
+    const int ch = (R + 31) / 32;
+    const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
+    int sum = 0;
+#pragma unroll 1
+    for (int s = i0; s < i1; ++s) sum += ccol[s];
+    int total;
+    int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
+    for (int s = i0; s < i1; ++s) { recv[s] = pre; pre += ccol[s]; }
+    if (lane == 0) recv[R] = total;
+  }
+}
+
 struct Plan2Params {
   SolveParams sp;
   TailParams tp;
-  int n_solve;   // solver blocks come first: block i < n_solve is (plan i / M, domain i % M)
+  int n_solve;   // blocks [0, n_solve): solver, (plan i / M, domain i % M)
+  int n_rank;    // the next n_rank blocks: rank blocks, (plan i / R, rank i % R); then per-token
 };
 
 template <bool LPT, bool VEC>
 __global__ void __launch_bounds__(kSolveThreads) plan2_kernel(const Plan2Params p) {
   extern __shared__ __align__(16) unsigned char smem[];
-  const int i = blockIdx.x;
+  int i = blockIdx.x;
   if (i < p.n_solve) {
     solve_body<LPT>(p.sp, smem, i % p.sp.d.M, i / p.sp.d.M);
-  } else {
-    const int t = i - p.n_solve, tiles = p.tp.tiles, R = p.tp.d.R;
-    tail_body<VEC>(p.tp, smem, t % tiles, (t / tiles) % R, t / (tiles * R));
+    return;
   }
+  i -= p.n_solve;
+  if (i < p.n_rank) {
+    if (!LPT) rank_body(p.sp, smem, i % p.sp.d.R, i / p.sp.d.R);
+    return;
+  }
+  i -= p.n_rank;
+  const int tiles = p.tp.tiles, R = p.tp.d.R;
+  tail_body<VEC>(p.tp, smem, i % tiles, (i / tiles) % R, i / (tiles * R));
 }
 
 }  // namespace
 
 size_t plan2_smem_bytes(const Dims& d, int tiles) {
-  return std::max(tail_layout(d, kPlan2TileIds, tiles).total, solve_smem_bytes(d));
+  return std::max(std::max(tail_layout(d, tiles).total, rank_layout(d).total), solve_smem_bytes(d));
+}
+
+long long plan2_blocks(const Dims& d, int tiles, int batch) {
+  return ((long long)d.M + d.R + (long long)tiles * d.R) * batch;
 }
 
 cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream) {
@@ -569,7 +862,8 @@ cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch,
   p.sp = sp;
   p.tp = tp;
   p.n_solve = sp.d.M * batch;
-  const dim3 grid(p.n_solve + tp.tiles * tp.d.R * batch), block(kSolveThreads);
+  p.n_rank = sp.d.R * batch;
+  const dim3 grid((unsigned)plan2_blocks(sp.d, tp.tiles, batch)), block(kSolveThreads);
   const size_t smem = plan2_smem_bytes(tp.d, tp.tiles);
   const bool pdl = tp.pdl != 0;
   if (sp.stage1_lpt)

@@ -14,7 +14,7 @@ constexpr int kRankCap = 128;   // stage 1 ranks up to this many candidates of a
 
 struct SolveLayout {
   size_t cand, col_main, col_rep, stat, mrank, mlocal, host_lo, host_hi, col_expert, col_cr, hostcol,
-      sdom, col_rank, D, qd, U, L, used, cnt, win_e, win_v, est, total;
+      sdom, col_rank, D, qd, U, L, used, cnt, win_e, win_v, est, nwin, total;
 };
 
 // The static block: everything that depends only on the handle and the domain, laid out in the
@@ -55,6 +55,7 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   o.win_v = at;      at += sizeof(int) * (size_t)d.G * d.N;   //             and their demand
   at = (at + 7) & ~(size_t)7;
   o.est = at;        at += sizeof(long long) * (size_t)d.G;   //             estimated rank loads
+  o.nwin = at;       at += sizeof(int) * (size_t)d.M;         // replicas inter-node placement made, per domain
   o.total = (at + 15) & ~(size_t)15;
   return o;
 }
@@ -141,6 +142,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   int* win_e = reinterpret_cast<int*>(smem + lay.win_e);
   int* win_v = reinterpret_cast<int*>(smem + lay.win_v);
   long long* est = reinterpret_cast<long long*>(smem + lay.est);
+  int* nwin = reinterpret_cast<int*>(smem + lay.nwin);
   short* hostcol = reinterpret_cast<short*>(smem + lay.hostcol);
   const short* sdom = reinterpret_cast<const short*>(smem + lay.sdom);
   const short* col_rank = reinterpret_cast<const short*>(smem + lay.col_rank);   // rank of a column
@@ -153,6 +155,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   copy_async(reinterpret_cast<int*>(smem + lay.stat),
              p.ws.solve_static + (size_t)dm * solve_static_ints(d), (int)solve_static_ints(d), tid, nt);
   if (tid < G) used[tid] = 0;
+  if (tid < M) nwin[tid] = 0;
 #pragma unroll 1
   for (int i = tid; i < R * G; i += nt) cnt[i] = 0;
   if (!p.acc) {
@@ -288,9 +291,23 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
       if (LPT && dd == dm)
         lpt_deal(col_main, est, win_e, win_v, used, col_expert, col_cr, hostcol, n_win, G, R, E, e_loc,
                  s_phys, p.stage1_slots, p.cost_rank_inter, lane);
+      if (lane == 0) nwin[dd] = n_win;
     }
   }
   __syncthreads();
+  // Two-kernel chain: when inter-node placement used every slot of every domain, the refinement
+  // cannot act (a move needs a target with a free slot) and the whole plan follows in closed form
+  // from the routing matrix and this placement.  The rank blocks of the grid produce it then,
+  // spread over R blocks instead of M, and this block has nothing left to do.
+  if (p.acc && !LPT) {
+    bool closed = true;
+    if (N > 0) {
+      if (M == 1 || p.stage1_slots != N) closed = false;
+#pragma unroll 1
+      for (int dd = 0; dd < M; ++dd) closed = closed && nwin[dd] == G * N;
+    }
+    if (closed) return;
+  }
 
   // ---- second batch of asynchronous copies: the routing-matrix columns of this domain's replicas ----
 #pragma unroll 1

@@ -220,6 +220,7 @@ size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 // second kernel of the two-kernel chain: solver blocks first, per-token blocks after them
 constexpr int kPlan2TileIds = kSolveThreads * kIdsPerThread;   // one block shape for both roles
 size_t plan2_smem_bytes(const Dims& d, int tiles);
+long long plan2_blocks(const Dims& d, int tiles, int batch);   // blocks of its grid
 cudaError_t configure_plan2(size_t smem);
 cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream);
 size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
