@@ -45,7 +45,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 enum WsSlot {
   W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
   W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC,
-  W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_DONE, W_SLOTS
+  W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_DONE, W_PLACE_REC, W_SLOTS
 };
 static_assert(W_SLOTS <= 32, "offset table size");
 
@@ -75,6 +75,7 @@ void carve(topoep_ctx* h) {
   sz[W_ACC_DEMAND0] = sz[W_ACC_DEMAND1] = 4 * B * (size_t)d.M * E;
   sz[W_EPOCH] = 16;
   sz[W_DONE] = 4 * B * (size_t)d.M;
+  sz[W_PLACE_REC] = 8 * B * (size_t)d.M * ((size_t)d.G * d.N + 1);
   size_t at = 0;
   for (int i = 0; i < W_SLOTS; ++i) { h->off[i] = at; at += align_up(sz[i]); }
   h->ws_bytes = at;
@@ -282,6 +283,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.acc_demand[1] = at<int32_t>(dev_ptr, h->off[W_ACC_DEMAND1]);
   w.epoch = at<unsigned>(dev_ptr, h->off[W_EPOCH]);
   w.done_flags = at<unsigned>(dev_ptr, h->off[W_DONE]);
+  w.place_rec = at<unsigned long long>(dev_ptr, h->off[W_PLACE_REC]);
 
   cudaError_t e;
   const size_t E = h->d.E;

@@ -2,23 +2,28 @@
 // one (layer, microbatch) plan at a time sits in front of every MoE layer, so its latency, not
 // its throughput, is what counts).
 //
-// Chain: accumulating histogram -> this kernel.  One grid, three kinds of blocks:
+// Chain: accumulating histogram -> this kernel.  One grid, four kinds of blocks:
 //
+//   placement blocks (plan, domain)        inter-node placement of one domain, published;
 //   solver blocks    (plan, domain)        the body of the solver kernel;
 //   rank blocks      (plan, rank)          the plan in closed form, one rank's share of it;
 //   per-token blocks (plan, source, tile)  the per-token assignment of one tile.
 //
-// Every block recomputes the inter-node placement of every domain from the demand D (the
-// paper's "every rank recomputes, no broadcast" idea, applied per block).  If that placement
-// used every replica slot, intra-node refinement cannot act: a move needs a target with a free
-// slot, because an expert has at most one instance per domain after inter-node placement.  Then
-// the plan is a closed form of the routing matrix and the placement (paper, "Inter-node
-// placement": routing construction, loads), and
+// A placement block ranks the candidates of its domain with all its warps and publishes the
+// winners as a short record of 64-bit words, each tagged with the serial number of the call, so
+// a reader knows a word is this call's without any other handshake.  Rank and per-token blocks
+// poll the records of their plan (with a limit).  Code that runs once per block costs about 15
+// cycles per instruction on this machine, so a block does as little of it as possible: what M
+// blocks can compute once is not recomputed by hundreds.
+// If the placement used every replica slot, intra-node refinement cannot act: a move needs a
+// target with a free slot, because an expert has at most one instance per domain after
+// inter-node placement.  Then the plan is a closed form of the routing matrix and the placement
+// (paper, "Inter-node placement": routing construction, loads), and
 //   * a per-token block derives the routing table of its source from row s of the routing matrix
 //     and streams its tile without waiting for anybody: histogram -> per-token assignment is
 //     the critical path;
-//   * a rank block writes what belongs to rank r: row r of q and of the dispatch counts, its
-//     instance loads U, its rank load L, its receive offsets, its replica slots;
+//   * a rank block writes what belongs to rank r: row r of q, of the dispatch counts and of the
+//     send offsets, its instance loads U, its rank load L, its receive offsets, its replica slots;
 //   * the solver blocks return at once.
 // Otherwise (some slot is free) the rank blocks return at once, the solver blocks run placement,
 // routing and refinement as in the solver kernel and publish a flag each, and a per-token block
@@ -27,8 +32,7 @@
 // wait for nobody: the wait cannot starve them.
 //
 // From the routing table on, a per-token block does what the reroute kernel does: tile prefixes,
-// resolved tiles, stream, ranking tail.  The tile with index 0 of a row also writes the row's
-// send offsets.
+// resolved tiles, stream, ranking tail.
 #include <limits.h>
 
 #include <algorithm>
@@ -86,118 +90,161 @@ __device__ __forceinline__ void tail_scan2(const int* nz, int n, int* out_a, int
   __syncthreads();
 }
 
-// ---- inter-node placement of every domain, by the whole block --------------------------------
+// ---- placement blocks ----------------------------------------------------------------------------
 // (Paper, "Inter-node placement": the candidates of a domain -- main instance elsewhere, positive
 // benefit, i.e. demand above the threshold -- in descending order (D, then ascending e); the i-th
-// winner goes to rank i mod G, slot i / G.)  In: D[M][E] in shared memory, the hosting masks with
-// the main-domain bits set.  Out: the masks with the winners' bits added, win[dd * GN + i] = the
-// i-th winner of domain dd, nwin[dd] = their number.  A domain is handled by a team of
-// nwarps / M warps when there are that many: each warp compacts the candidates of its share of
-// the experts, then ranks its own candidates against all of the domain's.
-struct Placement {
-  int* D;                       // [M][E]  (the slot-by-slot path zeroes entries)
-  unsigned long long* cand;     // [nwarps][kP2RankCap]
-  int* subcnt;                  // [nwarps]
-  unsigned* hm_lo;              // [E] hosting domains 0..31
-  unsigned* hm_hi;              // [E] hosting domains 32..63
-  int* win;                     // [M][GN], -1 where no winner
-  int* nwin;                    // [M]
-};
+// winner goes to rank i mod G, slot i / G.)  Record of (plan, domain): GN + 1 words,
+//   word 0     = serial << 32 | number of winners
+//   word 1 + i = serial << 32 | i-th winner (0xffffffff: none)
+struct PlaceLayout { size_t cand, D, mdom, chunk, winl, total; };
 
-__device__ __forceinline__ void place_all_domains(const Placement& pl, int M, int E, int GN, int slots,
-                                                  int thr, int tid, int nt) {
+__host__ __device__ inline PlaceLayout place_layout(const Dims& d) {
+  auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
+  PlaceLayout o;
+  size_t at = 0;
+  o.cand = at;  at += sizeof(unsigned long long) * (size_t)kP2RankCap;
+  o.D = at;     at += sizeof(int) * pad4(d.E);
+  o.mdom = at;  at += sizeof(int) * pad4(d.E);
+  o.chunk = at; at += sizeof(int) * pad4((size_t)(d.E + 31) / 32 + 1);
+  o.winl = at;  at += sizeof(int) * pad4((size_t)d.G * d.N + 1);
+  o.total = at;
+  return o;
+}
+
+__device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* smem, int dm, int b) {
+  const Dims d = p.d;
+  const int M = d.M, G = d.G, E = d.E, GN = d.G * d.N, slots = G * p.stage1_slots;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
   const unsigned full = 0xffffffffu;
-  const int lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+  const PlaceLayout lay = place_layout(d);
+  unsigned long long* cand = reinterpret_cast<unsigned long long*>(smem + lay.cand);
+  int* Dd = reinterpret_cast<int*>(smem + lay.D);
+  int* mdom = reinterpret_cast<int*>(smem + lay.mdom);       // 1: main instance in this domain
+  int* chunk = reinterpret_cast<int*>(smem + lay.chunk);     // candidates per 32 experts
+  int* winl = reinterpret_cast<int*>(smem + lay.winl);
+  const int nchunks = (E + 31) / 32;
+#pragma unroll 2
+  for (int e = tid; e < E; e += nt) mdom[e] = __ldg(p.ws.main_rank + e) / G == dm ? 1 : 0;
+  for (int i = tid; i <= GN; i += nt) winl[i] = -1;
+  pdl_wait();
+  const unsigned serial = __ldcg(p.ws.epoch);
+  const int32_t* dA = p.ws.acc_demand[0] + ((size_t)b * M + dm) * E;
+  const int32_t* dB = p.ws.acc_demand[1] + ((size_t)b * M + dm) * E;
+#pragma unroll 2
+  for (int e = tid; e < E; e += nt) {
+    const int v = __ldcg(dA + e) + __ldcg(dB + e);
+    Dd[e] = v;
+    if (p.ws.demand) p.ws.demand[((size_t)b * M + dm) * E + e] = v;   // kept for inspection
+  }
+  __syncthreads();
+  int n_win = 0;
   if (M > 1 && slots > 0) {
-    const int wpd = M <= nwarps ? nwarps / M : 1;   // warps per domain
-    const int nteams = nwarps / wpd, team = warp / wpd, j = warp - team * wpd;
+    // candidates per chunk of 32 experts, then their places in the compacted list
 #pragma unroll 1
-    for (int dd0 = 0; dd0 < M; dd0 += nteams) {   // one trip when a domain has several warps
-      const int dd = dd0 + team;
-      const bool on = dd < M && team < nteams;
-      unsigned long long* cand = pl.cand + (size_t)warp * kP2RankCap;
-      int* Dd = pl.D + (on ? dd : 0) * E;
-      int n_c = 0;
-      if (on) {
+    for (int c = warp; c < nchunks; c += nwarps) {
+      const int e = c * 32 + lane;
+      const bool is = e < E && !mdom[e] && Dd[e] > p.cand_thr;
+      const unsigned m = __ballot_sync(full, is);
+      if (lane == 0) chunk[c] = __popc(m);
+    }
+    __syncthreads();
+    int total = 0;
 #pragma unroll 1
-        for (int e0 = j * 32; e0 < E; e0 += wpd * 32) {
-          const int e = e0 + lane;
-          int v = 0;
-          if (e < E) {
-            // bit dd is still the main-domain bit here: it is only set below, after the barrier
-            const unsigned hosted = dd < 32 ? pl.hm_lo[e] >> dd : pl.hm_hi[e] >> (dd - 32);
-            v = (hosted & 1u) ? 0 : Dd[e];
-            v = v > thr ? v : 0;
-          }
-          const unsigned m = __ballot_sync(full, v > 0);
-          const int at = n_c + __popc(m & lanemask_lt());
-          if (v > 0 && at < kP2RankCap)
-            cand[at] = ((unsigned long long)(unsigned)v << 32) | (unsigned)~(unsigned)e;
-          n_c += __popc(m);
-        }
-        if (lane == 0) pl.subcnt[warp] = n_c;
+    for (int c = lane; c < nchunks; c += 32) total += chunk[c];
+    total = __reduce_add_sync(full, total);
+    if (total <= kP2RankCap) {
+#pragma unroll 1
+      for (int c = warp; c < nchunks; c += nwarps) {
+        int before = 0;
+#pragma unroll 1
+        for (int u = lane; u < c; u += 32) before += chunk[u];
+        before = __reduce_add_sync(full, before);
+        const int e = c * 32 + lane;
+        const bool is = e < E && !mdom[e] && Dd[e] > p.cand_thr;
+        const unsigned m = __ballot_sync(full, is);
+        if (is)
+          cand[before + __popc(m & lanemask_lt())] =
+              ((unsigned long long)(unsigned)Dd[e] << 32) | (unsigned)~(unsigned)e;
       }
-      if (wpd > 1) __syncthreads(); else __syncwarp();
-      if (on) {
-        int total = 0;
+      __syncthreads();
+      // a warp takes a candidate, its lanes the others: rank = keys above its own
+      n_win = min(total, slots);
 #pragma unroll 1
-        for (int u = 0; u < wpd; ++u) total += pl.subcnt[team * wpd + u];
-        if (total <= kP2RankCap) {
-          // every candidate counts the keys of its domain above its own; rank < slots wins
+      for (int c = warp; c < total; c += nwarps) {
+        const unsigned long long mine = cand[c];
+        int rank = 0;
 #pragma unroll 1
-          for (int c0 = 0; c0 < n_c; c0 += 32) {
-            const int c = c0 + lane;
-            const unsigned long long mine = c < n_c ? cand[c] : 0ull;
-            int rank = 0;
-#pragma unroll 1
-            for (int u = 0; u < wpd; ++u) {
-              const unsigned long long* sub = pl.cand + (size_t)(team * wpd + u) * kP2RankCap;
-              const int n_u = pl.subcnt[team * wpd + u];
-#pragma unroll 4
-              for (int o = 0; o < n_u; ++o) rank += sub[o] > mine ? 1 : 0;
-            }
-            if (c < n_c && rank < slots) {
-              const int e = (int)~(unsigned)mine;
-              if (dd < 32) atomicOr(&pl.hm_lo[e], 1u << dd); else atomicOr(&pl.hm_hi[e], 1u << (dd - 32));
-              pl.win[dd * GN + rank] = e;
-            }
-          }
-          if (j == 0 && lane == 0) pl.nwin[dd] = min(total, slots);
-        } else if (j == 0) {
-          // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
-#pragma unroll 1
-          for (int e = lane; e < E; e += 32) {
-            const unsigned hosted = dd < 32 ? pl.hm_lo[e] >> dd : pl.hm_hi[e] >> (dd - 32);
-            if ((hosted & 1u) || Dd[e] <= thr) Dd[e] = 0;
-          }
-          __syncwarp();
-          int n_win = 0;
-#pragma unroll 1
-          for (int i = 0; i < slots; ++i) {
-            int bestD = 0, bestE = INT_MAX;
-#pragma unroll 1
-            for (int e = lane; e < E; e += 32) {
-              const int v = Dd[e];
-              if (v > bestD) { bestD = v; bestE = e; }   // ascending e: first hit is smallest
-            }
-            const int maxD = __reduce_max_sync(full, bestD);
-            if (maxD <= 0) break;
-            n_win = i + 1;
-            const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
-            if (lane == 0) {
-              Dd[e] = 0;   // taken
-              if (dd < 32) atomicOr(&pl.hm_lo[e], 1u << dd); else atomicOr(&pl.hm_hi[e], 1u << (dd - 32));
-              pl.win[dd * GN + i] = e;
-            }
-            __syncwarp();
-          }
-          if (lane == 0) pl.nwin[dd] = n_win;
-        }
+        for (int o0 = 0; o0 < total; o0 += 32)
+          rank += __popc(__ballot_sync(full, o0 + lane < total && cand[o0 + lane] > mine));
+        if (lane == 0 && rank < slots) winl[rank] = (int)~(unsigned)mine;
       }
-      if (wpd == 1) __syncwarp();
+    } else if (warp == 0) {
+      // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
+#pragma unroll 1
+      for (int e = lane; e < E; e += 32)
+        if (mdom[e] || Dd[e] <= p.cand_thr) Dd[e] = 0;
+      __syncwarp();
+#pragma unroll 1
+      for (int i = 0; i < slots; ++i) {
+        int bestD = 0, bestE = INT_MAX;
+#pragma unroll 1
+        for (int e = lane; e < E; e += 32) {
+          const int v = Dd[e];
+          if (v > bestD) { bestD = v; bestE = e; }   // ascending e: first hit is smallest
+        }
+        const int maxD = __reduce_max_sync(full, bestD);
+        if (maxD <= 0) break;
+        n_win = i + 1;
+        const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
+        if (lane == 0) { Dd[e] = 0; winl[i] = e; }
+        __syncwarp();
+      }
+      if (lane == 0) winl[GN] = n_win;   // hand the count to the publishing threads
+    }
+    __syncthreads();
+    if (total > kP2RankCap) n_win = winl[GN];
+  }
+  unsigned long long* rec = p.ws.place_rec + ((size_t)b * M + dm) * (GN + 1);
+  for (int i = tid; i <= GN; i += nt) {
+    const unsigned v = i == 0 ? (unsigned)n_win : (unsigned)winl[i - 1];
+    __stcg(rec + i, ((unsigned long long)serial << 32) | v);
+  }
+}
+
+// Readers of the placement records of plan b: poll until every word carries this call's serial
+// number (bounded), then win[dd * GN + i], nwin[dd] and the winners' bits in the hosting masks
+// (which hold the main-domain bits already).  False if the records did not arrive.
+__device__ __forceinline__ bool fetch_placement(const Workspace& ws, int b, unsigned serial, int M,
+                                                int GN, int* win, int* nwin, unsigned* hm_lo,
+                                                unsigned* hm_hi, int tid, int nt) {
+  const unsigned long long* rec = ws.place_rec + (size_t)b * M * (GN + 1);
+  const int words = M * (GN + 1);
+  bool all = false;
+#pragma unroll 1
+  for (unsigned it = 0; it < kFlagWaitLimit && !all; ++it) {
+    bool ok = true;
+#pragma unroll 1
+    for (int i = tid; i < words; i += nt) {
+      const unsigned long long w = __ldcg(rec + i);
+      ok = ok && (unsigned)(w >> 32) == serial;
+      const int dd = i / (GN + 1), k = i - dd * (GN + 1);
+      if (k == 0) nwin[dd] = (int)(unsigned)w; else win[dd * GN + k - 1] = (int)(unsigned)w;
+    }
+    all = __syncthreads_and(ok);
+  }
+  if (!all) {
+    if (tid == 0) atomicOr(ws.status, TOPOEP_FLAG_INTERNAL);
+    return false;
+  }
+#pragma unroll 1
+  for (int i = tid; i < M * GN; i += nt) {
+    const int dd = i / GN, k = i - dd * GN, e = win[i];
+    if (k < nwin[dd] && e >= 0) {
+      if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
     }
   }
   __syncthreads();
+  return true;
 }
 
 // Can the refinement act at all?  Only a target with a free slot can take a move.
@@ -239,12 +286,9 @@ __device__ __forceinline__ int replica_instance(const int* win, const int* nwin,
 
 // ---- per-token blocks -------------------------------------------------------------------------
 struct TailLayout {
-  // scratch with two lives: inter-node placement first, the ranking tail afterwards
-  size_t D, cand;              // life 1
-  size_t cnt, base, work;      // life 2
-  // tables that live from their construction to the end
+  size_t cnt, base, work;      // the ranking tail's counters, bases and work list
   size_t route, hdr, seg, cum, inst, tbase, tpre;
-  size_t rm, qrow, mr, ml, orow, hm_lo, hm_hi, win, nwin, subcnt, nz, single, sidx, seg_e, crow,
+  size_t rm, qrow, mr, ml, orow, hm_lo, hm_hi, win, nwin, nz, single, sidx, seg_e, crow,
       split_e, warp_tot, tc;
   size_t total;
 };
@@ -255,17 +299,9 @@ __host__ __device__ inline TailLayout tail_layout(const Dims& d, int tiles) {
   const size_t RN = (size_t)d.R * d.N, GN = (size_t)d.G * d.N;
   TailLayout o;
   size_t at = 0;
-  o.D = at;
-  size_t l1 = (sizeof(int) * pad4((size_t)d.M * d.E) + 15) & ~(size_t)15;
-  o.cand = o.D + l1;
-  l1 += sizeof(unsigned long long) * (size_t)kP2RankCap * kP2Warps;
-  o.cnt = at;
-  size_t l2 = sizeof(uint4) * (size_t)kSplitCap * rows;
-  o.base = at + l2;
-  l2 += sizeof(int) * (size_t)kSplitCap * rows;
-  o.work = at + l2;
-  l2 += sizeof(unsigned short) * (size_t)kPlan2TileIds;
-  at += ((l1 > l2 ? l1 : l2) + 15) & ~(size_t)15;
+  o.cnt = at;   at += sizeof(uint4) * (size_t)kSplitCap * rows;
+  o.base = at;  at += sizeof(int) * (size_t)kSplitCap * rows;
+  o.work = at;  at += (sizeof(unsigned short) * (size_t)kPlan2TileIds + 15) & ~(size_t)15;
   auto ints = [&](size_t n) { const size_t r = at; at += sizeof(int) * pad4(n); return r; };
   o.route = ints(d.E + 1);
   o.hdr = ints(4);
@@ -283,7 +319,6 @@ __host__ __device__ inline TailLayout tail_layout(const Dims& d, int tiles) {
   o.hm_hi = ints(d.E);
   o.win = ints((size_t)d.M * GN + 1);
   o.nwin = ints(d.M);
-  o.subcnt = ints(kP2Warps);
   o.nz = ints(d.E);
   o.single = ints(d.E);
   o.sidx = ints(d.E + 1);
@@ -306,8 +341,6 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   const int rows = 4 * nwarps;   // 128-id rows of the tile, in flat order
   const unsigned full = 0xffffffffu;
   const TailLayout lay = tail_layout(d, p.tiles);
-  int* Dsm = reinterpret_cast<int*>(smem + lay.D);
-  unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);
   uint4* cnt4 = reinterpret_cast<uint4*>(smem + lay.cnt);
   unsigned* cntw = reinterpret_cast<unsigned*>(smem + lay.cnt);
   int* base = reinterpret_cast<int*>(smem + lay.base);
@@ -328,7 +361,6 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   unsigned* hm_hi = reinterpret_cast<unsigned*>(smem + lay.hm_hi);
   int* win = reinterpret_cast<int*>(smem + lay.win);         // [M][G*N] stage-1 winners in order
   int* nwin = reinterpret_cast<int*>(smem + lay.nwin);       // [M]
-  int* subcnt = reinterpret_cast<int*>(smem + lay.subcnt);
   int* nz = reinterpret_cast<int*>(smem + lay.nz);           // [E]   instances with q > 0
   int* single = reinterpret_cast<int*>(smem + lay.single);   // [E]
   int* sidx = reinterpret_cast<int*>(smem + lay.sidx);       // [E+1] split index of e
@@ -358,17 +390,19 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     const int md = r / G;   // the expert's main domain hosts it from the start
     hm_lo[e] = md < 32 ? 1u << md : 0u;
     hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
+    route[e] = ml[e];       // most experts have one instance with a share: their main instance
   }
-#pragma unroll 1
-  for (int i = tid; i < M * GN; i += nt) win[i] = -1;
-#pragma unroll 1
-  for (int r = tid; r < R; r += nt) crow[r] = 0;
-  if (tid < M) nwin[tid] = 0;
-  if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
+  if (tid == 0) {
+    route[E] = -1;          // every id outside [0,E) is clamped onto this entry
+    hdr[0] = 0; hdr[1] = 0; hdr[2] = 0; hdr[3] = 0;
+  }
+  static_assert(kSplitCap % 8 == 0, "counter words per thread");
+#pragma unroll
+  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
   pdl_wait();
   // ---- one round of loads of what the histogram kernel wrote (read past L1): the row's tile
-  // counts, row s of the routing matrix and the demand -- one accumulator pair holds the sums, the
-  // other zeros, so the two are added
+  // counts and row s of the routing matrix -- one accumulator pair holds the sums, the other
+  // zeros, so the two are added -- and the first poll of the placement records
   const unsigned serial = __ldcg(p.ws.epoch);   // of this call: the histogram kernel advanced it
   {
     const unsigned short* src =
@@ -385,86 +419,67 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     const int32_t* oB = p.ws.acc_omega[1] + row * E;
 #pragma unroll 2
     for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
-    const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
-    const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
-#pragma unroll 4
-    for (int i = tid; i < M * E; i += nt) Dsm[i] = __ldcg(dA + i) + __ldcg(dB + i);
   }
+  const bool have_placement = fetch_placement(p.ws, b, serial, M, GN, win, nwin, hm_lo, hm_hi, tid, nt);
   cp_async_wait_all();
   __syncthreads();
-
-  const Placement pl = {Dsm, cand_all, subcnt, hm_lo, hm_hi, win, nwin};
-  place_all_domains(pl, M, E, GN, G * p.stage1_slots, p.cand_thr, tid, nt);
+  if (!have_placement) return;   // flagged; nothing sensible can be written
   int n_split, n_list;
 
-  if (plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) {
-    // ---- the routing table of source s straight from omega[s][.] and the placement: a thread
-    // takes an expert.  An expert hosted in the source's domain, or hosted once, has one instance
-    // with a share; otherwise its share is split over its instances, ascending domain.
+  const bool closed = plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt);
+  if (closed) {
+    // ---- the routing table of source s straight from omega[s][.] and the placement.  Every
+    // expert that won no replica keeps the entry set up front (its main instance).  Warp 0 walks
+    // the winners: a replica in the source's own domain takes everything; an expert the source's
+    // domain does not host is split over its instances (ascending domain), and the lane of its
+    // first replica builds the list.
+    if (warp == 0) {
+      int ns = 0, nl = 0;   // split experts and list entries so far (warp-uniform)
 #pragma unroll 1
-    for (int e = tid; e < E; e += nt) {
-      const int w = orow[e], md = mr[e] / G;
-      const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
-      const int n = __popcll(hm);
-      int nzv, sg = ml[e];
-      if (((hm >> ds) & 1ull) || n == 1) {
-        nzv = w > 0 ? 1 : 0;
-        if (md != ds && ((hm >> ds) & 1ull)) sg = replica_instance(win, nwin, ds, e, G, GN, s_phys, e_loc);
-      } else {
-        const int bs = w / n, rem = w - bs * n;
-        nzv = bs > 0 ? n : rem;
-        if (nzv == 1) {   // one unit: it goes to the instance at index (s+e) mod n
+      for (int i0 = 0; i0 < M * GN; i0 += 32) {
+        const int idx = i0 + lane;
+        const bool valid = idx < M * GN;
+        const int dd = valid ? idx / GN : 0, i = idx - dd * GN;
+        const int e = valid ? win[idx] : 0;
+        const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
+        const int md = mr[e] / G, n = __popcll(hm), w = orow[e];
+        if (valid && dd == ds) route[e] = (dd * G + i % G) * s_phys + e_loc + i / G;
+        // first replica domain of e = lowest hosting domain that is not its main's
+        const bool first = valid && !((hm >> ds) & 1ull) &&
+                           __ffsll((long long)(hm & ~(1ull << md))) - 1 == dd;
+        const int bs = w / n, rem = w - bs * n, start = (s + e) % n;
+        const int nzv = first ? (bs > 0 ? n : rem) : 0;
+        const bool split = nzv >= 2;
+        const unsigned sm = __ballot_sync(full, split);
+        int ltot;
+        const int lpre = warp_exclusive_scan(split ? nzv : 0, lane, &ltot);
+        if (first && nzv >= 1) {
+          const int si = ns + __popc(sm & lanemask_lt());
+          int k = nl + lpre, acc = 0;
+          if (split) { route[e] = -2 - si; seg[si] = k; split_e[si] = e; }
           unsigned long long m = hm;
 #pragma unroll 1
-          for (int t = (s + e) % n; t > 0; --t) m &= m - 1;
-          const int dd = __ffsll((long long)m) - 1;
-          if (dd != md) sg = replica_instance(win, nwin, dd, e, G, GN, s_phys, e_loc);
-        }
-      }
-      nz[e] = nzv;
-      single[e] = sg;
-    }
-    __syncthreads();
-    tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
-    n_split = sidx[E];
-    n_list = seg_e[E];
-#pragma unroll 1
-    for (int e = tid; e < E; e += nt) {
-      const bool split = nz[e] >= 2;
-      route[e] = split ? -2 - sidx[e] : single[e];
-      const int w = orow[e];
-      if (split) {
-        const int i = sidx[e], md = mr[e] / G;
-        seg[i] = seg_e[e];
-        split_e[i] = e;
-        unsigned long long m = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
-        const int n = __popcll(m), bs = w / n, rem = w - bs * n, start = (s + e) % n;
-        int k = seg_e[e], acc = 0;
-#pragma unroll 1
-        for (int idx = 0; idx < n; ++idx) {
-          const int dd = __ffsll((long long)m) - 1;
-          m &= m - 1;
-          int sh = idx - start;
-          if (sh < 0) sh += n;
-          const int v = bs + (sh < rem ? 1 : 0);
-          if (v > 0) {
-            const int pi = dd == md ? ml[e] : replica_instance(win, nwin, dd, e, G, GN, s_phys, e_loc);
-            acc += v;
-            cum[k] = acc;
-            inst[k] = pi;
-            ++k;
-            if (tile == 0) atomicAdd(&crow[pi / s_phys], v);
+          for (int t = 0; t < n; ++t) {
+            const int dx = __ffsll((long long)m) - 1;
+            m &= m - 1;
+            int sh = t - start;
+            if (sh < 0) sh += n;
+            const int v = bs + (sh < rem ? 1 : 0);
+            if (v > 0) {
+              const int pi = dx == md ? ml[e] : replica_instance(win, nwin, dx, e, G, GN, s_phys, e_loc);
+              if (split) { acc += v; cum[k] = acc; inst[k] = pi; ++k; }
+              else route[e] = pi;   // one unit: it goes to the instance at index (s+e) mod n
+            }
           }
         }
-      } else if (tile == 0 && w > 0) {
-        atomicAdd(&crow[single[e] / s_phys], w);
+        ns += __popc(sm);
+        nl += ltot;
       }
-    }
-    if (tid == 0) {
-      hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
-      seg[n_split] = n_list;
+      if (lane == 0) { hdr[0] = ns; hdr[1] = nl; seg[ns] = nl; }
     }
     __syncthreads();
+    n_split = hdr[0];
+    n_list = hdr[1];
   } else {
     // ---- the refinement decides q: wait for the solver blocks of this plan (bounded polls),
     // then row s of q and the replica map come from memory
@@ -594,7 +609,8 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     if (i < kSplitCap) tbase[i] = ex;
     if (res >= 0) route[e] = res;
   }
-  if (tile == 0) {
+  if (tile == 0 && !closed) {
+    // (the rank block of s writes these when the plan is closed-form)
     // row s of the routing matrix, kept for inspection and the summaries
 #pragma unroll 1
     for (int e = tid; e < E; e += nt) p.ws.omega[row * E + e] = orow[e];
@@ -613,10 +629,6 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
       if (lane == 0) send[R] = total;
     }
   }
-  // second life of the scratch region: the ranking counters (the placement is done with it)
-  static_assert(kSplitCap % 8 == 0, "counter words per thread");
-#pragma unroll
-  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
 
   // ---- stream: look up and store; split ids are remembered, pushed and patched below
@@ -658,18 +670,14 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
 
 // ---- rank blocks: the plan in closed form, rank r's share ---------------------------------------
 struct RankLayout {
-  size_t D, cand, subcnt, hm_lo, hm_hi, win, nwin, mr, mie, orow, colv, qrow, crow, ccol, U, total;
+  size_t hm_lo, hm_hi, win, nwin, mr, mie, orow, colv, qrow, crow, ccol, U, total;
 };
 
 __host__ __device__ inline RankLayout rank_layout(const Dims& d) {
   auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
   RankLayout o;
   size_t at = 0;
-  o.cand = at;
-  at += sizeof(unsigned long long) * (size_t)kP2RankCap * kP2Warps;
   auto ints = [&](size_t n) { const size_t r = at; at += sizeof(int) * pad4(n); return r; };
-  o.D = ints((size_t)d.M * d.E);
-  o.subcnt = ints(kP2Warps);
   o.hm_lo = ints(d.E);
   o.hm_hi = ints(d.E);
   o.win = ints((size_t)d.M * d.G * d.N + 1);
@@ -691,9 +699,6 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
   const int M = d.M, G = d.G, R = d.R, E = d.E, N = d.N, P = d.P, s_phys = d.s_phys, e_loc = d.e_loc;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
   const RankLayout lay = rank_layout(d);
-  int* Dsm = reinterpret_cast<int*>(smem + lay.D);
-  unsigned long long* cand_all = reinterpret_cast<unsigned long long*>(smem + lay.cand);
-  int* subcnt = reinterpret_cast<int*>(smem + lay.subcnt);
   unsigned* hm_lo = reinterpret_cast<unsigned*>(smem + lay.hm_lo);
   unsigned* hm_hi = reinterpret_cast<unsigned*>(smem + lay.hm_hi);
   int* win = reinterpret_cast<int*>(smem + lay.win);
@@ -703,6 +708,7 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
   int* orow = reinterpret_cast<int*>(smem + lay.orow);     // [E]   omega[r][.]  (r as a source)
   int* colv = reinterpret_cast<int*>(smem + lay.colv);     // [s_phys][R] omega[.][e] of my columns
   int* qrow = reinterpret_cast<int*>(smem + lay.qrow);     // [P]   q(r, instance) (r as a source)
+  int* crow = reinterpret_cast<int*>(smem + lay.crow);     // [R]   counts[r][.]
   int* ccol = reinterpret_cast<int*>(smem + lay.ccol);     // [R]   counts[.][r]
   int* U = reinterpret_cast<int*>(smem + lay.U);           // [s_phys] loads of my instances
   const int GN = G * N, dm = r / G, g = r - dm * G;
@@ -720,20 +726,14 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
 #pragma unroll 2
   for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
 #pragma unroll 1
-  for (int i = tid; i < M * GN; i += nt) win[i] = -1;
-#pragma unroll 1
   for (int i = tid; i < R; i += nt) ccol[i] = 0;
   if (tid < s_phys) U[tid] = 0;
-  if (tid < M) nwin[tid] = 0;
   __syncthreads();
   pdl_wait();
+  const unsigned serial = __ldcg(p.ws.epoch);
   const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E;
   const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E;
   {
-    const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
-    const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
-#pragma unroll 4
-    for (int i = tid; i < M * E; i += nt) Dsm[i] = __ldcg(dA + i) + __ldcg(dB + i);
 #pragma unroll 2
     for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + (size_t)r * E + e) + __ldcg(oB + (size_t)r * E + e);
     // my main columns: omega[s][e] for every source s
@@ -743,14 +743,7 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
       colv[i] = e < 0 ? 0 : __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
     }
   }
-  __syncthreads();
-  if (g == 0 && p.ws.demand) {   // domain demand, kept for inspection (debug tensor)
-#pragma unroll 1
-    for (int e = tid; e < E; e += nt) p.ws.demand[((size_t)b * M + dm) * E + e] = Dsm[dm * E + e];
-  }
-  __syncthreads();   // the placement may zero entries of D
-  const Placement pl = {Dsm, cand_all, subcnt, hm_lo, hm_hi, win, nwin};
-  place_all_domains(pl, M, E, GN, G * p.stage1_slots, p.cand_thr, tid, nt);
+  if (!fetch_placement(p.ws, b, serial, M, GN, win, nwin, hm_lo, hm_hi, tid, nt)) return;
   if (!plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) return;   // solver's job
 
   // my replica columns (every slot is taken): a second, short round of loads
@@ -775,9 +768,13 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
     int sum = 0;
 #pragma unroll 1
     for (int l = 0; l < s_phys; ++l) sum += qrow[rr * s_phys + l];
+    crow[rr] = sum;
     p.ws.counts[row * R + rr] = sum;
     p.out_counts[row * R + rr] = sum;
   }
+  // row r of the routing matrix, kept for inspection and the summaries
+#pragma unroll 1
+  for (int e = tid; e < E; e += nt) p.ws.omega[row * E + e] = orow[e];
   // my columns: q(s, my instance l) for every source s; instance loads U and counts[s][r]
 #pragma unroll 1
   for (int i = tid; i < s_phys * R; i += nt) {
@@ -806,6 +803,20 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
     p.ws.rank_load[row] = load;
     if (g == 0) p.ws.refine_iters[(size_t)b * M + dm] = 0;
   }
+  // send offsets of source r: exclusive scan of its dispatch counts, total appended
+  if (warp == 1 % (nt >> 5)) {
+    int32_t* send = p.out_offsets + (((size_t)b * 2 + 0) * R + r) * (R + 1);
+    const int ch = (R + 31) / 32;
+    const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
+    int sum = 0;
+#pragma unroll 1
+    for (int x = i0; x < i1; ++x) sum += crow[x];
+    int total;
+    int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
+    for (int x = i0; x < i1; ++x) { send[x] = pre; pre += crow[x]; }
+    if (lane == 0) send[R] = total;
+  }
   // receive offsets of rank r: exclusive scan over the sources, total appended
   if (warp == 0) {
     int32_t* recv = p.out_offsets + (((size_t)b * 2 + 1) * R + r) * (R + 1);
@@ -825,7 +836,8 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
 struct Plan2Params {
   SolveParams sp;
   TailParams tp;
-  int n_solve;   // blocks [0, n_solve): solver, (plan i / M, domain i % M)
+  int n_solve;   // blocks [0, n_solve): placement, (plan i / M, domain i % M); the next n_solve
+                 // blocks: solver, same numbering
   int n_rank;    // the next n_rank blocks: rank blocks, (plan i / R, rank i % R); then per-token
 };
 
@@ -833,6 +845,11 @@ template <bool LPT, bool VEC>
 __global__ void __launch_bounds__(kSolveThreads) plan2_kernel(const Plan2Params p) {
   extern __shared__ __align__(16) unsigned char smem[];
   int i = blockIdx.x;
+  if (i < p.n_solve) {
+    place_body(p.sp, smem, i % p.sp.d.M, i / p.sp.d.M);
+    return;
+  }
+  i -= p.n_solve;
   if (i < p.n_solve) {
     solve_body<LPT>(p.sp, smem, i % p.sp.d.M, i / p.sp.d.M);
     return;
@@ -850,11 +867,12 @@ __global__ void __launch_bounds__(kSolveThreads) plan2_kernel(const Plan2Params 
 }  // namespace
 
 size_t plan2_smem_bytes(const Dims& d, int tiles) {
-  return std::max(std::max(tail_layout(d, tiles).total, rank_layout(d).total), solve_smem_bytes(d));
+  return std::max(std::max(tail_layout(d, tiles).total, rank_layout(d).total),
+                  std::max(solve_smem_bytes(d), place_layout(d).total));
 }
 
 long long plan2_blocks(const Dims& d, int tiles, int batch) {
-  return ((long long)d.M + d.R + (long long)tiles * d.R) * batch;
+  return (2ll * d.M + d.R + (long long)tiles * d.R) * batch;
 }
 
 cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream) {

@@ -67,6 +67,9 @@ struct Workspace {
                                     //   sums in pair 0, 1; [3] histogram blocks that have started
   unsigned* done_flags;             // [max_batch][M] serial of the last call whose solver block
                                     //   (plan, domain) has finished
+  unsigned long long* place_rec;    // [max_batch][M][G*N + 1] inter-node placement of (plan,
+                                    //   domain) as published by its placement block: every
+                                    //   word = call serial << 32 | value
 };
 
 // Record of one (plan, source) written by the route kernel, read by the reroute kernel:
