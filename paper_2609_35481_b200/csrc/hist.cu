@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   const int nt = blockDim.x, tid = threadIdx.x;
   const unsigned lane = tid & 31;
   __shared__ unsigned call_state[3];   // ACC: serial of the previous call, plans in pair 0 / 1
-  if (ACC) pdl_trigger();
+  if (ACC) { TL_MIN(p.ws, 0); pdl_trigger(); }
 
   // workspace rows are indexed by the global source rank, the caller's buffer by its window
   const size_t row = (size_t)b * p.d.R + p.rank_first + s;
@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
       __threadfence();
       p.ws.epoch[0] = ep + 1u;
     }
+    TL_MAX(p.ws, 1);
   }
 }
 

@@ -123,10 +123,12 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
   int* chunk = reinterpret_cast<int*>(smem + lay.chunk);     // candidates per 32 experts
   int* winl = reinterpret_cast<int*>(smem + lay.winl);
   const int nchunks = (E + 31) / 32;
+  TL_MIN(p.ws, 2);
 #pragma unroll 2
   for (int e = tid; e < E; e += nt) mdom[e] = __ldg(p.ws.main_rank + e) / G == dm ? 1 : 0;
   for (int i = tid; i <= GN; i += nt) winl[i] = -1;
   pdl_wait();
+  TL_MIN(p.ws, 3);
   const unsigned serial = __ldcg(p.ws.epoch);
   const int32_t* dA = p.ws.acc_demand[0] + ((size_t)b * M + dm) * E;
   const int32_t* dB = p.ws.acc_demand[1] + ((size_t)b * M + dm) * E;
@@ -137,6 +139,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
     if (p.ws.demand) p.ws.demand[((size_t)b * M + dm) * E + e] = v;   // kept for inspection
   }
   __syncthreads();
+  TL_MAX(p.ws, 4);
   int n_win = 0;
   if (M > 1 && slots > 0) {
     // candidates per chunk of 32 experts, then their places in the compacted list
@@ -209,6 +212,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
     const unsigned v = i == 0 ? (unsigned)n_win : (unsigned)winl[i - 1];
     __stcg(rec + i, ((unsigned long long)serial << 32) | v);
   }
+  TL_MAX(p.ws, 5);
 }
 
 // Readers of the placement records of plan b: poll until every word carries this call's serial
@@ -376,6 +380,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   const int32_t* ids = p.ids + row * (size_t)p.n_ids + begin;
   int32_t* out = p.out_token_replica + row * (size_t)p.n_ids + begin;
   const int RN = R * N, GN = G * N, ds = s / G;
+  TL_MIN(p.ws, 6);
 
   // ---- before the histogram kernel is known to be complete: the ids (nobody's output) and the
   // handle's static tables
@@ -400,6 +405,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
 #pragma unroll
   for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
   pdl_wait();
+  TL_MIN(p.ws, 7);
   // ---- one round of loads of what the histogram kernel wrote (read past L1): the row's tile
   // counts and row s of the routing matrix -- one accumulator pair holds the sums, the other
   // zeros, so the two are added -- and the first poll of the placement records
@@ -424,6 +430,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   cp_async_wait_all();
   __syncthreads();
   if (!have_placement) return;   // flagged; nothing sensible can be written
+  TL_MAX(p.ws, 8);
   int n_split, n_list;
 
   const bool closed = plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt);
@@ -588,6 +595,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     __syncthreads();
   }
 
+  TL_MAX(p.ws, 9);
   // Cross-tile base of every split expert's stable rank, and the resolved tiles: when the ids of
   // the expert in this tile occupy ranks [ex, ex + tv) inside ONE instance's quota interval, they
   // all go to that instance and the tile ranks nothing for it.
@@ -631,6 +639,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   }
   __syncthreads();
 
+  TL_MAX(p.ws, 10);
   // ---- stream: look up and store; split ids are remembered, pushed and patched below
   const unsigned uE = (unsigned)E;
   unsigned split_mask = 0;
@@ -660,12 +669,15 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   }
   __syncthreads();   // also orders the stores above before the patches below
   const int n_work = hdr[2];
+  TL_MAX(p.ws, 11);
   if (n_work > 0) {
     const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
     const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, nullptr, tpre, ids, out,
                         rl, rows, n_split, n_list, n_work, p.ws.status, true};
     rank_and_patch(c, tid, nt, warp, nwarps);
   }
+  TL_MAX(p.ws, 12);
+  TL_MIN(p.ws, 13);
 }
 
 // ---- rank blocks: the plan in closed form, rank r's share ---------------------------------------
@@ -744,6 +756,7 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
     }
   }
   if (!fetch_placement(p.ws, b, serial, M, GN, win, nwin, hm_lo, hm_hi, tid, nt)) return;
+  TL_MAX(p.ws, 14);
   if (!plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) return;   // solver's job
 
   // my replica columns (every slot is taken): a second, short round of loads
@@ -831,6 +844,7 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
     for (int s = i0; s < i1; ++s) { recv[s] = pre; pre += ccol[s]; }
     if (lane == 0) recv[R] = total;
   }
+  TL_MAX(p.ws, 15);
 }
 
 struct Plan2Params {

@@ -559,6 +559,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   if (p.acc) {
     __threadfence();
     __syncthreads();
+    TL_MAX(p.ws, 16);
     if (tid == 0) {
       const unsigned serial = __ldcg(p.ws.epoch);
       asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ws.done_flags + (size_t)b * M + dm),

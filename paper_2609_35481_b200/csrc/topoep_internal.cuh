@@ -261,6 +261,22 @@ cudaError_t launch_empty(int count, cudaStream_t stream);
 // at once (a single plan), the early trigger lets every later kernel finish its prologue --
 // static tables, the ids of the reroute tiles -- before its predecessor is done (1-2 us more).
 // The histogram never triggers early: the reroute blocks would read the ids at the same time.
+// Phase stamps for tuning (compiled out unless TOPOEP_TIMELINE is defined): thread 0 of a block
+// folds the global nanosecond timer into slot `slot` of a table behind the status word -- the
+// earliest (TL_MIN) or latest (TL_MAX) block to pass the point.  The host reads the table.
+#ifdef TOPOEP_TIMELINE
+__device__ __forceinline__ unsigned long long tl_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define TL_MIN(ws, slot) do { if (threadIdx.x == 0) atomicMin(reinterpret_cast<unsigned long long*>((ws).status) + 2 + (slot), tl_now()); } while (0)
+#define TL_MAX(ws, slot) do { if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned long long*>((ws).status) + 2 + (slot), tl_now()); } while (0)
+#else
+#define TL_MIN(ws, slot) do { } while (0)
+#define TL_MAX(ws, slot) do { } while (0)
+#endif
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 // Lets the dependent kernel's blocks become resident now (they still stop at their pdl_wait()).
 __device__ __forceinline__ void pdl_trigger() {
