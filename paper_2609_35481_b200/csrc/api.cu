@@ -43,7 +43,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 enum WsSlot {
-  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
+  W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_MAIN_DOM, W_MAIN_INSTANCE, W_SLOT_P, W_SLOT_DD, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
   W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC,
   W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_DONE, W_PLACE_REC, W_SLOTS
 };
@@ -57,6 +57,9 @@ void carve(topoep_ctx* h) {
   sz[W_MAIN_LOCAL] = 4 * E;
   sz[W_MAIN_INST] = 4 * R * (size_t)std::max(d.e_loc, 1);
   sz[W_SOLVE_STATIC] = (size_t)d.M * solve_static_bytes(d);
+  sz[W_MAIN_DOM] = 4 * E;
+  sz[W_MAIN_INSTANCE] = 4 * E;
+  sz[W_SLOT_P] = sz[W_SLOT_DD] = 4 * (R * (size_t)d.N + 1);
   sz[W_STATUS] = 4;
   sz[W_OMEGA] = 4 * B * R * E;
   sz[W_OMEGA_M] = 4 * B * R * (size_t)std::max(d.e_loc, 1) * R;
@@ -262,6 +265,10 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.main_local = at<int32_t>(dev_ptr, h->off[W_MAIN_LOCAL]);
   w.main_inst_expert = at<int32_t>(dev_ptr, h->off[W_MAIN_INST]);
   w.solve_static = at<int32_t>(dev_ptr, h->off[W_SOLVE_STATIC]);
+  w.main_dom = at<int32_t>(dev_ptr, h->off[W_MAIN_DOM]);
+  w.main_inst = at<int32_t>(dev_ptr, h->off[W_MAIN_INSTANCE]);
+  w.slot_p = at<int32_t>(dev_ptr, h->off[W_SLOT_P]);
+  w.slot_dd = at<int32_t>(dev_ptr, h->off[W_SLOT_DD]);
   w.status = at<uint32_t>(dev_ptr, h->off[W_STATUS]);
   w.omega = at<int32_t>(dev_ptr, h->off[W_OMEGA]);
   w.omega_m = at<int32_t>(dev_ptr, h->off[W_OMEGA_M]);
@@ -308,6 +315,24 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
     e = cudaMemcpy(const_cast<int32_t*>(w.solve_static), blocks.data(), 4 * blocks.size(),
                    cudaMemcpyHostToDevice);
     if (e != cudaSuccess) goto fail;
+  }
+  {
+    const Dims& d = h->d;
+    const int GN = d.G * d.N;
+    std::vector<int32_t> mdom(E), minst(E), sp((size_t)d.M * GN + 1), sd((size_t)d.M * GN + 1);
+    for (size_t x = 0; x < E; ++x) {
+      mdom[x] = h->main_rank[x] / d.G;
+      minst[x] = h->main_rank[x] * d.s_phys + h->main_local[x];
+    }
+    for (int dd = 0; dd < d.M; ++dd)
+      for (int i = 0; i < GN; ++i) {
+        sp[(size_t)dd * GN + i] = (dd * d.G + i % d.G) * d.s_phys + d.e_loc + i / d.G;
+        sd[(size_t)dd * GN + i] = dd;
+      }
+    if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_dom), mdom.data(), 4 * E, cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+    if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_inst), minst.data(), 4 * E, cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+    if ((e = cudaMemcpy(const_cast<int32_t*>(w.slot_p), sp.data(), 4 * sp.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
+    if ((e = cudaMemcpy(const_cast<int32_t*>(w.slot_dd), sd.data(), 4 * sd.size(), cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
   }
   if ((e = cudaMemset(w.status, 0, 4)) != cudaSuccess) goto fail;
   // accumulators, serial number and flags of the two-kernel chain start at zero (each call

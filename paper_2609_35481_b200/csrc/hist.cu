@@ -252,7 +252,9 @@ size_t hist_smem_bytes(const Dims& d) { return sizeof(int) * ((size_t)d.E + 1); 
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream) {
   const dim3 grid(p.tiles, p.rank_count, batch);
   const size_t smem = hist_smem_bytes(p.d);
-  const bool wide = p.tile_ids >= 2048;   // 32 ids per thread once the CTA still has 2+ warps
+  // 32 ids per thread once the CTA still has 2+ warps; the accumulating form, used where latency
+  // counts, keeps the shorter per-thread chain of 16
+  const bool wide = p.tile_ids >= 2048 && !p.acc;
   const dim3 block(p.tile_ids / (wide ? 32 : 16));
   const bool pdl = p.pdl != 0;
   if (p.acc) {

@@ -124,7 +124,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
   int* winl = reinterpret_cast<int*>(smem + lay.winl);
   const int nchunks = (E + 31) / 32;
   TL_MIN(p.ws, 2);
-#pragma unroll 2
+#pragma unroll 1
   for (int e = tid; e < E; e += nt) mdom[e] = __ldg(p.ws.main_rank + e) / G == dm ? 1 : 0;
   for (int i = tid; i <= GN; i += nt) winl[i] = -1;
   pdl_wait();
@@ -132,7 +132,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
   const unsigned serial = __ldcg(p.ws.epoch);
   const int32_t* dA = p.ws.acc_demand[0] + ((size_t)b * M + dm) * E;
   const int32_t* dB = p.ws.acc_demand[1] + ((size_t)b * M + dm) * E;
-#pragma unroll 2
+#pragma unroll 1
   for (int e = tid; e < E; e += nt) {
     const int v = __ldcg(dA + e) + __ldcg(dB + e);
     Dd[e] = v;
@@ -218,21 +218,26 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
 // Readers of the placement records of plan b: poll until every word carries this call's serial
 // number (bounded), then win[dd * GN + i], nwin[dd] and the winners' bits in the hosting masks
 // (which hold the main-domain bits already).  False if the records did not arrive.
+// slot_dd[i] = domain of winner entry i (a table, set up before the wait: no divisions here).
 __device__ __forceinline__ bool fetch_placement(const Workspace& ws, int b, unsigned serial, int M,
-                                                int GN, int* win, int* nwin, unsigned* hm_lo,
-                                                unsigned* hm_hi, int tid, int nt) {
+                                                int GN, int* win, int* nwin, const int* slot_dd,
+                                                unsigned* hm_lo, unsigned* hm_hi, int tid, int nt) {
   const unsigned long long* rec = ws.place_rec + (size_t)b * M * (GN + 1);
-  const int words = M * (GN + 1);
   bool all = false;
 #pragma unroll 1
   for (unsigned it = 0; it < kFlagWaitLimit && !all; ++it) {
     bool ok = true;
 #pragma unroll 1
-    for (int i = tid; i < words; i += nt) {
-      const unsigned long long w = __ldcg(rec + i);
+    for (int i = tid; i < M * GN; i += nt) {   // winner i of domain dd is word dd + 1 + i
+      const unsigned long long w = __ldcg(rec + slot_dd[i] + 1 + i);
       ok = ok && (unsigned)(w >> 32) == serial;
-      const int dd = i / (GN + 1), k = i - dd * (GN + 1);
-      if (k == 0) nwin[dd] = (int)(unsigned)w; else win[dd * GN + k - 1] = (int)(unsigned)w;
+      win[i] = (int)(unsigned)w;
+    }
+#pragma unroll 1
+    for (int dd = tid; dd < M; dd += nt) {     // the count of domain dd is word dd * (GN + 1)
+      const unsigned long long w = __ldcg(rec + (size_t)dd * (GN + 1));
+      ok = ok && (unsigned)(w >> 32) == serial;
+      nwin[dd] = (int)(unsigned)w;
     }
     all = __syncthreads_and(ok);
   }
@@ -242,7 +247,7 @@ __device__ __forceinline__ bool fetch_placement(const Workspace& ws, int b, unsi
   }
 #pragma unroll 1
   for (int i = tid; i < M * GN; i += nt) {
-    const int dd = i / GN, k = i - dd * GN, e = win[i];
+    const int dd = slot_dd[i], k = i - dd * GN, e = win[i];
     if (k < nwin[dd] && e >= 0) {
       if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
     }
@@ -277,15 +282,17 @@ __device__ __forceinline__ int closed_q(int w, unsigned long long hm, int dd, in
   return bs + (sh < rem ? 1 : 0);
 }
 
-// Instance of the replica of e that inter-node placement put into domain dd.
-__device__ __forceinline__ int replica_instance(const int* win, const int* nwin, int dd, int e, int G,
-                                                int GN, int s_phys, int e_loc) {
+// Instance of the replica of e that inter-node placement put into domain dd.  slot_p[dd * GN + i]
+// is the instance of the i-th winner's slot (rank i mod G, slot i / G of the domain): a table,
+// because integer division costs dozens of instructions on the critical path.
+__device__ __forceinline__ int replica_instance(const int* win, const int* nwin, const int* slot_p,
+                                                int dd, int e, int GN) {
   const int* w = win + dd * GN;
   const int n = nwin[dd];
   int i = 0;
 #pragma unroll 1
   while (i < n - 1 && w[i] != e) ++i;
-  return (dd * G + i % G) * s_phys + e_loc + i / G;
+  return slot_p[dd * GN + i];
 }
 
 // ---- per-token blocks -------------------------------------------------------------------------
@@ -293,7 +300,7 @@ struct TailLayout {
   size_t cnt, base, work;      // the ranking tail's counters, bases and work list
   size_t route, hdr, seg, cum, inst, tbase, tpre;
   size_t rm, qrow, mr, ml, orow, hm_lo, hm_hi, win, nwin, nz, single, sidx, seg_e, crow,
-      split_e, warp_tot, tc;
+      split_e, warp_tot, mdom, slot_p, slot_dd, tc;
   size_t total;
 };
 
@@ -330,10 +337,141 @@ __host__ __device__ inline TailLayout tail_layout(const Dims& d, int tiles) {
   o.crow = ints(d.R);
   o.split_e = ints(d.E);
   o.warp_tot = ints(2 * kP2Warps);
+  o.mdom = ints(d.E);
+  o.slot_p = ints(RN + 1);
+  o.slot_dd = ints(RN + 1);
   o.tc = at;   // per-tile counts of the row, 16 bits each: [tiles][E]
   at += (sizeof(unsigned short) * (size_t)tiles * d.E + 15) & ~(size_t)15;
   o.total = at;
   return o;
+}
+
+// Shared-memory tables of a per-token block.
+struct TailSm {
+  int *route, *hdr, *seg, *cum, *inst, *rm, *qrow, *mr, *ml, *nz, *single, *sidx, *seg_e, *crow,
+      *split_e, *warp_tot;
+};
+
+// The refinement decides q (some replica slot was free after inter-node placement): wait for the
+// solver blocks of this plan (bounded polls), read row s of q and the replica map, and build the
+// routing table the way the route kernel does.
+__device__ __forceinline__ void slow_route(const TailParams& p, const TailSm& t, int tile, int s, int b,
+                                        unsigned serial) {
+  const Dims& d = p.d;
+  const int M = d.M, R = d.R, E = d.E, N = d.N, P = d.P, s_phys = d.s_phys, e_loc = d.e_loc;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = nt >> 5;
+  const unsigned full = 0xffffffffu;
+  const int RN = R * N;
+  const size_t row = (size_t)b * R + s;
+  int *route = t.route, *hdr = t.hdr, *seg = t.seg, *cum = t.cum, *inst = t.inst, *rm = t.rm,
+      *qrow = t.qrow, *mr = t.mr, *ml = t.ml, *nz = t.nz, *single = t.single, *sidx = t.sidx,
+      *seg_e = t.seg_e, *crow = t.crow, *split_e = t.split_e, *warp_tot = t.warp_tot;
+  int n_split, n_list;
+  // ---- the refinement decides q: wait for the solver blocks of this plan (bounded polls),
+  // then row s of q and the replica map come from memory
+  if (warp == 0) {
+    const unsigned* flags = p.ws.done_flags + (size_t)b * M;
+    bool done = false;
+#pragma unroll 1
+    for (unsigned it = 0; it < kFlagWaitLimit && !done; ++it) {
+      bool mine = true;
+#pragma unroll 1
+      for (int dd = lane; dd < M; dd += 32) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flags + dd) : "memory");
+        mine = mine && v == serial;
+      }
+      done = __all_sync(full, mine);
+    }
+    if (!done && lane == 0) atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i < RN; i += nt) rm[i] = __ldcg(p.ws.replica_map + (size_t)b * RN + i);
+#pragma unroll 1
+  for (int i = tid; i < P; i += nt) qrow[i] = __ldcg(p.ws.q + row * P + i);
+  __syncthreads();
+  // instances with a share, per expert; split experts and their lists
+#pragma unroll 1
+  for (int e = tid; e < E; e += nt) {
+    nz[e] = qrow[ml[e]] > 0 ? 1 : 0;
+    single[e] = ml[e];
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i < RN; i += nt) {
+    const int e = rm[i];
+    if (e >= 0 && qrow[(i / N) * s_phys + e_loc + i % N] > 0) atomicAdd(&nz[e], 1);
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int i = tid; i < RN; i += nt) {   // the one instance with a share, when it is a replica
+    const int e = rm[i];
+    const int pi = (i / N) * s_phys + e_loc + i % N;
+    if (e >= 0 && nz[e] == 1 && qrow[pi] > 0) single[e] = pi;
+  }
+  tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
+  n_split = sidx[E];
+  n_list = seg_e[E];
+#pragma unroll 1
+  for (int e = tid; e < E; e += nt) {
+    const bool split = nz[e] >= 2;
+    route[e] = split ? -2 - sidx[e] : single[e];
+    if (split) { seg[sidx[e]] = seg_e[e]; split_e[sidx[e]] = e; }
+  }
+  if (tid == 0) {
+    hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
+    seg[n_split] = n_list;
+  }
+  if (tile == 0) {   // dispatch counts of row s, for the send offsets below
+#pragma unroll 1
+    for (int r = tid; r < R; r += nt) {
+      int sum = 0;
+#pragma unroll 1
+      for (int l = 0; l < s_phys; ++l) sum += qrow[r * s_phys + l];
+      crow[r] = sum;
+    }
+  }
+  __syncthreads();
+  // Split lists, one warp per split expert: the instances with a share in ascending rank order
+  // (the replica slots are in rank order; the main instance goes in front of the first slot on
+  // a higher rank) with cumulative quotas.
+#pragma unroll 1
+  for (int i = warp; i < n_split; i += nwarps) {
+    const int e = split_e[i];
+    const int lb = seg_e[e], qm = qrow[ml[e]], rmain = mr[e];
+    int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
+#pragma unroll 1
+    for (int i0 = 0; i0 < RN; i0 += 32) {
+      const int slot = i0 + lane;
+      int v = 0, r = 0, pi = 0;
+      if (slot < RN && rm[slot] == e) {
+        r = slot / N;
+        pi = r * s_phys + e_loc + (slot - r * N);
+        v = max(qrow[pi], 0);
+      }
+      const unsigned m = __ballot_sync(full, v > 0);
+      if (m == 0) continue;
+      int tot;
+      const int ex = warp_exclusive_scan(v, lane, &tot);
+      const bool below_main = v > 0 && r < rmain;
+      main_pos += __popc(__ballot_sync(full, below_main));
+      main_below += __reduce_add_sync(full, below_main ? v : 0);
+      if (v > 0) {
+        const bool after_main = qm > 0 && rmain < r;
+        const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
+        cum[lb + pos] = carry_cum + ex + v + (after_main ? qm : 0);
+        inst[lb + pos] = pi;
+      }
+      carry_pos += __popc(m);
+      carry_cum += tot;
+    }
+    if (lane == 0 && qm > 0) {
+      cum[lb + main_pos] = main_below + qm;
+      inst[lb + main_pos] = ml[e];
+    }
+  }
+  __syncthreads();
 }
 
 template <bool VEC>
@@ -372,8 +510,13 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   int* crow = reinterpret_cast<int*>(smem + lay.crow);       // [R]   counts[s][.]
   int* split_e = reinterpret_cast<int*>(smem + lay.split_e); // [n_split] expert of split index i
   int* warp_tot = reinterpret_cast<int*>(smem + lay.warp_tot);
+  int* mdom = reinterpret_cast<int*>(smem + lay.mdom);       // [E]   main domain
+  int* slot_p = reinterpret_cast<int*>(smem + lay.slot_p);   // [M*GN] instance of a winner's slot
+  int* slot_dd = reinterpret_cast<int*>(smem + lay.slot_dd); // [M*GN] its domain
   unsigned short* tc = reinterpret_cast<unsigned short*>(smem + lay.tc);   // [tiles][E]
 
+  const TailSm t = {route, hdr, seg, cum, inst, rm, qrow, mr, ml, nz, single, sidx, seg_e, crow,
+                    split_e, warp_tot};
   const size_t row = (size_t)b * R + s;
   const int begin = tile * p.tile_ids;
   const int count = min(p.tile_ids, p.n_ids - begin);
@@ -387,16 +530,23 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   int4 x[kIdsPerThread / 4];
 #pragma unroll
   for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
-#pragma unroll 2
+#pragma unroll 1
   for (int e = tid; e < E; e += nt) {
-    const int r = __ldg(p.ws.main_rank + e);
-    mr[e] = r;
-    ml[e] = r * s_phys + __ldg(p.ws.main_local + e);
-    const int md = r / G;   // the expert's main domain hosts it from the start
+    const int md = __ldg(p.ws.main_dom + e), mi = __ldg(p.ws.main_inst + e);
+    mr[e] = __ldg(p.ws.main_rank + e);
+    ml[e] = mi;
+    mdom[e] = md;           // the expert's main domain hosts it from the start
     hm_lo[e] = md < 32 ? 1u << md : 0u;
     hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
-    route[e] = ml[e];       // most experts have one instance with a share: their main instance
+    route[e] = mi;          // most experts have one instance with a share: their main instance
   }
+  // tables of the winner slots: entry dd * GN + i sits on rank i mod G of domain dd, slot i / G
+#pragma unroll 1
+  for (int idx = tid; idx < M * GN; idx += nt) {
+    slot_dd[idx] = __ldg(p.ws.slot_dd + idx);
+    slot_p[idx] = __ldg(p.ws.slot_p + idx);
+  }
+  __syncthreads();
   if (tid == 0) {
     route[E] = -1;          // every id outside [0,E) is clamped onto this entry
     hdr[0] = 0; hdr[1] = 0; hdr[2] = 0; hdr[3] = 0;
@@ -415,18 +565,19 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
         reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + row * (size_t)p.max_tiles * E;
     const int n16 = (tile + 1) * E;   // the row's tiles up to and including this one
     if (E % 8 == 0) {
-#pragma unroll 4
+#pragma unroll 1
       for (int i = tid; i < n16 / 8; i += nt) cp_async16_cg(tc + 8 * i, src + 8 * i);
     } else {
-#pragma unroll 4
+#pragma unroll 1
       for (int i = tid; i < n16; i += nt) tc[i] = __ldcg(src + i);
     }
     const int32_t* oA = p.ws.acc_omega[0] + row * E;
     const int32_t* oB = p.ws.acc_omega[1] + row * E;
-#pragma unroll 2
+#pragma unroll 1
     for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
   }
-  const bool have_placement = fetch_placement(p.ws, b, serial, M, GN, win, nwin, hm_lo, hm_hi, tid, nt);
+  const bool have_placement =
+      fetch_placement(p.ws, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt);
   cp_async_wait_all();
   __syncthreads();
   if (!have_placement) return;   // flagged; nothing sensible can be written
@@ -437,47 +588,35 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   if (closed) {
     // ---- the routing table of source s straight from omega[s][.] and the placement.  Every
     // expert that won no replica keeps the entry set up front (its main instance).  Warp 0 walks
-    // the winners: a replica in the source's own domain takes everything; an expert the source's
-    // domain does not host is split over its instances (ascending domain), and the lane of its
-    // first replica builds the list.
+    // the winners once: a replica in the source's own domain takes everything; an expert that the
+    // source's domain does not host is shared out over its instances, and the entry of its first
+    // replica domain stands for it.  Then every warp takes such an entry, a lane per instance.
+    int* ent_k = rm;      // [M*GN] list start of the entry's expert (split), or -1: nothing to do
+    int* ent_si = qrow;   // [M*GN] its split index, or -1: a single unit, one instance gets it
     if (warp == 0) {
       int ns = 0, nl = 0;   // split experts and list entries so far (warp-uniform)
 #pragma unroll 1
       for (int i0 = 0; i0 < M * GN; i0 += 32) {
         const int idx = i0 + lane;
         const bool valid = idx < M * GN;
-        const int dd = valid ? idx / GN : 0, i = idx - dd * GN;
+        const int dd = valid ? slot_dd[idx] : 0;
         const int e = valid ? win[idx] : 0;
         const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
-        const int md = mr[e] / G, n = __popcll(hm), w = orow[e];
-        if (valid && dd == ds) route[e] = (dd * G + i % G) * s_phys + e_loc + i / G;
+        const int md = mdom[e], n = __popcll(hm), w = orow[e];
+        if (valid && dd == ds) route[e] = slot_p[idx];
         // first replica domain of e = lowest hosting domain that is not its main's
         const bool first = valid && !((hm >> ds) & 1ull) &&
                            __ffsll((long long)(hm & ~(1ull << md))) - 1 == dd;
-        const int bs = w / n, rem = w - bs * n, start = (s + e) % n;
-        const int nzv = first ? (bs > 0 ? n : rem) : 0;
+        const int nzv = first ? min(w, n) : 0;   // instances with a share: all n once w >= n
         const bool split = nzv >= 2;
         const unsigned sm = __ballot_sync(full, split);
         int ltot;
         const int lpre = warp_exclusive_scan(split ? nzv : 0, lane, &ltot);
-        if (first && nzv >= 1) {
+        if (valid) {
           const int si = ns + __popc(sm & lanemask_lt());
-          int k = nl + lpre, acc = 0;
-          if (split) { route[e] = -2 - si; seg[si] = k; split_e[si] = e; }
-          unsigned long long m = hm;
-#pragma unroll 1
-          for (int t = 0; t < n; ++t) {
-            const int dx = __ffsll((long long)m) - 1;
-            m &= m - 1;
-            int sh = t - start;
-            if (sh < 0) sh += n;
-            const int v = bs + (sh < rem ? 1 : 0);
-            if (v > 0) {
-              const int pi = dx == md ? ml[e] : replica_instance(win, nwin, dx, e, G, GN, s_phys, e_loc);
-              if (split) { acc += v; cum[k] = acc; inst[k] = pi; ++k; }
-              else route[e] = pi;   // one unit: it goes to the instance at index (s+e) mod n
-            }
-          }
+          ent_k[idx] = nzv >= 1 ? nl + lpre : -1;
+          ent_si[idx] = split ? si : -1;
+          if (split) { route[e] = -2 - si; seg[si] = nl + lpre; split_e[si] = e; }
         }
         ns += __popc(sm);
         nl += ltot;
@@ -487,114 +626,51 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     __syncthreads();
     n_split = hdr[0];
     n_list = hdr[1];
-  } else {
-    // ---- the refinement decides q: wait for the solver blocks of this plan (bounded polls),
-    // then row s of q and the replica map come from memory
-    if (warp == 0) {
-      const unsigned* flags = p.ws.done_flags + (size_t)b * M;
-      bool done = false;
 #pragma unroll 1
-      for (unsigned it = 0; it < kFlagWaitLimit && !done; ++it) {
-        bool mine = true;
+    for (int idx = warp; idx < M * GN; idx += nwarps) {
+      const int k0 = ent_k[idx];
+      if (k0 < 0) continue;
+      const int e = win[idx], si = ent_si[idx];
+      const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
+      const int md = mdom[e], n = __popcll(hm), w = orow[e];
+      const int bs = w / n, rem = w - bs * n, start = (s + e) % n;
+      int carry_pos = 0, carry_cum = 0;
 #pragma unroll 1
-        for (int dd = lane; dd < M; dd += 32) {
-          unsigned v;
-          asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flags + dd) : "memory");
-          mine = mine && v == serial;
+      for (int t0 = 0; t0 < n; t0 += 32) {   // lane t: the t-th hosting domain, ascending
+        const int t = t0 + lane;
+        int v = 0, pi = 0;
+        if (t < n) {
+          unsigned long long m = hm;
+#pragma unroll 1
+          for (int u = 0; u < t; ++u) m &= m - 1;
+          const int dx = __ffsll((long long)m) - 1;
+          int sh = t - start;
+          if (sh < 0) sh += n;
+          v = bs + (sh < rem ? 1 : 0);
+          if (v > 0) pi = dx == md ? ml[e] : replica_instance(win, nwin, slot_p, dx, e, GN);
         }
-        done = __all_sync(full, mine);
-      }
-      if (!done && lane == 0) atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
-    }
-    __syncthreads();
-#pragma unroll 4
-    for (int i = tid; i < RN; i += nt) rm[i] = __ldcg(p.ws.replica_map + (size_t)b * RN + i);
-#pragma unroll 4
-    for (int i = tid; i < P; i += nt) qrow[i] = __ldcg(p.ws.q + row * P + i);
-    __syncthreads();
-    // instances with a share, per expert; split experts and their lists
-#pragma unroll 1
-    for (int e = tid; e < E; e += nt) {
-      nz[e] = qrow[ml[e]] > 0 ? 1 : 0;
-      single[e] = ml[e];
-    }
-    __syncthreads();
-#pragma unroll 1
-    for (int i = tid; i < RN; i += nt) {
-      const int e = rm[i];
-      if (e >= 0 && qrow[(i / N) * s_phys + e_loc + i % N] > 0) atomicAdd(&nz[e], 1);
-    }
-    __syncthreads();
-#pragma unroll 1
-    for (int i = tid; i < RN; i += nt) {   // the one instance with a share, when it is a replica
-      const int e = rm[i];
-      const int pi = (i / N) * s_phys + e_loc + i % N;
-      if (e >= 0 && nz[e] == 1 && qrow[pi] > 0) single[e] = pi;
-    }
-    tail_scan2(nz, E, sidx, seg_e, warp_tot, tid, nt);
-    n_split = sidx[E];
-    n_list = seg_e[E];
-#pragma unroll 1
-    for (int e = tid; e < E; e += nt) {
-      const bool split = nz[e] >= 2;
-      route[e] = split ? -2 - sidx[e] : single[e];
-      if (split) { seg[sidx[e]] = seg_e[e]; split_e[sidx[e]] = e; }
-    }
-    if (tid == 0) {
-      hdr[0] = n_split; hdr[1] = n_list; hdr[2] = 0; hdr[3] = 0;
-      seg[n_split] = n_list;
-    }
-    if (tile == 0) {   // dispatch counts of row s, for the send offsets below
-#pragma unroll 1
-      for (int r = tid; r < R; r += nt) {
-        int sum = 0;
-#pragma unroll 1
-        for (int l = 0; l < s_phys; ++l) sum += qrow[r * s_phys + l];
-        crow[r] = sum;
-      }
-    }
-    __syncthreads();
-    // Split lists, one warp per split expert: the instances with a share in ascending rank order
-    // (the replica slots are in rank order; the main instance goes in front of the first slot on
-    // a higher rank) with cumulative quotas.
-#pragma unroll 1
-    for (int i = warp; i < n_split; i += nwarps) {
-      const int e = split_e[i];
-      const int lb = seg_e[e], qm = qrow[ml[e]], rmain = mr[e];
-      int carry_pos = 0, carry_cum = 0, main_pos = 0, main_below = 0;
-#pragma unroll 1
-      for (int i0 = 0; i0 < RN; i0 += 32) {
-        const int slot = i0 + lane;
-        int v = 0, r = 0, pi = 0;
-        if (slot < RN && rm[slot] == e) {
-          r = slot / N;
-          pi = r * s_phys + e_loc + (slot - r * N);
-          v = max(qrow[pi], 0);
-        }
-        const unsigned m = __ballot_sync(full, v > 0);
-        if (m == 0) continue;
+        const unsigned m2 = __ballot_sync(full, v > 0);
         int tot;
         const int ex = warp_exclusive_scan(v, lane, &tot);
-        const bool below_main = v > 0 && r < rmain;
-        main_pos += __popc(__ballot_sync(full, below_main));
-        main_below += __reduce_add_sync(full, below_main ? v : 0);
         if (v > 0) {
-          const bool after_main = qm > 0 && rmain < r;
-          const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
-          cum[lb + pos] = carry_cum + ex + v + (after_main ? qm : 0);
-          inst[lb + pos] = pi;
+          if (si >= 0) {
+            const int pos = k0 + carry_pos + __popc(m2 & lanemask_lt());
+            cum[pos] = carry_cum + ex + v;
+            inst[pos] = pi;
+          } else {
+            route[e] = pi;   // one unit: it goes to the instance at index (s+e) mod n
+          }
         }
-        carry_pos += __popc(m);
+        carry_pos += __popc(m2);
         carry_cum += tot;
-      }
-      if (lane == 0 && qm > 0) {
-        cum[lb + main_pos] = main_below + qm;
-        inst[lb + main_pos] = ml[e];
       }
     }
     __syncthreads();
+  } else {
+    slow_route(p, t, tile, s, b, serial);
+    n_split = hdr[0];
+    n_list = hdr[1];
   }
-
   TL_MAX(p.ws, 9);
   // Cross-tile base of every split expert's stable rank, and the resolved tiles: when the ids of
   // the expert in this tile occupy ranks [ex, ex + tv) inside ONE instance's quota interval, they
@@ -603,7 +679,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   for (int i = tid; i < n_split; i += nt) {
     const int e = split_e[i];
     int ex = 0;
-#pragma unroll 4
+#pragma unroll 1
     for (int t = 0; t < tile; ++t) ex += tc[(size_t)t * E + e];
     const int tv = tc[(size_t)tile * E + e];
     int lo = 0, res = -1;
@@ -682,7 +758,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
 
 // ---- rank blocks: the plan in closed form, rank r's share ---------------------------------------
 struct RankLayout {
-  size_t hm_lo, hm_hi, win, nwin, mr, mie, orow, colv, qrow, crow, ccol, U, total;
+  size_t hm_lo, hm_hi, win, nwin, mr, mie, orow, colv, qrow, crow, ccol, U, slot_dd, total;
 };
 
 __host__ __device__ inline RankLayout rank_layout(const Dims& d) {
@@ -702,6 +778,7 @@ __host__ __device__ inline RankLayout rank_layout(const Dims& d) {
   o.crow = ints(d.R);
   o.ccol = ints(d.R);
   o.U = ints(d.s_phys);
+  o.slot_dd = ints((size_t)d.R * d.N + 1);
   o.total = at;
   return o;
 }
@@ -723,11 +800,12 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
   int* crow = reinterpret_cast<int*>(smem + lay.crow);     // [R]   counts[r][.]
   int* ccol = reinterpret_cast<int*>(smem + lay.ccol);     // [R]   counts[.][r]
   int* U = reinterpret_cast<int*>(smem + lay.U);           // [s_phys] loads of my instances
+  int* slot_dd = reinterpret_cast<int*>(smem + lay.slot_dd);
   const int GN = G * N, dm = r / G, g = r - dm * G;
   const size_t row = (size_t)b * R + r;
 
   // static tables first: they name the experts of this rank's main columns
-#pragma unroll 2
+#pragma unroll 1
   for (int e = tid; e < E; e += nt) {
     const int m = __ldg(p.ws.main_rank + e);
     mr[e] = m;
@@ -735,10 +813,12 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
     hm_lo[e] = md < 32 ? 1u << md : 0u;
     hm_hi[e] = md < 32 ? 0u : 1u << (md - 32);
   }
-#pragma unroll 2
+#pragma unroll 1
   for (int i = tid; i < R * e_loc; i += nt) mie[i] = __ldg(p.ws.main_inst_expert + i);
 #pragma unroll 1
   for (int i = tid; i < R; i += nt) ccol[i] = 0;
+#pragma unroll 1
+  for (int i = tid; i < M * GN; i += nt) slot_dd[i] = i / GN;
   if (tid < s_phys) U[tid] = 0;
   __syncthreads();
   pdl_wait();
@@ -746,21 +826,21 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
   const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E;
   const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E;
   {
-#pragma unroll 2
+#pragma unroll 1
     for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + (size_t)r * E + e) + __ldcg(oB + (size_t)r * E + e);
     // my main columns: omega[s][e] for every source s
-#pragma unroll 2
+#pragma unroll 1
     for (int i = tid; i < e_loc * R; i += nt) {
       const int l = i / R, s = i - l * R, e = mie[r * e_loc + l];
       colv[i] = e < 0 ? 0 : __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
     }
   }
-  if (!fetch_placement(p.ws, b, serial, M, GN, win, nwin, hm_lo, hm_hi, tid, nt)) return;
+  if (!fetch_placement(p.ws, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt)) return;
   TL_MAX(p.ws, 14);
   if (!plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) return;   // solver's job
 
   // my replica columns (every slot is taken): a second, short round of loads
-#pragma unroll 2
+#pragma unroll 1
   for (int i = tid; i < N * R; i += nt) {
     const int j = i / R, s = i - j * R, e = win[dm * GN + j * G + g];
     colv[(e_loc + j) * R + s] = __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
@@ -856,7 +936,7 @@ struct Plan2Params {
 };
 
 template <bool LPT, bool VEC>
-__global__ void __launch_bounds__(kSolveThreads) plan2_kernel(const Plan2Params p) {
+__global__ void __launch_bounds__(kSolveThreads, 2) plan2_kernel(const Plan2Params p) {
   extern __shared__ __align__(16) unsigned char smem[];
   int i = blockIdx.x;
   if (i < p.n_solve) {

@@ -35,6 +35,13 @@ struct Workspace {
   const int32_t* main_local;        // [E] index l of e among the experts of its main rank
   const int32_t* main_inst_expert;  // [R][e_loc] expert of main instance l on rank r, -1 if none
   const int32_t* solve_static;      // [M][solve_static_ints]: per-domain static block of the solver
+  // static tables of the two-kernel chain (integer division is dozens of instructions on a path
+  // where every instruction counts, so whatever depends only on the handle is tabulated)
+  const int32_t* main_dom;          // [E] domain of the main rank
+  const int32_t* main_inst;         // [E] instance id of the main instance
+  const int32_t* slot_p;            // [M*G*N] instance of the slot the i-th winner of domain dd gets
+                                    //   (entry dd*G*N + i: rank i mod G, slot i / G of the domain)
+  const int32_t* slot_dd;           // [M*G*N] dd of the entry
   uint32_t* status;                 // [1]
   int32_t* omega;                   // [max_batch][R][E]
   int32_t* omega_m;                 // [max_batch][R*e_loc][R] omega transposed, one row per main
