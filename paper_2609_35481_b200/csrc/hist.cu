@@ -37,18 +37,13 @@ __device__ __forceinline__ void count_one(int* cnt, int e, unsigned E, unsigned 
 }
 
 // IPT ids per thread (IPT/4 int4 loads in flight per thread); blockDim.x = tile_ids / IPT.
-// ACC: first kernel of the three-kernel chain for small calls.  The tile's counts are also added
-// into the routing-matrix and demand accumulators (see Workspace), which replaces the omega
-// kernel, and the kernel lets its dependents become resident from the start.
-template <int MODE, int IPT, bool ACC>
+template <int MODE, int IPT>
 __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const HistParams p) {
   extern __shared__ int cnt[];   // [E + 1]: the last bin collects ignored ids
   const int E = p.d.E;
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int nt = blockDim.x, tid = threadIdx.x;
   const unsigned lane = tid & 31;
-  __shared__ unsigned call_state[3];   // ACC: serial of the previous call, plans in pair 0 / 1
-  if (ACC) { TL_MIN(p.ws, 0); pdl_trigger(); }
 
   // workspace rows are indexed by the global source rank, the caller's buffer by its window
   const size_t row = (size_t)b * p.d.R + p.rank_first + s;
@@ -58,19 +53,6 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   int4 x[IPT / 4];
 #pragma unroll
   for (int j = 0; j < IPT / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, p.vec_ok);
-  unsigned checked_in = 0;
-  if (ACC && tid == 0) {
-    // One thread per block reads the bookkeeping words (in flight together with the ids) and
-    // then checks in.  The block that checks in last knows that every block has read them, and
-    // moves them on at its end: this call's sums go to pair (serial & 1), the other pair gets
-    // cleared below, the serial number advances.  Whoever runs after this kernel sees the new
-    // values.
-    const unsigned ep = __ldcg(p.ws.epoch), d0 = __ldcg(p.ws.epoch + 1), d1 = __ldcg(p.ws.epoch + 2);
-    call_state[0] = ep; call_state[1] = d0; call_state[2] = d1;
-    __threadfence();
-    checked_in = atomicAdd(p.ws.epoch + 3, 1u);
-  }
-
   for (int e = tid; e <= E; e += nt) cnt[e] = 0;
   __syncthreads();
   unsigned mx = 0;
@@ -95,35 +77,91 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
     unsigned short* out = reinterpret_cast<unsigned short*>(p.ws.tile_cnt) + at;
     for (int e = tid; e < E; e += nt) out[e] = (unsigned short)cnt[e];
   }
-  if (ACC) {
-    // omega[s][e] and D[dom(s)][e] (paper, "System Model", Eq. Omega and Eq. D) by integer adds
-    const unsigned cur = call_state[0] & 1u, dirty0 = call_state[1], dirty1 = call_state[2];
-    int32_t* om = p.ws.acc_omega[cur] + row * E;
-    int32_t* dem = p.ws.acc_demand[cur] + ((size_t)b * p.d.M + (p.rank_first + s) / p.d.G) * E;
-    for (int e = tid; e < E; e += nt) {
-      const int c = cnt[e];
-      if (c != 0) { atomicAdd(om + e, c); atomicAdd(dem + e, c); }
-    }
-    // clear the sums the previous call left in the other pair (nobody reads them any more: this
-    // kernel is launched in plain stream order, after everything of the previous call)
-    const size_t dirty = min((size_t)(cur ? dirty0 : dirty1), (size_t)p.max_batch);
-    const size_t n_om = dirty * p.d.R * E, n_dem = dirty * p.d.M * E;
-    const size_t ctas = (size_t)gridDim.x * gridDim.y * gridDim.z;
-    const size_t cta = ((size_t)b * gridDim.y + s) * gridDim.x + tile;
-    int32_t* zo = p.ws.acc_omega[cur ^ 1u];
-    int32_t* zd = p.ws.acc_demand[cur ^ 1u];
-    for (size_t i = cta * nt + tid; i < n_om; i += ctas * nt) zo[i] = 0;
-    for (size_t i = cta * nt + tid; i < n_dem; i += ctas * nt) zd[i] = 0;
-    if (tid == 0 && checked_in == (unsigned)ctas - 1u) {
-      const unsigned ep = call_state[0];
-      p.ws.epoch[3] = 0u;
-      p.ws.epoch[1 + (ep & 1u)] = gridDim.z;
-      p.ws.epoch[1 + ((ep & 1u) ^ 1u)] = 0u;
-      __threadfence();
-      p.ws.epoch[0] = ep + 1u;
-    }
-    TL_MAX(p.ws, 1);
+}
+
+// First kernel of the two-kernel chain for small calls: the tile histogram, and the tile's counts
+// added straight into the routing-matrix and demand accumulators (see Workspace; paper, "System
+// Model", Eq. Omega and Eq. D) -- integer adds, so the sums do not depend on arrival order --
+// which replaces the omega kernel.  A lean kernel of its own: on this path the time goes into
+// fetching instructions, so it carries no variant it does not run.  One 8192-id tile per block,
+// 16 ids per thread; the dependents may become resident from the start.
+template <bool VEC>
+__global__ void __launch_bounds__(kPlan2TileIds / kIdsPerThread) hist_acc_kernel(const HistParams p) {
+  extern __shared__ int cnt[];   // [E + 1]: the last bin collects ignored ids
+  __shared__ unsigned call_state[3];   // serial of the previous call, plans with sums in pair 0 / 1
+  const int E = p.d.E;
+  const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
+  const int nt = blockDim.x, tid = threadIdx.x;
+  TL_MIN(p.ws, 0);
+  pdl_trigger();
+  const int row = b * p.d.R + s, dem_row = b * p.d.M + s / p.d.G;
+  const int begin = tile * kPlan2TileIds;
+  const int count = min(kPlan2TileIds, p.n_ids - begin);
+  const int32_t* ids = p.ids + (size_t)row * p.n_ids + begin;
+  int4 x[kIdsPerThread / 4];
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+  unsigned checked_in = 0;
+  if (tid == 0) {
+    // One thread per block reads the bookkeeping words (in flight together with the ids) and
+    // then checks in.  The block that checks in last knows that every block has read them, and
+    // moves them on at its end: this call's sums go to pair (serial & 1), the other pair gets
+    // cleared below, the serial number advances.  Whoever runs after this kernel sees the new
+    // values.
+    const unsigned ep = __ldcg(p.ws.epoch), d0 = __ldcg(p.ws.epoch + 1), d1 = __ldcg(p.ws.epoch + 2);
+    call_state[0] = ep; call_state[1] = d0; call_state[2] = d1;
+    __threadfence();
+    checked_in = atomicAdd(p.ws.epoch + 3, 1u);
   }
+#pragma unroll 1
+  for (int e = tid; e <= E; e += nt) cnt[e] = 0;
+  __syncthreads();
+  const unsigned uE = (unsigned)E;
+  unsigned mx = 0;
+#pragma unroll
+  for (int j = 0; j < kIdsPerThread / 4; ++j) {
+    const int v[4] = {x[j].x, x[j].y, x[j].z, x[j].w};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      mx = max(mx, (unsigned)(v[u] + 1));
+      atomicAdd(&cnt[min((unsigned)v[u], uE)], 1);   // ids outside [0,E) land on the spare bin
+    }
+  }
+  if (mx > uE) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);
+  __syncthreads();
+  // the tile's counts (16 bits each: a tile has fewer than 65536 ids), and the sums
+  const unsigned cur = call_state[0] & 1u;
+  unsigned short* tc = reinterpret_cast<unsigned short*>(p.ws.tile_cnt) +
+                       ((size_t)row * p.max_tiles + tile) * E;
+  int32_t* om = p.ws.acc_omega[cur] + (size_t)row * E;
+  int32_t* dem = p.ws.acc_demand[cur] + (size_t)dem_row * E;
+#pragma unroll 1
+  for (int e = tid; e < E; e += nt) {
+    const int c = cnt[e];
+    tc[e] = (unsigned short)c;
+    if (c != 0) { atomicAdd(om + e, c); atomicAdd(dem + e, c); }
+  }
+  // clear the sums the previous call left in the other pair (nobody reads them any more: this
+  // kernel is launched in plain stream order, after everything of the previous call)
+  const unsigned dirty = min(cur ? call_state[1] : call_state[2], (unsigned)p.max_batch);
+  const size_t n_om = (size_t)dirty * p.d.R * E, n_dem = (size_t)dirty * p.d.M * E;
+  const unsigned ctas = gridDim.x * gridDim.y * gridDim.z;
+  const unsigned cta = (b * gridDim.y + s) * gridDim.x + tile;
+  int32_t* zo = p.ws.acc_omega[cur ^ 1u];
+  int32_t* zd = p.ws.acc_demand[cur ^ 1u];
+#pragma unroll 1
+  for (size_t i = (size_t)cta * nt + tid; i < n_om; i += (size_t)ctas * nt) zo[i] = 0;
+#pragma unroll 1
+  for (size_t i = (size_t)cta * nt + tid; i < n_dem; i += (size_t)ctas * nt) zd[i] = 0;
+  if (tid == 0 && checked_in == ctas - 1u) {
+    const unsigned ep = call_state[0];
+    p.ws.epoch[3] = 0u;
+    p.ws.epoch[1 + (ep & 1u)] = gridDim.z;
+    p.ws.epoch[1 + ((ep & 1u) ^ 1u)] = 0u;
+    __threadfence();
+    p.ws.epoch[0] = ep + 1u;
+  }
+  TL_MAX(p.ws, 1);
 }
 
 // omega[b][s][e] = sum over the row's tiles (or a routing matrix handed in), written three ways
@@ -252,25 +290,20 @@ size_t hist_smem_bytes(const Dims& d) { return sizeof(int) * ((size_t)d.E + 1); 
 cudaError_t launch_hist(const HistParams& p, int batch, int mode, cudaStream_t stream) {
   const dim3 grid(p.tiles, p.rank_count, batch);
   const size_t smem = hist_smem_bytes(p.d);
-  // 32 ids per thread once the CTA still has 2+ warps; the accumulating form, used where latency
-  // counts, keeps the shorter per-thread chain of 16
-  const bool wide = p.tile_ids >= 2048 && !p.acc;
+  const bool wide = p.tile_ids >= 2048;   // 32 ids per thread once the CTA still has 2+ warps
   const dim3 block(p.tile_ids / (wide ? 32 : 16));
   const bool pdl = p.pdl != 0;
-  if (p.acc) {
-    if (mode == 1) {
-      return wide ? launch_kernel(hist_kernel<1, 32, true>, grid, block, smem, stream, pdl, p)
-                  : launch_kernel(hist_kernel<1, 16, true>, grid, block, smem, stream, pdl, p);
-    }
-    return wide ? launch_kernel(hist_kernel<0, 32, true>, grid, block, smem, stream, pdl, p)
-                : launch_kernel(hist_kernel<0, 16, true>, grid, block, smem, stream, pdl, p);
+  if (p.acc) {   // the lean kernel of the two-kernel chain (plain atomics, its own tile size)
+    const dim3 acc_block(kPlan2TileIds / kIdsPerThread);
+    return p.vec_ok ? launch_kernel(hist_acc_kernel<true>, grid, acc_block, smem, stream, pdl, p)
+                    : launch_kernel(hist_acc_kernel<false>, grid, acc_block, smem, stream, pdl, p);
   }
   if (mode == 1) {
-    return wide ? launch_kernel(hist_kernel<1, 32, false>, grid, block, smem, stream, pdl, p)
-                : launch_kernel(hist_kernel<1, 16, false>, grid, block, smem, stream, pdl, p);
+    return wide ? launch_kernel(hist_kernel<1, 32>, grid, block, smem, stream, pdl, p)
+                : launch_kernel(hist_kernel<1, 16>, grid, block, smem, stream, pdl, p);
   }
-  return wide ? launch_kernel(hist_kernel<0, 32, false>, grid, block, smem, stream, pdl, p)
-              : launch_kernel(hist_kernel<0, 16, false>, grid, block, smem, stream, pdl, p);
+  return wide ? launch_kernel(hist_kernel<0, 32>, grid, block, smem, stream, pdl, p)
+              : launch_kernel(hist_kernel<0, 16>, grid, block, smem, stream, pdl, p);
 }
 
 cudaError_t launch_omega(const OmegaParams& p, int batch, cudaStream_t stream) {
