@@ -197,6 +197,7 @@ def test_random_problems_with_policies_tunings_and_skew():
         pl.set_policy(B.POLICY_STAGE1_RANK, lpt)
         pl.set_tuning(B.KNOB_TILE_IDS, int(rng.choice([1024, 2048, 4096, 8192])))
         pl.set_tuning(B.KNOB_PDL, int(rng.integers(0, 4)))
+        pl.set_tuning(B.KNOB_CHAIN, int(rng.integers(0, 3)))
         gpu = run_gpu(pl, ids)
         ref = orc.plan(oracle_config(w, reserve_slots=reserve, stage1_rank=lpt, **over), ids)
         try:
@@ -242,6 +243,59 @@ def test_empty_batch_and_zero_tokens():
     assert pl.status() == 0
 
 
+# ---- the two kernel chains of topoep_plan ---------------------------------------------------
+CHAIN_CASES = [
+    ("tiny", dict(), 2),                                    # refinement acts: solver blocks + flags
+    ("tiny", dict(slots_per_rank=3), 3),
+    ("mid", dict(), 1),                                     # closed form: every slot taken
+    ("mid", dict(slots_per_rank=3), 2),
+    ("dsv3", dict(), 1),
+    ("dsv3", dict(slots_per_rank=3, tokens_per_rank=2048), 2),
+    ("dsv3", dict(tokens_per_rank=1027, top_k=3), 1),       # ragged tiles, scalar loads
+    ("mid", dict(nodes=1, gpus_per_node=8, experts=64, slots_per_rank=2, tokens_per_rank=1000), 2),
+    ("tiny", dict(slots_per_rank=0), 1),                    # no slots: closed form, no replicas
+    ("tiny", dict(nodes=8, gpus_per_node=1, tokens_per_rank=3000), 1),
+    ("tiny", dict(nodes=40, gpus_per_node=1, experts=80, slots_per_rank=2, top_k=4,
+                  tokens_per_rank=700, zipf_s=0.9, ffn=2), 2),   # hosting masks beyond bit 31
+    ("tiny", dict(nodes=3, gpus_per_node=4, experts=600, slots_per_rank=24, top_k=8,
+                  tokens_per_rank=4096, zipf_s=0.3, ffn=1, hidden=32), 1),   # > 128 candidates
+    ("scaleout", dict(tokens_per_rank=1024), 1),            # 128 ranks, 512 experts, 2 slots
+]
+
+
+@pytest.mark.parametrize("name,over,batch", CHAIN_CASES)
+def test_two_kernel_chain_equals_five_kernel_chain_and_the_oracle(name, over, batch):
+    """topoep_plan has two kernel chains (TOPOEP_KNOB_CHAIN): five kernels, or -- for small calls --
+    an accumulating histogram followed by one grid of placement, solver, rank and per-token blocks.
+    Both must give the oracle's plan bit for bit, call after call on one handle (the accumulators
+    of the second chain alternate between two pairs and clean up after themselves), also when the
+    chains alternate and when the batch size changes between calls."""
+    w = wl.CONFIGS[name].replace(**over)
+    ids = wl.make_topk_ids(w, seed=91, batch=batch)
+    ref = orc.plan(oracle_config(w), ids)
+    pl = make_planner(w, max_batch=batch)
+    for chain in (2, 2, 1, 2, 0, 2):
+        pl.set_tuning(B.KNOB_CHAIN, chain)
+        gpu = run_gpu(pl, ids)
+        assert_same(gpu, ref)
+        assert gpu["flags"] == ref.flags
+    if batch > 1:   # a smaller batch in between leaves sums of the larger one behind: cleared?
+        pl.set_tuning(B.KNOB_CHAIN, 2)
+        one = orc.plan(oracle_config(w), ids[:1])
+        for part, want in ((ids[:1], one), (ids, ref), (ids[:1], one), (ids[:1], one), (ids, ref)):
+            assert_same(run_gpu(pl, part), want)
+    # a stage call continues from stage calls, not from a plan of the two-kernel chain
+    dev = torch.from_numpy(ids).to(pl.device)
+    out = pl.plan(dev)
+    assert B.topoep_reroute(pl.handle, dev, w.tokens_per_rank, batch, out.token_replica, 0) == -6
+    # but the solver stage may start from the routing matrix the plan left behind
+    again = pl.solve(None, batch, tokens_per_rank=w.tokens_per_rank)
+    torch.cuda.synchronize()
+    assert np.array_equal(again.replica_map.cpu().numpy(), ref.replica_map)
+    assert np.array_equal(again.dispatch_offsets.cpu().numpy()[:, 1], ref.dispatch_offsets[:, 1])
+    assert pl.status() == 0
+
+
 # ---- determinism: reruns and launch configurations ----------------------------------------
 def test_bitwise_identical_across_reruns_and_tunings():
     w = wl.CONFIGS["dsv3"].replace(slots_per_rank=3)
@@ -254,6 +308,8 @@ def test_bitwise_identical_across_reruns_and_tunings():
             pl.set_tuning(B.KNOB_HIST_MODE, mode)
             # launch protocol: plain order, automatic, never early, always early
             pl.set_tuning(B.KNOB_PDL, (tile // 1024 + mode) % 4)
+            # kernel chain: by size, five kernels, two kernels
+            pl.set_tuning(B.KNOB_CHAIN, (tile // 2048 + mode) % 3)
             for rep in range(2):
                 again = run_gpu(pl, ids)
                 for key, val in base.items():
