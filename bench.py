@@ -35,19 +35,24 @@ if ROOT not in sys.path:
 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
-KERNELS_PER_PLAN = 5
-# DRAM read+write bytes per PLAN of the DeepSeek-V3-shaped layer from the committed ncu capture of a
-# 16-plan call (profiles/reroute_kernel_dsv3_batch16.md, profiles/hist_kernel_dsv3_batch16.md);
-# a launch's traffic is this times its plans (every CTA touches only its own tile and tables).
-NCU_TRAFFIC_PER_PLAN = {
-    "reroute": (137112320 + 85663744) / 16,
-    "hist": (134235136 + 6251776) / 16,
-}
+NOMINAL_HBM_GBS = 8000.0   # the figure the target statement names; context beside the measured peak
+REPEATS = 11               # timed replays of every graph: the median is reported, min and max beside it
+# DRAM bytes per PLAN of the DeepSeek-V3-shaped layer.  READS come from the committed ncu capture of
+# a 16-plan call (profiles/reroute_kernel_dsv3_batch16.md, profiles/hist_kernel_dsv3_batch16.md) and
+# grow in proportion to the plans of a call (every CTA reads only its own tile and its source's
+# tables).  WRITES do not scale from that capture: its 134 MB of output partly stayed dirty in the
+# 126 MB L2 at kernel end (85.7 MB reached DRAM), a constant, not a proportion -- a full-size call
+# writes 1.9 GB through the same L2, so its DRAM writes are its algorithmic output bytes (4 per
+# assignment for the reroute kernel; the tile counts of the histogram kernel: 16-bit, E per tile).
+NCU_READ_BYTES_PER_PLAN = {"reroute": 137112320 / 16, "hist": 134235136 / 16}
 
 
-def ncu_traffic(w, kernel):
-    if w.name in ("dsv3", "dsv3_batched") and kernel in NCU_TRAFFIC_PER_PLAN:
-        return int(NCU_TRAFFIC_PER_PLAN[kernel] * w.batch)
+def ncu_traffic(w, kernel, tile_ids=4096):
+    if w.name in ("dsv3", "dsv3_batched") and kernel in NCU_READ_BYTES_PER_PLAN:
+        per_plan_ids = w.assignments // w.batch
+        writes = {"reroute": 4 * per_plan_ids,
+                  "hist": 2 * w.experts * (per_plan_ids // tile_ids)}[kernel]
+        return int((NCU_READ_BYTES_PER_PLAN[kernel] + writes) * w.batch)
     return None
 
 
@@ -157,19 +162,39 @@ def oracle_config(w):
                             main_rank=w.main_rank())
 
 
-def time_oracle(w, ids, budget_s):
-    """Run the oracle plan by plan on `ids` [B][R][T][k] until the budget is used up."""
+def time_oracle(w, ids, budget_s, threads=1):
+    """Run the oracle plan by plan on `ids` [B][R][T][k] until the budget is used up.  With
+    threads > 1 the independent plans of the batch are dealt to that many host threads (the
+    oracle is a C routine behind ctypes, which releases the interpreter lock while it runs)."""
     import oracle as orc
     cfg = oracle_config(w)
-    done, t0 = 0, time.perf_counter()
-    while True:
-        b = done % ids.shape[0]
-        orc.plan(cfg, ids[b:b + 1], want_q=False)
-        done += 1
-        if time.perf_counter() - t0 >= budget_s:
-            break
-    dt = time.perf_counter() - t0
     per_plan = ids.shape[1] * ids.shape[2] * ids.shape[3]
+    t0 = time.perf_counter()
+    if threads <= 1:
+        done = 0
+        while True:
+            b = done % ids.shape[0]
+            orc.plan(cfg, ids[b:b + 1], want_q=False)
+            done += 1
+            if time.perf_counter() - t0 >= budget_s:
+                break
+        dt = time.perf_counter() - t0
+        return done * per_plan / dt, done, dt
+    from concurrent.futures import ThreadPoolExecutor
+    counts = [0] * threads
+
+    def worker(i):
+        n = 0
+        while time.perf_counter() - t0 < budget_s:
+            b = (i + n * threads) % ids.shape[0]
+            orc.plan(cfg, ids[b:b + 1], want_q=False)
+            n += 1
+        counts[i] = n
+
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        list(pool.map(worker, range(threads)))
+    dt = time.perf_counter() - t0
+    done = sum(counts)
     return done * per_plan / dt, done, dt
 
 
@@ -198,11 +223,16 @@ def run_reference(args, w):
     dt = time.perf_counter() - t0
     value = args.steps * ids.size / dt
     sample = "one plan of the %s shape with %d of %d tokens per rank per step" % (w.name, T, w.tokens_per_rank)
+    # the step this arm runs: ONE plan of the workload's shape with T tokens per rank
+    step_w = w.replace(tokens_per_rank=T, batch=1)
+    cfg_line = workload_config(step_w, 1, None)
+    cfg_line["workload"] = w.name
+    cfg_line["sampled_from"] = {"tokens_per_rank": w.tokens_per_rank, "plans_per_step": w.batch}
     line = {"impl": "reference", "metric": "topk_assignments_per_s", "value": value,
             "unit": "assignments/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-            "config": workload_config(w, 1, "n/a (CPU)"),
+            "config": cfg_line,
             "cpu_baseline": {"value": value, "unit": "assignments/s", "cores": 1, "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": "assignments/s", "h2d_bytes_per_step": 0,
@@ -212,18 +242,30 @@ def run_reference(args, w):
 
 
 def workload_config(w, nsets, l2_policy):
-    return {"workload": w.name, "nodes": w.nodes, "gpus_per_node": w.gpus_per_node,
-            "ranks": w.ranks, "experts": w.experts, "slots_per_rank": w.slots_per_rank,
-            "top_k": w.top_k, "tokens_per_rank": w.tokens_per_rank, "plans_per_step": w.batch,
-            "assignments_per_step": w.assignments, "main_map": w.main_map, "seed": wl.BASE_SEED,
-            "buffer_sets": nsets, "l2": l2_policy}
+    cfg = {"workload": w.name, "nodes": w.nodes, "gpus_per_node": w.gpus_per_node,
+           "ranks": w.ranks, "experts": w.experts, "slots_per_rank": w.slots_per_rank,
+           "top_k": w.top_k, "tokens_per_rank": w.tokens_per_rank, "plans_per_step": w.batch,
+           "assignments_per_step": w.assignments, "main_map": w.main_map, "seed": wl.BASE_SEED}
+    if l2_policy is not None:   # only the GPU arm has buffer sets and an L2 to defeat
+        cfg["buffer_sets"] = nsets
+        cfg["l2"] = l2_policy
+    return cfg
 
 
 # ------------------------------------------------------------------------------------------------
 # the CUDA arm
 # ------------------------------------------------------------------------------------------------
-def measure(w, K, W, rank, world, dev, args, stages=True):
-    """Device-timed K plans of workload w inside one captured CUDA graph, plus per-stage graphs."""
+def spread(ms_list, per):
+    """median / min / max of repeated timings, each divided by `per`, in microseconds."""
+    v = sorted(m / per * 1e3 for m in ms_list)
+    return {"median": round(v[len(v) // 2], 3), "min": round(v[0], 3), "max": round(v[-1], 3),
+            "repeats": len(v)}
+
+
+def measure(w, K, W, rank, world, dev, args, stages=True, chain=-1, warm_l2=False):
+    """Device-timed K plans of workload w inside one captured CUDA graph, plus per-stage graphs.
+    chain: TOPOEP_KNOB_CHAIN for the plan graph (-1: the library's choice).  warm_l2: one buffer
+    set only, so that every replay finds its ids in L2 (reported beside the rotating figures)."""
     import torch
     import torch.distributed as dist
     from paper_2609_35481_b200 import Planner, binding as B
@@ -231,8 +273,9 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
     # inputs: nsets distinct seeded batches, each with its own planner, workspace and outputs, so
     # that a rotation over them touches more than twice L2 before any buffer repeats
     ids_bytes = w.assignments * 4
-    nsets = int(max(1, min(32, -(-2 * L2_BYTES // (2 * ids_bytes)))))
-    l2_policy = ("inputs+outputs of one step exceed L2" if nsets == 1 else
+    nsets = 1 if warm_l2 else int(max(1, min(32, -(-2 * L2_BYTES // (2 * ids_bytes)))))
+    l2_policy = ("one buffer set: ids and outputs stay in L2 (warm)" if warm_l2 and 2 * ids_bytes < L2_BYTES
+                 else "inputs+outputs of one step exceed L2" if nsets == 1 else
                  "rotation over %d distinct input/output/workspace sets (%.0f MB) exceeds L2"
                  % (nsets, nsets * 2 * ids_bytes / 1e6))
     sets = []
@@ -248,6 +291,8 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
             pl.set_tuning(B.KNOB_HIST_MODE, args.hist_mode)
         if args.pdl >= 0:
             pl.set_tuning(B.KNOB_PDL, args.pdl)
+        if chain >= 0:
+            pl.set_tuning(B.KNOB_CHAIN, chain)
         ids_dev = torch.from_numpy(ids).to(dev)
         sets.append({"pl": pl, "ids_host": ids, "ids": ids_dev,
                      "out": pl.alloc_outputs(w.batch, w.tokens_per_rank)})
@@ -276,8 +321,13 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
                               s["out"].token_replica, sh)
         assert rc == 0, rc
 
+    kernels_per_plan = 2 if (chain == 2 or (chain != 1 and sets[0]["pl"].plans_with_two_kernels(w.tokens_per_rank, w.batch))) else 5
+
     def floor(i):
-        assert B.topoep_launch_floor(KERNELS_PER_PLAN, sh) == 0
+        assert B.topoep_launch_floor(kernels_per_plan, sh) == 0
+
+    def floor1(i):
+        assert B.topoep_launch_floor(1, sh) == 0
 
     def capture(fn, n):
         g = torch.cuda.CUDAGraph()
@@ -315,17 +365,22 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
 
     g_plan = capture(plan, K)
     g_plan.replay()                      # one untimed replay of the captured graph
-    ms_total = timed_replay(g_plan)      # EXACTLY K steps
+    plan_ms = [timed_replay(g_plan) for _ in range(REPEATS)]   # each replay: EXACTLY K steps
+    ms_total = sorted(plan_ms)[len(plan_ms) // 2]
     del g_plan
 
-    # per-stage times (same rotation; hist = tile histogram + omega, solve = solver + route
-    # tables, reroute) and the launch floor: the same number of empty kernels
-    stage_us = {}
-    names = (("hist", hist), ("solve", solve), ("reroute", reroute), ("floor", floor))
+    # per-stage times through the stage entry points (same rotation; hist = tile histogram + omega,
+    # solve = solver + route tables, reroute: the kernels of the five-kernel chain) and the launch
+    # floor: as many empty kernels as the plan has kernels, and one empty kernel
+    stage_us, stage_spread = {}, {}
+    names = (("hist", hist), ("solve", solve), ("reroute", reroute), ("floor", floor),
+             ("floor1", floor1))
     for name, fn in (names if stages else names[3:]):
         g = capture(fn, K)
         g.replay()
-        stage_us[name] = timed_replay(g) / K * 1e3
+        ms = [timed_replay(g) for _ in range(REPEATS)]
+        stage_spread[name] = spread(ms, K)
+        stage_us[name] = stage_spread[name]["median"]
         del g
     # leave every workspace consistent again (the stage graphs ran stages out of order)
     with torch.cuda.stream(stream):
@@ -334,7 +389,8 @@ def measure(w, K, W, rank, world, dev, args, stages=True):
     torch.cuda.synchronize(dev)
     return {"sets": sets, "nsets": nsets, "l2_policy": l2_policy, "stream": stream,
             "ms_total": ms_total, "ms_step": ms_total / K, "stage_us": stage_us,
-            "barrier": barrier}
+            "plan_spread": spread(plan_ms, K), "stage_spread": stage_spread,
+            "kernels_per_plan": kernels_per_plan, "barrier": barrier}
 
 
 def main():
@@ -353,7 +409,7 @@ def main():
     ap.add_argument("--tile-ids", type=int, default=0)
     ap.add_argument("--hist-mode", type=int, default=-1)
     ap.add_argument("--pdl", type=int, default=-1)
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -431,6 +487,7 @@ def main():
             ev_down[j].record(down)
 
     k_e2e = max(4, min(K, int(2.0 / max(ms_step * 1e-3 + max(h2d, d2h) / 20e9, 1e-6))))
+    s0["pl"].set_tuning(B.KNOB_CHAIN, 0)
     for i in range(4):
         e2e_step(i)
     torch.cuda.synchronize(dev)
@@ -536,22 +593,47 @@ def main():
         assert pl0.status() == 0
         del main, slots, gslots, acc
 
-    # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol
+    # ---- latency of ONE layer plan (the single-plan shape of the same layer), same protocol:
+    # the library's choice of chain (two kernels for a call this small), the five-kernel chain
+    # beside it, and both again with one buffer set (ids warm in L2)
     single = None
-    if w.batch > 1 and not args.no_single_plan:
+    if not args.no_single_plan:
         w1 = wl.CONFIGS["dsv3"] if w.name == "dsv3_batched" else w.replace(batch=1)
         for s_ in sets[1:]:
             s_["pl"].close()
+
+        def close_sets(m):
+            for s_ in m["sets"]:
+                s_["pl"].close()
+
         m1 = measure(w1, 200, 20, rank, world, dev, args)
+        us = m1["plan_spread"]["median"]
+        roof_us = 12 * w1.assignments / measured_peak_gbs()[0] / 1e3
         single = {"workload": w1.name, "steps": 200, "warmup": 20,
-                  "us_per_layer_plan": round(m1["ms_step"] * 1e3, 3),
-                  "kernel_us": {n: round(m1["stage_us"][n], 3) for n in ("hist", "solve", "reroute")},
-                  "launch_floor_us": round(m1["stage_us"]["floor"], 3),
-                  "vs_launch_floor": round(m1["ms_step"] * 1e3 / m1["stage_us"]["floor"], 2),
-                  "hbm_roofline_us": round(12 * w1.assignments / measured_peak_gbs()[0] / 1e3, 3),
+                  "us_per_layer_plan": us, "spread_us": m1["plan_spread"],
+                  "kernels_per_plan": m1["kernels_per_plan"],
+                  "launch_floor_us": m1["stage_us"]["floor"],
+                  "launch_floor_one_kernel_us": m1["stage_us"]["floor1"],
+                  "vs_launch_floor": round(us / m1["stage_us"]["floor"], 2),
+                  "hbm_roofline_us": round(roof_us, 3),
+                  "hbm_frac": round(roof_us / us, 4),
+                  "hbm_frac_8B": round(roof_us * 8 / 12 / us, 4),
+                  "hbm_frac_nominal": round(12 * w1.assignments / NOMINAL_HBM_GBS / 1e3 / us, 4),
+                  "five_kernel_stage_us": {n: m1["stage_us"][n] for n in ("hist", "solve", "reroute")},
                   "l2": m1["l2_policy"]}
-        for s_ in m1["sets"]:
-            s_["pl"].close()
+        close_sets(m1)
+        m5 = measure(w1, 200, 20, rank, world, dev, args, stages=False, chain=1)
+        single["five_kernel_chain"] = {"us_per_layer_plan": m5["plan_spread"]["median"],
+                                       "spread_us": m5["plan_spread"],
+                                       "launch_floor_us": m5["stage_us"]["floor"]}
+        close_sets(m5)
+        mw = measure(w1, 200, 20, rank, world, dev, args, stages=False, warm_l2=True)
+        single["warm_l2"] = {"us_per_layer_plan": mw["plan_spread"]["median"],
+                             "spread_us": mw["plan_spread"], "l2": mw["l2_policy"]}
+        close_sets(mw)
+        mw5 = measure(w1, 200, 20, rank, world, dev, args, stages=False, chain=1, warm_l2=True)
+        single["warm_l2"]["five_kernel_chain_us"] = mw5["plan_spread"]["median"]
+        close_sets(mw5)
     clocks = sampler.finish()
 
     # the e2e outputs came back to the host: check them against the device copies of the same plan
@@ -574,14 +656,22 @@ def main():
     else:
         dom_bytes = algo_bytes[dominant]
     achieved = dom_bytes / (stage_us[dominant] * 1e-6) / 1e9
+    plan_gbs = 12 * A / (ms_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": {"hist": "hist_kernel", "solve": "solve_kernel",
                                            "reroute": "reroute_kernel"}[dominant],
                 "achieved": round(achieved, 2), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "peak_source": "of " + peak_kind,
-                "traffic": ncu_traffic(w, dominant),
+                "frac_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
+                "traffic": ncu_traffic(w, dominant, args.tile_ids or 4096),
+                "traffic_note": "reads: ncu capture of a 16-plan call scaled by plans; writes: "
+                                "algorithmic output bytes (see the comment at NCU_READ_BYTES_PER_PLAN)",
                 "algorithmic_bytes_per_launch": dom_bytes,
                 "plan_bytes": 12 * A,
-                "plan_frac": round(12 * A / (ms_step * 1e-3) / 1e9 / peak, 4),
+                "plan_frac": round(plan_gbs / peak, 4),
+                # the whole plan against 8 B per assignment: ids read from DRAM once (second pass
+                # from L2), outputs written once -- the bound a chunked batch could approach
+                "plan_frac_8B": round(plan_gbs * 8 / 12 / peak, 4),
+                "plan_frac_nominal": round(plan_gbs / NOMINAL_HBM_GBS, 4),
                 "hbm_kernels": hbm_kernels,
                 "note": "peak is a plain read+write copy; a kernel with the same traffic mix can land "
                         "a few percent above it (the full-size parity tests run this launch configuration)"}
@@ -596,8 +686,11 @@ def main():
             "e2e": {"value": e2e_value, "unit": "assignments/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": k_e2e,
                     "us_per_layer_plan": ms_e2e * 1e3 / k_e2e / w.batch},
-            "gpu_launches": KERNELS_PER_PLAN * K,
+            "gpu_launches": m["kernels_per_plan"] * K,
+            "repeats": m["plan_spread"]["repeats"],
+            "us_per_step": m["plan_spread"],
             "kernel_us": {n: round(stage_us[n], 3) for n in ("hist", "solve", "reroute")},
+            "kernel_us_spread": {n: m["stage_spread"][n] for n in ("hist", "solve", "reroute")},
             "launch_floor_us": round(stage_us["floor"], 3),
             "vs_launch_floor": round(ms_step * 1e3 / stage_us["floor"], 2),
             "roofline": roofline}
@@ -609,11 +702,19 @@ def main():
         line["replica_transfer"] = transfer
 
     if rank == 0 and not args.no_cpu_baseline:
-        sample_ids = s0["ids_host"][:min(w.batch, 8)]
+        ncores = os.cpu_count() or 1
+        sample_ids = s0["ids_host"][:min(w.batch, max(8, ncores))]
         v, plans, dt = time_oracle(w, sample_ids, args.cpu_seconds)
         line["cpu_baseline"] = {"value": v, "unit": "assignments/s", "cores": 1, "kind": "oracle",
                                 "sample": "%d whole plans of the %s shape in %.1f s (host has %d cores)"
-                                          % (plans, w.name, dt, os.cpu_count() or 0)}
+                                          % (plans, w.name, dt, ncores)}
+        if w.batch > 1 and ncores > 1:
+            # the plans of a batch are independent: the same oracle, one plan per host thread
+            va, plans_a, dta = time_oracle(w, sample_ids, args.cpu_seconds, threads=ncores)
+            line["cpu_baseline_all_cores"] = {
+                "value": va, "unit": "assignments/s", "cores": ncores, "kind": "oracle",
+                "sample": "%d whole plans of the %s shape in %.1f s, independent plans dealt to "
+                          "%d host threads" % (plans_a, w.name, dta, ncores)}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

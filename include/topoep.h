@@ -423,6 +423,14 @@ int topoep_replica_grad_return(topoep_handle_t h, const int32_t* dev_replica_map
  */
 int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count);
 
+/*
+ * Number of kernels topoep_plan would enqueue for a call of this size with the
+ * current knobs: 5, or 2 for a small call (see TOPOEP_KNOB_CHAIN).  Needs the
+ * workspace (the answer depends on the device).  Negative status on a bad
+ * handle or size.  Not part of the method: for benchmarks and tests.
+ */
+int topoep_plan_kernels(topoep_handle_t h, int tokens_per_rank, int batch);
+
 /* Derived sizes: E_loc, S_phys, P.  Any output pointer may be NULL. */
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances);
 

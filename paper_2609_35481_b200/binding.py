@@ -23,7 +23,7 @@ EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_
            "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions", "topoep_dispatch_window",
            "topoep_summary", "topoep_read_status",
            "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_set_policy", "topoep_replica_pull", "topoep_replica_grad_return",
-           "topoep_get_layout",
+           "topoep_get_layout", "topoep_plan_kernels",
            "topoep_launch_floor", "topoep_strerror")
 
 
@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
             fn.argtypes = [vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.topoep_get_layout.restype = ci
         L.topoep_get_layout.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.topoep_plan_kernels.restype = ci
+        L.topoep_plan_kernels.argtypes = [vp, ci, ci]
         L.topoep_launch_floor.restype = ci
         L.topoep_launch_floor.argtypes = [ci, vp]
         L.topoep_strerror.restype = ctypes.c_char_p
@@ -258,6 +260,11 @@ def topoep_get_layout(h):
     a, b, c = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
     rc = lib().topoep_get_layout(h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
     return rc, a.value, b.value, c.value
+
+
+def topoep_plan_kernels(h, tokens_per_rank: int, batch: int) -> int:
+    """Kernels topoep_plan would enqueue for a call of this size (5, or 2 for a small call)."""
+    return lib().topoep_plan_kernels(h, tokens_per_rank, batch)
 
 
 def topoep_launch_floor(count: int, stream=0) -> int:

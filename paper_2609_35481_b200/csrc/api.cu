@@ -814,6 +814,12 @@ int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count) {
   return TOPOEP_OK;
 }
 
+int topoep_plan_kernels(topoep_handle_t h, int tokens_per_rank, int batch) {
+  const int rc = check_sizes(h, tokens_per_rank, batch);
+  if (rc != TOPOEP_OK) return rc;
+  return use_two_kernels(h, tokens_per_rank, batch) ? 2 : 5;
+}
+
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances) {
   if (!h) return TOPOEP_ERR_NULL;
   if (e_loc) *e_loc = h->d.e_loc;

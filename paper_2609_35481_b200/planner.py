@@ -261,6 +261,10 @@ class Planner:
         raw = self.workspace[off:off + batch * per].cpu().numpy()
         return torch.from_numpy(raw.view(np.int32).reshape((batch,) + shape).copy())
 
+    def plans_with_two_kernels(self, tokens_per_rank: int, batch: int) -> bool:
+        """True when topoep_plan would take its two-kernel chain for a call of this size."""
+        return B.topoep_plan_kernels(self.handle, tokens_per_rank, batch) == 2
+
     def set_policy(self, policy: int, value: int):
         """Policy variants change the plan (unlike tuning knobs); see topoep_set_policy."""
         rc = B.topoep_set_policy(self.handle, policy, value)
