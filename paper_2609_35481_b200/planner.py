@@ -179,7 +179,7 @@ class Planner:
                      out: Optional[PlanOutputs] = None) -> PlanOutputs:
         """One planning step of a process that owns a window of source ranks.
 
-        Every process of `group` (torch.distributed, NCCL) calls this with the ids of its own
+        Every process of `group` (torch.distributed; NCCL, or gloo through host memory) calls this with the ids of its own
         window [B][count][T][k]; windows are equal-sized and ordered by group rank.  The rows of
         the routing matrix are all-gathered (the only exchange: B*R*E int32, never the ids), every
         process solves the whole group's plan from the same matrix, and reroutes its own ids.
@@ -196,8 +196,16 @@ class Planner:
         if self.window != (me * cnt, cnt):
             self.set_rank_window(me * cnt, cnt)
         rows = self.histogram(my_topk_ids)                       # [B][cnt][E]
-        allrows = torch.empty((world,) + tuple(rows.shape), dtype=rows.dtype, device=self.device)
-        dist.all_gather_into_tensor(allrows, rows, group=group)
+        if dist.get_backend(group) == "gloo":
+            # a host-side group (tests, or processes that share one GPU): the rows travel through
+            # host memory, then return to the device
+            host = rows.cpu()
+            parts = [torch.empty_like(host) for _ in range(world)]
+            dist.all_gather(parts, host, group=group)
+            allrows = torch.stack(parts).to(self.device)
+        else:
+            allrows = torch.empty((world,) + tuple(rows.shape), dtype=rows.dtype, device=self.device)
+            dist.all_gather_into_tensor(allrows, rows, group=group)
         omega = allrows.permute(1, 0, 2, 3).reshape(Bn, self.R, self.E).contiguous()
         out = self.solve(omega, Bn, out=out, tokens_per_rank=T)
         rc = B.topoep_reroute(self.handle, my_topk_ids, T, Bn, out.token_replica,
