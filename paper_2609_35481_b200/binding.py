@@ -52,10 +52,15 @@ def lib() -> ctypes.CDLL:
         # Stale or missing library: compile it in-tree (nvcc, sm_100a).  There is no other
         # implementation to fall back to; a failed build raises.
         from . import build as _build
-        _build.build()
-        if not os.path.exists(LIB_PATH):
+        path = LIB_PATH
+        if os.environ.get("TOPOEP_CHECKED_BUILD") == "1":
+            # the tests' bounds-checked build of the same sources (same entry points)
+            path = _build.build_checked()
+        else:
+            _build.build()
+        if not os.path.exists(path):
             raise RuntimeError("libtopoep.so could not be built (there is no CPU fallback)")
-        L = ctypes.CDLL(LIB_PATH)
+        L = ctypes.CDLL(path)
         vp, ci, i32p = ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p
         L.topoep_create.restype = ci
         L.topoep_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, ci, i32p,

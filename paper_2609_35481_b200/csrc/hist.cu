@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kPlan2TileIds / kIdsPerThread) hist_acc_kernel
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       mx = max(mx, (unsigned)(v[u] + 1));
-      atomicAdd(&cnt[min((unsigned)v[u], uE)], 1);   // ids outside [0,E) land on the spare bin
+      atomicAdd(&cnt[CK(p.ws.status, (long long)min((unsigned)v[u], uE), E + 1)], 1);   // ids outside [0,E): the spare bin
     }
   }
   if (mx > uE) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);

@@ -166,7 +166,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
         const bool is = e < E && !mdom[e] && Dd[e] > p.cand_thr;
         const unsigned m = __ballot_sync(full, is);
         if (is)
-          cand[before + __popc(m & lanemask_lt())] =
+          cand[CK(p.ws.status, before + __popc(m & lanemask_lt()), kP2RankCap)] =
               ((unsigned long long)(unsigned)Dd[e] << 32) | (unsigned)~(unsigned)e;
       }
       __syncthreads();
@@ -179,7 +179,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
 #pragma unroll 1
         for (int o0 = 0; o0 < total; o0 += 32)
           rank += __popc(__ballot_sync(full, o0 + lane < total && cand[o0 + lane] > mine));
-        if (lane == 0 && rank < slots) winl[rank] = (int)~(unsigned)mine;
+        if (lane == 0 && rank < slots) winl[CK(p.ws.status, rank, GN)] = (int)~(unsigned)mine;
       }
     } else if (warp == 0) {
       // many candidates: pick the maximum slot by slot (non-candidates are zeroed first)
@@ -199,7 +199,7 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
         if (maxD <= 0) break;
         n_win = i + 1;
         const int e = __reduce_min_sync(full, bestD == maxD ? bestE : INT_MAX);
-        if (lane == 0) { Dd[e] = 0; winl[i] = e; }
+        if (lane == 0) { Dd[CK(p.ws.status, e, E)] = 0; winl[CK(p.ws.status, i, GN)] = e; }
         __syncwarp();
       }
       if (lane == 0) winl[GN] = n_win;   // hand the count to the publishing threads
@@ -219,8 +219,9 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
 // number (bounded), then win[dd * GN + i], nwin[dd] and the winners' bits in the hosting masks
 // (which hold the main-domain bits already).  False if the records did not arrive.
 // slot_dd[i] = domain of winner entry i (a table, set up before the wait: no divisions here).
-__device__ __forceinline__ bool fetch_placement(const Workspace& ws, int b, unsigned serial, int M,
-                                                int GN, int* win, int* nwin, const int* slot_dd,
+__device__ __forceinline__ bool fetch_placement(const Workspace& ws, int ws_experts, int b,
+                                                unsigned serial, int M, int GN, int* win,
+                                                int* nwin, const int* slot_dd,
                                                 unsigned* hm_lo, unsigned* hm_hi, int tid, int nt) {
   const unsigned long long* rec = ws.place_rec + (size_t)b * M * (GN + 1);
   bool all = false;
@@ -247,7 +248,8 @@ __device__ __forceinline__ bool fetch_placement(const Workspace& ws, int b, unsi
   }
 #pragma unroll 1
   for (int i = tid; i < M * GN; i += nt) {
-    const int dd = slot_dd[i], k = i - dd * GN, e = win[i];
+    const int dd = CK(ws.status, slot_dd[i], M), k = i - dd * GN;
+    const int e = win[i] < 0 ? -1 : CK(ws.status, win[i], ws_experts);
     if (k < nwin[dd] && e >= 0) {
       if (dd < 32) atomicOr(&hm_lo[e], 1u << dd); else atomicOr(&hm_hi[e], 1u << (dd - 32));
     }
@@ -292,7 +294,7 @@ __device__ __forceinline__ int replica_instance(const int* win, const int* nwin,
   int i = 0;
 #pragma unroll 1
   while (i < n - 1 && w[i] != e) ++i;
-  return slot_p[dd * GN + i];
+  return slot_p[dd * GN + (i < 0 ? 0 : i)];
 }
 
 // ---- per-token blocks -------------------------------------------------------------------------
@@ -577,7 +579,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
   }
   const bool have_placement =
-      fetch_placement(p.ws, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt);
+      fetch_placement(p.ws, E, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt);
   cp_async_wait_all();
   __syncthreads();
   if (!have_placement) return;   // flagged; nothing sensible can be written
@@ -600,7 +602,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
         const int idx = i0 + lane;
         const bool valid = idx < M * GN;
         const int dd = valid ? slot_dd[idx] : 0;
-        const int e = valid ? win[idx] : 0;
+        const int e = valid ? CK(p.ws.status, win[idx], E) : 0;
         const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
         const int md = mdom[e], n = __popcll(hm), w = orow[e];
         if (valid && dd == ds) route[e] = slot_p[idx];
@@ -616,12 +618,16 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
           const int si = ns + __popc(sm & lanemask_lt());
           ent_k[idx] = nzv >= 1 ? nl + lpre : -1;
           ent_si[idx] = split ? si : -1;
-          if (split) { route[e] = -2 - si; seg[si] = nl + lpre; split_e[si] = e; }
+          if (split) {
+            route[e] = -2 - si;
+            seg[CK(p.ws.status, si, E)] = nl + lpre;
+            split_e[CK(p.ws.status, si, E)] = e;
+          }
         }
         ns += __popc(sm);
         nl += ltot;
       }
-      if (lane == 0) { hdr[0] = ns; hdr[1] = nl; seg[ns] = nl; }
+      if (lane == 0) { hdr[0] = ns; hdr[1] = nl; seg[CK(p.ws.status, ns, E + 1)] = nl; }
     }
     __syncthreads();
     n_split = hdr[0];
@@ -630,7 +636,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     for (int idx = warp; idx < M * GN; idx += nwarps) {
       const int k0 = ent_k[idx];
       if (k0 < 0) continue;
-      const int e = win[idx], si = ent_si[idx];
+      const int e = CK(p.ws.status, win[idx], E), si = ent_si[idx];
       const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
       const int md = mdom[e], n = __popcll(hm), w = orow[e];
       const int bs = w / n, rem = w - bs * n, start = (s + e) % n;
@@ -654,7 +660,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
         const int ex = warp_exclusive_scan(v, lane, &tot);
         if (v > 0) {
           if (si >= 0) {
-            const int pos = k0 + carry_pos + __popc(m2 & lanemask_lt());
+            const int pos = CK(p.ws.status, k0 + carry_pos + __popc(m2 & lanemask_lt()), P);
             cum[pos] = carry_cum + ex + v;
             inst[pos] = pi;
           } else {
@@ -677,7 +683,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   // all go to that instance and the tile ranks nothing for it.
 #pragma unroll 1
   for (int i = tid; i < n_split; i += nt) {
-    const int e = split_e[i];
+    const int e = CK(p.ws.status, split_e[i], E);
     int ex = 0;
 #pragma unroll 1
     for (int t = 0; t < tile; ++t) ex += tc[(size_t)t * E + e];
@@ -685,8 +691,8 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     int lo = 0, res = -1;
 #pragma unroll 1
     for (int k = seg[i]; k < seg[i + 1]; ++k) {
-      const int hi = cum[k];
-      if (ex >= lo && ex + tv <= hi) { res = inst[k]; break; }
+      const int hi = cum[CK(p.ws.status, k, P)];
+      if (ex >= lo && ex + tv <= hi) { res = inst[CK(p.ws.status, k, P)]; break; }
       lo = hi;
     }
     tpre[i] = ex;
@@ -741,7 +747,8 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   while (split_mask) {
     const int k = __ffs(split_mask) - 1;
     split_mask &= split_mask - 1;
-    work[atomicAdd(hdr + 2, 1)] = (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
+    work[CK(p.ws.status, atomicAdd(hdr + 2, 1), kPlan2TileIds)] =
+        (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
   }
   __syncthreads();   // also orders the stores above before the patches below
   const int n_work = hdr[2];
@@ -835,21 +842,22 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
       colv[i] = e < 0 ? 0 : __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
     }
   }
-  if (!fetch_placement(p.ws, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt)) return;
+  if (!fetch_placement(p.ws, E, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt)) return;
   TL_MAX(p.ws, 14);
   if (!plan_is_closed_form(nwin, M, GN, N, p.stage1_slots, p.stage1_lpt)) return;   // solver's job
 
   // my replica columns (every slot is taken): a second, short round of loads
 #pragma unroll 1
   for (int i = tid; i < N * R; i += nt) {
-    const int j = i / R, s = i - j * R, e = win[dm * GN + j * G + g];
+    const int j = i / R, s = i - j * R, e = CK(p.ws.status, win[dm * GN + j * G + g], E);
     colv[(e_loc + j) * R + s] = __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
   }
   // meanwhile: row r of q (r as a source) and of the dispatch counts
 #pragma unroll 1
   for (int pi = tid; pi < P; pi += nt) {
     const int rr = pi / s_phys, l = pi - rr * s_phys, dd = rr / G;
-    const int e = l < e_loc ? mie[rr * e_loc + l] : win[dd * GN + (l - e_loc) * G + (rr - dd * G)];
+    const int e0 = l < e_loc ? mie[rr * e_loc + l] : win[dd * GN + (l - e_loc) * G + (rr - dd * G)];
+    const int e = e0 < 0 ? -1 : CK(p.ws.status, e0, E);
     int v = 0;
     if (e >= 0) v = closed_q(orow[e], ((unsigned long long)hm_hi[e] << 32) | hm_lo[e], dd, dm, r, e);
     qrow[pi] = v;
@@ -872,8 +880,9 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
 #pragma unroll 1
   for (int i = tid; i < s_phys * R; i += nt) {
     const int l = i / R, s = i - l * R;
-    const int e = l < e_loc ? mie[r * e_loc + l] : win[dm * GN + (l - e_loc) * G + g];
-    if (e < 0) continue;
+    const int e0 = l < e_loc ? mie[r * e_loc + l] : win[dm * GN + (l - e_loc) * G + g];
+    if (e0 < 0) continue;
+    const int e = CK(p.ws.status, e0, E);
     const int v = closed_q(colv[i], ((unsigned long long)hm_hi[e] << 32) | hm_lo[e], dm, s / G, s, e);
     if (v != 0) { atomicAdd(&U[l], v); atomicAdd(&ccol[s], v); }
   }

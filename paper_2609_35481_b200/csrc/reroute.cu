@@ -172,7 +172,8 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   while (split_mask) {   // ~3% of the ids on the benchmark workloads
     const int k = __ffs(split_mask) - 1;
     split_mask &= split_mask - 1;
-    work[atomicAdd(hdr + 2, 1)] = (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
+    work[CK(p.ws.status, atomicAdd(hdr + 2, 1), p.tile_ids)] =
+        (unsigned short)(4 * ((k >> 2) * nt + tid) + (k & 3));
   }
   __syncthreads();   // also orders the stores above before the patches below
   const int n_work = hdr[2];

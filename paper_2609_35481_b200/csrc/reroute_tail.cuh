@@ -55,7 +55,7 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
     // every item bumps the 4-bit counter of its (split expert, row, lane)
 #pragma unroll 1
     for (int w = tid; w < c.n_work; w += nt) {
-      const int pos = c.work[w];
+      const int pos = CK(c.status, c.work[w], rows * 128);
       const int i = -2 - c.route[__ldg(c.ids + pos)] - p0;
       if (i < 0 || i >= n_here) continue;
       const int vec = pos >> 2;                            // int4 index inside the tile
@@ -84,7 +84,7 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
     sync();
 #pragma unroll 1
     for (int w = tid; w < c.n_work; w += nt) {
-      const int pos = c.work[w], vec = pos >> 2;
+      const int pos = CK(c.status, c.work[w], rows * 128), vec = pos >> 2;
       const int e = __ldg(c.ids + pos);
       const int i = -2 - c.route[e] - p0;
       if (i < 0 || i >= n_here) continue;
@@ -103,6 +103,7 @@ __device__ __forceinline__ void rank_and_patch(const SplitCtx& c, int tid, int n
       int at = c.seg[p0 + i];
       const int end = c.seg[p0 + i + 1] - 1;
       while (at < end && rho >= c.cum[at]) ++at;
+      at = CK(c.status, at, c.n_list);
       broken |= rho >= c.cum[at];
       c.out[pos] = c.inst[at];
     }

@@ -193,15 +193,15 @@ __global__ void __launch_bounds__(kRouteThreads) route_kernel(const RouteParams 
       if (v > 0) {
         const bool after_main = qm > 0 && rmain < r;
         const int pos = carry_pos + __popc(m & lanemask_lt()) + (after_main ? 1 : 0);
-        cum_s[base + pos] = carry_cum + ex + v + (after_main ? qm : 0);
-        inst_s[base + pos] = pi;
+        cum_s[CK(p.ws.status, base + pos, P)] = carry_cum + ex + v + (after_main ? qm : 0);
+        inst_s[CK(p.ws.status, base + pos, P)] = pi;
       }
       carry_pos += __popc(m);
       carry_cum += tot;
     }
     if (lane == 0 && qm > 0) {
-      cum_s[base + main_pos] = main_below + qm;
-      inst_s[base + main_pos] = ml[e];
+      cum_s[CK(p.ws.status, base + main_pos, P)] = main_below + qm;
+      inst_s[CK(p.ws.status, base + main_pos, P)] = ml[e];
     }
     __syncwarp();
     const int n_e = nz[e];

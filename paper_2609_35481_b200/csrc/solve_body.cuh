@@ -453,11 +453,11 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
         if (lane == 0) atomicOr(p.ws.status, TOPOEP_FLAG_REFINE_CAP);
         break;
       }
-      const int e = (int)((mk >> 5) & 0x7fffffu), wt = (int)(mk & 31u);
-      const int cb = hostcol[gb * E + e];
+      const int e = CK(p.ws.status, (int)((mk >> 5) & 0x7fffffu), E), wt = (int)(mk & 31u);
+      const int cb = CK(p.ws.status, hostcol[gb * E + e], C);
       int ct = hostcol[wt * E + e];
       if (ct < 0) {   // create the replica in the target's next free slot
-        ct = wt * s_phys + e_loc + __shfl_sync(full, usedreg, wt);
+        ct = CK(p.ws.status, wt * s_phys + e_loc + __shfl_sync(full, usedreg, wt), C);
         if (lane == 0) {
           col_expert[ct] = e;
           col_cr[ct] = col_cr[cb];

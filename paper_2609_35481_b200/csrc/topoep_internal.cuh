@@ -268,6 +268,24 @@ cudaError_t launch_empty(int count, cudaStream_t stream);
 // at once (a single plan), the early trigger lets every later kernel finish its prologue --
 // static tables, the ids of the reroute tiles -- before its predecessor is done (1-2 us more).
 // The histogram never triggers early: the reroute blocks would read the ids at the same time.
+// Bounds-checked build (-DTOPOEP_CHECKED; a second library for the tests, never the product):
+// CK(status, i, n) wraps an index that is derived from DATA -- an expert id read from a record, an
+// instance id, a list position, a work-list entry.  An index outside [0, n) sets
+// TOPOEP_FLAG_INTERNAL in the status word and is clamped into range: nothing traps, nothing
+// faults, and the tests see the flag.  In the normal build CK is the index itself.
+#ifdef TOPOEP_CHECKED
+__device__ __forceinline__ int ck_index(uint32_t* status, long long i, long long n) {
+  if (i < 0 || i >= n) {
+    atomicOr(status, TOPOEP_FLAG_INTERNAL);
+    return (int)(i < 0 || n <= 0 ? 0 : n - 1);
+  }
+  return (int)i;
+}
+#define CK(status, i, n) ck_index((status), (i), (n))
+#else
+#define CK(status, i, n) (i)
+#endif
+
 // Phase stamps for tuning (compiled out unless TOPOEP_TIMELINE is defined): thread 0 of a block
 // folds the global nanosecond timer into slot `slot` of a table behind the status word -- the
 // earliest (TL_MIN) or latest (TL_MAX) block to pass the point.  The host reads the table.
