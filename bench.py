@@ -321,7 +321,7 @@ def measure(w, K, W, rank, world, dev, args, stages=True, chain=-1, warm_l2=Fals
                               s["out"].token_replica, sh)
         assert rc == 0, rc
 
-    kernels_per_plan = 2 if (chain == 2 or (chain != 1 and sets[0]["pl"].plans_with_two_kernels(w.tokens_per_rank, w.batch))) else 5
+    kernels_per_plan = B.topoep_plan_kernels(sets[0]["pl"].handle, w.tokens_per_rank, w.batch)
 
     def floor(i):
         assert B.topoep_launch_floor(kernels_per_plan, sh) == 0
@@ -409,6 +409,8 @@ def main():
     ap.add_argument("--tile-ids", type=int, default=0)
     ap.add_argument("--hist-mode", type=int, default=-1)
     ap.add_argument("--pdl", type=int, default=-1)
+    ap.add_argument("--chain", type=int, default=-1,
+                    help="TOPOEP_KNOB_CHAIN for the timed plan (default: the library's choice)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -438,7 +440,7 @@ def main():
 
     sampler = ClockSampler(local)
     sampler.start()
-    m = measure(w, K, W, rank, world, dev, args)
+    m = measure(w, K, W, rank, world, dev, args, chain=args.chain)
     sets, nsets, l2_policy, stream = m["sets"], m["nsets"], m["l2_policy"], m["stream"]
     ms_step, ms_total, stage_us = m["ms_step"], m["ms_total"], m["stage_us"]
     value = job_throughput(world, w.assignments, K, ms_total)

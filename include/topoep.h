@@ -136,13 +136,17 @@ enum {
                                    histogram, omega, solver, route tables, reroute);
                                    2: two whenever the tables fit shared memory (a
                                    histogram that also sums the routing matrix, then
-                                   one grid of solver blocks and per-token blocks;
-                                   a per-token block builds its source's route
-                                   table itself and, when inter-node placement used
-                                   every slot, does not wait for the solver); 0
+                                   one grid of placement, solver, rank and per-token
+                                   blocks; a per-token block builds its source's
+                                   route table itself and, when inter-node placement
+                                   used every slot, does not wait for the solver);
+                                   3: four whenever the tables fit (histogram, omega,
+                                   the same grid with one route block per source in
+                                   place of the per-token blocks, reroute); 0
                                    (default): two for calls small enough to be
                                    resident on the GPU at once, where latency
-                                   counts, else five                              */
+                                   counts; four for a single plan whose second grid
+                                   is resident at once; else five                 */
   TOPOEP_KNOB_TRANSFER_SELFTEST = 4 /* tests only (the one knob that does change
                                    output): 1 makes one block of the bulk engine
                                    wait for a copy it never issued, so its bounded
@@ -208,8 +212,8 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes);
  * Within a (plan, source, expert) group, assignments are ranked by flat index
  * t*k+j and dealt to the expert's instances in ascending rank order, each
  * taking q(s,e,r) of them.  Equivalent to topoep_histogram, topoep_solve and
- * topoep_reroute in a row: enqueues five kernels on `stream` (two for small
- * calls, see TOPOEP_KNOB_CHAIN); capturable in a CUDA graph.  Two plans on one
+ * topoep_reroute in a row: enqueues five kernels on `stream` (two or four for
+ * smaller calls, see TOPOEP_KNOB_CHAIN); capturable in a CUDA graph.  Two plans on one
  * handle must not overlap on the device.  The stage calls below continue from
  * stage calls: topoep_reroute after a topoep_plan returns TOPOEP_ERR_SIZE.
  */
@@ -425,7 +429,7 @@ int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count);
 
 /*
  * Number of kernels topoep_plan would enqueue for a call of this size with the
- * current knobs: 5, or 2 for a small call (see TOPOEP_KNOB_CHAIN).  Needs the
+ * current knobs: 5, 4 or 2 (see TOPOEP_KNOB_CHAIN).  Needs the
  * workspace (the answer depends on the device).  Negative status on a bad
  * handle or size.  Not part of the method: for benchmarks and tests.
  */

@@ -24,7 +24,8 @@ struct topoep_ctx {
   int transfer_ready, transfer_mode, sms;   // replica executor: configured?, copy engine, SM count
   int transfer_selftest;   // tests only: the bulk engine's bounded wait is made to run out once
   int max_tiles;
-  int chain;           // knob: 0 choose by size, 1 always five kernels, 2 two kernels when they fit
+  int chain;           // knob: 0 choose by size, 1 always five kernels, 2 two kernels when they fit,
+                       //   3 four kernels when they fit
   size_t plan2_smem;   // shared memory the second kernel of the two-kernel chain may use
   bool aux_valid;      // omega_m and demand in the workspace belong to the omega now there
   bool routes_valid;   // route tables in the workspace belong to the tile counts now there
@@ -76,7 +77,7 @@ void carve(topoep_ctx* h) {
   sz[W_SPLIT_REC] = 4 * B * R * (size_t)split_rec_layout(d.E, d.P, h->max_tiles).ints;
   sz[W_ACC_OMEGA0] = sz[W_ACC_OMEGA1] = 4 * B * R * E;
   sz[W_ACC_DEMAND0] = sz[W_ACC_DEMAND1] = 4 * B * (size_t)d.M * E;
-  sz[W_EPOCH] = 16;
+  sz[W_EPOCH] = 32;
   sz[W_DONE] = 4 * B * (size_t)d.M;
   sz[W_PLACE_REC] = 8 * B * (size_t)d.M * ((size_t)d.G * d.N + 1);
   size_t at = 0;
@@ -148,6 +149,7 @@ OmegaParams make_omega(topoep_ctx* h, const int32_t* src, int32_t* out_omega, in
   op.epw = 32 / gpad;
   op.rank_first = 0;
   op.rank_count = h->d.R;
+  op.bump_serial = 0;
   return op;
 }
 
@@ -355,7 +357,7 @@ fail:
 namespace {
 
 int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* out_omega,
-                 cudaStream_t stream, bool two = false) {
+                 cudaStream_t stream, bool two = false, bool four = false) {
   HistParams hp = make_hist(h, ids, T, out_omega);
   if (two) {   // the second kernel of the two-kernel chain has one block shape: its tile size
     hp.tile_ids = kPlan2TileIds;
@@ -370,6 +372,10 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
   if (e == cudaSuccess && !two) {
     OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles, batch);
+    op.bump_serial = four ? 1 : 0;   // the combined kernel follows: a new serial for its records
+    // ... and its blocks (few: the call is a single mid-size plan) may become resident while this
+    // small kernel runs, to fetch their static tables
+    if (four) op.pdl = h->pdl != 0 ? 2 : 0;
     if (h->rank_count != h->d.R) {
       // a window of ranks: plain tile sums, rank by rank; the demand and the transposed copy need
       // every rank's row and are derived later, from the gathered matrix handed to topoep_solve
@@ -396,6 +402,7 @@ SolveParams make_solve(topoep_ctx* h, int batch, int32_t* replica_map, int32_t* 
   sp.ws = h->ws;
   sp.pdl = chain_pdl(h, batch);
   sp.acc = 0;
+  sp.fused = 0;
   sp.max_iters = h->max_iters;
   sp.min_delta = h->min_delta;
   // 2 D S_tok - ||W|| > 0  <=>  D > floor(||W|| / (2 S_tok)); S_tok = 0 admits no candidate
@@ -470,17 +477,21 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   return TOPOEP_OK;
 }
 
-// Second kernel of the two-kernel chain: solver blocks and per-token blocks in one grid.
+// The combined kernel: placement, solver and rank blocks in one grid, and either the per-token
+// blocks (two-kernel chain: the accumulating histogram in front) or one route block per source
+// (four-kernel chain: histogram and omega kernels in front, reroute kernel behind).
 int enqueue_plan2(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* replica_map,
                   int32_t* token_replica, int32_t* counts, int32_t* offsets, int32_t* inst_counts,
-                  cudaStream_t stream) {
+                  bool route_only, cudaStream_t stream) {
   SolveParams sp = make_solve(h, batch, replica_map, counts, offsets, inst_counts);
   sp.pdl = h->pdl != 0;
-  sp.acc = 1;
+  sp.acc = route_only ? 0 : 1;
+  sp.fused = 1;
   TailParams tp;
   tp.d = h->d;
   tp.ws = h->ws;
   tp.pdl = h->pdl != 0;
+  tp.acc = sp.acc;
   tp.stage1_lpt = sp.stage1_lpt;
   tp.stage1_slots = sp.stage1_slots;
   tp.cand_thr = sp.cand_thr;
@@ -488,20 +499,21 @@ int enqueue_plan2(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* 
   tp.out_token_replica = token_replica;
   tp.out_offsets = offsets;
   tp.n_ids = T * h->d.k;
-  tp.tile_ids = kPlan2TileIds;
+  tp.tile_ids = h->hist_tile_ids;
   tp.tiles = std::max(1, (tp.n_ids + tp.tile_ids - 1) / tp.tile_ids);
   tp.max_tiles = h->max_tiles;
   tp.vec_ok = (tp.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0) &&
               ((reinterpret_cast<uintptr_t>(token_replica) & 15u) == 0);
-  const cudaError_t e = launch_plan2(sp, tp, batch, stream);
+  const cudaError_t e = launch_plan2(sp, tp, batch, route_only, stream);
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
+  if (route_only) h->routes_valid = true;
   return TOPOEP_OK;
 }
 
 // Which chain plans this call: two kernels when the per-token blocks' tables fit their shared
 // memory and (unless forced) the whole call is resident on the GPU at once.
 bool use_two_kernels(const topoep_ctx* h, int T, int batch) {
-  if (h->chain == 1 || T <= 0 || h->rank_count != h->d.R) return false;
+  if (h->chain == 1 || h->chain == 3 || T <= 0 || h->rank_count != h->d.R) return false;
   const long long n_ids = (long long)T * h->d.k;
   const long long tiles = std::max(1ll, (n_ids + kPlan2TileIds - 1) / kPlan2TileIds);
   if (tiles > h->max_tiles) return false;
@@ -510,6 +522,20 @@ bool use_two_kernels(const topoep_ctx* h, int T, int batch) {
   if (h->chain == 2) return true;
   const long long per_sm = std::max<long long>(1, std::min<long long>(2, (227 * 1024) / (long long)smem));
   return plan2_blocks(h->d, (int)tiles, batch) <= per_sm * h->d.sms;
+}
+
+// Four kernels (histogram, omega, the combined kernel with route blocks, reroute) for the other
+// calls, when the route blocks' tables fit shared memory.
+bool use_four_kernels(const topoep_ctx* h, int T, int batch) {
+  if (h->chain == 1 || h->chain == 2 || T <= 0 || h->rank_count != h->d.R) return false;
+  const long long n_ids = (long long)T * h->d.k;
+  const long long tiles = std::max(1ll, (n_ids + h->tile_ids - 1) / h->tile_ids);
+  if (plan2_route_smem_bytes(h->d, (int)tiles) > h->plan2_smem) return false;
+  if (h->chain == 3) return true;
+  // by size: only while the combined kernel's grid is resident at once (a single mid-size plan:
+  // 62 against 69 us at 128 ranks); with hundreds of plans its blocks cost more than the solver
+  // and route kernels they replace (1142 against 926 us for 232 plans)
+  return (2ll * h->d.M + 2ll * h->d.R) * batch <= 2ll * h->d.sms;
 }
 
 }  // namespace
@@ -572,7 +598,15 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
     rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, true);
     if (rc != TOPOEP_OK) return rc;
     return enqueue_plan2(h, dev_topk_ids, tokens_per_rank, batch, dev_replica_map, dev_token_replica,
-                         dev_dispatch_counts, dev_dispatch_offsets, dev_instance_counts, stream);
+                         dev_dispatch_counts, dev_dispatch_offsets, dev_instance_counts, false, stream);
+  }
+  if (use_four_kernels(h, tokens_per_rank, batch)) {
+    rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, false, true);
+    if (rc != TOPOEP_OK) return rc;
+    rc = enqueue_plan2(h, dev_topk_ids, tokens_per_rank, batch, dev_replica_map, dev_token_replica,
+                       dev_dispatch_counts, dev_dispatch_offsets, dev_instance_counts, true, stream);
+    if (rc != TOPOEP_OK) return rc;
+    return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
   }
   rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream);
   if (rc != TOPOEP_OK) return rc;
@@ -777,7 +811,7 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
       h->transfer_mode = value;
       return TOPOEP_OK;
     case TOPOEP_KNOB_CHAIN:
-      if (value < 0 || value > 2) return TOPOEP_ERR_ARG;
+      if (value < 0 || value > 3) return TOPOEP_ERR_ARG;
       h->chain = value;
       return TOPOEP_OK;
     case TOPOEP_KNOB_TRANSFER_SELFTEST:
@@ -817,7 +851,8 @@ int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count) {
 int topoep_plan_kernels(topoep_handle_t h, int tokens_per_rank, int batch) {
   const int rc = check_sizes(h, tokens_per_rank, batch);
   if (rc != TOPOEP_OK) return rc;
-  return use_two_kernels(h, tokens_per_rank, batch) ? 2 : 5;
+  return use_two_kernels(h, tokens_per_rank, batch) ? 2
+         : use_four_kernels(h, tokens_per_rank, batch) ? 4 : 5;
 }
 
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances) {

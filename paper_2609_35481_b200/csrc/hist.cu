@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
 template <bool VEC>
 __global__ void __launch_bounds__(kPlan2TileIds / kIdsPerThread) hist_acc_kernel(const HistParams p) {
   extern __shared__ int cnt[];   // [E + 1]: the last bin collects ignored ids
-  __shared__ unsigned call_state[3];   // serial of the previous call, plans with sums in pair 0 / 1
+  __shared__ unsigned call_state[4];   // pair serial, plans with sums in pair 0 / 1, plan-call serial
   const int E = p.d.E;
   const int tile = blockIdx.x, s = blockIdx.y, b = blockIdx.z;
   const int nt = blockDim.x, tid = threadIdx.x;
@@ -109,7 +109,8 @@ __global__ void __launch_bounds__(kPlan2TileIds / kIdsPerThread) hist_acc_kernel
     // cleared below, the serial number advances.  Whoever runs after this kernel sees the new
     // values.
     const unsigned ep = __ldcg(p.ws.epoch), d0 = __ldcg(p.ws.epoch + 1), d1 = __ldcg(p.ws.epoch + 2);
-    call_state[0] = ep; call_state[1] = d0; call_state[2] = d1;
+    const unsigned sn = __ldcg(p.ws.epoch + 4);
+    call_state[0] = ep; call_state[1] = d0; call_state[2] = d1; call_state[3] = sn;
     __threadfence();
     checked_in = atomicAdd(p.ws.epoch + 3, 1u);
   }
@@ -158,6 +159,7 @@ __global__ void __launch_bounds__(kPlan2TileIds / kIdsPerThread) hist_acc_kernel
     p.ws.epoch[3] = 0u;
     p.ws.epoch[1 + (ep & 1u)] = gridDim.z;
     p.ws.epoch[1 + ((ep & 1u) ^ 1u)] = 0u;
+    p.ws.epoch[4] = call_state[3] + 1u;
     __threadfence();
     p.ws.epoch[0] = ep + 1u;
   }
@@ -174,6 +176,8 @@ __global__ void __launch_bounds__(128) omega_kernel(const OmegaParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int dm = blockIdx.y, b = blockIdx.z;
   if (p.pdl == 2) pdl_trigger();
+  if (p.bump_serial && (blockIdx.x | blockIdx.y | blockIdx.z | threadIdx.x) == 0)
+    p.ws.epoch[4] = __ldcg(p.ws.epoch + 4) + 1u;   // one writer; read by the kernel after this one
   const int g = lane / epw, e = (blockIdx.x * 4 + warp) * epw + (lane - g * epw);
   const bool on = g < G && e < E;
   const int s = p.rank_first + dm * G + g;   // global source rank
@@ -218,6 +222,8 @@ __global__ void __launch_bounds__(128) omega4_kernel(const OmegaParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int dm = blockIdx.y, b = blockIdx.z;
   if (p.pdl == 2) pdl_trigger();
+  if (p.bump_serial && (blockIdx.x | blockIdx.y | blockIdx.z | threadIdx.x) == 0)
+    p.ws.epoch[4] = __ldcg(p.ws.epoch + 4) + 1u;   // one writer; read by the kernel after this one
   const int g = lane / epw, e = 4 * ((blockIdx.x * 4 + warp) * epw + (lane - g * epw));
   const bool on = g < G && e < E;
   const int s = p.rank_first + dm * G + g;   // global source rank

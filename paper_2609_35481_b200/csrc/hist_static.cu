@@ -111,7 +111,7 @@ extern "C" int topoep_histogram_static(const int32_t* dev_topk_ids, int batch, i
   hp.vec_ok = (n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(dev_topk_ids) & 15u) == 0);
   e = launch_hist(hp, batch, 0, stream);
   if (e == cudaSuccess) {
-    OmegaParams op = {};   // every rank its own "domain": plain tile sums into dev_omega
+    OmegaParams op = {};   // every rank its own "domain": plain tile sums into dev_omega (bump_serial 0)
     op.d.R = ranks;
     op.d.M = ranks;
     op.d.G = 1;

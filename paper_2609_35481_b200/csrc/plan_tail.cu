@@ -129,14 +129,20 @@ __device__ __forceinline__ void place_body(const SolveParams& p, unsigned char* 
   for (int i = tid; i <= GN; i += nt) winl[i] = -1;
   pdl_wait();
   TL_MIN(p.ws, 3);
-  const unsigned serial = __ldcg(p.ws.epoch);
-  const int32_t* dA = p.ws.acc_demand[0] + ((size_t)b * M + dm) * E;
-  const int32_t* dB = p.ws.acc_demand[1] + ((size_t)b * M + dm) * E;
+  const unsigned serial = __ldcg(p.ws.epoch + 4);
+  const size_t drow = ((size_t)b * M + dm) * E;
+  if (p.acc) {   // one accumulator pair holds the sums, the other zeros
+    const int32_t* dA = p.ws.acc_demand[0] + drow;
+    const int32_t* dB = p.ws.acc_demand[1] + drow;
 #pragma unroll 1
-  for (int e = tid; e < E; e += nt) {
-    const int v = __ldcg(dA + e) + __ldcg(dB + e);
-    Dd[e] = v;
-    if (p.ws.demand) p.ws.demand[((size_t)b * M + dm) * E + e] = v;   // kept for inspection
+    for (int e = tid; e < E; e += nt) {
+      const int v = __ldcg(dA + e) + __ldcg(dB + e);
+      Dd[e] = v;
+      p.ws.demand[drow + e] = v;   // kept for inspection
+    }
+  } else {       // the omega kernel left the demand in the workspace
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) Dd[e] = __ldcg(p.ws.demand + drow + e);
   }
   __syncthreads();
   TL_MAX(p.ws, 4);
@@ -302,7 +308,7 @@ struct TailLayout {
   size_t cnt, base, work;      // the ranking tail's counters, bases and work list
   size_t route, hdr, seg, cum, inst, tbase, tpre;
   size_t rm, qrow, mr, ml, orow, hm_lo, hm_hi, win, nwin, nz, single, sidx, seg_e, crow,
-      split_e, warp_tot, mdom, slot_p, slot_dd, tc;
+      split_e, warp_tot, mdom, slot_p, slot_dd, chunk_ns, chunk_nl, tc;
   size_t total;
 };
 
@@ -342,6 +348,8 @@ __host__ __device__ inline TailLayout tail_layout(const Dims& d, int tiles) {
   o.mdom = ints(d.E);
   o.slot_p = ints(RN + 1);
   o.slot_dd = ints(RN + 1);
+  o.chunk_ns = ints(RN / 32 + 2);
+  o.chunk_nl = ints(RN / 32 + 2);
   o.tc = at;   // per-tile counts of the row, 16 bits each: [tiles][E]
   at += (sizeof(unsigned short) * (size_t)tiles * d.E + 15) & ~(size_t)15;
   o.total = at;
@@ -476,7 +484,10 @@ __device__ __forceinline__ void slow_route(const TailParams& p, const TailSm& t,
   __syncthreads();
 }
 
-template <bool VEC>
+// ROUTE_ONLY: a route block of the four-kernel chain -- one per (plan, source): it builds the
+// same routing table, for every tile of the row, and writes it in the form reroute_kernel reads
+// (the role of route_kernel); `tile` is the row's last tile then.
+template <bool VEC, bool ROUTE_ONLY>
 __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* smem, int tile, int s,
                                           int b) {
   const Dims d = p.d;
@@ -515,6 +526,8 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   int* mdom = reinterpret_cast<int*>(smem + lay.mdom);       // [E]   main domain
   int* slot_p = reinterpret_cast<int*>(smem + lay.slot_p);   // [M*GN] instance of a winner's slot
   int* slot_dd = reinterpret_cast<int*>(smem + lay.slot_dd); // [M*GN] its domain
+  int* chunk_ns = reinterpret_cast<int*>(smem + lay.chunk_ns);   // split experts per 32 winners
+  int* chunk_nl = reinterpret_cast<int*>(smem + lay.chunk_nl);   // list entries per 32 winners
   unsigned short* tc = reinterpret_cast<unsigned short*>(smem + lay.tc);   // [tiles][E]
 
   const TailSm t = {route, hdr, seg, cum, inst, rm, qrow, mr, ml, nz, single, sidx, seg_e, crow,
@@ -530,8 +543,10 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   // ---- before the histogram kernel is known to be complete: the ids (nobody's output) and the
   // handle's static tables
   int4 x[kIdsPerThread / 4];
+  if (!ROUTE_ONLY) {
 #pragma unroll
-  for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+    for (int j = 0; j < kIdsPerThread / 4; ++j) x[j] = load_ids4(ids, j * nt + tid, count, VEC);
+  }
 #pragma unroll 1
   for (int e = tid; e < E; e += nt) {
     const int md = __ldg(p.ws.main_dom + e), mi = __ldg(p.ws.main_inst + e);
@@ -552,6 +567,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   if (tid == 0) {
     route[E] = -1;          // every id outside [0,E) is clamped onto this entry
     hdr[0] = 0; hdr[1] = 0; hdr[2] = 0; hdr[3] = 0;
+    seg[0] = 0;
   }
   static_assert(kSplitCap % 8 == 0, "counter words per thread");
 #pragma unroll
@@ -561,7 +577,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
   // ---- one round of loads of what the histogram kernel wrote (read past L1): the row's tile
   // counts and row s of the routing matrix -- one accumulator pair holds the sums, the other
   // zeros, so the two are added -- and the first poll of the placement records
-  const unsigned serial = __ldcg(p.ws.epoch);   // of this call: the histogram kernel advanced it
+  const unsigned serial = __ldcg(p.ws.epoch + 4);   // of this call: the histogram kernel advanced it
   {
     const unsigned short* src =
         reinterpret_cast<const unsigned short*>(p.ws.tile_cnt) + row * (size_t)p.max_tiles * E;
@@ -573,10 +589,15 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
 #pragma unroll 1
       for (int i = tid; i < n16; i += nt) tc[i] = __ldcg(src + i);
     }
-    const int32_t* oA = p.ws.acc_omega[0] + row * E;
-    const int32_t* oB = p.ws.acc_omega[1] + row * E;
+    if (p.acc) {
+      const int32_t* oA = p.ws.acc_omega[0] + row * E;
+      const int32_t* oB = p.ws.acc_omega[1] + row * E;
 #pragma unroll 1
-    for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
+      for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + e) + __ldcg(oB + e);
+    } else {
+#pragma unroll 1
+      for (int e = tid; e < E; e += nt) orow[e] = __ldcg(p.ws.omega + row * E + e);
+    }
   }
   const bool have_placement =
       fetch_placement(p.ws, E, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt);
@@ -595,17 +616,19 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     // replica domain stands for it.  Then every warp takes such an entry, a lane per instance.
     int* ent_k = rm;      // [M*GN] list start of the entry's expert (split), or -1: nothing to do
     int* ent_si = qrow;   // [M*GN] its split index, or -1: a single unit, one instance gets it
-    if (warp == 0) {
-      int ns = 0, nl = 0;   // split experts and list entries so far (warp-uniform)
+    // (32 winners per warp step; with more than 32 winners a first pass counts the split experts
+    // and list entries of every step, so that all warps can take steps in the second pass)
+    const int chunks = (M * GN + 31) >> 5;
 #pragma unroll 1
-      for (int i0 = 0; i0 < M * GN; i0 += 32) {
-        const int idx = i0 + lane;
+    for (int pass = chunks > 1 ? 0 : 1; pass < 2; ++pass) {
+#pragma unroll 1
+      for (int c = warp; c < chunks; c += nwarps) {
+        const int idx = c * 32 + lane;
         const bool valid = idx < M * GN;
         const int dd = valid ? slot_dd[idx] : 0;
         const int e = valid ? CK(p.ws.status, win[idx], E) : 0;
         const unsigned long long hm = ((unsigned long long)hm_hi[e] << 32) | hm_lo[e];
         const int md = mdom[e], n = __popcll(hm), w = orow[e];
-        if (valid && dd == ds) route[e] = slot_p[idx];
         // first replica domain of e = lowest hosting domain that is not its main's
         const bool first = valid && !((hm >> ds) & 1ull) &&
                            __ffsll((long long)(hm & ~(1ull << md))) - 1 == dd;
@@ -614,7 +637,19 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
         const unsigned sm = __ballot_sync(full, split);
         int ltot;
         const int lpre = warp_exclusive_scan(split ? nzv : 0, lane, &ltot);
+        if (pass == 0) {
+          if (lane == 0) { chunk_ns[c] = __popc(sm); chunk_nl[c] = ltot; }
+          continue;
+        }
+        int ns = 0, nl = 0;   // split experts and list entries of the earlier steps
+        if (chunks > 1) {
+#pragma unroll 1
+          for (int u = lane; u < c; u += 32) { ns += chunk_ns[u]; nl += chunk_nl[u]; }
+          ns = __reduce_add_sync(full, ns);
+          nl = __reduce_add_sync(full, nl);
+        }
         if (valid) {
+          if (dd == ds) route[e] = slot_p[idx];
           const int si = ns + __popc(sm & lanemask_lt());
           ent_k[idx] = nzv >= 1 ? nl + lpre : -1;
           ent_si[idx] = split ? si : -1;
@@ -624,12 +659,14 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
             split_e[CK(p.ws.status, si, E)] = e;
           }
         }
-        ns += __popc(sm);
-        nl += ltot;
+        if (c == chunks - 1 && lane == 0) {
+          hdr[0] = ns + __popc(sm);
+          hdr[1] = nl + ltot;
+          seg[CK(p.ws.status, ns + __popc(sm), E + 1)] = nl + ltot;
+        }
       }
-      if (lane == 0) { hdr[0] = ns; hdr[1] = nl; seg[CK(p.ws.status, ns, E + 1)] = nl; }
+      __syncthreads();
     }
-    __syncthreads();
     n_split = hdr[0];
     n_list = hdr[1];
 #pragma unroll 1
@@ -673,11 +710,77 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     }
     __syncthreads();
   } else {
-    slow_route(p, t, tile, s, b, serial);
+    slow_route(p, t, ROUTE_ONLY ? 0 : tile, s, b, serial);
     n_split = hdr[0];
     n_list = hdr[1];
   }
   TL_MAX(p.ws, 9);
+  if (ROUTE_ONLY) {
+    // ---- write the tables in the layout reroute_kernel reads: route[e]; the split record (header,
+    // list starts, cumulative quotas, instances); per tile and split expert the prefix over the
+    // earlier tiles, and for the first kSplitCap split experts also the resolved instance
+    const SplitRec rl = split_rec_layout(E, P, p.max_tiles);
+    int32_t* rec = p.ws.split_rec + row * (size_t)rl.ints;
+    int32_t* g_route = p.ws.route + row * E;
+#pragma unroll 1
+    for (int e = tid; e < E; e += nt) g_route[e] = route[e];
+#pragma unroll 1
+    for (int i = tid; i <= n_split; i += nt) rec[rl.seg + i] = seg[i];
+#pragma unroll 1
+    for (int k = tid; k < n_list; k += nt) {
+      rec[rl.cum + k] = cum[k];
+      rec[rl.inst + k] = inst[k];
+    }
+    if (tid == 0) { rec[0] = n_split; rec[1] = n_list; rec[2] = 0; rec[3] = 0; }
+    const size_t trow = row * (size_t)p.max_tiles * E;
+    const int tiles = p.tiles;
+#pragma unroll 1
+    for (int i = warp; i < n_split; i += nwarps) {   // a warp per split expert, a lane per tile
+      const int e = CK(p.ws.status, split_e[i], E);
+      int carry = 0;
+#pragma unroll 1
+      for (int t0 = 0; t0 < tiles; t0 += 32) {
+        const int tl = t0 + lane;
+        const int tv = tl < tiles ? tc[(size_t)tl * E + e] : 0;
+        int tot;
+        const int ex = carry + warp_exclusive_scan(tv, lane, &tot);
+        carry += tot;
+        if (tl < tiles) {
+          p.ws.tile_pref[trow + (size_t)tl * E + i] = ex;
+          if (i < kSplitCap) {
+            int lo = 0, res = -1;
+#pragma unroll 1
+            for (int k = seg[i]; k < seg[i + 1]; ++k) {
+              const int hi = cum[CK(p.ws.status, k, P)];
+              if (ex >= lo && ex + tv <= hi) { res = inst[CK(p.ws.status, k, P)]; break; }
+              lo = hi;
+            }
+            int32_t* t3 = rec + rl.tp + tl * 3 * kSplitCap + i;
+            t3[0] = ex;
+            t3[kSplitCap] = res;
+            t3[2 * kSplitCap] = e;
+          }
+        }
+      }
+    }
+    if (!closed) {
+      // send offsets of source s (the rank block of s writes them when the plan is closed-form)
+      if (warp == 0) {
+        int32_t* send = p.out_offsets + (((size_t)b * 2 + 0) * R + s) * (R + 1);
+        const int ch = (R + 31) / 32;
+        const int i0 = min(R, lane * ch), i1 = min(R, i0 + ch);
+        int sum = 0;
+#pragma unroll 1
+        for (int r = i0; r < i1; ++r) sum += crow[r];
+        int total;
+        int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
+        for (int r = i0; r < i1; ++r) { send[r] = pre; pre += crow[r]; }
+        if (lane == 0) send[R] = total;
+      }
+    }
+    return;
+  }
   // Cross-tile base of every split expert's stable rank, and the resolved tiles: when the ids of
   // the expert in this tile occupy ranks [ex, ex + tv) inside ONE instance's quota interval, they
   // all go to that instance and the tile ranks nothing for it.
@@ -699,7 +802,7 @@ __device__ __forceinline__ void tail_body(const TailParams& p, unsigned char* sm
     if (i < kSplitCap) tbase[i] = ex;
     if (res >= 0) route[e] = res;
   }
-  if (tile == 0 && !closed) {
+  if ((ROUTE_ONLY || tile == 0) && !closed) {
     // (the rank block of s writes these when the plan is closed-form)
     // row s of the routing matrix, kept for inspection and the summaries
 #pragma unroll 1
@@ -829,17 +932,21 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
   if (tid < s_phys) U[tid] = 0;
   __syncthreads();
   pdl_wait();
-  const unsigned serial = __ldcg(p.ws.epoch);
-  const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E;
+  const unsigned serial = __ldcg(p.ws.epoch + 4);
+  // the routing matrix of plan b: the sum of the two accumulator pairs (one holds the sums, the
+  // other zeros), or the matrix the omega kernel left in the workspace
+  const int32_t* oA = (p.acc ? p.ws.acc_omega[0] : p.ws.omega) + (size_t)b * R * E;
   const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E;
+  const bool two = p.acc != 0;
+  auto om = [&](size_t at) { return two ? __ldcg(oA + at) + __ldcg(oB + at) : __ldcg(oA + at); };
   {
 #pragma unroll 1
-    for (int e = tid; e < E; e += nt) orow[e] = __ldcg(oA + (size_t)r * E + e) + __ldcg(oB + (size_t)r * E + e);
+    for (int e = tid; e < E; e += nt) orow[e] = om((size_t)r * E + e);
     // my main columns: omega[s][e] for every source s
 #pragma unroll 1
     for (int i = tid; i < e_loc * R; i += nt) {
       const int l = i / R, s = i - l * R, e = mie[r * e_loc + l];
-      colv[i] = e < 0 ? 0 : __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
+      colv[i] = e < 0 ? 0 : om((size_t)s * E + e);
     }
   }
   if (!fetch_placement(p.ws, E, b, serial, M, GN, win, nwin, slot_dd, hm_lo, hm_hi, tid, nt)) return;
@@ -850,7 +957,7 @@ __device__ __forceinline__ void rank_body(const SolveParams& p, unsigned char* s
 #pragma unroll 1
   for (int i = tid; i < N * R; i += nt) {
     const int j = i / R, s = i - j * R, e = CK(p.ws.status, win[dm * GN + j * G + g], E);
-    colv[(e_loc + j) * R + s] = __ldcg(oA + (size_t)s * E + e) + __ldcg(oB + (size_t)s * E + e);
+    colv[(e_loc + j) * R + s] = om((size_t)s * E + e);
   }
   // meanwhile: row r of q (r as a source) and of the dispatch counts
 #pragma unroll 1
@@ -941,10 +1048,11 @@ struct Plan2Params {
   TailParams tp;
   int n_solve;   // blocks [0, n_solve): placement, (plan i / M, domain i % M); the next n_solve
                  // blocks: solver, same numbering
-  int n_rank;    // the next n_rank blocks: rank blocks, (plan i / R, rank i % R); then per-token
+  int n_rank;    // then the per-token blocks (two-kernel chain) or n_rank route blocks (four-kernel
+                 // chain); the LAST n_rank blocks: rank blocks, (plan i / R, rank i % R)
 };
 
-template <bool LPT, bool VEC>
+template <bool LPT, bool VEC, bool ROUTE_ONLY>
 __global__ void __launch_bounds__(kSolveThreads, 2) plan2_kernel(const Plan2Params p) {
   extern __shared__ __align__(16) unsigned char smem[];
   int i = blockIdx.x;
@@ -958,13 +1066,17 @@ __global__ void __launch_bounds__(kSolveThreads, 2) plan2_kernel(const Plan2Para
     return;
   }
   i -= p.n_solve;
-  if (i < p.n_rank) {
+  // The blocks on the critical path come next (blocks start in index order, a few dozen per
+  // microsecond when they are this large); the rank blocks, which nobody waits for, come last.
+  const int n_front = (int)gridDim.x - 2 * p.n_solve - p.n_rank;
+  if (i >= n_front) {
+    i -= n_front;
     if (!LPT) rank_body(p.sp, smem, i % p.sp.d.R, i / p.sp.d.R);
     return;
   }
-  i -= p.n_rank;
   const int tiles = p.tp.tiles, R = p.tp.d.R;
-  tail_body<VEC>(p.tp, smem, i % tiles, (i / tiles) % R, i / (tiles * R));
+  if (ROUTE_ONLY) tail_body<VEC, true>(p.tp, smem, tiles - 1, i % R, i / R);
+  else tail_body<VEC, false>(p.tp, smem, i % tiles, (i / tiles) % R, i / (tiles * R));
 }
 
 }  // namespace
@@ -974,33 +1086,45 @@ size_t plan2_smem_bytes(const Dims& d, int tiles) {
                   std::max(solve_smem_bytes(d), place_layout(d).total));
 }
 
+size_t plan2_route_smem_bytes(const Dims& d, int tiles) { return plan2_smem_bytes(d, tiles); }
+
 long long plan2_blocks(const Dims& d, int tiles, int batch) {
   return (2ll * d.M + d.R + (long long)tiles * d.R) * batch;
 }
 
-cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream) {
+cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, bool route_only,
+                         cudaStream_t stream) {
   Plan2Params p;
   p.sp = sp;
   p.tp = tp;
   p.n_solve = sp.d.M * batch;
   p.n_rank = sp.d.R * batch;
-  const dim3 grid((unsigned)plan2_blocks(sp.d, tp.tiles, batch)), block(kSolveThreads);
+  const long long blocks = route_only ? (2ll * sp.d.M + 2ll * sp.d.R) * batch
+                                      : plan2_blocks(sp.d, tp.tiles, batch);
+  const dim3 grid((unsigned)blocks), block(kSolveThreads);
   const size_t smem = plan2_smem_bytes(tp.d, tp.tiles);
   const bool pdl = tp.pdl != 0;
+  if (route_only) {   // no ids in these blocks: the VEC variants differ by nothing they run
+    return sp.stage1_lpt ? launch_kernel(plan2_kernel<true, false, true>, grid, block, smem, stream, pdl, p)
+                         : launch_kernel(plan2_kernel<false, false, true>, grid, block, smem, stream, pdl, p);
+  }
   if (sp.stage1_lpt)
-    return tp.vec_ok ? launch_kernel(plan2_kernel<true, true>, grid, block, smem, stream, pdl, p)
-                     : launch_kernel(plan2_kernel<true, false>, grid, block, smem, stream, pdl, p);
-  return tp.vec_ok ? launch_kernel(plan2_kernel<false, true>, grid, block, smem, stream, pdl, p)
-                   : launch_kernel(plan2_kernel<false, false>, grid, block, smem, stream, pdl, p);
+    return tp.vec_ok ? launch_kernel(plan2_kernel<true, true, false>, grid, block, smem, stream, pdl, p)
+                     : launch_kernel(plan2_kernel<true, false, false>, grid, block, smem, stream, pdl, p);
+  return tp.vec_ok ? launch_kernel(plan2_kernel<false, true, false>, grid, block, smem, stream, pdl, p)
+                   : launch_kernel(plan2_kernel<false, false, false>, grid, block, smem, stream, pdl, p);
 }
 
 cudaError_t configure_plan2(size_t smem) {
   cudaError_t e;
   const int n = (int)smem;
-  if ((e = cudaFuncSetAttribute(plan2_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, n)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(plan2_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(plan2_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, n)) != cudaSuccess) return e;
-  return cudaFuncSetAttribute(plan2_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, n);
+  const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<true, true, false>, attr, n)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<true, false, false>, attr, n)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<false, true, false>, attr, n)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<false, false, false>, attr, n)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(plan2_kernel<true, false, true>, attr, n)) != cudaSuccess) return e;
+  return cudaFuncSetAttribute(plan2_kernel<false, false, true>, attr, n);
 }
 
 }  // namespace topoep

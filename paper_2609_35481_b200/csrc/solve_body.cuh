@@ -299,7 +299,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   // cannot act (a move needs a target with a free slot) and the whole plan follows in closed form
   // from the routing matrix and this placement.  The rank blocks of the grid produce it then,
   // spread over R blocks instead of M, and this block has nothing left to do.
-  if (p.acc && !LPT) {
+  if (p.fused && !LPT) {
     bool closed = true;
     if (N > 0) {
       if (M == 1 || p.stage1_slots != N) closed = false;
@@ -556,12 +556,12 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   // Two-kernel chain: tell the per-token blocks of this grid that wait for the refinement that
   // this domain's results are in memory (the serial number of the call is the flag value, so the
   // flags never need clearing).
-  if (p.acc) {
+  if (p.fused) {
     __threadfence();
     __syncthreads();
     TL_MAX(p.ws, 16);
     if (tid == 0) {
-      const unsigned serial = __ldcg(p.ws.epoch);
+      const unsigned serial = __ldcg(p.ws.epoch + 4);
       asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.ws.done_flags + (size_t)b * M + dm),
                    "r"(serial)
                    : "memory");

@@ -69,9 +69,11 @@ struct Workspace {
   // the other only zeros: readers add the two and need not know which is which.
   int32_t* acc_omega[2];            // [max_batch][R][E] each
   int32_t* acc_demand[2];           // [max_batch][M][E] each
-  unsigned* epoch;                  // [0] calls so far (the serial number of the running call once
-                                    //   its histogram kernel is complete); [1], [2] plans with
-                                    //   sums in pair 0, 1; [3] histogram blocks that have started
+  unsigned* epoch;                  // [0] calls of the accumulating histogram so far (its parity
+                                    //   names the pair in use); [1], [2] plans with sums in pair
+                                    //   0, 1; [3] histogram blocks that have started; [4] serial
+                                    //   number of the running plan call, advanced by the kernel in
+                                    //   front of the combined kernel: the tag of records and flags
   unsigned* done_flags;             // [max_batch][M] serial of the last call whose solver block
                                     //   (plan, domain) has finished
   unsigned long long* place_rec;    // [max_batch][M][G*N + 1] inter-node placement of (plan,
@@ -127,6 +129,8 @@ struct OmegaParams {
   Workspace ws;
   int pdl;   // launched with programmatic dependent launch
   int rank_first, rank_count;   // window of source ranks the caller's id buffers cover
+  int bump_serial;            // advance the plan-call serial (this kernel runs in front of the
+                              //   combined kernel of the four-kernel chain)
   const int32_t* src_omega;   // given routing matrix [B][R][E], or NULL: sum the tile counts
   int32_t* out_omega;         // optional caller copy of omega [B][R][E]
   int tiles, max_tiles;
@@ -146,7 +150,9 @@ struct SolveParams {
   int32_t* out_counts;        // [B][R][R]
   int32_t* out_offsets;       // [B][2][R][R+1]
   int32_t* out_inst_counts;   // [B][P] or NULL
-  int acc;            // two-kernel chain: demand and columns come from the accumulators
+  int acc;            // demand and columns come from the accumulators (two-kernel chain)
+  int fused;          // the block runs inside the combined kernel: it returns at once when the
+                      //   plan is closed-form, and publishes a flag when it is done
 };
 
 // Per-token blocks of the second kernel of the two-kernel chain: per tile, the source's routing
@@ -161,6 +167,8 @@ struct TailParams {
   int32_t* out_offsets;       // [B][2][R][R+1]: the send half is written here
   int n_ids, tiles, max_tiles, tile_ids;
   int vec_ok;
+  int acc;         // row s of the routing matrix comes from the accumulators (two-kernel chain),
+                   //   else from the matrix the omega kernel left in the workspace
 };
 
 struct RouteParams {
@@ -230,9 +238,13 @@ size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 // second kernel of the two-kernel chain: solver blocks first, per-token blocks after them
 constexpr int kPlan2TileIds = kSolveThreads * kIdsPerThread;   // one block shape for both roles
 size_t plan2_smem_bytes(const Dims& d, int tiles);
-long long plan2_blocks(const Dims& d, int tiles, int batch);   // blocks of its grid
+long long plan2_blocks(const Dims& d, int tiles, int batch);   // blocks of its grid (two-kernel chain)
 cudaError_t configure_plan2(size_t smem);
-cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, cudaStream_t stream);
+// route_only: per-source route blocks that write the tables reroute_kernel reads (four-kernel
+// chain) in place of the per-token blocks (two-kernel chain)
+cudaError_t launch_plan2(const SolveParams& sp, const TailParams& tp, int batch, bool route_only,
+                         cudaStream_t stream);
+size_t plan2_route_smem_bytes(const Dims& d, int tiles);
 size_t pos_rank_smem_bytes(const Dims& d, int tile_ids);
 size_t pos_prefix_smem_bytes(const Dims& d);
 

@@ -47,7 +47,7 @@ def main():
         ids = wl.make_topk_ids(w, seed=17, batch=batch).copy()
         ids[0, 0, :1, :] = -1                     # some padding
         ref = orc.plan(oracle_config(w), ids)
-        for chain in (1, 2):
+        for chain in (1, 2, 3):
             pl = make_planner(w, max_batch=batch)
             pl.set_tuning(B.KNOB_CHAIN, chain)
             for rep in range(2):

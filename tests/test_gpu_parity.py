@@ -197,7 +197,7 @@ def test_random_problems_with_policies_tunings_and_skew():
         pl.set_policy(B.POLICY_STAGE1_RANK, lpt)
         pl.set_tuning(B.KNOB_TILE_IDS, int(rng.choice([1024, 2048, 4096, 8192])))
         pl.set_tuning(B.KNOB_PDL, int(rng.integers(0, 4)))
-        pl.set_tuning(B.KNOB_CHAIN, int(rng.integers(0, 3)))
+        pl.set_tuning(B.KNOB_CHAIN, int(rng.integers(0, 4)))
         gpu = run_gpu(pl, ids)
         ref = orc.plan(oracle_config(w, reserve_slots=reserve, stage1_rank=lpt, **over), ids)
         try:
@@ -264,17 +264,19 @@ CHAIN_CASES = [
 
 
 @pytest.mark.parametrize("name,over,batch", CHAIN_CASES)
-def test_two_kernel_chain_equals_five_kernel_chain_and_the_oracle(name, over, batch):
-    """topoep_plan has two kernel chains (TOPOEP_KNOB_CHAIN): five kernels, or -- for small calls --
-    an accumulating histogram followed by one grid of placement, solver, rank and per-token blocks.
-    Both must give the oracle's plan bit for bit, call after call on one handle (the accumulators
-    of the second chain alternate between two pairs and clean up after themselves), also when the
-    chains alternate and when the batch size changes between calls."""
+def test_kernel_chains_agree_with_one_another_and_the_oracle(name, over, batch):
+    """topoep_plan has three kernel chains (TOPOEP_KNOB_CHAIN): five kernels; for small calls an
+    accumulating histogram followed by one grid of placement, solver, rank and per-token blocks;
+    for a single mid-size plan histogram, omega, the same grid with route blocks in place of the
+    per-token blocks, and the reroute kernel.  All must give the oracle's plan bit for bit, call
+    after call on one handle (the accumulators of the second chain alternate between two pairs and
+    clean up after themselves; records and flags are told apart by the call's serial number), also
+    when the chains alternate and when the batch size changes between calls."""
     w = wl.CONFIGS[name].replace(**over)
     ids = wl.make_topk_ids(w, seed=91, batch=batch)
     ref = orc.plan(oracle_config(w), ids)
     pl = make_planner(w, max_batch=batch)
-    for chain in (2, 2, 1, 2, 0, 2):
+    for chain in (2, 2, 1, 3, 2, 0, 3, 3, 2):
         pl.set_tuning(B.KNOB_CHAIN, chain)
         gpu = run_gpu(pl, ids)
         assert_same(gpu, ref)
@@ -285,6 +287,7 @@ def test_two_kernel_chain_equals_five_kernel_chain_and_the_oracle(name, over, ba
         for part, want in ((ids[:1], one), (ids, ref), (ids[:1], one), (ids[:1], one), (ids, ref)):
             assert_same(run_gpu(pl, part), want)
     # a stage call continues from stage calls, not from a plan of the two-kernel chain
+    pl.set_tuning(B.KNOB_CHAIN, 2)
     dev = torch.from_numpy(ids).to(pl.device)
     out = pl.plan(dev)
     assert B.topoep_reroute(pl.handle, dev, w.tokens_per_rank, batch, out.token_replica, 0) == -6
@@ -308,8 +311,8 @@ def test_bitwise_identical_across_reruns_and_tunings():
             pl.set_tuning(B.KNOB_HIST_MODE, mode)
             # launch protocol: plain order, automatic, never early, always early
             pl.set_tuning(B.KNOB_PDL, (tile // 1024 + mode) % 4)
-            # kernel chain: by size, five kernels, two kernels
-            pl.set_tuning(B.KNOB_CHAIN, (tile // 2048 + mode) % 3)
+            # kernel chain: by size, five kernels, two kernels, four kernels
+            pl.set_tuning(B.KNOB_CHAIN, (tile // 1024 + mode) % 4)
             for rep in range(2):
                 again = run_gpu(pl, ids)
                 for key, val in base.items():
