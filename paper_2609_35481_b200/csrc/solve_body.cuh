@@ -423,28 +423,35 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
       const int gb = __ffs(__ballot_sync(full, Lreg == Lb)) - 1;   // busiest, lowest id on ties
       const int Lt = __shfl_sync(full, Lreg, gt);
       const bool has_slot = __shfl_sync(full, usedreg, gt) < N;
-      int bd = 0, bl = INT_MAX;
+      int bd = 0;
       unsigned bk = 0xffffffffu;
-      if (lane_on && gt != gb) {
-        const int half = (Lb - Lt) >> 1;                         // half-gap bound
-        if (half >= p.min_delta) {
+      const int half = (Lb - Lt) >> 1;                           // half-gap bound
+      const bool on = lane_on && gt != gb && half >= p.min_delta;
+      // Selects instead of branches: one warp runs this loop alone, so a taken branch costs more
+      // than the handful of wasted table reads of a lane that has no candidate.
 #pragma unroll 1
-          for (int l = k0; l < s_phys; l += kstep) {
-            const int cb = gb * s_phys + l;
-            const int e = col_expert[cb];
-            const int u = U[cb];
-            if (e < 0 || u <= 0) continue;
-            const int hc = hostcol[gt * E + e];
-            if (hc < 0 && !has_slot) continue;                   // neither hosts e nor has a slot
-            const int delta = min(u, half);
-            if (delta < p.min_delta) continue;
-            const unsigned cr = hc >= 0 ? 0u : (unsigned)col_cr[cb];
-            const unsigned key = (cr << 28) | ((unsigned)e << 5) | (unsigned)gt;
-            if (delta > bd || (delta == bd && key < bk)) { bd = delta; bk = key; }
-          }
-          bl = Lt;
-        }
+      for (int l = k0; l < s_phys; l += 2 * kstep) {
+        const int cb0 = gb * s_phys + l;
+        const bool two = l + kstep < s_phys;
+        const int cb1 = two ? cb0 + kstep : cb0;
+        const int e0 = col_expert[cb0], e1 = col_expert[cb1];
+        const int u0 = U[cb0], u1 = U[cb1];
+        const unsigned cr0 = (unsigned)col_cr[cb0], cr1 = (unsigned)col_cr[cb1];
+        const int hc0 = hostcol[gt * E + max(e0, 0)];
+        const int hc1 = hostcol[gt * E + max(e1, 0)];
+        const int d0 = min(u0, half), d1 = min(u1, half);
+        const bool ok0 = on && e0 >= 0 && u0 > 0 && (hc0 >= 0 || has_slot) && d0 >= p.min_delta;
+        const bool ok1 = on && two && e1 >= 0 && u1 > 0 && (hc1 >= 0 || has_slot) && d1 >= p.min_delta;
+        const unsigned key0 = ((hc0 >= 0 ? 0u : cr0) << 28) | ((unsigned)e0 << 5) | (unsigned)gt;
+        const unsigned key1 = ((hc1 >= 0 ? 0u : cr1) << 28) | ((unsigned)e1 << 5) | (unsigned)gt;
+        const bool b0 = ok0 && (d0 > bd || (d0 == bd && key0 < bk));
+        bd = b0 ? d0 : bd;
+        bk = b0 ? key0 : bk;
+        const bool b1 = ok1 && (d1 > bd || (d1 == bd && key1 < bk));
+        bd = b1 ? d1 : bd;
+        bk = b1 ? key1 : bk;
       }
+      const int bl = on ? Lt : INT_MAX;
       const int md = __reduce_max_sync(full, bd);
       if (md <= 0) break;
       const int ml = __reduce_min_sync(full, bd == md ? bl : INT_MAX);
@@ -473,23 +480,50 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
       const int rb = dm * G + gb, rt = dm * G + wt;
       const int qrt = qd[rt * QS + cb], qrb = qd[rb * QS + cb];
       const int i0 = min(R, lane * chunk), i1 = min(R, i0 + chunk);
-      int sum = 0;
-#pragma unroll 1
-      for (int s = i0; s < i1; ++s) sum += qd[s * QS + cb];
-      int total;
-      int pre = warp_exclusive_scan(sum, lane, &total);
-#pragma unroll 1
-      for (int s = i0; s < i1; ++s) {
-        const int v = qd[s * QS + cb];
-        int before = qrt + pre - (rt < s ? qrt : 0) - (rb < s ? qrb : 0);
-        if (s == rt) before = 0;
-        if (s == rb) before = total - qrb;
-        const int take = min(max(md - before, 0), v);
-        if (take > 0) {
-          qd[s * QS + cb] = v - take;
-          qd[s * QS + ct] += take;
+      if (chunk <= 4) {
+        // up to 128 ranks: a lane's sources fit in registers, so both columns are read with
+        // independent loads before the scan instead of one dependent load per source after it
+        int v[4], w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int s = i0 + j;
+          v[j] = s < i1 ? qd[s * QS + cb] : 0;
+          w[j] = s < i1 ? qd[s * QS + ct] : 0;
         }
-        pre += v;
+        int total;
+        int pre = warp_exclusive_scan(v[0] + v[1] + v[2] + v[3], lane, &total);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int s = i0 + j;
+          int before = qrt + pre - (rt < s ? qrt : 0) - (rb < s ? qrb : 0);
+          before = s == rt ? 0 : before;
+          before = s == rb ? total - qrb : before;
+          const int take = min(max(md - before, 0), v[j]);
+          if (s < i1 && take > 0) {
+            qd[s * QS + cb] = v[j] - take;
+            qd[s * QS + ct] = w[j] + take;
+          }
+          pre += v[j];
+        }
+      } else {
+        int sum = 0;
+#pragma unroll 1
+        for (int s = i0; s < i1; ++s) sum += qd[s * QS + cb];
+        int total;
+        int pre = warp_exclusive_scan(sum, lane, &total);
+#pragma unroll 1
+        for (int s = i0; s < i1; ++s) {
+          const int v = qd[s * QS + cb];
+          int before = qrt + pre - (rt < s ? qrt : 0) - (rb < s ? qrb : 0);
+          if (s == rt) before = 0;
+          if (s == rb) before = total - qrb;
+          const int take = min(max(md - before, 0), v);
+          if (take > 0) {
+            qd[s * QS + cb] = v - take;
+            qd[s * QS + ct] += take;
+          }
+          pre += v;
+        }
       }
       if (lane == 0) { U[cb] -= md; U[ct] += md; }
       if (lane == gb) Lreg -= md;
