@@ -147,6 +147,17 @@ enum {
                                    resident on the GPU at once, where latency
                                    counts; four for a single plan whose second grid
                                    is resident at once; else five                 */
+  TOPOEP_KNOB_PACKED_IDS = 6,   /* five-kernel chain of topoep_plan with at most 256
+                                   experts: the histogram also writes a one-byte
+                                   copy of every id into the workspace and the
+                                   reroute kernel reads that instead of the 4-byte
+                                   ids a second time (a tile that holds padding or
+                                   an invalid id is read in full again).  0
+                                   (default): when the ids of the call exceed the
+                                   L2 cache; 1: never; 2: whenever possible       */
+  TOPOEP_KNOB_REROUTE_TILES = 7,/* consecutive tiles of one source a block of the
+                                   reroute kernel walks when it reads the one-byte
+                                   copy: 1..64, default 4                         */
   TOPOEP_KNOB_TRANSFER_SELFTEST = 4 /* tests only (the one knob that does change
                                    output): 1 makes one block of the bulk engine
                                    wait for a copy it never issued, so its bounded

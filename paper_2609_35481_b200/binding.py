@@ -18,6 +18,7 @@ OK = 0
 FLAG_BAD_ID, FLAG_REFINE_CAP, FLAG_INTERNAL = 1, 2, 4
 T_OMEGA, T_Q, T_RANK_LOAD, T_REFINE_ITERS, T_D, T_U = 0, 1, 2, 3, 4, 5
 KNOB_TILE_IDS, KNOB_HIST_MODE, KNOB_PDL, KNOB_TRANSFER_MODE, KNOB_TRANSFER_SELFTEST, KNOB_CHAIN = 0, 1, 2, 3, 4, 5
+KNOB_PACKED_IDS, KNOB_REROUTE_TILES = 6, 7
 
 EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_set_workspace",
            "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions", "topoep_dispatch_window",

@@ -26,6 +26,9 @@ struct topoep_ctx {
   int max_tiles;
   int chain;           // knob: 0 choose by size, 1 always five kernels, 2 two kernels when they fit,
                        //   3 four kernels when they fit
+  int reroute_tiles_per_block;   // multi-tile reroute kernel: tiles of a source per block
+  int pack_ids;        // knob: 0 choose by size, 1 never, 2 whenever possible (one-byte id copy)
+  int l2_bytes;        // L2 size of the device the workspace lives on
   size_t plan2_smem;   // shared memory the second kernel of the two-kernel chain may use
   bool aux_valid;      // omega_m and demand in the workspace belong to the omega now there
   bool routes_valid;   // route tables in the workspace belong to the tile counts now there
@@ -45,7 +48,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 enum WsSlot {
   W_MAIN_RANK, W_MAIN_LOCAL, W_MAIN_INST, W_SOLVE_STATIC, W_MAIN_DOM, W_MAIN_INSTANCE, W_SLOT_P, W_SLOT_DD, W_STATUS, W_OMEGA, W_OMEGA_M, W_DEMAND, W_TILE_CNT, W_TILE_PREF, W_Q, W_LOAD,
-  W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC,
+  W_ITERS, W_INST_COUNTS, W_REPLICA_MAP, W_COUNTS, W_ROUTE, W_SPLIT_REC, W_IDS8, W_TILE_FLAG,
   W_ACC_OMEGA0, W_ACC_OMEGA1, W_ACC_DEMAND0, W_ACC_DEMAND1, W_EPOCH, W_DONE, W_PLACE_REC, W_SLOTS
 };
 static_assert(W_SLOTS <= 32, "offset table size");
@@ -75,6 +78,9 @@ void carve(topoep_ctx* h) {
   sz[W_COUNTS] = 4 * B * R * R;
   sz[W_ROUTE] = 4 * B * R * E;
   sz[W_SPLIT_REC] = 4 * B * R * (size_t)split_rec_layout(d.E, d.P, h->max_tiles).ints;
+  // one byte per id, only where a byte holds an expert id; rows keep the 4-byte rows' alignment / 4
+  sz[W_IDS8] = E <= 256 ? B * R * (size_t)h->max_tokens * d.k : 0;
+  sz[W_TILE_FLAG] = 4 * B * R * (size_t)h->max_tiles;
   sz[W_ACC_OMEGA0] = sz[W_ACC_OMEGA1] = 4 * B * R * E;
   sz[W_ACC_DEMAND0] = sz[W_ACC_DEMAND1] = 4 * B * (size_t)d.M * E;
   sz[W_EPOCH] = 32;
@@ -117,6 +123,7 @@ HistParams make_hist(topoep_ctx* h, const int32_t* ids, int T, int32_t* out_omeg
   p.rank_first = h->rank_first;
   p.rank_count = h->rank_count;
   p.acc = 0;
+  p.pack = 0;
   p.max_batch = h->max_batch;
   return p;
 }
@@ -224,6 +231,9 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->max_batch = max_batch;
   h->tile_ids = 4096;
   h->chain = 0;
+  h->pack_ids = 0;
+  h->reroute_tiles_per_block = 4;
+  h->l2_bytes = 0;
   h->plan2_smem = 0;
   h->aux_valid = false;
   h->routes_valid = false;
@@ -293,6 +303,8 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   w.epoch = at<unsigned>(dev_ptr, h->off[W_EPOCH]);
   w.done_flags = at<unsigned>(dev_ptr, h->off[W_DONE]);
   w.place_rec = at<unsigned long long>(dev_ptr, h->off[W_PLACE_REC]);
+  w.ids8 = h->d.E <= 256 ? at<unsigned char>(dev_ptr, h->off[W_IDS8]) : nullptr;
+  w.tile_flag = at<int32_t>(dev_ptr, h->off[W_TILE_FLAG]);
 
   cudaError_t e;
   const size_t E = h->d.E;
@@ -301,6 +313,7 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) goto fail;
     if ((e = cudaDeviceGetAttribute(&h->d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) goto fail;
     h->sms = h->d.sms;
+    if ((e = cudaDeviceGetAttribute(&h->l2_bytes, cudaDevAttrL2CacheSize, dev)) != cudaSuccess) goto fail;
   }
   if ((e = cudaMemcpy(const_cast<int32_t*>(w.main_rank), h->main_rank.data(), 4 * E,
                       cudaMemcpyHostToDevice)) != cudaSuccess) goto fail;
@@ -357,7 +370,7 @@ fail:
 namespace {
 
 int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* out_omega,
-                 cudaStream_t stream, bool two = false, bool four = false) {
+                 cudaStream_t stream, bool two = false, bool four = false, bool pack = false) {
   HistParams hp = make_hist(h, ids, T, out_omega);
   if (two) {   // the second kernel of the two-kernel chain has one block shape: its tile size
     hp.tile_ids = kPlan2TileIds;
@@ -369,6 +382,7 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
   h->routes_valid = false;
   h->aux_valid = !two && h->rank_count == h->d.R;
   hp.acc = two ? 1 : 0;
+  hp.pack = pack ? 1 : 0;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
   if (e == cudaSuccess && !two) {
     OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles, batch);
@@ -456,7 +470,7 @@ int enqueue_solve(topoep_ctx* h, const int32_t* omega, int batch, int32_t* repli
 }
 
 int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* token_replica,
-                    cudaStream_t stream) {
+                    cudaStream_t stream, bool packed = false) {
   if (T == 0) return TOPOEP_OK;
   RerouteParams rp;
   rp.d = h->d;
@@ -472,9 +486,25 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   rp.max_tiles = h->max_tiles;
   rp.vec_ok = (rp.n_ids % 4 == 0) && ((reinterpret_cast<uintptr_t>(ids) & 15u) == 0) &&
               ((reinterpret_cast<uintptr_t>(token_replica) & 15u) == 0);
+  rp.packed = packed && rp.vec_ok ? 1 : 0;
+  rp.tiles_per_block = std::max(1, std::min(rp.tiles, h->reroute_tiles_per_block));
   const cudaError_t e = launch_reroute(rp, batch, stream);
   if (e != cudaSuccess) { h->last_cuda = e; return TOPOEP_ERR_CUDA; }
   return TOPOEP_OK;
+}
+
+// Five-kernel chain of a topoep_plan call: should the histogram leave a one-byte copy of the ids
+// for the reroute kernel?  It trades 1 byte written + 1 byte read per assignment for the second
+// 4-byte read, which pays once the ids no longer survive in L2 between the two kernels.  Needs
+// E <= 256, 16-byte aligned buffers and whole groups of four ids per row.
+bool use_packed_ids(const topoep_ctx* h, const int32_t* ids, const int32_t* token_replica, int T,
+                    int batch) {
+  if (h->pack_ids == 1 || !h->ws.ids8 || T == 0) return false;
+  const long long n_ids = (long long)T * h->d.k;
+  if (n_ids % 4 != 0 || (reinterpret_cast<uintptr_t>(ids) & 15u) || (reinterpret_cast<uintptr_t>(token_replica) & 15u))
+    return false;
+  if (h->pack_ids == 2) return true;
+  return 4ll * n_ids * h->d.R * batch > (long long)h->l2_bytes;
 }
 
 // The combined kernel: placement, solver and rank blocks in one grid, and either the per-token
@@ -608,12 +638,13 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
     if (rc != TOPOEP_OK) return rc;
     return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
   }
-  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream);
+  const bool pack = use_packed_ids(h, dev_topk_ids, dev_token_replica, tokens_per_rank, batch);
+  rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, false, false, pack);
   if (rc != TOPOEP_OK) return rc;
   rc = enqueue_solve(h, nullptr, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
                      dev_instance_counts, stream);
   if (rc != TOPOEP_OK) return rc;
-  return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
+  return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream, pack);
 }
 
 size_t topoep_dispatch_scratch_bytes(topoep_handle_t h, int tokens_per_rank, int batch) {
@@ -817,6 +848,14 @@ int topoep_set_tuning(topoep_handle_t h, int knob, int value) {
     case TOPOEP_KNOB_TRANSFER_SELFTEST:
       if (value != 0 && value != 1) return TOPOEP_ERR_ARG;
       h->transfer_selftest = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_PACKED_IDS:
+      if (value < 0 || value > 2) return TOPOEP_ERR_ARG;
+      h->pack_ids = value;
+      return TOPOEP_OK;
+    case TOPOEP_KNOB_REROUTE_TILES:
+      if (value < 1 || value > 64) return TOPOEP_ERR_ARG;
+      h->reroute_tiles_per_block = value;
       return TOPOEP_OK;
     default:
       return TOPOEP_ERR_ARG;

@@ -65,7 +65,31 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread) hist_kernel(const
   }
   pdl_wait();   // the ids are nobody's output; everything written below may still be in use
   if (mx > (unsigned)E) atomicOr(p.ws.status, TOPOEP_FLAG_BAD_ID);
-  __syncthreads();
+  if (p.pack) {
+    // One-byte copy of the tile for the reroute kernel of a large call (E <= 256, rows of whole
+    // 16-byte groups): the low byte of every id, four per word, same flat order.  Streaming
+    // stores: the copy is read once, long after it has left L2.  An id outside [0, E) (padding
+    // or invalid) cannot be told from a valid one in a byte: the tile is flagged and the reroute
+    // kernel reads its 4-byte ids.
+    unsigned* dst = reinterpret_cast<unsigned*>(p.ws.ids8 + row * (size_t)p.n_ids + begin);
+    const unsigned uE = (unsigned)E;
+    int outside = 0;
+#pragma unroll
+    for (int j = 0; j < IPT / 4; ++j) {
+      const int vec = j * nt + tid;
+      const unsigned lo = __byte_perm((unsigned)x[j].x, (unsigned)x[j].y, 0x0040);
+      const unsigned hi = __byte_perm((unsigned)x[j].z, (unsigned)x[j].w, 0x0040);
+      if (4 * vec < count) {
+        __stcs(dst + vec, __byte_perm(lo, hi, 0x5410));
+        outside |= ((unsigned)x[j].x >= uE) | ((unsigned)x[j].y >= uE) | ((unsigned)x[j].z >= uE) |
+                   ((unsigned)x[j].w >= uE);
+      }
+    }
+    outside = __syncthreads_or(outside);
+    if (tid == 0) p.ws.tile_flag[row * (size_t)p.max_tiles + tile] = outside;
+  } else {
+    __syncthreads();
+  }
   const size_t at = (row * (size_t)p.max_tiles + tile) * E;
   if (!p.ws.tile_cnt16) {
     int32_t* out = p.ws.tile_cnt + at;

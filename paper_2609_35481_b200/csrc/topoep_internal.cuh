@@ -79,6 +79,13 @@ struct Workspace {
   unsigned long long* place_rec;    // [max_batch][M][G*N + 1] inter-node placement of (plan,
                                     //   domain) as published by its placement block: every
                                     //   word = call serial << 32 | value
+  unsigned char* ids8;              // [max_batch][R][max ids per row] one-byte copy of the ids of a
+                                    //   large topoep_plan call (E <= 256 only, else NULL): the
+                                    //   histogram writes it, the reroute kernel reads it instead
+                                    //   of the 4-byte ids
+  int32_t* tile_flag;               // [max_batch][R][max_tiles] 1: the tile holds an id outside
+                                    //   [0, E) (padding or invalid), which one byte cannot tell
+                                    //   from a valid id: reroute reads that tile's 4-byte ids
 };
 
 // Record of one (plan, source) written by the route kernel, read by the reroute kernel:
@@ -122,6 +129,7 @@ struct HistParams {
   int vec_ok;           // rows are 16-byte aligned and n_ids % 4 == 0
   int acc;              // two-kernel chain: also add the tile counts into the accumulators
   int max_batch;        // plans the accumulators are sized for
+  int pack;             // also write the one-byte copy of the ids and the per-tile flag
 };
 
 struct OmegaParams {
@@ -189,6 +197,8 @@ struct RerouteParams {
   int32_t* out_token_replica;
   int n_ids, tiles, max_tiles, tile_ids;
   int vec_ok;
+  int packed;   // read the one-byte copy the histogram of this call left in the workspace
+  int tiles_per_block;   // ... in the multi-tile kernel: consecutive tiles of a source per block
 };
 
 struct PosParams {

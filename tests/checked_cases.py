@@ -47,13 +47,15 @@ def main():
         ids = wl.make_topk_ids(w, seed=17, batch=batch).copy()
         ids[0, 0, :1, :] = -1                     # some padding
         ref = orc.plan(oracle_config(w), ids)
-        for chain in (1, 2, 3):
+        for chain, packed in ((1, 1), (1, 2), (2, 0), (3, 0)):
             pl = make_planner(w, max_batch=batch)
             pl.set_tuning(B.KNOB_CHAIN, chain)
+            pl.set_tuning(B.KNOB_PACKED_IDS, packed)   # 2: the one-byte id copy and the multi-tile reroute kernel
+            pl.set_tuning(B.KNOB_REROUTE_TILES, 3)
             for rep in range(2):
                 gpu = run_gpu(pl, ids)
                 assert_same(gpu, ref)
-                assert gpu["flags"] == ref.flags == 0, (name, over, chain, gpu["flags"])
+                assert gpu["flags"] == ref.flags == 0, (name, over, chain, packed, gpu["flags"])
             # the dispatch permutation and the replica copies on the same plan
             out = pl.plan(torch.from_numpy(ids).to(pl.device))
             send, recv, off = pl.dispatch_positions(out.token_replica)

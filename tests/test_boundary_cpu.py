@@ -84,6 +84,10 @@ def test_calls_without_workspace_or_handle_fail_cleanly():
     assert B.topoep_set_workspace(h, None, 1 << 20) == -1
     assert B.topoep_set_tuning(h, 99, 0) == -10
     assert B.topoep_set_tuning(h, B.KNOB_TILE_IDS, 2048) == 0
+    assert B.topoep_set_tuning(h, B.KNOB_PACKED_IDS, 2) == 0
+    assert B.topoep_set_tuning(h, B.KNOB_PACKED_IDS, 3) == -10
+    assert B.topoep_set_tuning(h, B.KNOB_REROUTE_TILES, 64) == 0
+    assert B.topoep_set_tuning(h, B.KNOB_REROUTE_TILES, 0) == -10
     B.topoep_destroy(h)
     assert B.topoep_workspace_bytes(None) == 0
     assert B.topoep_plan(None, 0, 0, 0, 0, 0, 0, 0, 0, 0) == -1

@@ -198,6 +198,8 @@ def test_random_problems_with_policies_tunings_and_skew():
         pl.set_tuning(B.KNOB_TILE_IDS, int(rng.choice([1024, 2048, 4096, 8192])))
         pl.set_tuning(B.KNOB_PDL, int(rng.integers(0, 4)))
         pl.set_tuning(B.KNOB_CHAIN, int(rng.integers(0, 4)))
+        pl.set_tuning(B.KNOB_PACKED_IDS, int(rng.integers(0, 3)))
+        pl.set_tuning(B.KNOB_REROUTE_TILES, int(rng.integers(1, 6)))
         gpu = run_gpu(pl, ids)
         ref = orc.plan(oracle_config(w, reserve_slots=reserve, stage1_rank=lpt, **over), ids)
         try:
@@ -299,6 +301,49 @@ def test_kernel_chains_agree_with_one_another_and_the_oracle(name, over, batch):
     assert pl.status() == 0
 
 
+# ---- the one-byte copy of the ids (five-kernel chain, E <= 256) ---------------------------------
+PACKED_CASES = [
+    ("tiny", {}, 3, "clean"),
+    ("mid", dict(slots_per_rank=3), 2, "padded"),
+    ("dsv3", dict(tokens_per_rank=3000, slots_per_rank=2), 2, "invalid"),
+    ("tiny", dict(tokens_per_rank=778, top_k=6, slots_per_rank=2), 2, "padded"),
+    ("tiny", dict(experts=30, tokens_per_rank=2048, slots_per_rank=2), 2, "padded"),   # E % 4 != 0
+    ("tiny", dict(tokens_per_rank=777, top_k=5), 2, "clean"),   # rows of 3885 ids: not whole groups of four
+    ("dsv3", dict(experts=224, tokens_per_rank=1536), 2, "padded"),
+    ("mid", dict(experts=512, nodes=2, tokens_per_rank=1024), 2, "clean"),   # E > 256: no copy exists
+]
+
+
+@pytest.mark.parametrize("name,over,batch,dirt", PACKED_CASES)
+def test_one_byte_id_copy_matches_the_oracle(name, over, batch, dirt):
+    """With at most 256 experts the histogram of a large topoep_plan call leaves a one-byte copy of
+    the ids for the reroute kernel (TOPOEP_KNOB_PACKED_IDS; here forced on for small calls).  A
+    tile with padding (-1) or an invalid id cannot be expressed in bytes and is read again in
+    full; rows that are not whole groups of four ids and configs with more experts fall back to
+    the plain kernels.  Every variant must give the oracle's plan, bit for bit."""
+    w = wl.CONFIGS[name].replace(**over)
+    ids = wl.make_topk_ids(w, seed=7, batch=batch).copy()
+    if dirt in ("padded", "invalid"):
+        ids[0, 1, -37:, :] = -1                                          # tail tokens of one rank
+        ids[batch - 1, w.ranks - 1, w.tokens_per_rank // 2:, :] = -1     # half a rank
+    if dirt == "invalid":
+        ids[0, 2, 5, 0] = w.experts
+        ids[1, 0, 100, 1] = 1 << 20
+        ids[1, 3, 7, 2] = -7
+    ref = orc.plan(oracle_config(w), ids)
+    for tile, tiles_per_block in ((1024, 1), (1024, 3), (4096, 4), (8192, 2)):
+        pl = make_planner(w, max_batch=batch)
+        pl.set_tuning(B.KNOB_CHAIN, 1)
+        pl.set_tuning(B.KNOB_PACKED_IDS, 2)
+        pl.set_tuning(B.KNOB_TILE_IDS, tile)
+        pl.set_tuning(B.KNOB_REROUTE_TILES, tiles_per_block)
+        for rep in range(2):   # the second call finds the first one's copy and flags in the workspace
+            gpu = run_gpu(pl, ids)
+            assert_same(gpu, ref)
+            assert gpu["flags"] == ref.flags
+        pl.close()
+
+
 # ---- determinism: reruns and launch configurations ----------------------------------------
 def test_bitwise_identical_across_reruns_and_tunings():
     w = wl.CONFIGS["dsv3"].replace(slots_per_rank=3)
@@ -313,6 +358,10 @@ def test_bitwise_identical_across_reruns_and_tunings():
             pl.set_tuning(B.KNOB_PDL, (tile // 1024 + mode) % 4)
             # kernel chain: by size, five kernels, two kernels, four kernels
             pl.set_tuning(B.KNOB_CHAIN, (tile // 1024 + mode) % 4)
+            # one-byte id copy for the reroute kernel: by size, never, whenever possible; and the
+            # tiles a block of that kernel walks
+            pl.set_tuning(B.KNOB_PACKED_IDS, (tile // 2048 + mode) % 3)
+            pl.set_tuning(B.KNOB_REROUTE_TILES, 1 + (tile // 1024 + 3 * mode) % 5)
             for rep in range(2):
                 again = run_gpu(pl, ids)
                 for key, val in base.items():
