@@ -35,24 +35,28 @@ if ROOT not in sys.path:
 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+NCU_REROUTE_ROWS_READ_16 = 42320896   # dram__bytes_read.sum of reroute_rows_kernel, 16 plans
+NCU_HIST_PACK_READ_16 = 134238720     # ... of hist_kernel when it also writes the byte copy
 NOMINAL_HBM_GBS = 8000.0   # the figure the target statement names; context beside the measured peak
 REPEATS = 11               # timed replays of every graph: the median is reported, min and max beside it
-# DRAM bytes per PLAN of the DeepSeek-V3-shaped layer.  READS come from the committed ncu capture of
-# a 16-plan call (profiles/reroute_kernel_dsv3_batch16.md, profiles/hist_kernel_dsv3_batch16.md) and
-# grow in proportion to the plans of a call (every CTA reads only its own tile and its source's
-# tables).  WRITES do not scale from that capture: its 134 MB of output partly stayed dirty in the
-# 126 MB L2 at kernel end (85.7 MB reached DRAM), a constant, not a proportion -- a full-size call
-# writes 1.9 GB through the same L2, so its DRAM writes are its algorithmic output bytes (4 per
-# assignment for the reroute kernel; the tile counts of the histogram kernel: 16-bit, E per tile).
-NCU_READ_BYTES_PER_PLAN = {"reroute": 137112320 / 16, "hist": 134235136 / 16}
+# DRAM bytes per PLAN of the DeepSeek-V3-shaped layer.  READS come from the committed ncu captures of
+# a 16-plan call (profiles/reroute_kernel_dsv3_batch16.md, profiles/hist_kernel_dsv3_batch16.md and,
+# for calls that keep a one-byte copy of the ids, profiles/byte_copy_kernels_dsv3_batch16.md) and
+# grow in proportion to the plans of a call (every CTA reads only its own tiles and its source's
+# tables).  WRITES do not scale from those captures: the 134 MB of output partly stayed dirty in the
+# 126 MB L2 at kernel end, a constant, not a proportion -- a full-size call writes 1.9 GB through
+# the same L2, so its DRAM writes are its output bytes (reroute: 4 per assignment; histogram: the
+# 16-bit tile counts, E per tile, and with the byte copy 1 per assignment).
+NCU_READ_BYTES_PER_PLAN = {("reroute", False): 137112320 / 16, ("hist", False): 134235136 / 16,
+                           ("reroute", True): NCU_REROUTE_ROWS_READ_16 / 16, ("hist", True): NCU_HIST_PACK_READ_16 / 16}
 
 
-def ncu_traffic(w, kernel, tile_ids=4096):
-    if w.name in ("dsv3", "dsv3_batched") and kernel in NCU_READ_BYTES_PER_PLAN:
+def ncu_traffic(w, kernel, tile_ids=4096, byte_copy=False):
+    if w.name in ("dsv3", "dsv3_batched") and (kernel, byte_copy) in NCU_READ_BYTES_PER_PLAN:
         per_plan_ids = w.assignments // w.batch
         writes = {"reroute": 4 * per_plan_ids,
-                  "hist": 2 * w.experts * (per_plan_ids // tile_ids)}[kernel]
-        return int((NCU_READ_BYTES_PER_PLAN[kernel] + writes) * w.batch)
+                  "hist": 2 * w.experts * (per_plan_ids // tile_ids) + (per_plan_ids if byte_copy else 0)}[kernel]
+        return int((NCU_READ_BYTES_PER_PLAN[(kernel, byte_copy)] + writes) * w.batch)
     return None
 
 
@@ -293,6 +297,8 @@ def measure(w, K, W, rank, world, dev, args, stages=True, chain=-1, warm_l2=Fals
             pl.set_tuning(B.KNOB_PDL, args.pdl)
         if chain >= 0:
             pl.set_tuning(B.KNOB_CHAIN, chain)
+        if args.packed_ids >= 0:
+            pl.set_tuning(B.KNOB_PACKED_IDS, args.packed_ids)
         ids_dev = torch.from_numpy(ids).to(dev)
         sets.append({"pl": pl, "ids_host": ids, "ids": ids_dev,
                      "out": pl.alloc_outputs(w.batch, w.tokens_per_rank)})
@@ -322,6 +328,7 @@ def measure(w, K, W, rank, world, dev, args, stages=True, chain=-1, warm_l2=Fals
         assert rc == 0, rc
 
     kernels_per_plan = B.topoep_plan_kernels(sets[0]["pl"].handle, w.tokens_per_rank, w.batch)
+    byte_copy = B.topoep_plan_byte_copy(sets[0]["pl"].handle, w.tokens_per_rank, w.batch) == 1
 
     def floor(i):
         assert B.topoep_launch_floor(kernels_per_plan, sh) == 0
@@ -390,7 +397,7 @@ def measure(w, K, W, rank, world, dev, args, stages=True, chain=-1, warm_l2=Fals
     return {"sets": sets, "nsets": nsets, "l2_policy": l2_policy, "stream": stream,
             "ms_total": ms_total, "ms_step": ms_total / K, "stage_us": stage_us,
             "plan_spread": spread(plan_ms, K), "stage_spread": stage_spread,
-            "kernels_per_plan": kernels_per_plan, "barrier": barrier}
+            "kernels_per_plan": kernels_per_plan, "byte_copy": byte_copy, "barrier": barrier}
 
 
 def main():
@@ -411,6 +418,8 @@ def main():
     ap.add_argument("--pdl", type=int, default=-1)
     ap.add_argument("--chain", type=int, default=-1,
                     help="TOPOEP_KNOB_CHAIN for the timed plan (default: the library's choice)")
+    ap.add_argument("--packed-ids", type=int, default=-1,
+                    help="TOPOEP_KNOB_PACKED_IDS (default: the library's choice; 1 = never)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -645,33 +654,56 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     A = w.assignments
     algo_bytes = {"hist": 4 * A, "reroute": 8 * A, "solve": None}
+    byte_copy = m["byte_copy"]
+    # what the two streaming kernels move when the histogram leaves a one-byte copy of the ids for
+    # the reroute kernel: 4 + 1 and 1 + 4 bytes per assignment instead of 4 and 4 + 4
+    moved_bytes = {"hist": 5 * A, "reroute": 5 * A} if byte_copy else {"hist": 4 * A, "reroute": 8 * A}
     dominant = max(("hist", "solve", "reroute"), key=lambda n: stage_us[n])
     hbm_kernels = {n: {"us": round(stage_us[n], 3),
                        "achieved_gbs": round(algo_bytes[n] / (stage_us[n] * 1e-6) / 1e9, 1),
-                       "frac": round(algo_bytes[n] / (stage_us[n] * 1e-6) / 1e9 / peak, 4)}
+                       "frac": round(algo_bytes[n] / (stage_us[n] * 1e-6) / 1e9 / peak, 4),
+                       "moved_gbs": round(moved_bytes[n] / (stage_us[n] * 1e-6) / 1e9, 1),
+                       "frac_moved": round(moved_bytes[n] / (stage_us[n] * 1e-6) / 1e9 / peak, 4)}
                    for n in ("hist", "reroute")}
     if dominant == "solve":
         # latency-bound: a few CTAs of serial integer work; judged against the launch floor, and
         # reported here with the bytes it has to touch (omega in, q and layout out)
         dom_bytes = 4 * w.batch * (w.ranks * w.experts + w.ranks * sets[0]["pl"].P
                                    + 3 * w.ranks * w.ranks)
+        dom_moved = dom_bytes
     else:
         dom_bytes = algo_bytes[dominant]
-    achieved = dom_bytes / (stage_us[dominant] * 1e-6) / 1e9
+        dom_moved = moved_bytes[dominant]
+    # With the byte copy the dominant kernel's bytes are the ones it moves (its input IS the copy);
+    # the 12 B-per-assignment definition of the whole plan stays in plan_frac, and the kernel's
+    # figure under that definition in frac_12B_definition.
+    achieved = dom_moved / (stage_us[dominant] * 1e-6) / 1e9
     plan_gbs = 12 * A / (ms_step * 1e-3) / 1e9
+    plan_moved = (10 if byte_copy else 12) * A
     roofline = {"bound": "hbm", "kernel": {"hist": "hist_kernel", "solve": "solve_kernel",
-                                           "reroute": "reroute_kernel"}[dominant],
+                                           "reroute": "reroute_rows_kernel" if byte_copy else "reroute_kernel"}[dominant],
                 "achieved": round(achieved, 2), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "peak_source": "of " + peak_kind,
                 "frac_nominal": round(achieved / NOMINAL_HBM_GBS, 4),
-                "traffic": ncu_traffic(w, dominant, args.tile_ids or 4096),
+                "traffic": ncu_traffic(w, dominant, args.tile_ids or 4096, byte_copy),
                 "traffic_note": "reads: ncu capture of a 16-plan call scaled by plans; writes: "
-                                "algorithmic output bytes (see the comment at NCU_READ_BYTES_PER_PLAN)",
-                "algorithmic_bytes_per_launch": dom_bytes,
+                                "output bytes (see the comment at NCU_READ_BYTES_PER_PLAN)",
+                "algorithmic_bytes_per_launch": dom_moved,
+                "byte_copy": byte_copy,
+                "bytes_per_launch_12B_definition": dom_bytes,
+                "frac_12B_definition": round(dom_bytes / (stage_us[dominant] * 1e-6) / 1e9 / peak, 4),
+                "byte_copy_note": "the 12 B-per-assignment definition of a plan counts a second 4-byte read "
+                                  "of every id by the reroute kernel; with at most 256 experts the histogram "
+                                  "kernel leaves a one-byte copy instead, so the plan moves 10 B per "
+                                  "assignment (histogram 4 + 1, reroute 1 + 4) and fractions of the 12 B "
+                                  "definition can exceed 1; achieved and frac count the bytes the kernel "
+                                  "moves" if byte_copy else None,
                 "plan_bytes": 12 * A,
                 "plan_frac": round(plan_gbs / peak, 4),
+                "plan_moved_bytes": plan_moved,
+                "plan_frac_moved": round(plan_gbs * plan_moved / (12 * A) / peak, 4),
                 # the whole plan against 8 B per assignment: ids read from DRAM once (second pass
-                # from L2), outputs written once -- the bound a chunked batch could approach
+                # from L2), outputs written once
                 "plan_frac_8B": round(plan_gbs * 8 / 12 / peak, 4),
                 "plan_frac_nominal": round(plan_gbs / NOMINAL_HBM_GBS, 4),
                 "hbm_kernels": hbm_kernels,

@@ -147,7 +147,8 @@ enum {
                                    resident on the GPU at once, where latency
                                    counts; four for a single plan whose second grid
                                    is resident at once; else five                 */
-  TOPOEP_KNOB_PACKED_IDS = 6,   /* five-kernel chain of topoep_plan with at most 256
+  TOPOEP_KNOB_PACKED_IDS = 6,   /* five-kernel chain (topoep_plan, or the stage calls
+                                   on the same id buffer) with at most 256
                                    experts: the histogram also writes a one-byte
                                    copy of every id into the workspace and the
                                    reroute kernel reads that instead of the 4-byte
@@ -445,6 +446,14 @@ int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count);
  * handle or size.  Not part of the method: for benchmarks and tests.
  */
 int topoep_plan_kernels(topoep_handle_t h, int tokens_per_rank, int batch);
+
+/*
+ * 1 when a topoep_plan call of this size, with the current knobs, leaves a
+ * one-byte copy of the ids for its reroute kernel (TOPOEP_KNOB_PACKED_IDS;
+ * given 16-byte aligned id and output buffers), else 0.  Needs the workspace
+ * (the rule looks at the device's L2 size); negative error code otherwise.
+ */
+int topoep_plan_byte_copy(topoep_handle_t h, int tokens_per_rank, int batch);
 
 /* Derived sizes: E_loc, S_phys, P.  Any output pointer may be NULL. */
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances);

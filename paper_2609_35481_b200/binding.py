@@ -24,7 +24,7 @@ EXPORTS = ("topoep_create", "topoep_destroy", "topoep_workspace_bytes", "topoep_
            "topoep_plan", "topoep_histogram", "topoep_histogram_static", "topoep_solve", "topoep_reroute", "topoep_dispatch_scratch_bytes", "topoep_dispatch_positions", "topoep_dispatch_window",
            "topoep_summary", "topoep_read_status",
            "topoep_debug_tensor", "topoep_set_tuning", "topoep_set_rank_window", "topoep_set_policy", "topoep_replica_pull", "topoep_replica_grad_return",
-           "topoep_get_layout", "topoep_plan_kernels",
+           "topoep_get_layout", "topoep_plan_kernels", "topoep_plan_byte_copy",
            "topoep_launch_floor", "topoep_strerror")
 
 
@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
         L.topoep_get_layout.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.topoep_plan_kernels.restype = ci
         L.topoep_plan_kernels.argtypes = [vp, ci, ci]
+        L.topoep_plan_byte_copy.restype = ci
+        L.topoep_plan_byte_copy.argtypes = [vp, ci, ci]
         L.topoep_launch_floor.restype = ci
         L.topoep_launch_floor.argtypes = [ci, vp]
         L.topoep_strerror.restype = ctypes.c_char_p
@@ -271,6 +273,11 @@ def topoep_get_layout(h):
 def topoep_plan_kernels(h, tokens_per_rank: int, batch: int) -> int:
     """Kernels topoep_plan would enqueue for a call of this size (5, or 2 for a small call)."""
     return lib().topoep_plan_kernels(h, tokens_per_rank, batch)
+
+
+def topoep_plan_byte_copy(h, tokens_per_rank: int, batch: int) -> int:
+    """1 when a plan call of this size leaves a one-byte copy of the ids for its reroute kernel."""
+    return lib().topoep_plan_byte_copy(h, tokens_per_rank, batch)
 
 
 def topoep_launch_floor(count: int, stream=0) -> int:

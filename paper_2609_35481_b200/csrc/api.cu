@@ -27,6 +27,7 @@ struct topoep_ctx {
   int chain;           // knob: 0 choose by size, 1 always five kernels, 2 two kernels when they fit,
                        //   3 four kernels when they fit
   int reroute_tiles_per_block;   // multi-tile reroute kernel: tiles of a source per block
+  const int32_t* packed_src;   // ids whose one-byte copy the workspace holds (NULL: none)
   int pack_ids;        // knob: 0 choose by size, 1 never, 2 whenever possible (one-byte id copy)
   int l2_bytes;        // L2 size of the device the workspace lives on
   size_t plan2_smem;   // shared memory the second kernel of the two-kernel chain may use
@@ -232,6 +233,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->tile_ids = 4096;
   h->chain = 0;
   h->pack_ids = 0;
+  h->packed_src = nullptr;
   h->reroute_tiles_per_block = 4;
   h->l2_bytes = 0;
   h->plan2_smem = 0;
@@ -360,6 +362,8 @@ int topoep_set_workspace(topoep_handle_t h, void* dev_ptr, size_t bytes) {
   if ((e = configure_route(route_smem_bytes(h->d))) != cudaSuccess) goto fail;
   if ((e = configure_reroute(reroute_smem_bytes(h->d, kMaxTileIds))) != cudaSuccess) goto fail;
   if ((e = cudaDeviceSynchronize()) != cudaSuccess) goto fail;
+  h->packed_src = nullptr;   // a new workspace holds no copy of anybody's ids
+  h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;
   h->have_ws = true;
   return TOPOEP_OK;
 fail:
@@ -383,6 +387,7 @@ int enqueue_hist(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t* o
   h->aux_valid = !two && h->rank_count == h->d.R;
   hp.acc = two ? 1 : 0;
   hp.pack = pack ? 1 : 0;
+  h->packed_src = pack ? ids : nullptr;
   cudaError_t e = launch_hist(hp, batch, h->hist_mode, stream);
   if (e == cudaSuccess && !two) {
     OmegaParams op = make_omega(h, nullptr, out_omega, hp.tiles, batch);
@@ -493,16 +498,14 @@ int enqueue_reroute(topoep_ctx* h, const int32_t* ids, int T, int batch, int32_t
   return TOPOEP_OK;
 }
 
-// Five-kernel chain of a topoep_plan call: should the histogram leave a one-byte copy of the ids
-// for the reroute kernel?  It trades 1 byte written + 1 byte read per assignment for the second
+// Five-kernel chain (topoep_plan, or topoep_histogram ... topoep_reroute): should the histogram
+// leave a one-byte copy of the ids for the reroute kernel?  It trades 1 byte written + 1 byte read per assignment for the second
 // 4-byte read, which pays once the ids no longer survive in L2 between the two kernels.  Needs
 // E <= 256, 16-byte aligned buffers and whole groups of four ids per row.
-bool use_packed_ids(const topoep_ctx* h, const int32_t* ids, const int32_t* token_replica, int T,
-                    int batch) {
-  if (h->pack_ids == 1 || !h->ws.ids8 || T == 0) return false;
+bool use_packed_ids(const topoep_ctx* h, const int32_t* ids, int T, int batch) {
+  if (h->pack_ids == 1 || !h->ws.ids8 || T == 0 || h->rank_count != h->d.R) return false;
   const long long n_ids = (long long)T * h->d.k;
-  if (n_ids % 4 != 0 || (reinterpret_cast<uintptr_t>(ids) & 15u) || (reinterpret_cast<uintptr_t>(token_replica) & 15u))
-    return false;
+  if (n_ids % 4 != 0 || (reinterpret_cast<uintptr_t>(ids) & 15u)) return false;
   if (h->pack_ids == 2) return true;
   return 4ll * n_ids * h->d.R * batch > (long long)h->l2_bytes;
 }
@@ -577,7 +580,8 @@ int topoep_histogram(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_
   if (batch == 0) return TOPOEP_OK;
   if (!dev_topk_ids && tokens_per_rank > 0) return TOPOEP_ERR_NULL;
   if (!aligned4(dev_topk_ids) || !aligned4(dev_omega)) return TOPOEP_ERR_ALIGN;
-  return enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, dev_omega, stream);
+  const bool pack = use_packed_ids(h, dev_topk_ids, tokens_per_rank, batch);
+  return enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, dev_omega, stream, false, false, pack);
 }
 
 int topoep_solve(topoep_handle_t h, const int32_t* dev_omega, int batch, int32_t* dev_replica_map,
@@ -606,7 +610,9 @@ int topoep_reroute(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_pe
     return TOPOEP_ERR_SIZE;
   if (tokens_per_rank > 0 && (!dev_topk_ids || !dev_token_replica)) return TOPOEP_ERR_NULL;
   if (!aligned4(dev_topk_ids) || !aligned4(dev_token_replica)) return TOPOEP_ERR_ALIGN;
-  return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
+  // the one-byte copy the histogram call left, if it was made from these very ids
+  const bool packed = h->packed_src != nullptr && h->packed_src == dev_topk_ids;
+  return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream, packed);
 }
 
 int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_rank, int batch,
@@ -638,7 +644,7 @@ int topoep_plan(topoep_handle_t h, const int32_t* dev_topk_ids, int tokens_per_r
     if (rc != TOPOEP_OK) return rc;
     return enqueue_reroute(h, dev_topk_ids, tokens_per_rank, batch, dev_token_replica, stream);
   }
-  const bool pack = use_packed_ids(h, dev_topk_ids, dev_token_replica, tokens_per_rank, batch);
+  const bool pack = use_packed_ids(h, dev_topk_ids, tokens_per_rank, batch);
   rc = enqueue_hist(h, dev_topk_ids, tokens_per_rank, batch, nullptr, stream, false, false, pack);
   if (rc != TOPOEP_OK) return rc;
   rc = enqueue_solve(h, nullptr, batch, dev_replica_map, dev_dispatch_counts, dev_dispatch_offsets,
@@ -884,6 +890,7 @@ int topoep_set_rank_window(topoep_handle_t h, int first_rank, int rank_count) {
   h->rank_first = first_rank;
   h->rank_count = rank_count;
   h->hist_tile_ids = h->hist_tokens = h->hist_batch = -1;   // earlier tile counts no longer apply
+  h->packed_src = nullptr;
   return TOPOEP_OK;
 }
 
@@ -892,6 +899,14 @@ int topoep_plan_kernels(topoep_handle_t h, int tokens_per_rank, int batch) {
   if (rc != TOPOEP_OK) return rc;
   return use_two_kernels(h, tokens_per_rank, batch) ? 2
          : use_four_kernels(h, tokens_per_rank, batch) ? 4 : 5;
+}
+
+int topoep_plan_byte_copy(topoep_handle_t h, int tokens_per_rank, int batch) {
+  const int rc = check_sizes(h, tokens_per_rank, batch);
+  if (rc != TOPOEP_OK) return rc;
+  if (use_two_kernels(h, tokens_per_rank, batch) || use_four_kernels(h, tokens_per_rank, batch)) return 0;
+  // alignment aside: the query has no buffers
+  return use_packed_ids(h, nullptr, tokens_per_rank, batch) ? 1 : 0;
 }
 
 int topoep_get_layout(topoep_handle_t h, int* e_loc, int* s_phys, int* instances) {

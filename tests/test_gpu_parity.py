@@ -385,10 +385,16 @@ def test_histogram_entry_point_matches_bincount():
             assert np.array_equal(om[b, s], np.bincount(ids[b, s].ravel(), minlength=w.experts))
 
 
-def test_stage_entry_points_equal_the_fused_plan():
+@pytest.mark.parametrize("packed", [1, 2])
+def test_stage_entry_points_equal_the_fused_plan(packed):
+    """packed = 2: the histogram call leaves the one-byte copy of the ids and the reroute call, given
+    the same buffer, reads it; given another buffer with the same ids it reads that one."""
     w = wl.CONFIGS["mid"].replace(slots_per_rank=3)
-    ids = wl.make_topk_ids(w, seed=13, batch=2)
+    ids = wl.make_topk_ids(w, seed=13, batch=2).copy()
+    ids[1, 5, -100:, :] = -1
     pl = make_planner(w, max_batch=2)
+    pl.set_tuning(B.KNOB_CHAIN, 1)
+    pl.set_tuning(B.KNOB_PACKED_IDS, packed)
     dev = torch.from_numpy(ids).to(pl.device)
     fused = pl.plan(dev)
     out = pl.alloc_outputs(2, w.tokens_per_rank)
@@ -407,6 +413,10 @@ def test_stage_entry_points_equal_the_fused_plan():
     for name in ("replica_map", "token_replica", "dispatch_counts", "dispatch_offsets",
                  "instance_counts"):
         assert torch.equal(getattr(out, name), getattr(fused, name)), name
+    out.token_replica.fill_(-9)
+    assert B.topoep_reroute(pl.handle, dev.clone(), T, 2, out.token_replica, 0) == 0
+    torch.cuda.synchronize()
+    assert torch.equal(out.token_replica, fused.token_replica)
     assert pl.status() == 0
 
 
