@@ -47,7 +47,6 @@ namespace {
 
 constexpr int kP2RankCap = 128;                  // candidates of a domain ranked all-pairs
 constexpr int kP2Warps = kSolveThreads / 32;     // every block of this kernel has this shape
-constexpr unsigned kFlagWaitLimit = 1u << 20;    // polls (roughly a second) for a solver block
 
 __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gmem_src) {
   const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -378,8 +377,9 @@ __device__ __forceinline__ void slow_route(const TailParams& p, const TailSm& t,
       *seg_e = t.seg_e, *crow = t.crow, *split_e = t.split_e, *warp_tot = t.warp_tot;
   int n_split, n_list;
   // ---- the refinement decides q: wait for the solver blocks of this plan (bounded polls),
-  // then row s of q and the replica map come from memory
-  if (warp == 0) {
+  // then row s of q and the replica map come from memory.  Warp 1 polls: warp 0 would share its
+  // scheduler with the refinement warp of a solver block on the same SM.
+  if (warp == 1) {
     const unsigned* flags = p.ws.done_flags + (size_t)b * M;
     bool done = false;
 #pragma unroll 1
@@ -392,6 +392,9 @@ __device__ __forceinline__ void slow_route(const TailParams& p, const TailSm& t,
         mine = mine && v == serial;
       }
       done = __all_sync(full, mine);
+      // the waiting warp shares its scheduler with the solver block's refinement warp when the
+      // two blocks sit on one SM: poll at intervals, not back to back
+      if (!done) __nanosleep(500);
     }
     if (!done && lane == 0) atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
   }

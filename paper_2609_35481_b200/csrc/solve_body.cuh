@@ -31,7 +31,6 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   auto pad4 = [](size_t ints) { return (ints + 3) & ~(size_t)3; };
   SolveLayout o;
   size_t at = 0;
-  o.cand = at;       at += sizeof(unsigned long long) * (size_t)kRankCap * (kSolveThreads / 32);
   o.col_main = at;   at += sizeof(int) * pad4((size_t)d.G * d.e_loc * d.R);   // [G*e_loc][R]
   o.col_rep = at;    at += sizeof(int) * pad4((size_t)d.G * d.N * d.R);       // [G*N][R]
   o.stat = at;
@@ -46,7 +45,15 @@ __host__ __device__ inline SolveLayout solve_layout(const Dims& d) {
   o.col_rank = at;   at += sizeof(short) * (size_t)d.C;
   at = o.stat + sizeof(int) * solve_static_ints(d);
   o.D = at;          at += sizeof(int) * pad4((size_t)d.M * d.E);
-  o.qd = at;         at += sizeof(int) * (size_t)d.R * d.qstride;
+  // the candidate lists of inter-node placement (one per warp) are dead before the first q is
+  // written: they share the q block's bytes, so that at 128 ranks two blocks still fit an SM
+  o.qd = at;
+  o.cand = at;
+  {
+    const size_t q_bytes = sizeof(int) * (size_t)d.R * d.qstride;
+    const size_t cand_bytes = sizeof(unsigned long long) * (size_t)kRankCap * (kSolveThreads / 32);
+    at += ((q_bytes > cand_bytes ? q_bytes : cand_bytes) + 15) & ~(size_t)15;
+  }
   o.U = at;          at += sizeof(int) * (size_t)d.C;
   o.L = at;          at += sizeof(int) * (size_t)d.G;
   o.used = at;       at += sizeof(int) * (size_t)d.G;
@@ -148,6 +155,14 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   const short* col_rank = reinterpret_cast<const short*>(smem + lay.col_rank);   // rank of a column
 
   const int32_t* om_m = p.ws.omega_m + (size_t)b * R * e_loc * R;   // rows = main instances
+  // In the combined kernel the placement blocks publish inter-node placement: this block reads
+  // the records instead of loading the demand of every domain and ranking every domain's
+  // candidates again (the least-loaded-rank policy needs the demand values: it keeps doing so).
+  // The records are staged where the demand would have been.
+  const int GNw = G * N;
+  // Worth the wait for the records only where the demand is large (many domains, many experts):
+  // a small one is loaded and ranked sooner than the placement blocks' result arrives.
+  const bool from_records = p.fused && !LPT && GNw + 1 <= E && M > 1 && p.stage1_slots > 0 && M * E >= 4096;
 
   // ---- first batch of asynchronous copies: the static block of this domain first (main-rank tables,
   // hosting masks and column tables as they are before any replica exists), then -- once the
@@ -160,7 +175,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   for (int i = tid; i < R * G; i += nt) cnt[i] = 0;
   if (!p.acc) {
     pdl_wait();
-    copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
+    if (!from_records) copy_async(D, p.ws.demand + (size_t)b * M * E, M * E, tid, nt);
     copy_async(col_main, om_m + (size_t)dm * G * e_loc * R, G * e_loc * R, tid, nt);
     cp_async_wait_all();
     __syncthreads();
@@ -173,8 +188,10 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
     pdl_wait();
     const int32_t* dA = p.ws.acc_demand[0] + (size_t)b * M * E;
     const int32_t* dB = p.ws.acc_demand[1] + (size_t)b * M * E;
+    if (!from_records) {
 #pragma unroll 4
-    for (int i = tid; i < M * E; i += nt) D[i] = __ldcg(dA + i) + __ldcg(dB + i);
+      for (int i = tid; i < M * E; i += nt) D[i] = __ldcg(dA + i) + __ldcg(dB + i);
+    }
     // main columns: a warp step covers 8 columns x 4 sources (blocked main maps: one sector each)
     const int32_t* oA = p.ws.acc_omega[0] + (size_t)b * R * E;
     const int32_t* oB = p.ws.acc_omega[1] + (size_t)b * R * E;
@@ -190,7 +207,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
       }
     }
     __syncthreads();
-    if (p.ws.demand) {   // kept for inspection (debug tensor); row dm by this CTA
+    if (p.ws.demand && !from_records) {   // kept for inspection (debug tensor); row dm by this CTA
 #pragma unroll 1
       for (int e = tid; e < E; e += nt) p.ws.demand[((size_t)b * M + dm) * E + e] = D[dm * E + e];
     }
@@ -200,7 +217,42 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   // Candidates in descending (b, then ascending e) order == descending (D, ascending e) for a
   // uniform ||W|| and S_tok; the i-th goes to rank i mod G, slot i / G (fewest used slots first,
   // ties to the lower rank).
-  if (M > 1 && p.stage1_slots > 0) {
+  if (from_records) {
+    const unsigned serial = __ldcg(p.ws.epoch + 4);
+    const unsigned long long* rec = p.ws.place_rec + (size_t)b * M * (GNw + 1);
+    int* recs = D;   // [M][GN + 1]: count, winners in rank order
+    bool all = false;
+#pragma unroll 1
+    for (unsigned it = 0; it < kFlagWaitLimit && !all; ++it) {
+      bool ok = true;
+#pragma unroll 1
+      for (int i = tid; i < M * (GNw + 1); i += nt) {
+        const unsigned long long w = __ldcg(rec + i);
+        ok = ok && (unsigned)(w >> 32) == serial;
+        recs[i] = (int)(unsigned)w;
+      }
+      all = __syncthreads_and(ok);
+    }
+    if (!all && tid == 0) atomicOr(p.ws.status, TOPOEP_FLAG_INTERNAL);
+    // hosting masks of every domain's winners; this domain's winners into its columns: the i-th
+    // to rank i mod G, slot i / G
+#pragma unroll 1
+    for (int i = tid; i < M * GNw; i += nt) {
+      const int dd = i / GNw, k = i - dd * GNw;
+      const int n = all ? min(max(recs[dd * (GNw + 1)], 0), GNw) : 0;
+      if (k == 0) nwin[dd] = n;
+      if (k >= n) continue;
+      const int e = CK(p.ws.status, recs[dd * (GNw + 1) + 1 + k], E);
+      if (dd < 32) atomicOr(&host_lo[e], 1u << dd); else atomicOr(&host_hi[e], 1u << (dd - 32));
+      if (dd == dm) {
+        const int g = k % G, j = k / G, col = g * s_phys + e_loc + j;
+        col_expert[col] = e;
+        col_cr[col] = p.cost_rank_inter;   // its main lies in another domain
+        hostcol[g * E + e] = (short)col;
+        atomicMax(&used[g], j + 1);
+      }
+    }
+  } else if (M > 1 && p.stage1_slots > 0) {
     const int slots = G * p.stage1_slots;   // all N per rank unless some are reserved
 #pragma unroll 1
     for (int dd = warp; dd < M; dd += nwarps) {
@@ -309,6 +361,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
     if (closed) return;
   }
 
+  TL_MAX(p.ws, 20);   // inter-node placement known
   // ---- second batch of asynchronous copies: the routing-matrix columns of this domain's replicas ----
 #pragma unroll 1
   for (int i = warp; i < G * N; i += nwarps) {
@@ -404,6 +457,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   }
   __syncthreads();
 
+  TL_MAX(p.ws, 21);   // routing constructed, loads known
   // ---- intra-node refinement: warp 0, one commit per iteration ------------------------------
   if (warp == 0) {
     int it = 0;
@@ -536,6 +590,7 @@ __device__ __forceinline__ void solve_body(const SolveParams& p, unsigned char* 
   }
   __syncthreads();
 
+  TL_MAX(p.ws, 22);   // refinement done
   // ---- results of this domain ----------------------------------------------------------------
 #pragma unroll 1
   for (int idx = tid; idx < G * N; idx += nt) {

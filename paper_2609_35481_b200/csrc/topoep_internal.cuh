@@ -246,6 +246,7 @@ void solve_static_fill(const Dims& d, int dm, const int32_t* main_rank, const in
 size_t route_smem_bytes(const Dims& d);
 size_t reroute_smem_bytes(const Dims& d, int tile_ids);
 // second kernel of the two-kernel chain: solver blocks first, per-token blocks after them
+constexpr unsigned kFlagWaitLimit = 1u << 20;   // polls (roughly a second) for a record or flag of another block
 constexpr int kPlan2TileIds = kSolveThreads * kIdsPerThread;   // one block shape for both roles
 size_t plan2_smem_bytes(const Dims& d, int tiles);
 long long plan2_blocks(const Dims& d, int tiles, int batch);   // blocks of its grid (two-kernel chain)
