@@ -36,13 +36,19 @@ def _check(res):
 
 
 @pytest.mark.parametrize("name,chain,batch", [("dsv3", 0, 1), ("dsv3", 1, 1), ("tiny", 2, 2),
-                                              ("scaleout", 0, 1), ("mid", 3, 2)])
+                                              ("scaleout", 0, 1), ("mid", 3, 2), ("dsv3", 11, 2)])
 def test_captured_plan_is_kernel_nodes_only(name, chain, batch):
+    # chain 11: five kernels with the one-byte copy of the ids (histogram writes, reroute reads it)
+    packed = chain == 11
+    chain = 1 if packed else chain
     rt = _cudart()
     w = wl.CONFIGS[name]
     ids = wl.make_topk_ids(w, seed=5, batch=batch)
     pl = make_planner(w, max_batch=batch)
     pl.set_tuning(B.KNOB_CHAIN, chain)
+    if packed:
+        pl.set_tuning(B.KNOB_PACKED_IDS, 2)
+        assert B.topoep_plan_byte_copy(pl.handle, w.tokens_per_rank, batch) == 1
     dev_ids = torch.from_numpy(ids).to(pl.device)
     out = pl.alloc_outputs(batch, w.tokens_per_rank)
     pl.plan(dev_ids, out)                        # first call outside capture
@@ -60,6 +66,13 @@ def test_captured_plan_is_kernel_nodes_only(name, chain, batch):
     assert n == B.topoep_plan_kernels(pl.handle, w.tokens_per_rank, batch)
     # by size: two kernels for a small plan, four for a single 128-rank plan; forced otherwise
     assert n == {("dsv3", 0): 2, ("dsv3", 1): 5, ("tiny", 2): 2, ("scaleout", 0): 4, ("mid", 3): 4}[(name, chain)]
+    if packed:   # the captured launches are the byte-copy pair, not the plain kernels
+        from torch.profiler import ProfilerActivity, profile
+        with profile(activities=[ProfilerActivity.CUDA]) as prof:
+            pl.plan(dev_ids, out)
+            torch.cuda.synchronize()
+        launched = [e.name for e in prof.events() if str(e.device_type).endswith("CUDA")]
+        assert any("reroute_rows_kernel" in k for k in launched), launched
     # the graph still does the work: instantiate, replay, compare with the oracle
     exe = _check(rt.cudaGraphInstantiate(graph, 0))
     out.token_replica.fill_(-7)
