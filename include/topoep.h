@@ -158,7 +158,7 @@ enum {
                                    L2 cache; 1: never; 2: whenever possible       */
   TOPOEP_KNOB_REROUTE_TILES = 7,/* consecutive tiles of one source a block of the
                                    reroute kernel walks when it reads the one-byte
-                                   copy: 1..64, default 4                         */
+                                   copy: 1..64, default 2                         */
   TOPOEP_KNOB_TRANSFER_SELFTEST = 4 /* tests only (the one knob that does change
                                    output): 1 makes one block of the bulk engine
                                    wait for a copy it never issued, so its bounded

@@ -234,7 +234,7 @@ int topoep_create(topoep_handle_t* out, int nodes, int gpus_per_node, int expert
   h->chain = 0;
   h->pack_ids = 0;
   h->packed_src = nullptr;
-  h->reroute_tiles_per_block = 4;
+  h->reroute_tiles_per_block = 2;
   h->l2_bytes = 0;
   h->plan2_smem = 0;
   h->aux_valid = false;

@@ -255,8 +255,6 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
       for (int e = tid; e < E; e += nt) cp_async4(route + e, g_route + e);
     }
   }
-#pragma unroll
-  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) route[E] = -1;   // an id outside [0,E) (re-read tiles) is clamped onto this entry
 
 #pragma unroll 1
@@ -287,15 +285,31 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
     if (tid == 0) hdr[2 + (cur ^ 1)] = 0;   // the next tile's work counter; nobody reads it now
     // A split expert whose ids of THIS tile all fall inside one instance's quota interval is not
     // split here: its table entry becomes that instance, else (again) the split mark.
+    int marks = 0;   // does the table hold a split mark for this tile?
     if (n_split > 0) {   // uniform
+      int mine = 0;
       if (tid < kSplitCap && tid < n_split) {
         const int res = tbase[kSplitCap + tid], e = tbase[2 * kSplitCap + tid];
-        if (e >= 0) route[e] = res >= 0 ? res : -2 - tid;
+        if (e >= 0) { route[e] = res >= 0 ? res : -2 - tid; mine = res < 0; }
       }
-      __syncthreads();
+      marks = __syncthreads_or(mine) | (n_split > kSplitCap);
     }
     int* n_work_p = hdr + 2 + cur;
-    if (!reread) {
+    if (!reread && !marks) {
+      // Nine tiles in ten: every id is a valid expert and no entry of the table is a split mark
+      // (each split expert's ids of this tile lie inside one instance's quota): look up, store.
+      const char* rb = reinterpret_cast<const char*>(route);
+#pragma unroll
+      for (int j = 0; j < kIdsPerThread / 4; ++j) {
+        const int vec = j * nt + tid;
+        const unsigned w = xb[j];
+        const int t0 = *reinterpret_cast<const int*>(rb + ((w << 2) & 0x3fcu));
+        const int t1 = *reinterpret_cast<const int*>(rb + ((w >> 6) & 0x3fcu));
+        const int t2 = *reinterpret_cast<const int*>(rb + ((w >> 14) & 0x3fcu));
+        const int t3 = *reinterpret_cast<const int*>(rb + ((w >> 22) & 0x3fcu));
+        if (4 * vec < count) __stcs(reinterpret_cast<int4*>(out) + vec, make_int4(t0, t1, t2, t3));
+      }
+    } else if (!reread) {
       // Every id of the tile is a valid expert (the histogram saw none outside [0, E)), so a table
       // entry is an instance (>= 0) or a split mark (< 0): no clamp, and the sign alone tells the
       // split ids.  Their marks are stored as they are: each of them is patched below.  The byte
@@ -340,17 +354,19 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
           if (t[u] < -1) work[CK(p.ws.status, atomicAdd(n_work_p, 1), p.tile_ids)] = (unsigned short)(4 * vec + u);
       }
     }
-    __syncthreads();   // also orders the stores above before the patches below
-    const int n_work = *n_work_p;
-    if (n_work > 0) {   // uniform
-      const int32_t* g_tp = p.ws.tile_pref + (row * (size_t)p.max_tiles + tile) * E;
-      const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, rec, g_tp, ids, out,
-                          rl, rows, n_split, hdr[1], n_work, p.ws.status, false};
-      rank_and_patch(c, tid, nt, warp, nwarps);
-      // fresh counters for the next tile that ranks (its first pass expects them zeroed)
-      __syncthreads();
+    if (reread || marks) {   // uniform: something may have been pushed
+      __syncthreads();   // also orders the stores above before the patches below
+      const int n_work = *n_work_p;
+      if (n_work > 0) {   // uniform
+        const int32_t* g_tp = p.ws.tile_pref + (row * (size_t)p.max_tiles + tile) * E;
+        const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, rec, g_tp, ids, out,
+                            rl, rows, n_split, hdr[1], n_work, p.ws.status, false};
+        // the ranking's first pass expects its counters zeroed: only the tiles that rank pay for it
 #pragma unroll
-      for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
+        for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        rank_and_patch(c, tid, nt, warp, nwarps);
+      }
     }
 #pragma unroll
     for (int j = 0; j < kIdsPerThread / 4; ++j) xb[j] = xn[j];
