@@ -125,11 +125,6 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
       for (int e = tid; e < E; e += nt) cp_async4(route + e, g_route + e);
     }
   }
-  // rows = blockDim.x / 8, so the kSplitCap * rows counter words are exactly kSplitCap / 8 per
-  // thread: straight-line stores (a counted loop here cost a hundred instructions per warp)
-  static_assert(kSplitCap % 8 == 0, "counter words per thread");
-#pragma unroll
-  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) route[E] = -1;   // every id outside [0,E) is clamped onto this entry
   cp_async_wait_all();           // hdr[2], the work-list length, arrives as the record's zero
   __syncthreads();
@@ -137,12 +132,36 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   // route kernel checked the tile's rank interval against the quotas) is not split here: its
   // table entry becomes that instance and its ids stream like everyone else's.  Only tiles that
   // straddle a quota boundary -- about one in ten on the benchmark workloads -- rank anything.
+  int marks = 0;   // does the table still hold a split mark for this tile?
   if (hdr[0] > 0) {   // uniform: the source has split experts at all
+    int mine = 0;
     if (tid < kSplitCap) {
       const int res = tbase[kSplitCap + tid], e = tbase[2 * kSplitCap + tid];
-      if (tid < hdr[0] && res >= 0 && e >= 0) route[e] = res;
+      if (tid < hdr[0] && e >= 0) {
+        if (res >= 0) route[e] = res; else mine = 1;
+      }
     }
-    __syncthreads();
+    marks = __syncthreads_or(mine) | (hdr[0] > kSplitCap);
+  }
+  if (!marks) {
+    // Most tiles: no entry of the table is a split mark, so every entry is an instance or the -1
+    // of an ignored id: look up, store, done (no mask of split ids, no work list, no barrier).
+    const unsigned uE = (unsigned)E;
+#pragma unroll
+    for (int j = 0; j < kIdsPerThread / 4; ++j) {
+      const int vec = j * nt + tid;
+      const int4 r = make_int4(route[min((unsigned)x[j].x, uE)], route[min((unsigned)x[j].y, uE)],
+                               route[min((unsigned)x[j].z, uE)], route[min((unsigned)x[j].w, uE)]);
+      if (VEC) {
+        if (4 * vec < count) __stcs(reinterpret_cast<int4*>(out) + vec, r);
+      } else {
+        if (4 * vec + 0 < count) out[4 * vec + 0] = r.x;
+        if (4 * vec + 1 < count) out[4 * vec + 1] = r.y;
+        if (4 * vec + 2 < count) out[4 * vec + 2] = r.z;
+        if (4 * vec + 3 < count) out[4 * vec + 3] = r.w;
+      }
+    }
+    return;
   }
 
   // Stream: look up and store.  An ignored id and a split id both store -1 for now; the split
@@ -180,6 +199,13 @@ __global__ void __launch_bounds__(kMaxTileIds / kIdsPerThread, TOPOEP_REROUTE_MI
   const int n_work = hdr[2];
   if (n_work == 0) return;
 
+  // The ranking's first pass expects its counters zeroed: only the tiles that rank pay for it.
+  // rows = blockDim.x / 8, so the kSplitCap * rows counter words are exactly kSplitCap / 8 per
+  // thread: straight-line stores (a counted loop here cost a hundred instructions per warp).
+  static_assert(kSplitCap % 8 == 0, "counter words per thread");
+#pragma unroll
+  for (int u = 0; u < kSplitCap / 8; ++u) cnt4[u * nt + tid] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
   const SplitCtx c = {cnt4, cntw, base, route, seg, cum, inst, tbase, work, rec, g_tp, ids, out,
                       rl, rows, hdr[0], hdr[1], n_work, p.ws.status, false};
   rank_and_patch(c, tid, nt, warp, nwarps);
