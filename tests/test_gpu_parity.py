@@ -210,6 +210,49 @@ def test_random_problems_with_policies_tunings_and_skew():
         pl.close()
 
 
+def test_random_many_domain_problems_through_the_combined_kernel():
+    """Many domains and experts (M * E >= 4096): there the solver blocks of the combined kernel read
+    the published inter-node placement instead of ranking every domain's demand again.  Random
+    shapes, main maps, padding and slot reservations through the two- and four-kernel chains."""
+    rng = np.random.default_rng(33)
+    done = 0
+    while done < 40:
+        M, G = int(rng.integers(4, 33)), int(rng.integers(1, 9))
+        R = M * G
+        E = int(rng.integers(max(1, 4096 // M), 1200))
+        N = int(rng.integers(0, 4))
+        k = int(rng.integers(1, 9))
+        T = int(rng.integers(1, 1500))
+        Bn = int(rng.integers(1, 3))
+        main = rng.integers(0, R, size=E).astype(np.int32)
+        tok, W = int(rng.integers(1, 64)), int(rng.integers(0, 2000))
+        skew = float(rng.uniform(0.5, 3.0))
+        ids = np.minimum((rng.random((Bn, R, T, k)) ** skew * E).astype(np.int32), E - 1)
+        if rng.random() < 0.3:
+            ids[rng.random(ids.shape) < 0.02] = -1
+        w = wl.Workload("rnd", M, G, E, N, k, T)
+        reserve = int(rng.integers(0, N + 1))
+        over = dict(main_rank=main, token_bytes=tok, expert_bytes=W,
+                    c_intra=int(rng.integers(0, 3)), c_inter=int(rng.integers(0, 9)))
+        try:
+            pl = make_planner(w, max_batch=Bn, **over)
+        except Exception:
+            continue   # a shape the library refuses (tables beyond shared memory)
+        pl.set_policy(B.POLICY_RESERVE_SLOTS, reserve)
+        chain = int(rng.choice([0, 2, 3]))
+        pl.set_tuning(B.KNOB_CHAIN, chain)
+        ref = orc.plan(oracle_config(w, reserve_slots=reserve, **over), ids)
+        for rep in range(2):
+            gpu = run_gpu(pl, ids)
+            try:
+                assert_same(gpu, ref)
+            except AssertionError as err:
+                raise AssertionError("%s: %s" % ((M, G, E, N, k, T, Bn, chain, reserve), err))
+            assert gpu["flags"] == ref.flags
+        pl.close()
+        done += 1
+
+
 def test_invalid_and_padded_ids():
     w = wl.CONFIGS["tiny"].replace(slots_per_rank=2)
     ids = wl.make_topk_ids(w, seed=4, batch=2).copy()
